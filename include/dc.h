@@ -1,0 +1,210 @@
+/*
+ * dc.h -- C ABI of libdepthc: merging runs of convolutions into one convolution and
+ * running the merged network's layers on an NVIDIA B200 (sm_100a).
+ *
+ * Source of the operations: arXiv 2301.12187, "Efficient Latency-Aware CNN Depth
+ * Compression via Two-Stage Dynamic Programming" -- Sec. 3 (merging two convolutions,
+ * f_{theta2}(f_{theta1}(X)) = f_{theta2 (*) theta1}(X)), Eq. 1 (theta^_i is the merge
+ * of the run s_{i-1}+1..s_i), Sec. 2 / Sec. 5.1 (BN fused into the preceding
+ * convolution), App. E.1 (skip addition folded into a single merged convolution),
+ * App. E.2 (all zero padding of a run moved to its first convolution).
+ *
+ * Conventions
+ *   - Feature maps are NHWC, dense, row-major: x[n][h][w][c].  dtype DC_F32 (float) or
+ *     DC_BF16 (bfloat16 storage, fp32 accumulation).
+ *   - Kernels handed in are fp32 [c_out][c_in/groups][k][k]; groups is 1 (dense) or
+ *     c_in == c_out (depthwise).  Square odd k, symmetric zero padding, dilation 1.
+ *   - Forward: y[n,Y,X,o] = act( b[o] + sum_{i,u,v} W[o,i,u,v] * x[n, Y*s+u-p, X*s+v-p, i] ),
+ *     zero outside the image, H_out = floor((H + 2p - k)/s) + 1  (cross-correlation).
+ *   - Every tensor pointer is a DEVICE pointer aligned to 16 bytes unless the argument is
+ *     documented as a host pointer.  Descriptor structs (dc_layer, dc_geom, ...) are HOST
+ *     memory and are only read during the call.
+ *   - Ownership: the caller owns every buffer, workspaces included.  The library never
+ *     allocates or frees device memory.
+ *   - Every call enqueues work on `stream` and returns without synchronising, except
+ *     dc_workspace_status and the *_host entry points, which say so.
+ *   - Errors: a dc_status is returned; argument and shape errors are detected on the host
+ *     before anything is launched.  Device-side waits are bounded; a wait that runs out
+ *     latches DC_ERR_TIMEOUT in the first word of the caller's workspace (read it with
+ *     dc_workspace_status) and the kernel returns without hanging.
+ */
+#ifndef DC_H_
+#define DC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *dc_stream; /* a cudaStream_t; NULL is the legacy default stream */
+
+typedef enum {
+  DC_OK = 0,
+  DC_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, bad enum, n <= 0 ...          */
+  DC_ERR_SHAPE = 2,         /* layer shapes do not connect, kernel larger than padded image    */
+  DC_ERR_UNSUPPORTED = 3,   /* even k, groups other than 1 or c, shape outside a kernel's range */
+  DC_ERR_NOT_MERGEABLE = 4, /* skip group without stride 1, c_in == c_out and 2p == k-1        */
+  DC_ERR_WORKSPACE = 5,     /* workspace missing or too small                                  */
+  DC_ERR_ALIGNMENT = 6,     /* a tensor pointer is not 16-byte aligned                         */
+  DC_ERR_CUDA = 7,          /* a CUDA runtime/driver call failed                               */
+  DC_ERR_TIMEOUT = 8        /* a bounded device-side wait ran out                              */
+} dc_status;
+
+typedef enum { DC_F32 = 0, DC_BF16 = 1 } dc_dtype;
+typedef enum { DC_ACT_IDENTITY = 0, DC_ACT_RELU6 = 1 } dc_act;
+typedef enum { DC_ALGO_AUTO = 0, DC_ALGO_TCGEN05 = 1, DC_ALGO_SIMT = 2 } dc_algo;
+
+/* One convolution of a run, optionally followed by an eval-mode batch-norm (Sec. 3: f_theta_l). */
+typedef struct {
+  int c_in, c_out, groups;   /* groups == 1 dense; groups == c_in == c_out depthwise            */
+  int k, stride, pad;
+  const float *weight;       /* device, fp32 [c_out][c_in/groups][k][k]                         */
+  const float *bias;         /* device, fp32 [c_out], or NULL                                   */
+  const float *bn_gamma, *bn_beta, *bn_mean, *bn_var; /* device fp32 [c_out]; all NULL: no BN   */
+  float bn_eps;
+} dc_layer;
+
+/* Skip addition y = run[first..last](x) + x inside a run (App. E.1).  Groups are disjoint and
+ * listed in increasing order. */
+typedef struct { int first, last; } dc_residual;
+
+/* Geometry of one convolution (merged or not). */
+typedef struct { int c_in, c_out, groups, k, stride, pad; } dc_geom;
+
+/* An unmerged inverted-residual block: expand 1x1 (optional) -> depthwise -> project 1x1 (+x). */
+typedef struct {
+  int c_in, c_hidden, c_out;
+  int has_expand;            /* 0: the block starts at the depthwise layer (c_hidden == c_in)   */
+  int dw_k, dw_stride, dw_pad;
+  int has_residual;          /* add the block input to the projection (stride 1, c_in == c_out) */
+  dc_act act_expand, act_dw; /* activation after expand and after depthwise                     */
+  const void *w_expand;      /* packed by dc_pack_weights for the call's dtype, or NULL         */
+  const float *b_expand;
+  const float *w_dw;         /* packed depthwise weights fp32 [k][k][c_hidden]                  */
+  const float *b_dw;
+  const void *w_project;     /* packed by dc_pack_weights for the call's dtype                  */
+  const float *b_project;
+} dc_block;
+
+const char *dc_status_string(dc_status s);
+
+/*
+ * BN fusion (Sec. 2 "TensorRT", Sec. 5.1 "Evaluation"): w_out[o,.] = g[o]*W[o,.],
+ * b_out[o] = beta[o] + (bias[o] - mean[o])*g[o], g = gamma/sqrt(var + eps); without BN it copies
+ * W and the bias (zeros if NULL).  w_out: device fp32, same shape as layer->weight; b_out: device
+ * fp32 [c_out].  fp32 arithmetic.
+ */
+dc_status dc_fold_bn(const dc_layer *layer, float *w_out, float *b_out, dc_stream stream);
+
+/*
+ * Host only: geometry of the merged convolution of a run (Sec. 3, Eq. 1) and the bytes of
+ * device workspace dc_merge_chain needs for it.  k' = k1 + (k2-1) s1, s' = s1 s2,
+ * p' = p1 + p2 s1, folded along the run.  Checks that shapes connect (DC_ERR_SHAPE), that
+ * each skip group has stride 1, c_in == c_out and 2p == k-1 (DC_ERR_NOT_MERGEABLE, App. E.1),
+ * odd k and groups in {1, c} (DC_ERR_UNSUPPORTED).  No device pointer is dereferenced.
+ */
+dc_status dc_merge_query(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                         dc_geom *merged, size_t *workspace_bytes);
+
+/* Host only: bytes of the packed-weight buffer dc_conv_forward / dc_dwconv_forward read for a
+ * convolution of this geometry and dtype. */
+dc_status dc_packed_bytes(const dc_geom *g, dc_dtype dtype, size_t *bytes);
+
+/*
+ * Merge a run of convolutions whose intermediate activations are identities into one
+ * convolution (Sec. 3; Eq. 1; App. E.1 for skips; App. E.2: the result equals the run with
+ * all its zero padding applied before the first layer).  BN is folded per layer, depthwise
+ * layers act as diagonal kernels, each skip group is merged first and gets an identity tap at
+ * its centre, pieces are composed left to right:
+ *   W'[o,i,u1+s1*u2,v1+s1*v2] += W2[o,c,u2,v2] * W1[c,i,u1,v1],  b' = b2 + (sum_taps W2) b1.
+ * Outputs (device): w_merged fp32 [c_out][c_in][k'][k'], b_merged fp32 [c_out]; if w_packed is
+ * not NULL also the packed copy for packed_dtype (size from dc_packed_bytes).  workspace: device,
+ * at least the bytes dc_merge_query reports.  fp32 FMA arithmetic throughout.
+ */
+dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                         float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
+                         void *workspace, size_t workspace_bytes, dc_stream stream);
+
+/*
+ * Repack fp32 [c_out][c_in/groups][k][k] weights (device) into the layout the forward kernels
+ * read.  Dense, DC_F32: fp32 [k][k][c_in][c_out].  Dense, DC_BF16: bfloat16 (round to nearest
+ * even) in the K-chunked operand layout of the tensor-core kernel, zero padded (opaque; size
+ * from dc_packed_bytes).  Depthwise, either dtype: fp32 [k][k][c].
+ */
+dc_status dc_pack_weights(const float *w, const dc_geom *g, dc_dtype dtype, void *w_packed,
+                          dc_stream stream);
+
+/* Host only: bytes of workspace dc_conv_forward needs (a status word plus padding). */
+size_t dc_conv_workspace_bytes(void);
+
+/*
+ * Forward pass of one dense convolution (the merged layer f_{theta^_i} of Eq. 1, or an
+ * unmerged 1x1 / stem / head layer):  y = act(conv(x) + bias + residual).
+ * x: [n][h][w][c_in], y: [n][h_out][w_out][c_out], residual: same shape as y or NULL, all of
+ * `dtype`; w_packed from dc_merge_chain / dc_pack_weights for the same dtype; bias fp32 [c_out]
+ * or NULL.  DC_BF16 runs as an implicit GEMM on the tensor cores (fp32 accumulate) when the
+ * shape allows (c_in, c_out multiples of 8, stride 1 or 2, ...), else on CUDA cores; DC_F32
+ * runs on CUDA cores in fp32.  workspace: device, >= dc_conv_workspace_bytes(), zeroed once by
+ * the caller.
+ */
+dc_status dc_conv_forward(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                          const float *bias, dc_act act, const void *residual, void *y,
+                          dc_dtype dtype, void *workspace, size_t workspace_bytes, dc_stream stream);
+
+/* As dc_conv_forward with the kernel family forced; DC_ERR_UNSUPPORTED if it cannot run the shape. */
+dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, const dc_geom *g,
+                               const void *w_packed, const float *bias, dc_act act,
+                               const void *residual, void *y, dc_dtype dtype, void *workspace,
+                               size_t workspace_bytes, dc_stream stream, dc_algo algo);
+
+/*
+ * Forward pass of one depthwise convolution (the layers the merge leaves alone):
+ * y[n,Y,X,c] = act( bias[c] + sum_{u,v} w[u][v][c] * x[n, Y*s+u-p, X*s+v-p, c] ).
+ * w: fp32 [k][k][c] (dc_pack_weights with groups == c), bias fp32 [c] or NULL.
+ */
+dc_status dc_dwconv_forward(const void *x, int n, int h, int w, int c, int k, int stride, int pad,
+                            const float *w_packed, const float *bias, dc_act act, void *y,
+                            dc_dtype dtype, dc_stream stream);
+
+/* Host only: workspace bytes dc_block_forward needs for this input size. */
+dc_status dc_block_workspace_bytes(int n, int h, int w, const dc_block *blk, dc_dtype dtype,
+                                   size_t *bytes);
+
+/*
+ * Forward pass of one unmerged inverted-residual block: expand 1x1 + act, depthwise + act,
+ * project 1x1, plus the block input when has_residual (the skip addition that stays explicit
+ * when the block is not merged into a single convolution, App. E.1).
+ */
+dc_status dc_block_forward(const void *x, int n, int h, int w, const dc_block *blk, void *y,
+                           dc_dtype dtype, void *workspace, size_t workspace_bytes,
+                           dc_stream stream);
+
+/*
+ * Synchronises `stream`, then returns the status latched in the first word of `workspace`
+ * (DC_OK or DC_ERR_TIMEOUT) and clears it.
+ */
+dc_status dc_workspace_status(void *workspace, dc_stream stream);
+
+/* Host only: bytes of device workspace dc_chain_forward_host needs. */
+dc_status dc_chain_host_workspace_bytes(const dc_layer *layers, int n_layers, const dc_residual *res,
+                                        int n_res, int n, int h, int w, dc_dtype dtype,
+                                        size_t *bytes);
+
+/*
+ * The whole path from HOST buffers: copy the run's parameters and the input to the device,
+ * merge the run (dc_merge_chain), run the merged convolution (dc_conv_forward) and copy the
+ * output back.  In `layers` every pointer is a HOST pointer here.  x_host / y_host: host
+ * NHWC buffers of `dtype` (pinned memory makes the copies asynchronous).  workspace: device.
+ * Synchronises the stream before returning.
+ */
+dc_status dc_chain_forward_host(const dc_layer *layers, int n_layers, const dc_residual *res,
+                                int n_res, const void *x_host, int n, int h, int w, dc_act act,
+                                void *y_host, dc_dtype dtype, void *workspace,
+                                size_t workspace_bytes, dc_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DC_H_ */

@@ -1,0 +1,140 @@
+// Shared declarations of the CUDA library (host planning structs, K-order of the packed
+// bf16 operand, small helpers).  Internal: the public contract is include/dc.h.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dc.h"
+
+#define DC_CUDA_OK(expr)                        \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) return DC_ERR_CUDA; \
+  } while (0)
+
+static inline bool dc_aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t dc_round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
+static inline int dc_floor_div2(int a) { return (a >= 0) ? a / 2 : -((-a + 1) / 2); }
+
+static inline int dc_out_extent(int h, int k, int s, int p) {
+  int a = h + 2 * p - k;
+  return a < 0 ? 0 : a / s + 1;
+}
+
+// ----------------------------------------------------------------------------------------------
+// K order of the packed bf16 weights (B operand) and of the activation planes (A operand).
+//
+// The reduction index of the implicit GEMM is cut into chunks of 8 input channels (16 bytes).
+// A chunk entry is (column parity pc, channel chunk cc, tap row r, tap column s).  The input
+// channels are processed in `ng` groups of `cg` chunks; inside a group the entries are ordered
+// by (pc, cc, r, s) -- the order in which their shared-memory addresses increase -- and padded
+// with one all-zero entry when their count is odd, because one tensor-core instruction consumes
+// two entries (K = 16).  Stride 1 has a single parity; stride 2 splits the taps by the parity
+// of the input column they read.
+// ----------------------------------------------------------------------------------------------
+struct KOrder {
+  int k, stride, pad;
+  int c_in, cch;      // input channels, chunks of 8 (rounded up)
+  int cg, ng;         // chunks per group, groups
+  int taps;           // k*k
+  int pcs;            // 1 (stride 1) or 2 (stride 2)
+  int ns[2];          // tap columns of each parity
+  int s0[2];          // first tap column of each parity
+  int e;              // entries per group = cg * taps
+  int e_pad;          // e rounded up to even
+  int n_pad;          // output channels rounded up to 16
+};
+
+static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
+  ko->k = g->k; ko->stride = g->stride; ko->pad = g->pad;
+  ko->c_in = g->c_in;
+  ko->cch = dc_div_up(g->c_in, 8);
+  ko->taps = g->k * g->k;
+  ko->n_pad = (int)dc_round_up((size_t)g->c_out, 16);
+  ko->pcs = (g->stride == 2) ? 2 : 1;
+  if (ko->pcs == 1) {
+    ko->ns[0] = g->k; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
+  } else {
+    for (int pc = 0; pc < 2; ++pc) {
+      ko->s0[pc] = (g->pad + pc) & 1;
+      ko->ns[pc] = (ko->s0[pc] >= g->k) ? 0 : (g->k - ko->s0[pc] + 1) / 2;
+    }
+  }
+  // largest divisor of cch that is <= 8 and keeps one group's weights for <= 256 output
+  // channels within 64 KB of shared memory
+  int n_tile = ko->n_pad < 256 ? ko->n_pad : 256;
+  int best = 1;
+  for (int d = 1; d <= 8 && d <= ko->cch; ++d) {
+    if (ko->cch % d) continue;
+    if ((size_t)d * ko->taps * n_tile * 16 <= 64 * 1024) best = d;
+  }
+  ko->cg = best;
+  ko->ng = ko->cch / best;
+  ko->e = ko->cg * ko->taps;
+  ko->e_pad = (ko->e + 1) & ~1;
+}
+
+// entry index within a group -> (pc, ccg, r, s); returns false for the zero padding entry
+__host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
+                                                        int *r, int *s) {
+  if (e >= ko.e) return false;
+  if (ko.pcs == 1) {
+    *pc = 0;
+    *ccg = e / ko.taps;
+    int t = e - *ccg * ko.taps;
+    *r = t / ko.k;
+    *s = t - *r * ko.k;
+    return true;
+  }
+  int per0 = ko.k * ko.ns[0];
+  int n0 = ko.cg * per0;
+  int p = (e < n0) ? 0 : 1;
+  int ee = (p == 0) ? e : e - n0;
+  int per = ko.k * ko.ns[p];
+  *pc = p;
+  *ccg = ee / per;
+  int rem = ee - *ccg * per;
+  *r = rem / ko.ns[p];
+  *s = ko.s0[p] + 2 * (rem - *r * ko.ns[p]);
+  return true;
+}
+
+// (channel chunk cc in [0,cch), tap r, s) -> position of that chunk in the packed weights,
+// in units of chunk planes (n_pad * 8 elements each)
+__host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
+  int grp = cc / ko.cg, ccg = cc - grp * ko.cg;
+  int e;
+  if (ko.pcs == 1) {
+    e = ccg * ko.taps + r * ko.k + s;
+  } else {
+    int p = ((s - ko.pad) & 1);
+    int per = ko.k * ko.ns[p];
+    int base = (p == 0) ? 0 : ko.cg * ko.k * ko.ns[0];
+    e = base + ccg * per + r * ko.ns[p] + (s - ko.s0[p]) / 2;
+  }
+  return grp * ko.e_pad + e;
+}
+
+__device__ __forceinline__ float dc_act_apply(float v, int act) {
+  return act == DC_ACT_RELU6 ? fminf(fmaxf(v, 0.f), 6.f) : v;
+}
+
+// Workspace header written by kernels with bounded waits.
+struct DcWsHeader {
+  unsigned int status;      // 0 or DC_ERR_TIMEOUT
+  unsigned int where;       // which wait gave up
+  unsigned int pad[62];
+};
+
+// internal launchers (defined in the .cu files)
+dc_status dc_launch_conv_simt(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y,
+                              dc_dtype dtype, cudaStream_t stream);
+dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                            const float *bias, dc_act act, const void *residual, void *y,
+                            void *workspace, cudaStream_t stream);
+bool dc_conv_tc_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_validate_geom(const dc_geom *g);

@@ -1,0 +1,260 @@
+// CUDA-core convolution kernels: the fp32 accuracy path of the dense convolution, a generic
+// bf16 dense convolution for shapes the tensor-core kernel does not take, and the depthwise
+// stencil.  NHWC, fp32 accumulation.
+#include "common.cuh"
+
+// ----------------------------------------------------------------------------------------------
+// dense, fp32: one thread = one output pixel x 4 consecutive output channels.
+// weights fp32 [k][k][c_in][c_out]: threads of a pixel read consecutive output channels.
+// ----------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_conv_dense_f32(const float *__restrict__ x, const float *__restrict__ w,
+                                                        const float *__restrict__ bias,
+                                                        const float *__restrict__ residual, float *__restrict__ y,
+                                                        int n, int h, int wd, int ho, int wo, dc_geom g, int act) {
+  const int noc = (g.c_out + 3) / 4;
+  const long long total = (long long)n * ho * wo * noc;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int oc = (int)(idx % noc) * 4;
+    long long pix = idx / noc;
+    const int X = (int)(pix % wo), Y = (int)((pix / wo) % ho), img = (int)(pix / ((long long)wo * ho));
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int u = 0; u < g.k; ++u) {
+      const int yy = Y * g.stride + u - g.pad;
+      if (yy < 0 || yy >= h) continue;
+      for (int v = 0; v < g.k; ++v) {
+        const int xx = X * g.stride + v - g.pad;
+        if (xx < 0 || xx >= wd) continue;
+        const float *xp = x + (((size_t)img * h + yy) * wd + xx) * g.c_in;
+        const float *wp = w + ((size_t)(u * g.k + v) * g.c_in) * g.c_out + oc;
+        for (int c = 0; c < g.c_in; ++c) {
+          const float xv = xp[c];
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (oc + q < g.c_out) acc[q] = fmaf(xv, wp[(size_t)c * g.c_out + q], acc[q]);
+        }
+      }
+    }
+    const size_t obase = (((size_t)img * ho + Y) * wo + X) * g.c_out + oc;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (oc + q < g.c_out) {
+        float v = acc[q] + (bias ? bias[oc + q] : 0.f);
+        if (residual) v += residual[obase + q];
+        y[obase + q] = dc_act_apply(v, act);
+      }
+  }
+}
+
+// ----------------------------------------------------------------------------------------------
+// dense, bf16 storage: one thread = one output pixel x one output channel; the packed weights
+// are the chunk planes [plane][n_pad][8] of KOrder, so threads of a pixel read consecutive
+// 16-byte chunks.  fp32 accumulation, one rounding at the store.
+// ----------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_conv_dense_bf16(const __nv_bfloat16 *__restrict__ x,
+                                                         const __nv_bfloat16 *__restrict__ w,
+                                                         const float *__restrict__ bias,
+                                                         const __nv_bfloat16 *__restrict__ residual,
+                                                         __nv_bfloat16 *__restrict__ y, int n, int h, int wd,
+                                                         int ho, int wo, dc_geom g, KOrder ko, int act) {
+  const long long total = (long long)n * ho * wo * g.c_out;
+  const bool vec = (g.c_in % 8) == 0;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int o = (int)(idx % g.c_out);
+    long long pix = idx / g.c_out;
+    const int X = (int)(pix % wo), Y = (int)((pix / wo) % ho), img = (int)(pix / ((long long)wo * ho));
+    float acc = 0.f;
+    for (int u = 0; u < g.k; ++u) {
+      const int yy = Y * g.stride + u - g.pad;
+      if (yy < 0 || yy >= h) continue;
+      for (int v = 0; v < g.k; ++v) {
+        const int xx = X * g.stride + v - g.pad;
+        if (xx < 0 || xx >= wd) continue;
+        const __nv_bfloat16 *xp = x + (((size_t)img * h + yy) * wd + xx) * g.c_in;
+        for (int cc = 0; cc < ko.cch; ++cc) {
+          const int plane = dc_korder_encode(ko, cc, u, v);
+          const uint4 wv = *reinterpret_cast<const uint4 *>(w + ((size_t)plane * ko.n_pad + o) * 8);
+          const __nv_bfloat16 *wb = reinterpret_cast<const __nv_bfloat16 *>(&wv);
+          if (vec) {
+            const uint4 xv = *reinterpret_cast<const uint4 *>(xp + cc * 8);
+            const __nv_bfloat16 *xb = reinterpret_cast<const __nv_bfloat16 *>(&xv);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc = fmaf(__bfloat162float(xb[q]), __bfloat162float(wb[q]), acc);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              if (cc * 8 + q < g.c_in) acc = fmaf(__bfloat162float(xp[cc * 8 + q]), __bfloat162float(wb[q]), acc);
+          }
+        }
+      }
+    }
+    const size_t oi = (((size_t)img * ho + Y) * wo + X) * g.c_out + o;
+    float vout = acc + (bias ? bias[o] : 0.f);
+    if (residual) vout += __bfloat162float(residual[oi]);
+    y[oi] = __float2bfloat16_rn(dc_act_apply(vout, act));
+  }
+}
+
+static inline int simt_blocks(long long total, int threads, int cap) {
+  long long b = (total + threads - 1) / threads;
+  if (b > cap) b = cap;
+  if (b < 1) b = 1;
+  return (int)b;
+}
+
+dc_status dc_launch_conv_simt(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y,
+                              dc_dtype dtype, cudaStream_t stream) {
+  const int ho = dc_out_extent(h, g->k, g->stride, g->pad), wo = dc_out_extent(w, g->k, g->stride, g->pad);
+  if (dtype == DC_F32) {
+    long long total = (long long)n * ho * wo * ((g->c_out + 3) / 4);
+    k_conv_dense_f32<<<simt_blocks(total, 128, 148 * 64), 128, 0, stream>>>(
+        (const float *)x, (const float *)w_packed, bias, (const float *)residual, (float *)y, n, h, w, ho, wo, *g,
+        (int)act);
+  } else {
+    KOrder ko;
+    dc_korder_init(&ko, g);
+    long long total = (long long)n * ho * wo * g->c_out;
+    k_conv_dense_bf16<<<simt_blocks(total, 128, 148 * 64), 128, 0, stream>>>(
+        (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_packed, bias, (const __nv_bfloat16 *)residual,
+        (__nv_bfloat16 *)y, n, h, w, ho, wo, *g, ko, (int)act);
+  }
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+// ----------------------------------------------------------------------------------------------
+// depthwise stencil.  One thread = one output pixel x VEC consecutive channels (16 bytes of
+// storage: 8 bf16 or 4 fp32), so a warp reads and writes whole 128-byte lines of the NHWC map.
+// weights fp32 [k][k][c].
+// ----------------------------------------------------------------------------------------------
+template <typename T> struct DwVec;
+template <> struct DwVec<float> {
+  static constexpr int V = 4;
+  __device__ static void load(const float *p, float *o) {
+    float4 v = *reinterpret_cast<const float4 *>(p);
+    o[0] = v.x; o[1] = v.y; o[2] = v.z; o[3] = v.w;
+  }
+  __device__ static void store(float *p, const float *o) {
+    *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
+  }
+  __device__ static float ld1(const float *p) { return *p; }
+  __device__ static void st1(float *p, float v) { *p = v; }
+};
+template <> struct DwVec<__nv_bfloat16> {
+  static constexpr int V = 8;
+  __device__ static void load(const __nv_bfloat16 *p, float *o) {
+    uint4 v = *reinterpret_cast<const uint4 *>(p);
+    const __nv_bfloat162 *b = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { float2 f = __bfloat1622float2(b[q]); o[2 * q] = f.x; o[2 * q + 1] = f.y; }
+  }
+  __device__ static void store(__nv_bfloat16 *p, const float *o) {
+    uint4 v;
+    __nv_bfloat162 *b = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) b[q] = __floats2bfloat162_rn(o[2 * q], o[2 * q + 1]);
+    *reinterpret_cast<uint4 *>(p) = v;
+  }
+  __device__ static float ld1(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+  __device__ static void st1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_dwconv_vec(const T *__restrict__ x, const float *__restrict__ w,
+                                                    const float *__restrict__ bias, T *__restrict__ y, int n, int h,
+                                                    int wd, int c, int ho, int wo, int k, int stride, int pad,
+                                                    int act) {
+  constexpr int V = DwVec<T>::V;
+  const int cv = c / V;
+  const long long total = (long long)n * ho * wo * cv;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int c0 = (int)(idx % cv) * V;
+    long long pix = idx / cv;
+    const int X = (int)(pix % wo), Y = (int)((pix / wo) % ho), img = (int)(pix / ((long long)wo * ho));
+    float acc[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) acc[q] = bias ? bias[c0 + q] : 0.f;
+    for (int u = 0; u < k; ++u) {
+      const int yy = Y * stride + u - pad;
+      if (yy < 0 || yy >= h) continue;
+      for (int v = 0; v < k; ++v) {
+        const int xx = X * stride + v - pad;
+        if (xx < 0 || xx >= wd) continue;
+        float xv[V];
+        DwVec<T>::load(x + (((size_t)img * h + yy) * wd + xx) * c + c0, xv);
+        const float *wp = w + (size_t)(u * k + v) * c + c0;
+#pragma unroll
+        for (int q = 0; q < V; q += 4) {
+          const float4 wv = *reinterpret_cast<const float4 *>(wp + q);
+          acc[q] = fmaf(xv[q], wv.x, acc[q]);
+          acc[q + 1] = fmaf(xv[q + 1], wv.y, acc[q + 1]);
+          acc[q + 2] = fmaf(xv[q + 2], wv.z, acc[q + 2]);
+          acc[q + 3] = fmaf(xv[q + 3], wv.w, acc[q + 3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < V; ++q) acc[q] = dc_act_apply(acc[q], act);
+    DwVec<T>::store(y + (((size_t)img * ho + Y) * wo + X) * c + c0, acc);
+  }
+}
+
+// any channel count: one thread = one output element
+template <typename T>
+__global__ void k_dwconv_scalar(const T *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias,
+                                T *__restrict__ y, int n, int h, int wd, int c, int ho, int wo, int k, int stride,
+                                int pad, int act) {
+  const long long total = (long long)n * ho * wo * c;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int ch = (int)(idx % c);
+    long long pix = idx / c;
+    const int X = (int)(pix % wo), Y = (int)((pix / wo) % ho), img = (int)(pix / ((long long)wo * ho));
+    float acc = bias ? bias[ch] : 0.f;
+    for (int u = 0; u < k; ++u) {
+      const int yy = Y * stride + u - pad;
+      if (yy < 0 || yy >= h) continue;
+      for (int v = 0; v < k; ++v) {
+        const int xx = X * stride + v - pad;
+        if (xx < 0 || xx >= wd) continue;
+        acc = fmaf(DwVec<T>::ld1(x + (((size_t)img * h + yy) * wd + xx) * c + ch), w[(size_t)(u * k + v) * c + ch], acc);
+      }
+    }
+    DwVec<T>::st1(y + idx, dc_act_apply(acc, act));
+  }
+}
+
+template <typename T>
+static dc_status launch_dw(const void *x, int n, int h, int w, int c, int k, int stride, int pad, const float *wp,
+                           const float *bias, dc_act act, void *y, cudaStream_t st) {
+  const int ho = dc_out_extent(h, k, stride, pad), wo = dc_out_extent(w, k, stride, pad);
+  constexpr int V = DwVec<T>::V;
+  if (c % V == 0) {
+    long long total = (long long)n * ho * wo * (c / V);
+    k_dwconv_vec<T><<<simt_blocks(total, 256, 148 * 32), 256, 0, st>>>((const T *)x, wp, bias, (T *)y, n, h, w, c, ho,
+                                                                      wo, k, stride, pad, (int)act);
+  } else {
+    long long total = (long long)n * ho * wo * c;
+    k_dwconv_scalar<T><<<simt_blocks(total, 256, 148 * 32), 256, 0, st>>>((const T *)x, wp, bias, (T *)y, n, h, w, c,
+                                                                         ho, wo, k, stride, pad, (int)act);
+  }
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+extern "C" dc_status dc_dwconv_forward(const void *x, int n, int h, int w, int c, int k, int stride, int pad,
+                                       const float *w_packed, const float *bias, dc_act act, void *y,
+                                       dc_dtype dtype, dc_stream stream) {
+  if (!x || !y || !w_packed) return DC_ERR_INVALID_ARG;
+  if (n <= 0 || h <= 0 || w <= 0 || c <= 0 || k <= 0 || stride <= 0 || pad < 0) return DC_ERR_INVALID_ARG;
+  if (dtype != DC_F32 && dtype != DC_BF16) return DC_ERR_INVALID_ARG;
+  if (act != DC_ACT_IDENTITY && act != DC_ACT_RELU6) return DC_ERR_INVALID_ARG;
+  if (k % 2 == 0) return DC_ERR_UNSUPPORTED;
+  if (dc_out_extent(h, k, stride, pad) <= 0 || dc_out_extent(w, k, stride, pad) <= 0) return DC_ERR_SHAPE;
+  if (!dc_aligned16(x) || !dc_aligned16(y) || !dc_aligned16(w_packed) || (bias && !dc_aligned16(bias)))
+    return DC_ERR_ALIGNMENT;
+  if (dtype == DC_F32)
+    return launch_dw<float>(x, n, h, w, c, k, stride, pad, w_packed, bias, act, y, (cudaStream_t)stream);
+  return launch_dw<__nv_bfloat16>(x, n, h, w, c, k, stride, pad, w_packed, bias, act, y, (cudaStream_t)stream);
+}

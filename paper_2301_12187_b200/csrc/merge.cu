@@ -1,0 +1,475 @@
+// BN folding, composition of a run of convolutions into one convolution, and weight repacking.
+// fp32 FMA arithmetic on CUDA cores: the merged weights must match an fp64 evaluation of the
+// same formula to 1e-5 relative, which rules out reduced-precision tensor-core math.
+#include <vector>
+
+#include "common.cuh"
+
+// ----------------------------------------------------------------------------------------------
+// kernels
+// ----------------------------------------------------------------------------------------------
+
+#define DC_FOLD_MAX 16
+struct FoldTable {
+  const float *w[DC_FOLD_MAX], *b[DC_FOLD_MAX], *gamma[DC_FOLD_MAX], *beta[DC_FOLD_MAX],
+      *mean[DC_FOLD_MAX], *var[DC_FOLD_MAX];
+  float *w_out[DC_FOLD_MAX], *b_out[DC_FOLD_MAX];
+  float eps[DC_FOLD_MAX];
+  int c_out[DC_FOLD_MAX], per_out[DC_FOLD_MAX];
+  int n;
+};
+
+// blockIdx.y = layer; grid-stride over that layer's weights.  g = gamma / sqrt(var + eps).
+__global__ void k_fold_bn(const __grid_constant__ FoldTable t) {
+  const int l = blockIdx.y;
+  const int per = t.per_out[l];
+  const int total = t.c_out[l] * per;
+  const bool has_bn = t.gamma[l] != nullptr;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int o = i / per;
+    float g = 1.f;
+    if (has_bn) g = t.gamma[l][o] / sqrtf(t.var[l][o] + t.eps[l]);
+    t.w_out[l][i] = g * t.w[l][i];
+    if (i - o * per == 0) {
+      float b = t.b[l] ? t.b[l][o] : 0.f;
+      t.b_out[l][o] = has_bn ? fmaf(b - t.mean[l][o], g, t.beta[l][o]) : b;
+    }
+  }
+}
+
+// One piece of a run while it is being merged: a dense kernel [c_out][c_in][k][k] or a diagonal
+// (depthwise) one [c][k][k], with its bias and accumulated stride.
+struct Piece {
+  const float *w;
+  const float *b;
+  int c_in, c_out, k, stride, diag;
+};
+
+// dense (second) o dense (first):  out[o][j] = sum_r A[o][r] * B[r][j] with
+//   r = (c, u2, v2),  j = (i, u', v'),  A = W2 as stored,
+//   B[r][j] = W1[c][i][u' - s1*u2][v' - s1*v2]  (0 when the tap falls outside W1).
+// 64x64 output tile, 16-deep slices, 256 threads, 4x4 outputs per thread.
+__global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece second, float *out, int kk) {
+  __shared__ float As[16][64 + 4];
+  __shared__ float Bs[16][64 + 4];
+  const int k1 = first.k, k2 = second.k, s1 = first.stride;
+  const int c0 = first.c_in, c1 = first.c_out, c2 = second.c_out;
+  const int R = c1 * k2 * k2, J = c0 * kk * kk;
+  const int o0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+  const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+  float acc[4][4] = {};
+  for (int r0 = 0; r0 < R; r0 += 16) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      int e = t + 256 * q;
+      int row = e / 16, rr = e % 16;
+      int o = o0 + row, r = r0 + rr;
+      As[rr][row] = (o < c2 && r < R) ? second.w[(size_t)o * R + r] : 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      int e = t + 256 * q;
+      int rr = e / 64, jj = e % 64;
+      int r = r0 + rr, j = j0 + jj;
+      float v = 0.f;
+      if (r < R && j < J) {
+        int c = r / (k2 * k2), t2 = r - c * k2 * k2;
+        int u2 = t2 / k2, v2 = t2 - u2 * k2;
+        int i = j / (kk * kk), tp = j - i * kk * kk;
+        int up = tp / kk, vp = tp - up * kk;
+        int u1 = up - s1 * u2, v1 = vp - s1 * v2;
+        if (u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1)
+          v = first.w[(((size_t)c * c0 + i) * k1 + u1) * k1 + v1];
+      }
+      Bs[rr][jj] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int rr = 0; rr < 16; ++rr) {
+      float a[4], b[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) { a[q] = As[rr][ty * 4 + q]; b[q] = Bs[rr][tx * 4 + q]; }
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[p][q] = fmaf(a[p], b[q], acc[p][q]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int p = 0; p < 4; ++p)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      int o = o0 + ty * 4 + p, j = j0 + tx * 4 + q;
+      if (o < c2 && j < J) out[(size_t)o * J + j] = acc[p][q];
+    }
+}
+
+// Compositions in which at least one operand is diagonal: one thread per output element.
+//   second diag, first dense: out[o,i,u',v'] = sum_{u2,v2} W2[o,u2,v2] * W1[o,i,u1,v1]
+//   second dense, first diag: out[o,i,u',v'] = sum_{u2,v2} W2[o,i,u2,v2] * W1[i,u1,v1]
+//   both diag:                out[c,u',v']   = sum_{u2,v2} W2[c,u2,v2]   * W1[c,u1,v1]
+__global__ void k_compose_diag(Piece first, Piece second, float *out, int kk, int total) {
+  const int k1 = first.k, k2 = second.k, s1 = first.stride;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    int vp = idx % kk, up = (idx / kk) % kk, rest = idx / (kk * kk);
+    int o, i;
+    if (first.diag && second.diag) { o = rest; i = rest; }
+    else { i = rest % first.c_in; o = rest / first.c_in; }
+    float acc = 0.f;
+    for (int u2 = 0; u2 < k2; ++u2) {
+      int u1 = up - s1 * u2;
+      if (u1 < 0 || u1 >= k1) continue;
+      for (int v2 = 0; v2 < k2; ++v2) {
+        int v1 = vp - s1 * v2;
+        if (v1 < 0 || v1 >= k1) continue;
+        float w2 = second.diag ? second.w[((size_t)o * k2 + u2) * k2 + v2]
+                               : second.w[(((size_t)o * second.c_in + i) * k2 + u2) * k2 + v2];
+        float w1 = first.diag ? first.w[((size_t)i * k1 + u1) * k1 + v1]
+                              : first.w[(((size_t)o * first.c_in + i) * k1 + u1) * k1 + v1];
+        acc = fmaf(w2, w1, acc);
+      }
+    }
+    out[idx] = acc;
+  }
+}
+
+// b'[o] = b2[o] + sum_c (sum_taps W2[o,c]) * b1[c]; one warp per output channel.
+__global__ void k_compose_bias(Piece first, Piece second, float *out) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
+  if (warp >= second.c_out) return;
+  const int o = warp, t2 = second.k * second.k;
+  float acc = 0.f;
+  if (second.diag) {
+    if (lane == 0) {
+      float ws = 0.f;
+      for (int t = 0; t < t2; ++t) ws += second.w[(size_t)o * t2 + t];
+      acc = ws * first.b[o];
+    }
+  } else {
+    for (int c = lane; c < second.c_in; c += 32) {
+      float ws = 0.f;
+      for (int t = 0; t < t2; ++t) ws += second.w[((size_t)o * second.c_in + c) * t2 + t];
+      acc = fmaf(ws, first.b[c], acc);
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+  if (lane == 0) out[o] = second.b[o] + acc;
+}
+
+// identity kernel of a skip addition: +1 on the centre tap of every (c, c) pair
+__global__ void k_add_identity(float *w, int c, int k, int diag) {
+  int o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= c) return;
+  int ctr = (k - 1) / 2;
+  size_t idx = diag ? ((size_t)o * k + ctr) * k + ctr : (((size_t)o * c + o) * k + ctr) * k + ctr;
+  w[idx] += 1.f;
+}
+
+__global__ void k_lift_diag(const float *wd, float *w, int c, int k) {
+  int total = c * c * k * k;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    int t = idx % (k * k), i = (idx / (k * k)) % c, o = idx / (k * k * c);
+    w[idx] = (o == i) ? wd[(size_t)o * k * k + t] : 0.f;
+  }
+}
+
+__global__ void k_copy(const float *src, float *dst, int n) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = src[i];
+}
+
+// fp32 [o][i][u][v] -> fp32 [u][v][i][o]
+__global__ void k_pack_f32(const float *w, float *out, int c_out, int c_in, int k) {
+  int total = c_out * c_in * k * k;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    int o = idx % c_out, i = (idx / c_out) % c_in, t = idx / (c_out * c_in);
+    out[idx] = w[((size_t)o * c_in + i) * k * k + t];
+  }
+}
+
+// depthwise fp32 [c][1][k][k] -> fp32 [k][k][c]
+__global__ void k_pack_dw(const float *w, float *out, int c, int k) {
+  int total = c * k * k;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    int ch = idx % c, t = idx / c;
+    out[idx] = w[(size_t)ch * k * k + t];
+  }
+}
+
+// fp32 [o][i][u][v] -> bf16 chunk planes [group][entry][n_pad][8] in the K order of KOrder
+__global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrder ko) {
+  const int total = ko.ng * ko.e_pad * ko.n_pad * 8;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    int c8 = idx % 8, o = (idx / 8) % ko.n_pad, plane = idx / (8 * ko.n_pad);
+    int grp = plane / ko.e_pad, e = plane - grp * ko.e_pad;
+    int pc, ccg, r, s;
+    float v = 0.f;
+    if (dc_korder_decode(ko, e, &pc, &ccg, &r, &s)) {
+      int c = (grp * ko.cg + ccg) * 8 + c8;
+      if (o < c_out && c < ko.c_in) v = w[(((size_t)o * ko.c_in + c) * ko.k + r) * ko.k + s];
+    }
+    out[idx] = __float2bfloat16_rn(v);
+  }
+}
+
+// ----------------------------------------------------------------------------------------------
+// host: validation and geometry
+// ----------------------------------------------------------------------------------------------
+
+dc_status dc_validate_geom(const dc_geom *g) {
+  if (!g) return DC_ERR_INVALID_ARG;
+  if (g->c_in <= 0 || g->c_out <= 0 || g->k <= 0 || g->stride <= 0 || g->pad < 0 || g->groups <= 0)
+    return DC_ERR_INVALID_ARG;
+  if (g->k % 2 == 0) return DC_ERR_UNSUPPORTED;
+  if (!(g->groups == 1 || (g->groups == g->c_in && g->c_in == g->c_out))) return DC_ERR_UNSUPPORTED;
+  return DC_OK;
+}
+
+static dc_status validate_layer(const dc_layer *L) {
+  dc_geom g = {L->c_in, L->c_out, L->groups, L->k, L->stride, L->pad};
+  dc_status st = dc_validate_geom(&g);
+  if (st != DC_OK) return st;
+  if (!L->weight) return DC_ERR_INVALID_ARG;
+  int nbn = (L->bn_gamma != nullptr) + (L->bn_beta != nullptr) + (L->bn_mean != nullptr) + (L->bn_var != nullptr);
+  if (nbn != 0 && nbn != 4) return DC_ERR_INVALID_ARG;
+  return DC_OK;
+}
+
+static size_t piece_elems(int c_in, int c_out, int k, int diag) {
+  return diag ? (size_t)c_out * k * k : (size_t)c_out * c_in * k * k;
+}
+
+static int find_group(const dc_residual *res, int n_res, int first) {
+  for (int i = 0; i < n_res; ++i)
+    if (res[i].first == first) return i;
+  return -1;
+}
+
+static dc_status check_chain(const dc_layer *layers, int n, const dc_residual *res, int n_res,
+                             dc_geom *merged) {
+  if (!layers || n <= 0 || n_res < 0 || (n_res > 0 && !res)) return DC_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    dc_status st = validate_layer(&layers[i]);
+    if (st != DC_OK) return st;
+    if (i > 0 && layers[i].c_in != layers[i - 1].c_out) return DC_ERR_SHAPE;
+  }
+  int prev_last = -1;
+  for (int gi = 0; gi < n_res; ++gi) {
+    if (res[gi].first < 0 || res[gi].last >= n || res[gi].first > res[gi].last) return DC_ERR_INVALID_ARG;
+    if (res[gi].first <= prev_last) return DC_ERR_INVALID_ARG;
+    prev_last = res[gi].last;
+    int k = 1, s = 1, p = 0;
+    for (int i = res[gi].first; i <= res[gi].last; ++i) {
+      k += (layers[i].k - 1) * s;
+      p += layers[i].pad * s;
+      s *= layers[i].stride;
+    }
+    if (s != 1 || layers[res[gi].first].c_in != layers[res[gi].last].c_out || 2 * p != k - 1)
+      return DC_ERR_NOT_MERGEABLE;
+  }
+  int k = 1, s = 1, p = 0;
+  for (int i = 0; i < n; ++i) {
+    k += (layers[i].k - 1) * s;
+    p += layers[i].pad * s;
+    s *= layers[i].stride;
+  }
+  if (merged) {
+    merged->c_in = layers[0].c_in;
+    merged->c_out = layers[n - 1].c_out;
+    merged->groups = 1;
+    merged->k = k; merged->stride = s; merged->pad = p;
+  }
+  return DC_OK;
+}
+
+// Bump allocator over the caller's workspace (256-byte granules); with base == nullptr it only counts.
+struct Bump {
+  char *base; size_t off;
+  float *take(size_t elems) {
+    size_t bytes = dc_round_up(elems * sizeof(float), 256);
+    float *p = base ? reinterpret_cast<float *>(base + off) : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+static inline int blocks_for(size_t total, int threads) {
+  size_t b = (total + threads - 1) / threads;
+  return (int)(b > 65535 ? 65535 : (b == 0 ? 1 : b));
+}
+
+// Composes second o first into a new piece; launches when `go`.
+static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool go, cudaStream_t st) {
+  Piece out;
+  out.c_in = first.c_in; out.c_out = second.c_out;
+  out.k = first.k + (second.k - 1) * first.stride;
+  out.stride = first.stride * second.stride;
+  out.diag = first.diag && second.diag;
+  size_t elems = piece_elems(out.c_in, out.c_out, out.k, out.diag);
+  float *w = bump.take(elems);
+  float *b = bump.take(out.c_out);
+  out.w = w; out.b = b;
+  if (go) {
+    if (!first.diag && !second.diag) {
+      dim3 grid(dc_div_up(out.c_in * out.k * out.k, 64), dc_div_up(out.c_out, 64));
+      k_compose_dense_dense<<<grid, 256, 0, st>>>(first, second, w, out.k);
+    } else {
+      k_compose_diag<<<blocks_for(elems, 256), 256, 0, st>>>(first, second, w, out.k, (int)elems);
+    }
+    k_compose_bias<<<dc_div_up(out.c_out * 32, 128), 128, 0, st>>>(first, second, b);
+  }
+  return out;
+}
+
+// One walk drives both the size query (go == false: nothing is dereferenced or launched) and the
+// launches (go == true: the caller has already checked workspace_bytes against the query).
+static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *res, int n_res,
+                            float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
+                            void *workspace, cudaStream_t st, bool go, dc_geom *merged, size_t *need) {
+  dc_geom mg;
+  dc_status s = check_chain(layers, n, res, n_res, &mg);
+  if (s != DC_OK) return s;
+  if (merged) *merged = mg;
+  Bump bump{go ? (char *)workspace : nullptr, 0};
+
+  // 1. fold every layer
+  std::vector<Piece> folded(n);
+  for (int l0 = 0; l0 < n; l0 += DC_FOLD_MAX) {
+    FoldTable t;
+    int cnt = n - l0 < DC_FOLD_MAX ? n - l0 : DC_FOLD_MAX;
+    t.n = cnt;
+    size_t max_total = 1;
+    for (int j = 0; j < cnt; ++j) {
+      const dc_layer &L = layers[l0 + j];
+      int diag = L.groups != 1;
+      size_t elems = piece_elems(L.c_in, L.c_out, L.k, diag);
+      float *w = bump.take(elems), *b = bump.take(L.c_out);
+      t.w[j] = L.weight; t.b[j] = L.bias; t.gamma[j] = L.bn_gamma; t.beta[j] = L.bn_beta;
+      t.mean[j] = L.bn_mean; t.var[j] = L.bn_var; t.eps[j] = L.bn_eps;
+      t.w_out[j] = w; t.b_out[j] = b;
+      t.c_out[j] = L.c_out; t.per_out[j] = (int)(elems / L.c_out);
+      if (elems > max_total) max_total = elems;
+      folded[l0 + j] = Piece{w, b, L.c_in, L.c_out, L.k, L.stride, diag};
+    }
+    if (go) {
+      int bx = blocks_for(max_total, 256);
+      dim3 grid(bx > 64 ? 64 : bx, cnt);
+      k_fold_bn<<<grid, 256, 0, st>>>(t);
+    }
+  }
+
+  // 2. compose: skip groups first (with their identity tap), then left to right
+  Piece acc{};
+  bool have = false;
+  int i = 0;
+  while (i < n) {
+    Piece piece;
+    int gi = find_group(res, n_res, i);
+    if (gi < 0) {
+      piece = folded[i];
+      ++i;
+    } else {
+      piece = folded[res[gi].first];
+      for (int j = res[gi].first + 1; j <= res[gi].last; ++j) piece = compose(piece, folded[j], bump, go, st);
+      if (go)
+        k_add_identity<<<dc_div_up(piece.c_out, 128), 128, 0, st>>>(const_cast<float *>(piece.w), piece.c_out,
+                                                                   piece.k, piece.diag);
+      i = res[gi].last + 1;
+    }
+    if (!have) { acc = piece; have = true; }
+    else acc = compose(acc, piece, bump, go, st);
+  }
+  if (need) *need = bump.off + 256;
+  if (!go) return DC_OK;
+
+  // 3. deliver: dense fp32 result, bias, optional packed copy
+  size_t elems = (size_t)mg.c_out * mg.c_in * mg.k * mg.k;
+  if (acc.diag) k_lift_diag<<<blocks_for(elems, 256), 256, 0, st>>>(acc.w, w_merged, mg.c_out, mg.k);
+  else k_copy<<<blocks_for(elems, 256), 256, 0, st>>>(acc.w, w_merged, (int)elems);
+  k_copy<<<1, 256, 0, st>>>(acc.b, b_merged, mg.c_out);
+  if (w_packed) {
+    dc_status ps = dc_pack_weights(w_merged, &mg, packed_dtype, w_packed, (dc_stream)st);
+    if (ps != DC_OK) return ps;
+  }
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+// ----------------------------------------------------------------------------------------------
+// exported
+// ----------------------------------------------------------------------------------------------
+
+extern "C" dc_status dc_fold_bn(const dc_layer *layer, float *w_out, float *b_out, dc_stream stream) {
+  if (!layer || !w_out || !b_out) return DC_ERR_INVALID_ARG;
+  dc_status s = validate_layer(layer);
+  if (s != DC_OK) return s;
+  if (!dc_aligned16(layer->weight) || !dc_aligned16(w_out) || !dc_aligned16(b_out)) return DC_ERR_ALIGNMENT;
+  FoldTable t;
+  t.n = 1;
+  size_t elems = piece_elems(layer->c_in, layer->c_out, layer->k, layer->groups != 1);
+  t.w[0] = layer->weight; t.b[0] = layer->bias; t.gamma[0] = layer->bn_gamma; t.beta[0] = layer->bn_beta;
+  t.mean[0] = layer->bn_mean; t.var[0] = layer->bn_var; t.eps[0] = layer->bn_eps;
+  t.w_out[0] = w_out; t.b_out[0] = b_out; t.c_out[0] = layer->c_out; t.per_out[0] = (int)(elems / layer->c_out);
+  int bx = blocks_for(elems, 256);
+  dim3 grid(bx > 256 ? 256 : bx, 1);
+  k_fold_bn<<<grid, 256, 0, (cudaStream_t)stream>>>(t);
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+extern "C" dc_status dc_merge_query(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                                    dc_geom *merged, size_t *workspace_bytes) {
+  return merge_walk(layers, n_layers, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr, false,
+                    merged, workspace_bytes);
+}
+
+extern "C" dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                                    float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
+                                    void *workspace, size_t workspace_bytes, dc_stream stream) {
+  if (!w_merged || !b_merged) return DC_ERR_INVALID_ARG;
+  if (packed_dtype != DC_F32 && packed_dtype != DC_BF16) return DC_ERR_INVALID_ARG;
+  size_t need = 0;
+  dc_status s = merge_walk(layers, n_layers, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr,
+                           false, nullptr, &need);
+  if (s != DC_OK) return s;
+  if (!workspace || workspace_bytes < need) return DC_ERR_WORKSPACE;
+  if (!dc_aligned16(w_merged) || !dc_aligned16(b_merged) || !dc_aligned16(workspace) ||
+      (w_packed && !dc_aligned16(w_packed)))
+    return DC_ERR_ALIGNMENT;
+  for (int i = 0; i < n_layers; ++i)
+    if (!dc_aligned16(layers[i].weight)) return DC_ERR_ALIGNMENT;
+  return merge_walk(layers, n_layers, res, n_res, w_merged, b_merged, w_packed, packed_dtype, workspace,
+                    (cudaStream_t)stream, true, nullptr, nullptr);
+}
+
+extern "C" dc_status dc_packed_bytes(const dc_geom *g, dc_dtype dtype, size_t *bytes) {
+  dc_status s = dc_validate_geom(g);
+  if (s != DC_OK) return s;
+  if (!bytes || (dtype != DC_F32 && dtype != DC_BF16)) return DC_ERR_INVALID_ARG;
+  if (g->groups != 1) { *bytes = (size_t)g->c_out * g->k * g->k * sizeof(float); return DC_OK; }
+  if (dtype == DC_F32) { *bytes = (size_t)g->c_out * g->c_in * g->k * g->k * sizeof(float); return DC_OK; }
+  KOrder ko;
+  dc_korder_init(&ko, g);
+  *bytes = (size_t)ko.ng * ko.e_pad * ko.n_pad * 8 * sizeof(__nv_bfloat16);
+  return DC_OK;
+}
+
+extern "C" dc_status dc_pack_weights(const float *w, const dc_geom *g, dc_dtype dtype, void *w_packed,
+                                     dc_stream stream) {
+  dc_status s = dc_validate_geom(g);
+  if (s != DC_OK) return s;
+  if (!w || !w_packed || (dtype != DC_F32 && dtype != DC_BF16)) return DC_ERR_INVALID_ARG;
+  if (!dc_aligned16(w) || !dc_aligned16(w_packed)) return DC_ERR_ALIGNMENT;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (g->groups != 1) {
+    size_t total = (size_t)g->c_out * g->k * g->k;
+    k_pack_dw<<<blocks_for(total, 256), 256, 0, st>>>(w, (float *)w_packed, g->c_out, g->k);
+  } else if (dtype == DC_F32) {
+    size_t total = (size_t)g->c_out * g->c_in * g->k * g->k;
+    k_pack_f32<<<blocks_for(total, 256), 256, 0, st>>>(w, (float *)w_packed, g->c_out, g->c_in, g->k);
+  } else {
+    KOrder ko;
+    dc_korder_init(&ko, g);
+    size_t total = (size_t)ko.ng * ko.e_pad * ko.n_pad * 8;
+    k_pack_bf16<<<blocks_for(total, 256), 256, 0, st>>>(w, (__nv_bfloat16 *)w_packed, g->c_out, ko);
+  }
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
