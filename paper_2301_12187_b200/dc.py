@@ -1,0 +1,294 @@
+"""ctypes binding of libdepthc (include/dc.h).  Argument marshalling only: every step of the
+path runs in the library's CUDA kernels.  torch is used for device memory and streams.
+
+The functions carry the names of the C entry points without the `dc_` prefix.  Importing this
+module does not load the library; the first call does, and raises if it cannot.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdepthc.so")
+
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_NOT_MERGEABLE, ERR_WORKSPACE, ERR_ALIGNMENT, \
+    ERR_CUDA, ERR_TIMEOUT = range(9)
+F32, BF16 = 0, 1
+ACT_IDENTITY, ACT_RELU6 = 0, 1
+ALGO_AUTO, ALGO_TCGEN05, ALGO_SIMT = 0, 1, 2
+
+_FP = C.POINTER(C.c_float)
+
+
+class Layer(C.Structure):
+    _fields_ = [("c_in", C.c_int), ("c_out", C.c_int), ("groups", C.c_int),
+                ("k", C.c_int), ("stride", C.c_int), ("pad", C.c_int),
+                ("weight", C.c_void_p), ("bias", C.c_void_p),
+                ("bn_gamma", C.c_void_p), ("bn_beta", C.c_void_p),
+                ("bn_mean", C.c_void_p), ("bn_var", C.c_void_p), ("bn_eps", C.c_float)]
+
+
+class Residual(C.Structure):
+    _fields_ = [("first", C.c_int), ("last", C.c_int)]
+
+
+class Geom(C.Structure):
+    _fields_ = [("c_in", C.c_int), ("c_out", C.c_int), ("groups", C.c_int),
+                ("k", C.c_int), ("stride", C.c_int), ("pad", C.c_int)]
+
+    def as_tuple(self):
+        return (self.c_in, self.c_out, self.groups, self.k, self.stride, self.pad)
+
+
+class Block(C.Structure):
+    _fields_ = [("c_in", C.c_int), ("c_hidden", C.c_int), ("c_out", C.c_int), ("has_expand", C.c_int),
+                ("dw_k", C.c_int), ("dw_stride", C.c_int), ("dw_pad", C.c_int), ("has_residual", C.c_int),
+                ("act_expand", C.c_int), ("act_dw", C.c_int),
+                ("w_expand", C.c_void_p), ("b_expand", C.c_void_p), ("w_dw", C.c_void_p),
+                ("b_dw", C.c_void_p), ("w_project", C.c_void_p), ("b_project", C.c_void_p)]
+
+
+EXPORTS = {
+    "dc_status_string": (C.c_char_p, [C.c_int]),
+    "dc_fold_bn": (C.c_int, [C.POINTER(Layer), C.c_void_p, C.c_void_p, C.c_void_p]),
+    "dc_merge_query": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int,
+                                 C.POINTER(Geom), C.POINTER(C.c_size_t)]),
+    "dc_packed_bytes": (C.c_int, [C.POINTER(Geom), C.c_int, C.POINTER(C.c_size_t)]),
+    "dc_merge_chain": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
+                                 C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "dc_pack_weights": (C.c_int, [C.c_void_p, C.POINTER(Geom), C.c_int, C.c_void_p, C.c_void_p]),
+    "dc_conv_workspace_bytes": (C.c_size_t, []),
+    "dc_conv_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Geom), C.c_void_p,
+                                  C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                  C.c_size_t, C.c_void_p]),
+    "dc_conv_forward_algo": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Geom), C.c_void_p,
+                                       C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                       C.c_size_t, C.c_void_p, C.c_int]),
+    "dc_dwconv_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                    C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p]),
+    "dc_block_workspace_bytes": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(Block), C.c_int,
+                                           C.POINTER(C.c_size_t)]),
+    "dc_block_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Block), C.c_void_p,
+                                   C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "dc_workspace_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "dc_chain_host_workspace_bytes": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int,
+                                                C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]),
+    "dc_chain_forward_host": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
+                                        C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p,
+                                        C.c_size_t, C.c_void_p]),
+}
+
+_lib = None
+
+
+class DcError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        try:
+            msg = lib().dc_status_string(status).decode()
+        except Exception:  # pragma: no cover
+            msg = "?"
+        super().__init__("%s: status %d (%s)" % (what, status, msg))
+
+
+def lib():
+    """Load libdepthc.so (building it with nvcc first if it is missing or stale).  Never falls
+    back to anything else: without the library every call raises."""
+    global _lib
+    if _lib is None:
+        from . import build as _build
+        try:
+            path = _build.build()
+        except Exception as e:
+            raise RuntimeError("libdepthc.so is missing and could not be built: %r" % (e,))
+        L = C.CDLL(path)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def _check(st: int, what: str):
+    if st != OK:
+        raise DcError(st, what)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream=None) -> Optional[int]:
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream or None
+
+
+def dtype_code(torch_dtype) -> int:
+    import torch
+    if torch_dtype == torch.float32:
+        return F32
+    if torch_dtype == torch.bfloat16:
+        return BF16
+    raise ValueError("dtype must be float32 or bfloat16")
+
+
+def geom(c_in, c_out, groups, k, stride, pad) -> Geom:
+    return Geom(c_in, c_out, groups, k, stride, pad)
+
+
+class DeviceLayer:
+    """One conv(+BN) with its parameters held as fp32 device tensors; `.c` is the dc_layer."""
+
+    def __init__(self, spec, device="cuda"):
+        import torch
+        self.spec = spec
+        self.tensors = {}
+
+        def up(a):
+            if a is None:
+                return None
+            return torch.from_numpy(a).to(device=device, dtype=torch.float32).contiguous()
+
+        self.weight = up(spec.weight)
+        self.bias = up(spec.bias)
+        self.bn = None if spec.bn is None else tuple(up(t) for t in spec.bn)
+        bn = self.bn or (None, None, None, None)
+        self.c = Layer(spec.c_in, spec.c_out, spec.groups, spec.k, spec.stride, spec.pad,
+                       _ptr(self.weight), _ptr(self.bias), _ptr(bn[0]), _ptr(bn[1]), _ptr(bn[2]),
+                       _ptr(bn[3]), float(spec.eps))
+
+
+def layer_array(layers: Sequence) -> "C.Array":
+    """ctypes array of dc_layer from DeviceLayer objects or Layer structs."""
+    arr = (Layer * len(layers))()
+    for i, L in enumerate(layers):
+        arr[i] = L.c if isinstance(L, DeviceLayer) else L
+    return arr
+
+
+def _res_array(residuals):
+    residuals = list(residuals or [])
+    arr = (Residual * max(1, len(residuals)))()
+    for i, (f, l) in enumerate(residuals):
+        arr[i] = Residual(f, l)
+    return arr, len(residuals)
+
+
+# --------------------------------------------------------------------------- entry points
+
+
+def status_string(st: int) -> str:
+    return lib().dc_status_string(st).decode()
+
+
+def fold_bn(layer, w_out, b_out, stream=None):
+    c = layer.c if isinstance(layer, DeviceLayer) else layer
+    _check(lib().dc_fold_bn(C.byref(c), _ptr(w_out), _ptr(b_out), _stream(stream)), "dc_fold_bn")
+
+
+def merge_query(layers, residuals=()) -> Tuple[Geom, int]:
+    arr = layer_array(layers)
+    res, n_res = _res_array(residuals)
+    g = Geom()
+    nbytes = C.c_size_t(0)
+    _check(lib().dc_merge_query(arr, len(layers), res, n_res, C.byref(g), C.byref(nbytes)), "dc_merge_query")
+    return g, int(nbytes.value)
+
+
+def packed_bytes(g: Geom, dtype: int) -> int:
+    nbytes = C.c_size_t(0)
+    _check(lib().dc_packed_bytes(C.byref(g), dtype, C.byref(nbytes)), "dc_packed_bytes")
+    return int(nbytes.value)
+
+
+def merge_chain(layers, residuals, w_merged, b_merged, w_packed, packed_dtype, workspace, stream=None):
+    arr = layer_array(layers)
+    res, n_res = _res_array(residuals)
+    _check(lib().dc_merge_chain(arr, len(layers), res, n_res, _ptr(w_merged), _ptr(b_merged),
+                                _ptr(w_packed), packed_dtype, _ptr(workspace),
+                                workspace.numel() * workspace.element_size(), _stream(stream)),
+           "dc_merge_chain")
+
+
+def pack_weights(w, g: Geom, dtype: int, w_packed, stream=None):
+    _check(lib().dc_pack_weights(_ptr(w), C.byref(g), dtype, _ptr(w_packed), _stream(stream)),
+           "dc_pack_weights")
+
+
+def conv_workspace_bytes() -> int:
+    return int(lib().dc_conv_workspace_bytes())
+
+
+def conv_forward(x, g: Geom, w_packed, bias, act, residual, y, workspace, stream=None, algo=ALGO_AUTO):
+    n, h, w, _ = x.shape
+    _check(lib().dc_conv_forward_algo(_ptr(x), n, h, w, C.byref(g), _ptr(w_packed), _ptr(bias), act,
+                                      _ptr(residual), _ptr(y), dtype_code(x.dtype), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream), algo),
+           "dc_conv_forward")
+
+
+def dwconv_forward(x, k, stride, pad, w_packed, bias, act, y, stream=None):
+    n, h, w, c = x.shape
+    _check(lib().dc_dwconv_forward(_ptr(x), n, h, w, c, k, stride, pad, _ptr(w_packed), _ptr(bias), act,
+                                   _ptr(y), dtype_code(x.dtype), _stream(stream)), "dc_dwconv_forward")
+
+
+def block_workspace_bytes(n, h, w, blk: Block, dtype: int) -> int:
+    nbytes = C.c_size_t(0)
+    _check(lib().dc_block_workspace_bytes(n, h, w, C.byref(blk), dtype, C.byref(nbytes)),
+           "dc_block_workspace_bytes")
+    return int(nbytes.value)
+
+
+def block_forward(x, blk: Block, y, workspace, stream=None):
+    n, h, w, _ = x.shape
+    _check(lib().dc_block_forward(_ptr(x), n, h, w, C.byref(blk), _ptr(y), dtype_code(x.dtype),
+                                  _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream)), "dc_block_forward")
+
+
+def workspace_status(workspace, stream=None) -> int:
+    return int(lib().dc_workspace_status(_ptr(workspace), _stream(stream)))
+
+
+def host_layer_array(specs) -> Tuple["C.Array", list]:
+    """dc_layer array whose pointers are HOST pointers (numpy float32), for chain_forward_host."""
+    import numpy as np
+    keep = []
+    arr = (Layer * len(specs))()
+
+    def hp(a):
+        if a is None:
+            return None
+        a = np.ascontiguousarray(a, dtype=np.float32)
+        keep.append(a)
+        return a.ctypes.data
+
+    for i, s in enumerate(specs):
+        bn = s.bn or (None, None, None, None)
+        arr[i] = Layer(s.c_in, s.c_out, s.groups, s.k, s.stride, s.pad, hp(s.weight), hp(s.bias),
+                       hp(bn[0]), hp(bn[1]), hp(bn[2]), hp(bn[3]), float(s.eps))
+    return arr, keep
+
+
+def chain_host_workspace_bytes(host_layers, n_layers, residuals, n, h, w, dtype: int) -> int:
+    res, n_res = _res_array(residuals)
+    nbytes = C.c_size_t(0)
+    _check(lib().dc_chain_host_workspace_bytes(host_layers, n_layers, res, n_res, n, h, w, dtype,
+                                               C.byref(nbytes)), "dc_chain_host_workspace_bytes")
+    return int(nbytes.value)
+
+
+def chain_forward_host(host_layers, n_layers, residuals, x_host, act, y_host, workspace, stream=None):
+    """x_host / y_host: CPU torch tensors (pinned for asynchronous copies), NHWC."""
+    res, n_res = _res_array(residuals)
+    n, h, w, _ = x_host.shape
+    _check(lib().dc_chain_forward_host(host_layers, n_layers, res, n_res, _ptr(x_host), n, h, w, act,
+                                       _ptr(y_host), dtype_code(x_host.dtype), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)),
+           "dc_chain_forward_host")

@@ -1,0 +1,310 @@
+"""GPU parity: every C-ABI entry point against the fp64 oracle on the same seeded inputs.
+
+Tolerances (rel-L2 = ||a-b||/||b||, b the oracle): merged weights and bias 1e-5 (fp32 FMA merge);
+conv outputs 1e-4 in fp32 and 2e-2 in bf16 (bf16 rounding of the merged weights, of the input and
+of the output; fp32 accumulation)."""
+import numpy as np
+import pytest
+
+from oracle import dc_oracle as O
+from paper_2301_12187_b200 import inputs as I
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL_W, TOL_F32, TOL_BF16 = 1e-5, 1e-4, 2e-2
+
+
+@pytest.fixture(scope="module")
+def dc():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_12187_b200 import dc as _dc
+    _dc.lib()
+    return _dc
+
+
+def dev(a, dtype=torch.float32):
+    return torch.from_numpy(np.ascontiguousarray(a)).to("cuda", dtype=dtype).contiguous()
+
+
+def nchw(t):
+    return t.float().cpu().numpy().astype(np.float64).transpose(0, 3, 1, 2)
+
+
+def new_ws(dc, nbytes=None):
+    return torch.zeros(max(nbytes or 0, dc.conv_workspace_bytes()), dtype=torch.uint8, device="cuda")
+
+
+def run_merge(dc, specs, residuals, packed_dtype=None):
+    layers = [dc.DeviceLayer(s) for s in specs]
+    g, ws_bytes = dc.merge_query(layers, residuals)
+    wm = torch.empty((g.c_out, g.c_in, g.k, g.k), dtype=torch.float32, device="cuda")
+    bm = torch.empty((g.c_out,), dtype=torch.float32, device="cuda")
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    packed = None
+    if packed_dtype is not None:
+        packed = torch.empty(dc.packed_bytes(g, packed_dtype), dtype=torch.uint8, device="cuda")
+    dc.merge_chain(layers, residuals, wm, bm, packed, packed_dtype if packed_dtype is not None else dc.F32, ws)
+    torch.cuda.synchronize()
+    return g, wm, bm, packed
+
+
+def run_conv(dc, x, g, packed, bias, act, residual=None, algo=0):
+    n, h, w, _ = x.shape
+    ho, wo = O.out_extent(h, g.k, g.stride, g.pad), O.out_extent(w, g.k, g.stride, g.pad)
+    y = torch.full((n, ho, wo, g.c_out), float("nan"), dtype=x.dtype, device="cuda")
+    ws = new_ws(dc)
+    dc.conv_forward(x, g, packed, bias, act, residual, y, ws, algo=algo)
+    assert dc.workspace_status(ws) == dc.OK
+    return y
+
+
+def small_chain(name, rng_seed=0):
+    """Reduced-size versions of the four single-span topologies plus harder ones."""
+    mk = I.make_layer
+    s = rng_seed
+    if name == "t0":
+        return [mk(s, 0, 16, 96, 1, 1, 0), mk(s, 1, 96, 96, 3, 1, 1, depthwise=True), mk(s, 2, 96, 24, 1, 1, 0)], []
+    if name == "t1":
+        return [mk(s, 0, 24, 144, 1, 1, 0), mk(s, 1, 144, 144, 3, 1, 1, depthwise=True), mk(s, 2, 144, 24, 1, 1, 0)], [(0, 2)]
+    if name == "t2":
+        return [mk(s, 0, 24, 144, 1, 1, 0), mk(s, 1, 144, 144, 3, 2, 1, depthwise=True), mk(s, 2, 144, 32, 1, 1, 0)], []
+    if name == "t3":
+        L = []
+        for b in range(2):
+            L += [mk(s, 3 * b, 32, 192, 1, 1, 0), mk(s, 3 * b + 1, 192, 192, 3, 1, 1, depthwise=True),
+                  mk(s, 3 * b + 2, 192, 32, 1, 1, 0)]
+        return L, [(0, 2), (3, 5)]
+    if name == "dense_pair":
+        return [mk(s, 0, 8, 16, 3, 1, 1), mk(s, 1, 16, 8, 3, 1, 1, with_bn=False)], []
+    if name == "s2_first":
+        return [mk(s, 0, 8, 16, 3, 2, 1), mk(s, 1, 16, 16, 1, 1, 0), mk(s, 2, 16, 24, 1, 1, 0)], []
+    if name == "dw_first":
+        return [mk(s, 0, 16, 16, 3, 1, 1, depthwise=True), mk(s, 1, 16, 16, 3, 1, 1, depthwise=True),
+                mk(s, 2, 16, 8, 1, 1, 0)], [(0, 0)]
+    if name == "dw_only":
+        return [mk(s, 0, 8, 8, 3, 1, 1, depthwise=True), mk(s, 1, 8, 8, 3, 2, 1, depthwise=True)], []
+    if name == "single":
+        return [mk(s, 0, 8, 24, 3, 1, 1)], []
+    if name == "skip_mid":
+        return [mk(s, 0, 8, 16, 1, 1, 0), mk(s, 1, 16, 16, 3, 1, 1, depthwise=True), mk(s, 2, 16, 40, 1, 1, 0)], [(1, 1)]
+    raise KeyError(name)
+
+
+CHAINS = ["t0", "t1", "t2", "t3", "dense_pair", "s2_first", "dw_first", "dw_only", "single", "skip_mid"]
+
+
+def test_fold_bn(dc):
+    for spec in (I.make_layer(3, 0, 24, 40, 3, 1, 1), I.make_layer(3, 1, 32, 32, 3, 1, 1, depthwise=True),
+                 I.make_layer(3, 2, 8, 8, 1, 1, 0, with_bn=False)):
+        lay = dc.DeviceLayer(spec)
+        w = torch.empty_like(lay.weight)
+        b = torch.empty(spec.c_out, device="cuda")
+        dc.fold_bn(lay, w, b)
+        Wo, bo = O.fold_bn(spec)
+        assert O.rel_l2(w.cpu().numpy(), Wo) < 1e-6 and O.rel_l2(b.cpu().numpy(), bo) < 1e-6 or \
+            (spec.bn is None and np.all(bo == 0) and float(b.abs().max()) == 0)
+
+
+@pytest.mark.parametrize("name", CHAINS)
+def test_merge_chain_weights(dc, name):
+    specs, res = small_chain(name)
+    g, wm, bm, _ = run_merge(dc, specs, res)
+    W, b, k, s, p = O.merge_formula(specs, res)
+    assert (g.k, g.stride, g.pad, g.c_in, g.c_out) == (k, s, p, W.shape[1], W.shape[0])
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W
+    assert O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+
+
+@pytest.mark.parametrize("name", CHAINS)
+def test_merged_conv_fp32_equals_sequential_chain(dc, name):
+    specs, res = small_chain(name, rng_seed=1)
+    g, wm, bm, packed = run_merge(dc, specs, res, packed_dtype=dc.F32)
+    x = I.make_input(1, (2, 13, 11, specs[0].c_in))
+    y = run_conv(dc, dev(x), g, packed, bm, dc.ACT_IDENTITY)
+    ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, res)
+    assert y.shape[1:3] == ref.shape[2:]
+    assert O.rel_l2(nchw(y), ref) <= TOL_F32
+
+
+def test_config0_tiny_fp32(dc):
+    case = I.chain_case(0)
+    g, wm, bm, packed = run_merge(dc, case.layers, case.residuals, packed_dtype=dc.F32)
+    W, b, k, s, p = O.merge_formula(case.layers, case.residuals)
+    assert (g.c_in, g.c_out, g.k, g.stride, g.pad) == (16, 24, 3, 1, 1)
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    x = case.x()
+    y = run_conv(dc, dev(x), g, packed, bm, dc.ACT_IDENTITY)
+    ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), case.layers, case.residuals)
+    assert O.rel_l2(nchw(y), ref) <= TOL_F32
+    # the chain with its original per-layer padding agrees inside and differs on the border ring
+    orig = O.chain_forward_original(x.transpose(0, 3, 1, 2), case.layers, case.residuals)
+    assert O.rel_l2(nchw(y)[:, :, 1:-1, 1:-1], orig[:, :, 1:-1, 1:-1]) <= TOL_F32
+    assert O.rel_l2(nchw(y), orig) > 1e-3
+
+
+BF16_SHAPES = [
+    # (name, n, h, w) -- spatial sizes that span several tiles and leave ragged tails
+    ("t1", 3, 19, 23), ("t2", 2, 22, 18), ("t3", 2, 17, 21), ("t0", 1, 9, 40), ("s2_first", 2, 30, 14),
+    ("dense_pair", 2, 12, 70), ("single", 3, 8, 8), ("skip_mid", 1, 33, 9),
+]
+
+
+@pytest.mark.parametrize("algo", ["simt", "auto"])
+@pytest.mark.parametrize("name,n,h,w", BF16_SHAPES)
+def test_merged_conv_bf16_equals_sequential_chain(dc, name, n, h, w, algo):
+    specs, res = small_chain(name, rng_seed=2)
+    g, wm, bm, packed = run_merge(dc, specs, res, packed_dtype=dc.BF16)
+    x = I.make_input(2, (n, h, w, specs[0].c_in), bf16=True)
+    for act in (dc.ACT_IDENTITY, dc.ACT_RELU6):
+        y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bm, act,
+                     algo=dc.ALGO_SIMT if algo == "simt" else dc.ALGO_AUTO)
+        ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, res,
+                                        final_act="relu6" if act else None)
+        assert not torch.isnan(y.float()).any()
+        assert O.rel_l2(nchw(y), ref) <= TOL_BF16
+
+
+@pytest.mark.parametrize("algo", ["simt", "auto"])
+@pytest.mark.parametrize("c_in,c_out,k,s,p,n,h,w", [
+    (32, 16, 1, 1, 0, 2, 14, 14), (96, 24, 1, 1, 0, 1, 20, 12), (160, 320, 1, 1, 0, 2, 7, 7),
+    (320, 1280, 1, 1, 0, 1, 7, 7), (3, 32, 3, 2, 1, 2, 32, 32), (16, 96, 1, 1, 0, 1, 24, 24),
+    (96, 144, 5, 2, 2, 1, 20, 20), (64, 384, 1, 1, 0, 3, 14, 14), (24, 40, 7, 1, 3, 1, 16, 16),
+    (40, 24, 3, 1, 0, 1, 12, 12), (20, 12, 3, 1, 1, 1, 10, 10),
+])
+def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, algo):
+    spec = I.make_layer(5, 0, c_in, c_out, k, s, p)
+    lay = dc.DeviceLayer(spec)
+    wf = torch.empty_like(lay.weight)
+    bf = torch.empty(c_out, device="cuda")
+    dc.fold_bn(lay, wf, bf)
+    g = dc.geom(c_in, c_out, 1, k, s, p)
+    packed = torch.empty(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
+    dc.pack_weights(wf, g, dc.BF16, packed)
+    x = I.make_input(6, (n, h, w, c_in), bf16=True)
+    ho, wo = O.out_extent(h, k, s, p), O.out_extent(w, k, s, p)
+    r = I.round_bf16(I.normal(7, 99, (n, ho, wo, c_out)))
+    y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bf, dc.ACT_RELU6, residual=dev(r, torch.bfloat16),
+                 algo=dc.ALGO_SIMT if algo == "simt" else dc.ALGO_AUTO)
+    Wf, bfo = O.fold_bn(spec)
+    ref = O.relu6(O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p) + r.transpose(0, 3, 1, 2))
+    assert O.rel_l2(nchw(y), ref) <= TOL_BF16
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("c,k,s,p,n,h,w", [(32, 3, 1, 1, 2, 12, 12), (96, 3, 2, 1, 1, 15, 17),
+                                           (144, 3, 1, 1, 1, 9, 30), (20, 5, 1, 2, 1, 8, 8),
+                                           (6, 3, 2, 1, 2, 7, 7), (960, 3, 1, 1, 2, 7, 7)])
+def test_dwconv(dc, dtype, c, k, s, p, n, h, w):
+    spec = I.make_layer(8, 0, c, c, k, s, p, depthwise=True)
+    lay = dc.DeviceLayer(spec)
+    wf = torch.empty_like(lay.weight)
+    bf = torch.empty(c, device="cuda")
+    dc.fold_bn(lay, wf, bf)
+    g = dc.geom(c, c, c, k, s, p)
+    packed = torch.empty(dc.packed_bytes(g, dc.F32) // 4, dtype=torch.float32, device="cuda")
+    dc.pack_weights(wf, g, dc.F32, packed)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    x = I.make_input(9, (n, h, w, c), bf16=(dtype == "bf16"))
+    ho, wo = O.out_extent(h, k, s, p), O.out_extent(w, k, s, p)
+    y = torch.empty((n, ho, wo, c), dtype=tdt, device="cuda")
+    dc.dwconv_forward(dev(x, tdt), k, s, p, packed, bf, dc.ACT_RELU6, y)
+    Wf, bfo = O.fold_bn(spec)
+    ref = O.relu6(O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p, groups=c))
+    assert O.rel_l2(nchw(y), ref) <= (TOL_F32 if dtype == "f32" else TOL_BF16)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("c_in,c_out,t,s,n,h,w", [(24, 24, 6, 1, 2, 14, 14), (16, 24, 6, 2, 1, 16, 16),
+                                                  (32, 16, 1, 1, 1, 12, 12)])
+def test_block_forward(dc, dtype, c_in, c_out, t, s, n, h, w):
+    specs = I.inverted_residual(10, 0, c_in, c_out, t, s, block=0)
+    code = dc.F32 if dtype == "f32" else dc.BF16
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    keep, packed, biases = [], [], []
+    for spec in specs:
+        lay = dc.DeviceLayer(spec)
+        wf = torch.empty_like(lay.weight)
+        bf = torch.empty(spec.c_out, device="cuda")
+        dc.fold_bn(lay, wf, bf)
+        g = dc.geom(spec.c_in, spec.c_out, spec.groups, spec.k, spec.stride, spec.pad)
+        pk = torch.empty(dc.packed_bytes(g, code), dtype=torch.uint8, device="cuda")
+        dc.pack_weights(wf, g, code, pk)
+        packed.append(pk)
+        biases.append(bf)
+        keep.append((lay, wf))
+    has_exp = t != 1
+    res = s == 1 and c_in == c_out
+    if has_exp:
+        pe, pd, pp = packed
+        be, bd, bp = biases
+    else:
+        (pd, pp), (bd, bp) = packed, biases
+        pe = be = None
+    blk = dc.Block(c_in, c_in * t, c_out, int(has_exp), 3, s, 1, int(res), dc.ACT_RELU6, dc.ACT_RELU6,
+                   pe.data_ptr() if has_exp else None, be.data_ptr() if has_exp else None,
+                   pd.data_ptr(), bd.data_ptr(), pp.data_ptr(), bp.data_ptr())
+    x = I.make_input(11, (n, h, w, c_in), bf16=(dtype == "bf16"))
+    ho = O.out_extent(h, 3, s, 1)
+    wo = O.out_extent(w, 3, s, 1)
+    y = torch.empty((n, ho, wo, c_out), dtype=tdt, device="cuda")
+    ws = new_ws(dc, dc.block_workspace_bytes(n, h, w, blk, code))
+    dc.block_forward(dev(x, tdt), blk, y, ws)
+    assert dc.workspace_status(ws) == dc.OK
+    cur = x.transpose(0, 3, 1, 2).astype(np.float64)
+    skip = cur
+    for spec in specs:
+        Wf, bfo = O.fold_bn(spec)
+        cur = O.conv_direct(cur, Wf, bfo, spec.k, spec.stride, spec.pad, spec.groups)
+        if spec.act == "relu6":
+            cur = O.relu6(cur)
+    if res:
+        cur = cur + skip
+    # bf16: three roundings of the intermediate maps on the GPU side -> 3x the single-layer budget
+    assert O.rel_l2(nchw(y), cur) <= (TOL_F32 if dtype == "f32" else 3 * TOL_BF16)
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+def test_full_size_configs_on_sampled_images(dc, idx):
+    """The batch-64/128 workloads in the launch configuration the benchmark times; the oracle
+    runs the sequential chain on the first two and the last image."""
+    case = I.chain_case(idx)
+    g, wm, bm, packed = run_merge(dc, case.layers, case.residuals, packed_dtype=dc.BF16)
+    W, b, k, s, p = O.merge_formula(case.layers, case.residuals)
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    x = case.x()
+    y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bm, dc.ACT_IDENTITY)
+    assert not torch.isnan(y.float()).any()
+    sel = [0, 1, x.shape[0] - 1]
+    ref = O.chain_forward_reordered(x[sel].transpose(0, 3, 1, 2), case.layers, case.residuals)
+    assert O.rel_l2(nchw(y[sel]), ref) <= TOL_BF16
+    # every image: the output is finite and has the scale of the sampled ones
+    norms = y.float().pow(2).mean(dim=(1, 2, 3)).sqrt().cpu().numpy()
+    assert np.all(np.isfinite(norms)) and norms.min() > 0.5 * norms[sel].min() and norms.max() < 2 * norms[sel].max()
+
+
+def test_host_entry_point_matches_device_path(dc):
+    case = I.chain_case(1, batch=4)
+    arr, keep = dc.host_layer_array(case.layers)
+    n, h, w, c = case.x_shape
+    nbytes = dc.chain_host_workspace_bytes(arr, len(case.layers), case.residuals, n, h, w, dc.BF16)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    xh = torch.from_numpy(case.x()).to(torch.bfloat16).pin_memory()
+    yh = torch.empty((n, h, w, 24), dtype=torch.bfloat16).pin_memory()
+    dc.chain_forward_host(arr, len(case.layers), case.residuals, xh, dc.ACT_IDENTITY, yh, ws)
+    assert dc.workspace_status(ws) == dc.OK
+    ref = O.chain_forward_reordered(case.x().transpose(0, 3, 1, 2), case.layers, case.residuals)
+    assert O.rel_l2(yh.float().numpy().transpose(0, 3, 1, 2), ref) <= TOL_BF16
+
+
+def test_empty_and_degenerate_inputs_are_rejected_or_handled(dc):
+    g = dc.geom(8, 8, 1, 3, 1, 1)
+    packed = torch.zeros(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
+    x = torch.zeros((1, 1, 1, 8), dtype=torch.bfloat16, device="cuda")
+    y = run_conv(dc, x, g, packed, None, dc.ACT_IDENTITY)            # 1x1 image, all taps but one in the padding
+    assert y.shape == (1, 1, 1, 8) and float(y.float().abs().max()) == 0.0
+    with pytest.raises(dc.DcError) as e:
+        dc.conv_forward(torch.zeros((1, 2, 2, 8), dtype=torch.bfloat16, device="cuda"), dc.geom(8, 8, 1, 5, 1, 0),
+                        packed, None, 0, None, y, new_ws(dc))
+    assert e.value.status == dc.ERR_SHAPE
