@@ -1,5 +1,5 @@
 // Dense convolution forward as an implicit GEMM on the 5th-generation tensor cores (sm_100a):
-// tcgen05.mma with the accumulator in tensor memory, operands staged in shared memory by TMA.
+// tcgen05.mma with the accumulator in tensor memory, operands staged in shared memory.
 //
 // GEMM view.  M = output pixels of a tile, N = output channels, K = (tap, input channel).
 // The activation tile is loaded ONCE per (tile, channel group) as a haloed patch and kept in
@@ -16,11 +16,19 @@
 // "start + LBO": any two chunk entries whose addresses increase can be paired, which is how
 // channel counts that are not multiples of 16 (24 = 3 chunks) avoid padding.
 //
-// Roles per CTA (192 threads): warp 0 lane 0 issues TMA loads into a ring of stages; warp 1
-// lane 0 issues the MMAs and owns the tensor-memory allocation; warps 2..5 read accumulators
-// back (tcgen05.ld), add bias / skip input, apply the activation and store bf16 NHWC.
-// Accumulators are double buffered so the epilogue of tile i overlaps the MMAs of tile i+1.
-// Every wait is bounded: when one runs out the CTA latches DC_ERR_TIMEOUT and leaves.
+// Staging.  Activations: four producer warps gather the patch with 16-byte cp.async copies
+// (global reads of a warp are contiguous; the scatter into planes happens on the shared-memory
+// side; halo pixels are zero-filled).  A tiled TMA copy cannot produce this layout at speed: its
+// innermost box row would be 16 bytes, and one request per 16 bytes measured 27 us for a 19 MB
+// problem.  Weights: one 3-D TMA tile per (output-channel tile, channel group), resident for the
+// whole kernel when they fit.  Output: the epilogue converts to bf16 into a dense shared-memory
+// tile and one bulk copy (cp.async.bulk shared -> global) writes it when the tile is contiguous
+// in global memory; otherwise 16-byte stores.
+//
+// Roles per CTA (288 threads): warps 0-3 producers, warp 4 lane 0 issues the MMAs and warp 4
+// owns the tensor-memory allocation, warps 5-8 epilogue.  Accumulators are double buffered so the
+// epilogue of tile i overlaps the MMAs of tile i+1.  Every wait is bounded: when one runs out the
+// CTA latches DC_ERR_TIMEOUT in the caller's workspace and leaves.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -28,23 +36,27 @@
 namespace {
 
 constexpr int kMaxStages = 8;
-constexpr int kThreads = 192;
+constexpr int kProducerThreads = 128;
+constexpr int kThreads = 288;
+constexpr int kMaxPieces = 16;          // 16-byte pieces of one patch row handled by one producer thread
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 
 struct TcParams {
-  int n_img, h, w, ho, wo, c_out;
-  int stride;
+  int n_img, h, w, ho, wo, c_in, c_out;
+  int k, stride;
   int tw, th, nxt;            // tile width / height in outputs, x tiles per row
   int P, mb;                  // GEMM-row pitch per output row, 128-row blocks per tile
   int n_tile, nnt;            // output channels per pass, passes
   int units_per_nt, total_units;
   int cg, ng, e_pad, cch, pcs;
-  int wbox, rbox;             // TMA box: patch columns, rows
-  int plane_bytes, region_bytes, a_stage_bytes, b_stage_bytes;
+  int wbox, rbox;             // patch columns (per parity), rows
+  int plane_stride, region_bytes, a_stage_bytes, b_stage_bytes;
   int stages, b_resident;
   int act;
-  int cx0, cy0;               // patch origin: x = xt*tw + cx0, y = y0*stride + cy0
+  int cx0, cy0;               // patch origin: x = xt*tw + cx0 (parity-plane columns), y = y0*stride + cy0
   int acc_cols, tmem_cols;
+  int bulk_out, out_tile_bytes;
+  int off_b, off_a, off_out, off_bias;  // offsets in dynamic shared memory
   int smem_bytes;
   KOrder ko;
 };
@@ -64,8 +76,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// raises the transaction count the current phase waits for; not an arrival
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try(uint64_t *bar, uint32_t parity) {
   uint32_t done;
@@ -102,14 +115,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
   return mbar_wait_slow(bar, parity, abort_flag, ws, site);
 }
 
-__device__ __forceinline__ void tma_load_5d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2),
-      "r"(c3), "r"(c4)
-      : "memory");
-}
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
@@ -118,6 +123,39 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, u
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+// 16-byte asynchronous copy global -> shared; src_bytes == 0 writes zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+// the mbarrier receives one arrival from this thread once all its earlier cp.async copies have landed
+__device__ __forceinline__ void cp_async_arrive(uint64_t *bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// contiguous shared -> global bulk copy (bytes multiple of 16), tracked by the thread's bulk group
+__device__ __forceinline__ void bulk_store(void *gdst, uint32_t ssrc, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(ssrc), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// barrier over the 128 epilogue threads that also tells every one of them whether all passed `ok`
+__device__ __forceinline__ bool epi_all(bool ok) {
+  uint32_t all;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(all)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return all != 0;
 }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
@@ -140,13 +178,24 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate));
 }
 // arrive on an mbarrier once every MMA issued so far by this thread has completed
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t *v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(addr)
+      : "memory");
 }
 // 32 lanes x 16 consecutive fp32 columns: thread i of the warp receives lane (base lane + i)
 __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t *v) {
@@ -160,7 +209,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t *v) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // shared-memory operand descriptor, K-major, no swizzle: 14-bit start>>4, LBO>>4 at bit 16,
-// SBO>>4 at bit 32, descriptor version 1 at bit 46
+// SBO>>4 at bit 32 (128 bytes between 8-row groups), descriptor version 1 at bit 46
 __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes) {
   const uint32_t lo = ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
   const uint32_t hi = (128u >> 4) | (1u << 14);
@@ -172,6 +221,8 @@ struct Tile {
   int nt, img, xt, y0, th;
 };
 
+// Units are output row segments ordered (nt, img, xt, y); a CTA owns a contiguous range of them
+// and cuts it into tiles of up to p.th rows that never cross an image or column-strip boundary.
 __device__ __forceinline__ Tile decode_tile(const TcParams &p, int cur, int end) {
   Tile t;
   t.nt = cur / p.units_per_nt;
@@ -189,65 +240,61 @@ __device__ __forceinline__ Tile decode_tile(const TcParams &p, int cur, int end)
 
 // ------------------------------------------------------------------------------------------ kernel
 __global__ void __launch_bounds__(kThreads, 1)
-k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-          const __grid_constant__ TcParams p, const float *__restrict__ bias,
+k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcParams p,
+          const __nv_bfloat16 *__restrict__ x, const float *__restrict__ bias,
           const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_accfull[2], bar_accempty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ uint32_t abort_s;
-  __shared__ uint32_t a_off[128];   // per instruction j: byte offset of its first chunk in the stage
-  __shared__ uint32_t a_lbo[128];   // per instruction j: byte distance to its second chunk
+  // per instruction j: low word of its A descriptor relative to the stage base:
+  // (offset of first chunk >> 4) | (distance to second chunk >> 4) << 16
+  __shared__ uint32_t a_desc_lo[128];
 
-  // dynamic shared memory: [B stages][A stages][slack], 1024-byte aligned base
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  const int nb = p.b_resident ? 1 : p.stages;
-  uint8_t *smem_b = smem;
-  uint8_t *smem_a = smem + (size_t)nb * p.b_stage_bytes;
+  uint8_t *smem_b = smem + p.off_b;
+  uint8_t *smem_a = smem + p.off_a;
+  uint8_t *smem_out = smem + p.off_out;
+  uint8_t *smem_zero = smem_a + (size_t)p.stages * p.a_stage_bytes;   // always-zero plane + slack
+  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile uint32_t *abort_flag = &abort_s;
+  const bool odd_entries = (p.ko.e & 1) != 0;
 
   // ---- set-up
   if (threadIdx.x == 0) {
     abort_s = 0;
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&bar_full[s], kProducerThreads); mbar_init(&bar_empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&bar_accfull[a], 1); mbar_init(&bar_accempty[a], 128); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tensormap(&map_a);
     prefetch_tensormap(&map_b);
   }
-  // chunk-pair table: entry e -> byte offset of its 16-byte column in an A stage
-  for (int j = threadIdx.x; j < p.e_pad / 2; j += kThreads) {
-    uint32_t off[2];
-    for (int q = 0; q < 2; ++q) {
-      int e = 2 * j + q, pc, ccg, r, s;
-      if (dc_korder_decode(p.ko, e, &pc, &ccg, &r, &s)) {
-        int sx = (p.stride == 1) ? s : ((s - p.ko.pad) >> 1) - ((-p.ko.pad) >> 1);
-        off[q] = (uint32_t)(pc * p.region_bytes + ccg * p.plane_bytes + (r * p.wbox + sx) * 16);
-      } else {
-        off[q] = off[0] + 16;  // zero-weight padding entry: any finite data will do
-      }
-    }
-    a_off[j] = off[0];
-    a_lbo[j] = off[1] - off[0];
-  }
-  // the bytes between the end of the planes and the end of each region are never written by
-  // TMA but can be read through the padding entry: make them zero once
-  {
-    const int used = p.cg * p.plane_bytes, padb = p.region_bytes - used;
-    const int nreg = p.stages * p.pcs;
-    for (int i = threadIdx.x; i < nreg * (padb / 4); i += kThreads) {
-      int reg = i / (padb / 4), wd = i - reg * (padb / 4);
-      int st = reg / p.pcs, pc = reg - st * p.pcs;
-      *reinterpret_cast<uint32_t *>(smem_a + (size_t)st * p.a_stage_bytes + pc * p.region_bytes + used + wd * 4) = 0u;
-    }
-  }
-  if (warp == 1) {
+  if (warp == 4) {
     tmem_alloc(&tmem_base_s, (uint32_t)p.tmem_cols);
     tmem_relinquish();
   }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (threadIdx.x >= 5 * 32) {
+    const int t = threadIdx.x - 5 * 32;
+    // chunk-pair table: entry e -> byte offset of its 16-byte column in an A stage
+    for (int j = t; j < p.e_pad / 2; j += 128) {
+      uint32_t off[2] = {0u, 16u};
+      for (int q = 0; q < 2; ++q) {
+        int e = 2 * j + q, pc, ccg, r, s;
+        if (dc_korder_decode(p.ko, e, &pc, &ccg, &r, &s)) {
+          int sx = (p.stride == 1) ? s : ((s - p.ko.pad) >> 1) - ((-p.ko.pad) >> 1);
+          off[q] = (uint32_t)(pc * p.region_bytes + ccg * p.plane_stride + (r * p.wbox + sx) * 16);
+        }
+      }
+      // the padding entry of an odd count gets its distance at issue time (it points at the zero plane)
+      a_desc_lo[j] = (off[0] >> 4) | (((off[1] - off[0]) >> 4) << 16);
+    }
+    for (int i = t; i < p.nnt * p.n_tile; i += 128) bias_s[i] = (bias && i < p.c_out) ? bias[i] : 0.f;
+    // the zero plane: second chunk of the padding entry, and the landing zone of reads past the last stage
+    uint4 *z = reinterpret_cast<uint4 *>(smem_zero);
+    for (int i = t; i < (p.mb * 2048 + 1024) / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  fence_proxy_async();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -256,40 +303,82 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   const int cta_begin = (int)((long long)p.total_units * blockIdx.x / gridDim.x);
   const int cta_end = (int)((long long)p.total_units * (blockIdx.x + 1) / gridDim.x);
 
-  if (warp == 0) {
-    // ================================================================== producer (TMA)
-    if (lane == 0) {
-      const uint32_t a_bytes = (uint32_t)(p.pcs * p.cg * p.plane_bytes);
-      uint32_t it = 0;
-      bool b_loaded = false;
-      for (int cur = cta_begin; cur < cta_end;) {
-        const Tile t = decode_tile(p, cur, cta_end);
-        cur += t.th;
-        const int cx = t.xt * p.tw + p.cx0, cy = t.y0 * p.stride + p.cy0;
-        for (int grp = 0; grp < p.ng; ++grp, ++it) {
-          const int s = it % p.stages;
-          const uint32_t ph = (it / p.stages) & 1;
-          if (!mbar_wait(&bar_empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) goto producer_done;
+  if (warp < 4) {
+    // ================================================================== producers (cp.async + TMA for weights)
+    const int ptid = threadIdx.x;
+    const int row_pieces = p.wbox * p.pcs * p.cg;
+    const int C2 = p.c_in * 2;
+    const int npieces = (ptid < row_pieces) ? (row_pieces - ptid + kProducerThreads - 1) / kProducerThreads : 0;
+    int src_off[kMaxPieces], gx_rel[kMaxPieces];
+    uint32_t dst_off[kMaxPieces];
+#pragma unroll
+    for (int i = 0; i < kMaxPieces; ++i) {
+      if (i >= npieces) break;
+      const int q = ptid + i * kProducerThreads;
+      const int ccg = q % p.cg;
+      const int t = q / p.cg;
+      const int pc = t % p.pcs;
+      const int col = t / p.pcs;
+      gx_rel[i] = (p.stride == 1) ? col : 2 * col + pc;
+      src_off[i] = gx_rel[i] * C2 + ccg * 16;
+      dst_off[i] = (uint32_t)(pc * p.region_bytes + ccg * p.plane_stride + col * 16);
+    }
+    const uint32_t a_base0 = smem_u32(smem_a);
+    const long long row_stride = (long long)p.w * C2;
+    const uint32_t drow_stride = (uint32_t)p.wbox * 16u;
+    uint32_t it = 0;
+    bool b_loaded = false, ok = true;
+    for (int cur = cta_begin; cur < cta_end && ok;) {
+      const Tile t = decode_tile(p, cur, cta_end);
+      cur += t.th;
+      const int gx0 = (t.xt * p.tw + p.cx0) * p.stride;
+      const int gy0 = t.y0 * p.stride + p.cy0;
+      const int rows = (t.th - 1) * p.stride + p.k;
+      const int r_lo = gy0 < 0 ? -gy0 : 0;                       // patch rows [r_lo, r_hi) lie inside the image
+      const int r_hi = (p.h - gy0 < rows) ? p.h - gy0 : rows;
+      const char *tile_base = reinterpret_cast<const char *>(x) + (size_t)t.img * p.h * row_stride +
+                              ((long long)gy0 * p.w + gx0) * C2;
+      for (int grp = 0; grp < p.ng; ++grp, ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (it / p.stages) & 1;
+        if (!mbar_wait(&bar_empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) { ok = false; break; }
+        if (ptid == 0) {
+          // a weight tile rides along on the same barrier as transaction bytes
           const bool load_b = !p.b_resident || !b_loaded;
-          mbar_expect_tx(&bar_full[s], a_bytes + (load_b ? (uint32_t)p.b_stage_bytes : 0u));
-          uint8_t *dst = smem_a + (size_t)s * p.a_stage_bytes;
-          for (int pc = 0; pc < p.pcs; ++pc)
-            tma_load_5d(dst + pc * p.region_bytes, &map_a, &bar_full[s], 0, cx, cy, t.img, pc * p.cch + grp * p.cg);
           if (load_b) {
+            mbar_expect_tx(&bar_full[s], (uint32_t)p.b_stage_bytes);
             tma_load_3d(smem_b + (size_t)(p.b_resident ? 0 : s) * p.b_stage_bytes, &map_b, &bar_full[s], 0,
                         t.nt * p.n_tile, grp * p.e_pad);
             b_loaded = true;
           }
         }
+        const uint32_t stage = a_base0 + (uint32_t)s * p.a_stage_bytes;
+        const char *grp_base = tile_base + grp * p.cg * 16;
+#pragma unroll
+        for (int i = 0; i < kMaxPieces; ++i) {
+          if (i >= npieces) break;
+          const int gx = gx0 + gx_rel[i];
+          const bool cv = (gx >= 0) && (gx < p.w);
+          const char *src = grp_base + src_off[i];
+          uint32_t dst = stage + dst_off[i];
+          for (int r = 0; r < rows; ++r) {
+            const bool v = cv && (r >= r_lo) && (r < r_hi);
+            cp_async16(dst, v ? (const void *)src : (const void *)x, v ? 16u : 0u);
+            src += row_stride;
+            dst += drow_stride;
+          }
+        }
+        cp_async_arrive(&bar_full[s]);           // arrives by itself when this thread's copies have landed
       }
     }
-  producer_done:;
-  } else if (warp == 1) {
+    cp_async_wait_all();                         // nothing of this thread is in flight when the CTA leaves
+  } else if (warp == 4) {
     // ================================================================== MMA issuer
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) | (8u << 24);
-      const uint32_t b_lbo = (uint32_t)p.n_tile * 16u;
+      const uint32_t desc_hi = (128u >> 4) | (1u << 14);
       const int npairs = p.e_pad / 2;
+      const uint32_t zero_addr = smem_u32(smem_zero);
       uint32_t it = 0, tile_i = 0;
       for (int cur = cta_begin; cur < cta_end; ++tile_i) {
         const Tile t = decode_tile(p, cur, cta_end);
@@ -304,14 +393,25 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1;
           if (!mbar_wait(&bar_full[s], ph, abort_flag, ws, 0x30000u | s)) goto mma_done;
+          fence_proxy_async();
           tc_fence_after();
           const uint32_t a_base = smem_u32(smem_a + (size_t)s * p.a_stage_bytes);
           const uint32_t b_base = smem_u32(smem_b + (size_t)(p.b_resident ? 0 : s) * p.b_stage_bytes);
+          const uint32_t b_lo0 = ((b_base >> 4) & 0x3FFFu) | ((uint32_t)p.n_tile << 16);
+          const uint32_t b_step = 2u * (uint32_t)p.n_tile;
+          // last pair of an odd entry count: second chunk = zero plane (same block offset on both sides)
+          const uint32_t last = (uint32_t)(npairs - 1);
+          const uint32_t first_off = (a_desc_lo[last] & 0x3FFFu) << 4;
+          const uint32_t pad_lo = (first_off >> 4) | (((zero_addr - a_base - first_off) >> 4) << 16);
           for (int b = 0; b < nblk; ++b) {
             const uint32_t d = d0 + (uint32_t)(b * p.n_tile);
+            const uint32_t a_add = (a_base >> 4) + (uint32_t)b * 128u;
+#pragma unroll 4
             for (int j = 0; j < npairs; ++j) {
-              const uint64_t ad = make_desc(a_base + a_off[j] + (uint32_t)b * 2048u, a_lbo[j]);
-              const uint64_t bd = make_desc(b_base + (uint32_t)(2 * j) * b_lbo, b_lbo);
+              uint32_t lo = a_desc_lo[j];
+              if (odd_entries && (uint32_t)j == last) lo = pad_lo;
+              const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
+              const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
               umma_bf16(d, ad, bd, idesc, (grp | j) != 0 ? 1u : 0u);
             }
           }
@@ -324,6 +424,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   } else {
     // ================================================================== epilogue (4 warps)
     const int q = warp & 3;                      // tensor-memory lane quadrant this warp may read
+    const bool elected = (threadIdx.x == 5 * 32);
     uint32_t tile_i = 0;
     for (int cur = cta_begin; cur < cta_end; ++tile_i) {
       const Tile t = decode_tile(p, cur, cta_end);
@@ -333,7 +434,10 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       const int x0 = t.xt * p.tw;
       const int tw_valid = (p.wo - x0 < p.tw) ? p.wo - x0 : p.tw;
       const uint32_t a = tile_i & 1, aph = (tile_i >> 1) & 1;
-      if (!mbar_wait(&bar_accfull[a], aph, abort_flag, ws, 0x40000u | a)) break;
+      uint8_t *obuf = smem_out + (size_t)a * p.out_tile_bytes;
+      if (p.bulk_out && elected) bulk_wait_read1();   // the store that last used this buffer has read it
+      // all 128 epilogue threads pass or leave together, so nobody is left alone at a named barrier
+      if (!epi_all(mbar_wait(&bar_accfull[a], aph, abort_flag, ws, 0x40000u | a))) break;
       tc_fence_after();
       const int ch_base = t.nt * p.n_tile;
       for (int b = 0; b < nblk; ++b) {
@@ -342,27 +446,30 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         const bool valid = (m < rows) && (xx < tw_valid) && (yy < t.th);
         const size_t pix = ((size_t)t.img * p.ho + (t.y0 + yy)) * p.wo + (x0 + xx);
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * (uint32_t)p.acc_cols + (uint32_t)(b * p.n_tile);
-        for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+        __nv_bfloat16 *gout = y + pix * p.c_out;
+        const __nv_bfloat16 *gres = residual ? residual + pix * p.c_out : nullptr;
+        uint8_t *sout = obuf + (size_t)(yy * p.tw + xx) * p.c_out * 2;
+        for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
           if (ch_base + c0 >= p.c_out) break;    // uniform across the warp
-          uint32_t v[16];
-          tmem_ld16(taddr + (uint32_t)c0, v);
+          uint32_t v[32];
+          const bool wide = (c0 + 32 <= p.n_tile);
+          if (wide) tmem_ld32(taddr + (uint32_t)c0, v);
+          else tmem_ld16(taddr + (uint32_t)c0, v);
           tmem_ld_wait();
           if (valid) {
 #pragma unroll
-            for (int hlf = 0; hlf < 2; ++hlf) {
-              const int ch = ch_base + c0 + hlf * 8;
-              if (ch < p.c_out) {
+            for (int e8 = 0; e8 < 4; ++e8) {
+              const int ch = ch_base + c0 + e8 * 8;
+              if ((e8 < 2 || wide) && ch < p.c_out) {
+                const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
+                const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
                 float f[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[hlf * 8 + i]);
-                if (bias) {
-                  const float4 b0 = *reinterpret_cast<const float4 *>(bias + ch);
-                  const float4 b1 = *reinterpret_cast<const float4 *>(bias + ch + 4);
-                  f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w;
-                  f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
-                }
-                if (residual) {
-                  const uint4 rv = *reinterpret_cast<const uint4 *>(residual + pix * p.c_out + ch);
+                f[0] = __uint_as_float(v[e8 * 8 + 0]) + b0.x; f[1] = __uint_as_float(v[e8 * 8 + 1]) + b0.y;
+                f[2] = __uint_as_float(v[e8 * 8 + 2]) + b0.z; f[3] = __uint_as_float(v[e8 * 8 + 3]) + b0.w;
+                f[4] = __uint_as_float(v[e8 * 8 + 4]) + b1.x; f[5] = __uint_as_float(v[e8 * 8 + 5]) + b1.y;
+                f[6] = __uint_as_float(v[e8 * 8 + 6]) + b1.z; f[7] = __uint_as_float(v[e8 * 8 + 7]) + b1.w;
+                if (gres) {
+                  const uint4 rv = *reinterpret_cast<const uint4 *>(gres + ch);
                   const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
 #pragma unroll
                   for (int i = 0; i < 4; ++i) {
@@ -375,7 +482,8 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                   ob[i] = __floats2bfloat162_rn(dc_act_apply(f[2 * i], p.act), dc_act_apply(f[2 * i + 1], p.act));
-                *reinterpret_cast<uint4 *>(y + pix * p.c_out + ch) = ov;
+                if (p.bulk_out) *reinterpret_cast<uint4 *>(sout + ch * 2) = ov;
+                else *reinterpret_cast<uint4 *>(gout + ch) = ov;
               }
             }
           }
@@ -383,7 +491,18 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       }
       tc_fence_before();
       mbar_arrive(&bar_accempty[a]);
+      if (p.bulk_out) {
+        fence_proxy_async();                     // the tile written above is read by the bulk copy engine
+        epi_barrier();
+        if (elected) {
+          const size_t pix0 = ((size_t)t.img * p.ho + t.y0) * p.wo + x0;
+          const uint32_t bytes = (uint32_t)(((p.ho == 1) ? tw_valid : t.th * p.tw) * p.c_out * 2);
+          bulk_store(y + pix0 * p.c_out, smem_u32(obuf), bytes);
+          bulk_commit();
+        }
+      }
     }
+    if (p.bulk_out && elected) bulk_wait_all();
   }
 
   // ---- teardown.  After a timeout, give copies and MMAs still in flight time to land before
@@ -394,7 +513,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 4) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
@@ -429,6 +548,14 @@ int sm_count() {
 
 constexpr int kSmemBudget = 200 * 1024;
 
+// plane stride in 16-byte units is made congruent to `want` mod 8 so that the cg chunks of one
+// pixel, written by neighbouring producer threads, fall into different bank groups
+int padded_plane_units(int units, int cg) {
+  int want = (cg == 3 || cg == 5 || cg == 7) ? cg : (cg >= 8 ? 1 : (8 / cg));
+  while ((units & 7) != (want & 7)) ++units;
+  return units;
+}
+
 // Chooses tiles, stages and the launch shape; false when the shape is outside this kernel's range.
 bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   if (g->groups != 1 || g->c_in % 8 || g->c_out % 8) return false;
@@ -444,7 +571,9 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   const bool flat = (g->k == 1 && g->stride == 1 && g->pad == 0);
 
   p->ko = ko;
+  p->k = g->k;
   p->stride = g->stride;
+  p->c_in = g->c_in;
   p->c_out = g->c_out;
   p->cg = ko.cg; p->ng = ko.ng; p->e_pad = ko.e_pad; p->cch = ko.cch; p->pcs = ko.pcs;
   p->nnt = dc_div_up(ko.n_pad, 256);
@@ -460,16 +589,13 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
     if (pixels >= (1ll << 31)) return false;
     p->n_img = 1; p->h = 1; p->w = (int)pixels; p->ho = 1; p->wo = (int)pixels;
     int mbf = mb_max < 2 ? mb_max : 2;
-    // keep at least ~4 tiles per SM when the map is small
-    while (mbf > 1 && pixels / (128 * mbf) < 4ll * n_sm) --mbf;
+    while (mbf > 1 && pixels / (128 * mbf) < 4ll * n_sm) --mbf;     // keep several tiles per SM
     p->tw = 128 * mbf; p->th = 1;
     p->wbox = p->tw; p->rbox = 1;
     p->P = p->tw;
     p->cx0 = 0; p->cy0 = 0;
   } else {
     p->n_img = n; p->h = h; p->w = w; p->ho = ho; p->wo = wo;
-    const int halo_lo = (g->stride == 1) ? 0 : 0;
-    (void)halo_lo;
     int nxt = dc_div_up(wo, 64);
     p->tw = dc_div_up(wo, nxt);
     if (g->stride == 1) {
@@ -481,7 +607,6 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
       p->P = 2 * p->wbox;
       p->cx0 = dc_floor_div2(-g->pad); p->cy0 = -g->pad;
     }
-    if (p->wbox > 256) return false;
     // rows per tile: bounded by the accumulator blocks, the image, shared memory, and a target
     // of about six tiles per CTA so that load, MMA and epilogue overlap
     long long total_rows = (long long)n * ho * dc_div_up(wo, p->tw) * p->nnt;
@@ -494,16 +619,17 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
     for (;; --th) {
       if (th < 1) return false;
       int rbox = (g->stride == 1) ? th + g->k - 1 : 2 * (th - 1) + g->k;
-      long long stage = (long long)ko.pcs * ko.cg * rbox * p->wbox * 16;
-      if (rbox <= 256 && stage <= 56 * 1024) { p->rbox = rbox; break; }
+      long long stage = (long long)ko.pcs * ko.cg * (rbox * p->wbox + 8) * 16;
+      if (stage <= 56 * 1024) { p->rbox = rbox; break; }
     }
     p->th = th;
   }
+  if (p->wbox * p->pcs * p->cg > kMaxPieces * kProducerThreads) return false;
   p->nxt = dc_div_up(p->wo, p->tw);
   p->mb = dc_div_up((p->th - 1) * p->P + p->tw, 128);
   if (p->mb > mb_max) return false;
-  p->plane_bytes = p->rbox * p->wbox * 16;
-  p->region_bytes = (int)dc_round_up((size_t)ko.cg * p->plane_bytes + 16, 128);
+  p->plane_stride = padded_plane_units(p->rbox * p->wbox + 1, ko.cg) * 16;
+  p->region_bytes = (int)dc_round_up((size_t)ko.cg * p->plane_stride, 128);
   p->a_stage_bytes = ko.pcs * p->region_bytes;
   p->acc_cols = p->mb * p->n_tile;
   int cols = 32;
@@ -515,16 +641,31 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   p->units_per_nt = (int)units;
   p->total_units = (int)(units * p->nnt);
 
-  // stages: as many as fit (2..kMaxStages), no more than a CTA will ever use
+  // output staging: one bulk copy per tile when the tile is contiguous in global memory
+  p->out_tile_bytes = (int)dc_round_up((size_t)p->th * p->tw * g->c_out * 2, 128);
+  p->bulk_out = (p->nnt == 1 && (flat || p->tw == p->wo) && p->out_tile_bytes <= 24 * 1024) ? 1 : 0;
+  if (!p->bulk_out) p->out_tile_bytes = 0;
+
+  // shared memory: [weights][bias][output tiles x2][activation stages][slack]
   const int slack = p->mb * 2048 + 1024;
+  const int bias_bytes = (int)dc_round_up((size_t)p->nnt * p->n_tile * 4, 128);
   int stages = kMaxStages;
   for (;; --stages) {
     if (stages < 2) return false;
-    long long tot = 1024ll + (long long)(p->b_resident ? 1 : stages) * p->b_stage_bytes +
-                    (long long)stages * p->a_stage_bytes + slack;
+    long long tot = 1024ll + (long long)(p->b_resident ? 1 : stages) * p->b_stage_bytes + bias_bytes +
+                    2ll * p->out_tile_bytes + (long long)stages * p->a_stage_bytes + slack;
     if (tot <= kSmemBudget) { p->smem_bytes = (int)tot; break; }
   }
+  // no point in more stages than a CTA has (tile, group) pairs
+  long long per_cta = ((long long)p->total_units / p->th / n_sm + 2) * p->ng;
+  if (stages > per_cta) stages = (int)per_cta;
+  if (stages < 2) stages = 2;
   p->stages = stages;
+  p->off_b = 0;
+  p->off_bias = (p->b_resident ? 1 : stages) * p->b_stage_bytes;
+  p->off_out = p->off_bias + bias_bytes;
+  p->off_a = p->off_out + 2 * p->out_tile_bytes;
+  p->smem_bytes = 1024 + p->off_a + stages * p->a_stage_bytes + slack;
   return true;
 }
 
@@ -545,26 +686,7 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) return DC_ERR_CUDA;
 
-  CUtensorMap map_a, map_b;
-  {
-    const cuuint64_t C2 = (cuuint64_t)g->c_in * 2;
-    cuuint64_t gdim[5], gstr[4];
-    if (p.stride == 1) {
-      gdim[0] = 8; gdim[1] = (cuuint64_t)p.w; gdim[2] = (cuuint64_t)p.h; gdim[3] = (cuuint64_t)p.n_img;
-      gdim[4] = (cuuint64_t)p.cch;
-      gstr[0] = C2; gstr[1] = C2 * p.w; gstr[2] = C2 * p.w * p.h; gstr[3] = 16;
-    } else {
-      gdim[0] = 8; gdim[1] = (cuuint64_t)p.w / 2; gdim[2] = (cuuint64_t)p.h; gdim[3] = (cuuint64_t)p.n_img;
-      gdim[4] = (cuuint64_t)2 * p.cch;
-      gstr[0] = 2 * C2; gstr[1] = C2 * p.w; gstr[2] = C2 * p.w * p.h; gstr[3] = 16;
-    }
-    cuuint32_t box[5] = {8, (cuuint32_t)p.wbox, (cuuint32_t)p.rbox, 1, (cuuint32_t)p.cg};
-    cuuint32_t es[5] = {1, 1, 1, 1, 1};
-    CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(x), gdim, gstr, box, es,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
-  }
+  CUtensorMap map_b;
   {
     cuuint64_t gdim[3] = {8, (cuuint64_t)p.ko.n_pad, (cuuint64_t)p.ng * p.e_pad};
     cuuint64_t gstr[2] = {16, (cuuint64_t)p.ko.n_pad * 16};
@@ -581,7 +703,8 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
     attr_set = true;
   }
   int grid = p.total_units < n_sm ? p.total_units : n_sm;
-  k_conv_tc<<<grid, kThreads, p.smem_bytes, stream>>>(map_a, map_b, p, bias, (const __nv_bfloat16 *)residual,
-                                                     (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  k_conv_tc<<<grid, kThreads, p.smem_bytes, stream>>>(map_b, p, (const __nv_bfloat16 *)x, bias,
+                                                     (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
+                                                     (DcWsHeader *)workspace);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
