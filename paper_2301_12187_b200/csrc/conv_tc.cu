@@ -59,6 +59,10 @@ struct TcParams {
   int off_b, off_a, off_out, off_bias;  // offsets in dynamic shared memory
   int smem_bytes;
   KOrder ko;
+  // per instruction j: low word of its A descriptor relative to the stage base:
+  // (offset of first chunk >> 4) | (distance to second chunk >> 4) << 16.  Lives in the kernel
+  // parameters (constant bank) so that the issuing warp reads it with uniform loads.
+  uint32_t a_desc_lo[128];
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -113,6 +117,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
   for (int i = 0; i < 16; ++i)
     if (mbar_try(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag, ws, site);
+}
+
+// Every lane of a converged warp waits (so each has observed the phase itself); the warp then
+// agrees on the outcome and stays converged.
+__device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          DcWsHeader *ws, uint32_t site) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, ws, site);
+  return __all_sync(0xffffffffu, ok) != 0;
+}
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b32 rx;\n\t"
+      "elect.sync rx|p, 0xffffffff;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2) {
@@ -208,13 +230,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t *v) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// shared-memory operand descriptor, K-major, no swizzle: 14-bit start>>4, LBO>>4 at bit 16,
-// SBO>>4 at bit 32 (128 bytes between 8-row groups), descriptor version 1 at bit 46
-__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes) {
-  const uint32_t lo = ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
-  const uint32_t hi = (128u >> 4) | (1u << 14);
-  return ((uint64_t)hi << 32) | lo;
-}
+// Shared-memory operand descriptors (K-major, no swizzle) are built inline: 14-bit start>>4,
+// LBO>>4 at bit 16, SBO>>4 at bit 32 (128 bytes between 8-row groups), version 1 at bit 46.
 
 // ------------------------------------------------------------------------------------------ tiles
 struct Tile {
@@ -247,9 +264,6 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
   __shared__ __align__(8) uint64_t bar_full[kMaxStages], bar_empty[kMaxStages], bar_accfull[2], bar_accempty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ uint32_t abort_s;
-  // per instruction j: low word of its A descriptor relative to the stage base:
-  // (offset of first chunk >> 4) | (distance to second chunk >> 4) << 16
-  __shared__ uint32_t a_desc_lo[128];
 
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t *smem_b = smem + p.off_b;
@@ -276,19 +290,6 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
   }
   if (threadIdx.x >= 5 * 32) {
     const int t = threadIdx.x - 5 * 32;
-    // chunk-pair table: entry e -> byte offset of its 16-byte column in an A stage
-    for (int j = t; j < p.e_pad / 2; j += 128) {
-      uint32_t off[2] = {0u, 16u};
-      for (int q = 0; q < 2; ++q) {
-        int e = 2 * j + q, pc, ccg, r, s;
-        if (dc_korder_decode(p.ko, e, &pc, &ccg, &r, &s)) {
-          int sx = (p.stride == 1) ? s : ((s - p.ko.pad) >> 1) - ((-p.ko.pad) >> 1);
-          off[q] = (uint32_t)(pc * p.region_bytes + ccg * p.plane_stride + (r * p.wbox + sx) * 16);
-        }
-      }
-      // the padding entry of an odd count gets its distance at issue time (it points at the zero plane)
-      a_desc_lo[j] = (off[0] >> 4) | (((off[1] - off[0]) >> 4) << 16);
-    }
     for (int i = t; i < p.nnt * p.n_tile; i += 128) bias_s[i] = (bias && i < p.c_out) ? bias[i] : 0.f;
     // the zero plane: second chunk of the padding entry, and the landing zone of reads past the last stage
     uint4 *z = reinterpret_cast<uint4 *>(smem_zero);
@@ -374,7 +375,9 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
     cp_async_wait_all();                         // nothing of this thread is in flight when the CTA leaves
   } else if (warp == 4) {
     // ================================================================== MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop converged and one elected lane issues: every operand is then
+    // warp-uniform (kernel parameters and loop counters), which keeps descriptor arithmetic cheap.
+    {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) | (8u << 24);
       const uint32_t desc_hi = (128u >> 4) | (1u << 14);
       const int npairs = p.e_pad / 2;
@@ -386,13 +389,13 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
         const int rows = (t.th - 1) * p.P + p.tw;
         const int nblk = (rows + 127) >> 7;
         const uint32_t a = tile_i & 1, aph = (tile_i >> 1) & 1;
-        if (!mbar_wait(&bar_accempty[a], aph ^ 1, abort_flag, ws, 0x20000u | a)) goto mma_done;
+        if (!warp_wait(&bar_accempty[a], aph ^ 1, abort_flag, ws, 0x20000u | a)) goto mma_done;
         tc_fence_after();
         const uint32_t d0 = tmem_base + a * (uint32_t)p.acc_cols;
         for (int grp = 0; grp < p.ng; ++grp, ++it) {
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1;
-          if (!mbar_wait(&bar_full[s], ph, abort_flag, ws, 0x30000u | s)) goto mma_done;
+          if (!warp_wait(&bar_full[s], ph, abort_flag, ws, 0x30000u | s)) goto mma_done;
           fence_proxy_async();
           tc_fence_after();
           const uint32_t a_base = smem_u32(smem_a + (size_t)s * p.a_stage_bytes);
@@ -401,23 +404,23 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
           const uint32_t b_step = 2u * (uint32_t)p.n_tile;
           // last pair of an odd entry count: second chunk = zero plane (same block offset on both sides)
           const uint32_t last = (uint32_t)(npairs - 1);
-          const uint32_t first_off = (a_desc_lo[last] & 0x3FFFu) << 4;
+          const uint32_t first_off = (p.a_desc_lo[last] & 0x3FFFu) << 4;
           const uint32_t pad_lo = (first_off >> 4) | (((zero_addr - a_base - first_off) >> 4) << 16);
           for (int b = 0; b < nblk; ++b) {
             const uint32_t d = d0 + (uint32_t)(b * p.n_tile);
             const uint32_t a_add = (a_base >> 4) + (uint32_t)b * 128u;
 #pragma unroll 4
             for (int j = 0; j < npairs; ++j) {
-              uint32_t lo = a_desc_lo[j];
+              uint32_t lo = p.a_desc_lo[j];
               if (odd_entries && (uint32_t)j == last) lo = pad_lo;
               const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
               const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
-              umma_bf16(d, ad, bd, idesc, (grp | j) != 0 ? 1u : 0u);
+              if (elect_one()) umma_bf16(d, ad, bd, idesc, (grp | j) != 0 ? 1u : 0u);
             }
           }
-          umma_commit(&bar_empty[s]);            // stage s may be refilled once these MMAs finish
+          if (elect_one()) umma_commit(&bar_empty[s]);   // stage s may be refilled once these MMAs finish
         }
-        umma_commit(&bar_accfull[a]);            // accumulator a is complete
+        if (elect_one()) umma_commit(&bar_accfull[a]);   // accumulator a is complete
       }
     }
   mma_done:;
@@ -666,6 +669,21 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   p->off_out = p->off_bias + bias_bytes;
   p->off_a = p->off_out + 2 * p->out_tile_bytes;
   p->smem_bytes = 1024 + p->off_a + stages * p->a_stage_bytes + slack;
+  // chunk-pair table: entry e -> byte offset of its 16-byte column in an A stage.  The padding
+  // entry of an odd count gets its distance at issue time (it points at the zero plane).
+  for (int j = 0; j < ko.e_pad / 2; ++j) {
+    uint32_t off[2] = {0u, 16u};
+    for (int q = 0; q < 2; ++q) {
+      int pc, ccg, r, s;
+      if (dc_korder_decode(ko, 2 * j + q, &pc, &ccg, &r, &s)) {
+        int sx = (g->stride == 1) ? s : dc_floor_div2(s - g->pad) - dc_floor_div2(-g->pad);
+        off[q] = (uint32_t)(pc * p->region_bytes + ccg * p->plane_stride + (r * p->wbox + sx) * 16);
+      } else if (q == 1) {
+        off[1] = off[0] + 16;
+      }
+    }
+    p->a_desc_lo[j] = (off[0] >> 4) | (((off[1] - off[0]) >> 4) << 16);
+  }
   return true;
 }
 
