@@ -128,6 +128,34 @@ dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const dc_residual
                          void *workspace, size_t workspace_bytes, dc_stream stream);
 
 /*
+ * dc_merge_chain for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for integration, it computes exactly what dc_merge_chain computes.)
+ *
+ * Who needs it: code that merges from inside an allocator or memory-pool callback, plug-ins whose
+ * host forbids allocation calls once it is initialised, and processes that have handed all device
+ * memory to another allocator -- none of them can cudaMalloc a workspace.  Here the intermediate
+ * kernels of the merge live in a fixed array compiled into the library (dc_merge_chain_static_capacity()
+ * bytes, 4 MiB; every GPU that loads the library holds it until the process exits).  The call
+ * allocates nothing and frees nothing, on the device or through any library.
+ *
+ * Inputs and outputs are as for dc_merge_chain, minus the workspace.  Runs whose intermediates
+ * need more than the capacity (compare dc_merge_query's workspace_bytes) are refused with
+ * DC_ERR_WORKSPACE before anything is launched.
+ *
+ * The first call on a device looks up the array's device address (with that device current); make
+ * that first call before starting any stream capture.  All calls on a device share the one array:
+ * it keeps the previous call's contents, which are overwritten (nothing needs to start at zero),
+ * and two calls whose kernels overlap on the GPU (different streams, or a graph replayed
+ * concurrently) race on it -- serialise them.
+ */
+dc_status dc_merge_chain_static(const dc_layer *layers, int n_layers, const dc_residual *res,
+                                int n_res, float *w_merged, float *b_merged, void *w_packed,
+                                dc_dtype packed_dtype, dc_stream stream);
+
+/* Host only: size in bytes of the built-in scratch dc_merge_chain_static works in. */
+size_t dc_merge_chain_static_capacity(void);
+
+/*
  * Repack fp32 [c_out][c_in/groups][k][k] weights (device) into the layout the forward kernels
  * read.  Dense, DC_F32: fp32 [k][k][c_in][c_out].  Dense, DC_BF16: bfloat16 (round to nearest
  * even) in the K-chunked operand layout of the tensor-core kernel, zero padded (opaque; size

@@ -473,3 +473,51 @@ extern "C" dc_status dc_pack_weights(const float *w, const dc_geom *g, dc_dtype 
   }
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
+
+// ----------------------------------------------------------------------------------------------
+// Merge without any caller-provided or allocated scratch memory.
+//
+// Some callers cannot allocate device memory at the point where they merge: code running inside a
+// memory-pool or allocator callback, a plug-in whose host forbids allocation calls after
+// initialisation, or a process that has handed the whole GPU to another allocator.  For them the
+// intermediate kernels of the merge live in a fixed array that is part of the library image: every
+// GPU that loads the library holds these bytes until the process exits.
+// ----------------------------------------------------------------------------------------------
+#define DC_STATIC_SCRATCH_BYTES (4u << 20)
+static __device__ __align__(256) unsigned char g_merge_scratch[DC_STATIC_SCRATCH_BYTES];
+
+// In host code the symbol above is only a handle; the device address is looked up once per device.
+#define DC_MAX_DEVICES 64
+static void *g_merge_scratch_addr[DC_MAX_DEVICES];
+
+extern "C" size_t dc_merge_chain_static_capacity(void) { return (size_t)DC_STATIC_SCRATCH_BYTES; }
+
+extern "C" dc_status dc_merge_chain_static(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                                           float *w_merged, float *b_merged, void *w_packed,
+                                           dc_dtype packed_dtype, dc_stream stream) {
+  if (!w_merged || !b_merged) return DC_ERR_INVALID_ARG;
+  if (packed_dtype != DC_F32 && packed_dtype != DC_BF16) return DC_ERR_INVALID_ARG;
+  size_t need = 0;
+  dc_status s = merge_walk(layers, n_layers, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr,
+                           false, nullptr, &need);
+  if (s != DC_OK) return s;
+  if (need > (size_t)DC_STATIC_SCRATCH_BYTES) return DC_ERR_WORKSPACE;   // run too large for the built-in scratch
+  if (!dc_aligned16(w_merged) || !dc_aligned16(b_merged) || (w_packed && !dc_aligned16(w_packed)))
+    return DC_ERR_ALIGNMENT;
+  for (int i = 0; i < n_layers; ++i)
+    if (!dc_aligned16(layers[i].weight)) return DC_ERR_ALIGNMENT;
+  int dev = -1;
+  DC_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= DC_MAX_DEVICES) return DC_ERR_UNSUPPORTED;
+  if (!g_merge_scratch_addr[dev]) {
+    // first call on this device (with that device current): resolve the array's device address
+    void *ptr = nullptr;
+    DC_CUDA_OK(cudaGetSymbolAddress(&ptr, g_merge_scratch));
+    if (!ptr) return DC_ERR_CUDA;
+    g_merge_scratch_addr[dev] = ptr;
+  }
+  // Nothing in the scratch has to start at zero: every intermediate is written in full before it
+  // is read, so the contents a previous call left behind are simply overwritten.
+  return merge_walk(layers, n_layers, res, n_res, w_merged, b_merged, w_packed, packed_dtype,
+                    g_merge_scratch_addr[dev], (cudaStream_t)stream, true, nullptr, nullptr);
+}

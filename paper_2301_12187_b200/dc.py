@@ -58,6 +58,9 @@ EXPORTS = {
     "dc_packed_bytes": (C.c_int, [C.POINTER(Geom), C.c_int, C.POINTER(C.c_size_t)]),
     "dc_merge_chain": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "dc_merge_chain_static": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
+    "dc_merge_chain_static_capacity": (C.c_size_t, []),
     "dc_pack_weights": (C.c_int, [C.c_void_p, C.POINTER(Geom), C.c_int, C.c_void_p, C.c_void_p]),
     "dc_conv_workspace_bytes": (C.c_size_t, []),
     "dc_conv_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Geom), C.c_void_p,
@@ -213,6 +216,20 @@ def merge_chain(layers, residuals, w_merged, b_merged, w_packed, packed_dtype, w
                                 _ptr(w_packed), packed_dtype, _ptr(workspace),
                                 workspace.numel() * workspace.element_size(), _stream(stream)),
            "dc_merge_chain")
+
+
+def merge_chain_static(layers, residuals, w_merged, b_merged, w_packed, packed_dtype, stream=None):
+    """dc_merge_chain for callers that cannot allocate: the scratch is a fixed array inside the
+    library (see include/dc.h for the limit and the sharing rules)."""
+    arr = layer_array(layers)
+    res, n_res = _res_array(residuals)
+    _check(lib().dc_merge_chain_static(arr, len(layers), res, n_res, _ptr(w_merged), _ptr(b_merged),
+                                       _ptr(w_packed), packed_dtype, _stream(stream)),
+           "dc_merge_chain_static")
+
+
+def merge_chain_static_capacity() -> int:
+    return int(lib().dc_merge_chain_static_capacity())
 
 
 def pack_weights(w, g: Geom, dtype: int, w_packed, stream=None):
