@@ -1,0 +1,115 @@
+"""Full depth-compressed MobileNetV2-1.0 forward (batch 128, 224x224, bf16) against the oracle.
+
+Per launch group: the GPU output of sampled images against the oracle applied to the GPU's own
+previous output (isolates each layer, 2e-2 each; 3 x 2e-2 for an unmerged block, which rounds two
+intermediate maps).  End to end: one image against the oracle's sequential network."""
+import numpy as np
+import pytest
+
+from oracle import dc_oracle as O
+from paper_2301_12187_b200 import inputs as I
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+
+
+def nchw(t):
+    return t.float().cpu().numpy().astype(np.float64).transpose(0, 3, 1, 2)
+
+
+def oracle_group(net, cn, op, x_prev, skip):
+    """What one launch group computes, by the oracle, from the map x_prev (NCHW fp64)."""
+    specs = [net.layers[i] for i in op.layers]
+    if op.kind == "block":
+        cur = x_prev
+        for s in specs:
+            Wf, bf = O.fold_bn(s)
+            cur = O.conv_direct(cur, Wf, bf, s.k, s.stride, s.pad, s.groups)
+            if s.act == "relu6":
+                cur = O.relu6(cur)
+        if net.blocks[specs[0].block]["residual"]:
+            cur = cur + x_prev
+        return cur
+    po = cn.plan_ops[op.plan_index[0]]
+    cur = O.chain_forward_reordered(x_prev, specs, po.residuals)
+    if skip is not None:
+        cur = cur + skip
+    return O.relu6(cur) if po.act == "relu6" else cur
+
+
+@pytest.fixture(scope="module")
+def run():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_12187_b200 import dc
+    from paper_2301_12187_b200.network import CompressedNetwork
+    net = I.mobilenet_v2(seed=0, batch=128)
+    acts, plan = I.plan_spans(net, seed=0)
+    cn = CompressedNetwork(net, acts, plan)
+    n_merged = cn.merge()
+    x_np = I.make_input(0, net.x_shape, bf16=True)
+    x = torch.from_numpy(x_np).to("cuda", dtype=torch.bfloat16)
+    y = cn.forward(x)
+    torch.cuda.synchronize()
+    assert cn.status() == dc.OK
+    return dict(dc=dc, net=net, cn=cn, x=x, x_np=x_np, y=y, n_merged=n_merged)
+
+
+def test_plan_covers_the_network_and_uses_every_kind_of_call(run):
+    cn = run["cn"]
+    kinds = {op.kind for op in cn.ops}
+    assert kinds >= {"conv", "dw"}
+    assert run["n_merged"] >= 8 and any(op.merged for op in cn.ops)
+    assert sorted(i for op in cn.ops for i in op.layers) == list(range(52))
+    assert tuple(run["y"].shape) == (128, 7, 7, 1280)
+    assert not torch.isnan(run["y"].float()).any()
+
+
+def test_each_launch_group_matches_the_oracle_on_sampled_images(run):
+    net, cn, x = run["net"], run["cn"], run["x"]
+    sel = [0, 127]
+    prev = x
+    worst = 0.0
+    for op in cn.ops:
+        skip = None
+        if op.kind != "block" and op.add_from == -1:
+            skip = nchw(x[sel])
+        elif op.kind != "block" and op.add_from >= 0:
+            skip = nchw(cn.ops[op.add_from].y[sel])
+        ref = oracle_group(net, cn, op, nchw(prev[sel]), skip)
+        err = O.rel_l2(nchw(op.y[sel]), ref)
+        tol = 3 * TOL if op.kind == "block" else TOL
+        assert err <= tol, ([net.layers[i].name for i in op.layers], op.kind, err)
+        worst = max(worst, err)
+        prev = op.y
+    print("worst per-group rel-L2: %.3e" % worst)
+
+
+def test_end_to_end_against_the_sequential_network(run):
+    net, cn, x = run["net"], run["cn"], run["x"]
+    cur = nchw(x[:1])
+    outs = []
+    for op in cn.ops:
+        skip = None
+        if op.kind != "block" and op.add_from == -1:
+            skip = nchw(x[:1])
+        elif op.kind != "block" and op.add_from >= 0:
+            skip = outs[op.add_from]
+        cur = oracle_group(net, cn, op, cur, skip)
+        outs.append(cur)
+    err = O.rel_l2(nchw(run["y"][:1]), cur)
+    print("end-to-end rel-L2 after %d launch groups: %.3e" % (len(cn.ops), err))
+    assert err <= TOL
+
+
+def test_graph_replay_reproduces_the_eager_result(run):
+    cn, x = run["cn"], run["x"]
+    ref = run["y"].clone()
+    g = cn.capture(x)
+    cn.ops[-1].y.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(cn.ops[-1].y, ref)
+    assert cn.status() == run["dc"].OK
