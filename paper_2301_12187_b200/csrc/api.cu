@@ -39,8 +39,11 @@ extern "C" dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, co
       (bias && !dc_aligned16(bias)) || (residual && !dc_aligned16(residual)))
     return DC_ERR_ALIGNMENT;
   cudaStream_t st = (cudaStream_t)stream;
-  const bool tc_ok = dtype == DC_BF16 && dc_conv_tc_supported(n, h, w, g);
-  if (algo == DC_ALGO_TCGEN05 && !tc_ok) return DC_ERR_UNSUPPORTED;
+  const bool fold_ok = dtype == DC_BF16 && dc_conv_fold_supported(n, h, w, g);
+  const bool tc_ok = dtype == DC_BF16 && !fold_ok && dc_conv_tc_supported(n, h, w, g);
+  if (algo == DC_ALGO_TCGEN05 && !tc_ok && !fold_ok) return DC_ERR_UNSUPPORTED;
+  if (fold_ok && algo != DC_ALGO_SIMT)
+    return dc_launch_conv_fold(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   if (tc_ok && algo != DC_ALGO_SIMT)
     return dc_launch_conv_tc(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   return dc_launch_conv_simt(x, n, h, w, g, w_packed, bias, act, residual, y, dtype, st);

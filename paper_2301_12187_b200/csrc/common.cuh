@@ -34,6 +34,13 @@ static inline int dc_out_extent(int h, int k, int s, int p) {
 // with one all-zero entry when their count is odd, because one tensor-core instruction consumes
 // two entries (K = 16).  Stride 1 has a single parity; stride 2 splits the taps by the parity
 // of the input column they read.
+//
+// "Fold" order (stride 1, k >= 3, few channels): the tap COLUMN s moves from K to N.  An entry is
+// (chunk cc, tap row r) and the operand has k * co8 rows n = s * co8 + o (co8 = output channels
+// rounded up to 8): one instruction then produces, for every tap column at once, the partial sums
+// Z[m][s][o] = sum_{r,c} x[m + r * pitch][c] * W[o][c][r][s], and the epilogue adds the k column
+// groups with a row shift, y[m][o] = sum_s Z[m + s][s][o].  This cuts the number of tensor-core
+// instructions per output by k, which is what bounds small-channel convolutions.
 // ----------------------------------------------------------------------------------------------
 struct KOrder {
   int k, stride, pad;
@@ -45,7 +52,9 @@ struct KOrder {
   int s0[2];          // first tap column of each parity
   int e;              // entries per group = cg * taps
   int e_pad;          // e rounded up to even
-  int n_pad;          // output channels rounded up to 16
+  int n_pad;          // operand rows rounded up to 16 (output channels, or k * co8 in fold order)
+  int fold;           // 1: fold order
+  int co8;            // output channels rounded up to 8
 };
 
 static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
@@ -54,7 +63,25 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->cch = dc_div_up(g->c_in, 8);
   ko->taps = g->k * g->k;
   ko->n_pad = (int)dc_round_up((size_t)g->c_out, 16);
+  ko->co8 = (int)dc_round_up((size_t)g->c_out, 8);
+  ko->fold = 0;
   ko->pcs = (g->stride == 2) ? 2 : 1;
+  if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch <= 8 && ko->co8 <= 32 &&
+      g->c_in % 8 == 0 && g->c_out % 8 == 0) {
+    // every column group is read back as 32 accumulator columns: the last one must fit as well
+    int rows = g->k * ko->co8;
+    if ((g->k - 1) * ko->co8 + 32 > rows) rows = (g->k - 1) * ko->co8 + 32;
+    const int n_pad = (int)dc_round_up((size_t)rows, 16);
+    if ((size_t)ko->cch * g->k * n_pad * 16 <= 64 * 1024) {
+      ko->fold = 1;
+      ko->n_pad = n_pad;
+      ko->ns[0] = g->k; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
+      ko->cg = ko->cch; ko->ng = 1;
+      ko->e = ko->cch * g->k;
+      ko->e_pad = (ko->e + 1) & ~1;
+      return;
+    }
+  }
   if (ko->pcs == 1) {
     ko->ns[0] = g->k; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
   } else {
@@ -81,6 +108,13 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
 __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
                                                         int *r, int *s) {
   if (e >= ko.e) return false;
+  if (ko.fold) {
+    *pc = 0;
+    *ccg = e / ko.k;
+    *r = e - *ccg * ko.k;
+    *s = -1;               // the tap column is part of the row index, not of the entry
+    return true;
+  }
   if (ko.pcs == 1) {
     *pc = 0;
     *ccg = e / ko.taps;
@@ -105,6 +139,7 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 // (channel chunk cc in [0,cch), tap r, s) -> position of that chunk in the packed weights,
 // in units of chunk planes (n_pad * 8 elements each)
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
+  if (ko.fold) return cc * ko.k + r;
   int grp = cc / ko.cg, ccg = cc - grp * ko.cg;
   int e;
   if (ko.pcs == 1) {
@@ -116,6 +151,11 @@ __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc,
     e = base + ccg * per + r * ko.ns[p] + (s - ko.s0[p]) / 2;
   }
   return grp * ko.e_pad + e;
+}
+
+// row of output channel o (and tap column s) inside a chunk plane of the packed weights
+__host__ __device__ static inline int dc_korder_row(const KOrder &ko, int s, int o) {
+  return ko.fold ? s * ko.co8 + o : o;
 }
 
 __device__ __forceinline__ float dc_act_apply(float v, int act) {
@@ -137,4 +177,8 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
                             const float *bias, dc_act act, const void *residual, void *y,
                             void *workspace, cudaStream_t stream);
 bool dc_conv_tc_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y,
+                              void *workspace, cudaStream_t stream);
+bool dc_conv_fold_supported(int n, int h, int w, const dc_geom *g);
 dc_status dc_validate_geom(const dc_geom *g);

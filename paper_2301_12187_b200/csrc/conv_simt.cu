@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(128) k_conv_dense_bf16(const __nv_bfloat16 *__
         const __nv_bfloat16 *xp = x + (((size_t)img * h + yy) * wd + xx) * g.c_in;
         for (int cc = 0; cc < ko.cch; ++cc) {
           const int plane = dc_korder_encode(ko, cc, u, v);
-          const uint4 wv = *reinterpret_cast<const uint4 *>(w + ((size_t)plane * ko.n_pad + o) * 8);
+          const uint4 wv = *reinterpret_cast<const uint4 *>(w + ((size_t)plane * ko.n_pad + dc_korder_row(ko, v, o)) * 8);
           const __nv_bfloat16 *wb = reinterpret_cast<const __nv_bfloat16 *>(&wv);
           if (vec) {
             const uint4 xv = *reinterpret_cast<const uint4 *>(xp + cc * 8);

@@ -205,6 +205,11 @@ __global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrde
     int pc, ccg, r, s;
     float v = 0.f;
     if (dc_korder_decode(ko, e, &pc, &ccg, &r, &s)) {
+      if (ko.fold) {                       // row = (tap column, output channel)
+        s = o / ko.co8;
+        o -= s * ko.co8;
+        if (s >= ko.k) o = c_out;          // padding rows
+      }
       int c = (grp * ko.cg + ccg) * 8 + c8;
       if (o < c_out && c < ko.c_in) v = w[(((size_t)o * ko.c_in + c) * ko.k + r) * ko.k + s];
     }

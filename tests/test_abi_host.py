@@ -75,9 +75,12 @@ def test_merge_query_rejects_bad_chains():
 def test_packed_bytes():
     assert dc.packed_bytes(dc.geom(24, 24, 1, 3, 1, 1), dc.F32) == 24 * 24 * 9 * 4
     assert dc.packed_bytes(dc.geom(96, 96, 96, 3, 1, 1), dc.BF16) == 96 * 9 * 4
-    # 27 chunk entries padded to 28, 24 output channels padded to 32, 16 bytes per (entry, channel)
-    assert dc.packed_bytes(dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == 28 * 32 * 16
-    assert dc.packed_bytes(dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == 100 * 32 * 16
+    # fold order: 3 chunks x 3 tap rows = 9 entries padded to 10; rows = 3 tap columns x 24 channels,
+    # padded to 80; 16 bytes per (entry, row)
+    assert dc.packed_bytes(dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == 10 * 80 * 16
+    assert dc.packed_bytes(dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == 20 * 160 * 16
+    # general order: 18 chunks x 9 taps in 3 groups of 6 chunks, 64 output channels
+    assert dc.packed_bytes(dc.geom(144, 64, 1, 3, 1, 1), dc.BF16) == 3 * 54 * 64 * 16
     assert dc.packed_bytes(dc.geom(3, 32, 1, 3, 2, 1), dc.BF16) == 10 * 32 * 16
     assert status_of(dc.packed_bytes, dc.geom(24, 24, 1, 4, 1, 1), dc.BF16) == dc.ERR_UNSUPPORTED
 
