@@ -29,25 +29,29 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
   asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ uint32_t mbar_try(uint64_t *bar, uint32_t parity) {
+// One probe of the phase; the hardware may park the warp for up to `hint_ns` before answering,
+// so a waiting warp does not compete for issue slots.
+__device__ __forceinline__ uint32_t mbar_try(uint64_t *bar, uint32_t parity, uint32_t hint_ns) {
   uint32_t done;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}"
       : "=r"(done)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
       : "memory");
   return done;
 }
 
-// Bounded wait.  Returns false when the wait ran out (or another role already gave up).
-static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                            DcWsHeader *ws, uint32_t site) {
+// Bounded wait.  Returns false when the wait ran out (or another role already gave up).  Not
+// inlined: the tensor-core kernels are sensitive to their instruction footprint and every wait
+// site shares this code.
+static __device__ __noinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                              DcWsHeader *ws, uint32_t site) {
+  if (mbar_try(bar, parity, 2000u)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
-    for (int i = 0; i < 32; ++i)
-      if (mbar_try(bar, parity)) return true;
+    if (mbar_try(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
     if (globaltimer_ns() - t0 > kWaitLimitNs) {
       *abort_flag = 1;
@@ -56,12 +60,6 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parit
       return false;
     }
   }
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          DcWsHeader *ws, uint32_t site) {
-  for (int i = 0; i < 16; ++i)
-    if (mbar_try(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, ws, site);
 }
 
 // Every lane of a converged warp waits (so each has observed the phase itself); the warp then
@@ -98,6 +96,16 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32
 // the mbarrier receives one arrival from this thread once all its earlier cp.async copies have landed
 __device__ __forceinline__ void cp_async_arrive(uint64_t *bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// waits until at most n (0..3) of this thread's committed cp.async groups are still in flight
+__device__ __forceinline__ void cp_async_wait_pending(int n) {
+  switch (n) {
+    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+  }
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
