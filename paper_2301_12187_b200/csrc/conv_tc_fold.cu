@@ -41,6 +41,7 @@ constexpr int kConsumerThreads = (1 + 4 * kGroups) * 32;
 constexpr int kThreads = kProducerThreads + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barriers: 1..kGroups epilogue groups, 7 all consumers
 constexpr int kMaxTiles = 96;
+constexpr int kMaxPairs = 16;                   // tensor-core instructions per 128-row block
 
 struct FoldParams {
   int n_img, h, w, ho, wo, c_in, c_out, co8;
@@ -56,7 +57,7 @@ struct FoldParams {
   int tmem_cols;
   int npairs, odd;
   uint32_t cch_inv;            // ceil(65536 / cch): q / cch == (q * cch_inv) >> 16 for q < 4096
-  uint32_t a_desc_lo[64];      // per instruction: (first chunk offset >> 4) | (distance >> 4) << 16
+  uint32_t a_desc_lo[kMaxPairs];      // per instruction: (first chunk offset >> 4) | (distance >> 4) << 16
 };
 
 // A tile = up to p.th output rows of one column strip of one image; c0 = index of its first
@@ -284,6 +285,8 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     const uint32_t a_base0 = smem_u32(smem_a);
     const long long row_stride = (long long)p.w * C2;
     const uint32_t drow_stride = (uint32_t)p.wbox * 16u;
+    int s = 0;
+    uint32_t ph = 0;
 #pragma unroll 1
     for (int it = 0; it < ntiles; ++it) {
       const Tile t = sh.tiles[it];
@@ -295,8 +298,6 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
       // pieces of a pixel row are contiguous in memory: piece q sits 16*q bytes after the row start
       const char *tile_base = reinterpret_cast<const char *>(x) + (size_t)t.img * p.h * row_stride +
                               ((long long)gy0 * p.w + gx0) * C2;
-      const int s = it % p.stages;
-      const uint32_t ph = (it / p.stages) & 1;
       if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
       if (ptid == 0 && it == 0) {
         // the weights ride on the first stage's barrier as transaction bytes and stay resident
@@ -321,6 +322,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
         for (; r < rows; ++r, dst += drow_stride) cp_async16(dst, x, 0u);
       }
       cp_async_arrive(&sh.full[s]);              // arrives by itself when this thread's copies have landed
+      if (++s == p.stages) { s = 0; ph ^= 1; }
     }
     cp_async_wait_all();                         // nothing of this thread is in flight when the CTA leaves
   } else {
@@ -351,11 +353,11 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
       const uint32_t last = (uint32_t)(p.npairs - 1);
       const uint32_t first_off = (p.a_desc_lo[last] & 0x3FFFu) << 4;
       bool ok = true;
+      int s = 0;                                 // stage and its phase, accumulator slot and its phase
+      uint32_t ph = 0, slot = 0, sph = 1;
 #pragma unroll 1
       for (int it = 0; it < ntiles && ok; ++it) {
         const Tile t = sh.tiles[it];
-        const int s = it % p.stages;
-        const uint32_t ph = (it / p.stages) & 1;
         if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
         tc_fence_after();
         const uint32_t a_base = smem_u32(smem_a + (size_t)s * p.a_stage_bytes);
@@ -363,23 +365,26 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
         const uint32_t pad_lo = (first_off >> 4) | (((zero_addr - a_base - first_off) >> 4) << 16);
 #pragma unroll 1
         for (int b = 0; b < t.nblk; ++b) {
-          const uint32_t c = (uint32_t)(t.c0 + b);
-          const uint32_t slot = c % p.slots, sph = (c / p.slots) & 1;
-          if (!warp_wait(&sh.slot_empty[slot], sph ^ 1, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
+          if (!warp_wait(&sh.slot_empty[slot], sph, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
           const uint32_t a_add = (a_base >> 4) + (uint32_t)(b * p.blk_rows);
-#pragma unroll 1
-          for (int j = 0; j < p.npairs; ++j) {
-            uint32_t lo = p.a_desc_lo[j];
-            if (p.odd && (uint32_t)j == last) lo = pad_lo;
-            const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
-            const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
-            if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+          // statically indexed so that the table entries are read straight from the constant bank
+#pragma unroll
+          for (int j = 0; j < kMaxPairs; ++j) {
+            if (j < p.npairs) {
+              uint32_t lo = p.a_desc_lo[j];
+              if (p.odd && (uint32_t)j == last) lo = pad_lo;
+              const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
+              const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
+              if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+            }
           }
           if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
+          if (++slot == (uint32_t)p.slots) { slot = 0; sph ^= 1; }
         }
         if (ok && elect_one()) umma_commit(&sh.empty[s]);      // the stage may be refilled once these MMAs finish
+        if (++s == p.stages) { s = 0; ph ^= 1; }
       }
     } else {
       switch (p.co8) {
@@ -454,7 +459,7 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->blk_rows = 128 - (g->k - 1);
   p->npairs = ko.e_pad / 2;
   p->odd = ko.e & 1;
-  if (p->npairs > 64) return false;
+  if (p->npairs > kMaxPairs) return false;
   p->slots = 512 / p->n_pad;
   if (p->slots > kMaxSlots) p->slots = kMaxSlots;
   if (p->slots < 2) return false;

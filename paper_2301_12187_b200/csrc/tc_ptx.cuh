@@ -43,12 +43,23 @@ __device__ __forceinline__ uint32_t mbar_try(uint64_t *bar, uint32_t parity, uin
   return done;
 }
 
-// Bounded wait.  Returns false when the wait ran out (or another role already gave up).  Not
-// inlined: the tensor-core kernels are sensitive to their instruction footprint and every wait
-// site shares this code.
-static __device__ __noinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                              DcWsHeader *ws, uint32_t site) {
-  if (mbar_try(bar, parity, 2000u)) return true;
+// Non-blocking probe of the phase (cheap: no suspension).
+__device__ __forceinline__ uint32_t mbar_test(uint64_t *bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return done;
+}
+
+// Slow path of the bounded wait: parks the warp in hardware between probes.  Not inlined: the
+// tensor-core kernels are sensitive to their instruction footprint and every wait site shares it.
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                                   DcWsHeader *ws, uint32_t site) {
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
     if (mbar_try(bar, parity, 20000u)) return true;
@@ -60,6 +71,13 @@ static __device__ __noinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, vo
       return false;
     }
   }
+}
+
+// Bounded wait.  Returns false when the wait ran out (or another role already gave up).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          DcWsHeader *ws, uint32_t site) {
+  if (mbar_test(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, ws, site);
 }
 
 // Every lane of a converged warp waits (so each has observed the phase itself); the warp then
