@@ -68,10 +68,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->pcs = (g->stride == 2) ? 2 : 1;
   if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch <= 8 && ko->co8 <= 32 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
-    // every column group is read back as 32 accumulator columns: the last one must fit as well
-    int rows = g->k * ko->co8;
-    if ((g->k - 1) * ko->co8 + 32 > rows) rows = (g->k - 1) * ko->co8 + 32;
-    const int n_pad = (int)dc_round_up((size_t)rows, 16);
+    const int n_pad = (int)dc_round_up((size_t)(g->k * ko->co8), 16);
     if ((size_t)ko->cch * g->k * n_pad * 16 <= 64 * 1024) {
       ko->fold = 1;
       ko->n_pad = n_pad;

@@ -21,25 +21,28 @@
 // small dynamic instruction count: the CTA's tiles are decoded once into a table, loops are not
 // unrolled, activation / skip-input variants are compiled separately.  Behind the activation
 // stages the unit is the 128-row block: blocks go round-robin over a ring of accumulator slots in
-// tensor memory, one warp issues the MMAs, two epilogue groups of four warps take alternate
-// blocks.  The valid outputs of a block are one contiguous range of the NHWC output when tiles
+// tensor memory, one warp issues the MMAs, four epilogue groups of four warps take the blocks
+// in turn.  The valid outputs of a block are one contiguous range of the NHWC output when tiles
 // span the image width, so each block leaves with one bulk copy.
 //
-// Roles (416 threads): warps 0-3 producers, warp 4 MMA issue (converged warp, elected lane) and
-// tensor-memory owner, warps 5-12 epilogue.  Waits are bounded (tc::mbar_wait).
+// Roles (640 threads): warps 0-2 producers, warp 3 MMA issue (converged warp, elected lane) and
+// tensor-memory owner, warps 4-19 epilogue (four groups).  Waits are bounded (tc::mbar_wait).
 #include "tc_ptx.cuh"
 
 namespace {
 using namespace tc;
 
 constexpr int kMaxStages = 8;
-constexpr int kMaxSlots = 4;
-constexpr int kProducerThreads = 128;
-constexpr int kGroups = 2;                       // epilogue groups of 4 warps
-constexpr int kFirstEpiWarp = 5;
+constexpr int kMaxSlots = 6;
+constexpr int kProducerThreads = 96;
+constexpr int kMmaWarp = kProducerThreads / 32;
+constexpr int kGroups = 4;                       // epilogue groups of 4 warps
+constexpr int kFirstEpiWarp = kMmaWarp + 1;
+static_assert(kFirstEpiWarp % 4 == 0, "epilogue warp w reads tensor-memory lane quadrant w mod 4");
 constexpr int kConsumerThreads = (1 + 4 * kGroups) * 32;
 constexpr int kThreads = kProducerThreads + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barriers: 1..kGroups epilogue groups, 7 all consumers
+static_assert(kGroups < kBarConsumers, "named barrier ids");
 constexpr int kMaxTiles = 96;
 constexpr int kMaxPairs = 16;                   // tensor-core instructions per 128-row block
 
@@ -52,11 +55,12 @@ struct FoldParams {
   int mb;                      // blocks per full tile
   int total_units;             // output row segments, ordered (img, xt, y)
   int plane_stride, a_stage_bytes, b_bytes;
-  int stages, slots, act, bulk_out, out_buf_bytes, xch_buf_floats;
+  int stages, slots, groups, act, bulk_out, out_buf_bytes, xch_buf_floats;
   int off_b, off_bias, off_out, off_xch, off_a, smem_bytes;
   int tmem_cols;
   int npairs, odd;
   uint32_t cch_inv;            // ceil(65536 / cch): q / cch == (q * cch_inv) >> 16 for q < 4096
+  uint32_t wbox_inv;           // ceil(2^20 / wbox): q / wbox == (q * wbox_inv) >> 20 for q < 4096
   uint32_t a_desc_lo[kMaxPairs];      // per instruction: (first chunk offset >> 4) | (distance >> 4) << 16
 };
 
@@ -100,7 +104,10 @@ __device__ __noinline__ void build_tiles(const FoldParams &p, Shared &sh, int be
 }
 
 // Epilogue of one group (4 warps = 128 threads, thread = GEMM row): blocks c = grp mod kGroups.
-// ACT and RES are compile-time so the per-pixel code carries no runtime switches.
+// ACT and RES are compile-time so the per-pixel code carries no runtime switches.  Per block the
+// group meets at two named barriers: after the cross-warp rows are in shared memory, and after the
+// block's pixels are staged for the bulk copy.  Exchange rows and staging buffer alternate between
+// two copies, so a block never waits for the previous block's readers.
 template <int CO8, int ACT, int RES>
 __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
                                               float *xch, uint8_t *smem_out, const __nv_bfloat16 *residual,
@@ -113,40 +120,45 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
   const int m = q * 32 + lane;
   const uint32_t tmem_row = sh.tmem_base + ((uint32_t)(q * 32) << 16);
   volatile uint32_t *abort_flag = &sh.abort;
-  uint8_t *obuf = smem_out + (size_t)grp * p.out_buf_bytes;
+  uint8_t *obuf0 = smem_out + (size_t)grp * 2 * p.out_buf_bytes;
   const int xch_q = (km1 * (km1 + 1) / 2) * 32;  // floats per quadrant: rows (s, lane < s), 32 channels each
   float *xg = xch + (size_t)grp * 2 * p.xch_buf_floats;
-  float bias_r[CO8];
-#pragma unroll
-  for (int o = 0; o < CO8; ++o) bias_r[o] = bias_s[o];
-  uint32_t mine = 0;                             // blocks this group has done
+  // accumulator slot and its phase for block c = grp, advanced by kGroups per block
+  uint32_t slot = (uint32_t)grp, sph = 0;
+  while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+  uint32_t next = (uint32_t)grp, mine = 0;       // next block of this group, blocks it has done
+  // A waiter may trail its barrier by one phase at most, so a slot must not complete twice before
+  // its group has looked: no more groups than slots take part.
+  if (grp >= p.groups) return;
+  const int ntiles = sh.ntiles;
 #pragma unroll 1
-  for (int ti = 0; ti < sh.ntiles; ++ti) {
+  for (int ti = 0; ti < ntiles; ++ti) {
     const Tile t = sh.tiles[ti];
 #pragma unroll 1
-    for (int b = 0; b < t.nblk; ++b) {
-      const uint32_t c = (uint32_t)(t.c0 + b);
-      if ((int)(c % kGroups) != grp) continue;
-      const uint32_t slot = c % p.slots, sph = (c / p.slots) & 1;
-      if (p.bulk_out && elected) bulk_wait_read0();          // this group's previous store has read its buffer
-      // the group passes or leaves together, so nobody is left alone at its named barrier
+    for (int b = (int)next - t.c0; b < t.nblk; b += p.groups, next += p.groups) {
+      // the group passes or leaves together, so nobody is left alone at a named barrier
       if (!bar_all(1 + grp, 128, mbar_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot))) return;
       tc_fence_after();
       const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
       float *xw = xg + (mine & 1) * p.xch_buf_floats;
+      uint8_t *obuf = obuf0 + (mine & 1) * p.out_buf_bytes;
       ++mine;
       float acc[CO8];
       {
-        uint32_t v[32];
-        tmem_ld32(taddr, v);
+        uint32_t v[CO8];
+        tmem_ld_cols<CO8>(taddr, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int o = 0; o < CO8; ++o) acc[o] = __uint_as_float(v[o]) + bias_r[o];
+        for (int o = 0; o < CO8; o += 4) {
+          const float4 bv = *reinterpret_cast<const float4 *>(bias_s + o);
+          acc[o] = __uint_as_float(v[o]) + bv.x; acc[o + 1] = __uint_as_float(v[o + 1]) + bv.y;
+          acc[o + 2] = __uint_as_float(v[o + 2]) + bv.z; acc[o + 3] = __uint_as_float(v[o + 3]) + bv.w;
+        }
       }
 #pragma unroll 1
       for (int s = 1; s <= km1; ++s) {
-        uint32_t v[32];
-        tmem_ld32(taddr + (uint32_t)(s * CO8), v);
+        uint32_t v[CO8];
+        tmem_ld_cols<CO8>(taddr + (uint32_t)(s * CO8), v);
         tmem_ld_wait();
         if (lane < s) {                          // rows owed to the previous warp
           float *dst = xw + q * xch_q + ((s - 1) * s / 2 + lane) * 32;
@@ -165,7 +177,11 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
-      bar_sync(1 + grp, 128);                    // exchange rows are visible (buffers alternate per block)
+      slot += (uint32_t)p.groups;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+      // the bulk copy that last read this staging buffer (two blocks ago) is done with it
+      if (p.bulk_out && elected) bulk_wait_read1();
+      bar_sync(1 + grp, 128);                    // exchange rows are visible, staging buffer is free
       if (q < 3 && lane + km1 >= 32) {
 #pragma unroll 1
         for (int s = 32 - lane; s <= km1; ++s) {
@@ -179,9 +195,9 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
       }
       const int pos0 = b * p.blk_rows;
       const int pos = pos0 + m;
-      const int yy = pos / p.wbox, xx = pos - yy * p.wbox;
+      const int yy = (int)(((uint32_t)pos * p.wbox_inv) >> 20), xx = pos - yy * p.wbox;
       // first valid pixel of the block (the bulk copy starts there)
-      int fy = pos0 / p.wbox, fx = pos0 - fy * p.wbox;
+      int fy = (int)(((uint32_t)pos0 * p.wbox_inv) >> 20), fx = pos0 - fy * p.wbox;
       if (fx >= p.tw) { ++fy; fx = 0; }
       if ((m < p.blk_rows) && (xx < t.tw_valid) && (yy < t.th)) {
         const size_t pix = ((size_t)t.img * p.ho + (t.y0 + yy)) * p.wo + (t.xt * p.tw + xx);
@@ -219,14 +235,14 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
           // the block's valid pixels are one contiguous range of the output
           int pos1 = pos0 + p.blk_rows - 1;
           if (pos1 > t.rows - 1) pos1 = t.rows - 1;
-          int ly = pos1 / p.wbox, lx = pos1 - ly * p.wbox;
+          int ly = (int)(((uint32_t)pos1 * p.wbox_inv) >> 20), lx = pos1 - ly * p.wbox;
           if (lx >= p.tw) lx = p.tw - 1;
           const int first = fy * p.tw + fx, last = ly * p.tw + lx;
           if (last >= first && fy < t.th) {
             const size_t pix0 = ((size_t)t.img * p.ho + t.y0) * p.wo + first;
             bulk_store(y + pix0 * p.c_out, smem_u32(obuf), (uint32_t)((last - first + 1) * p.c_out * 2));
-            bulk_commit();
           }
+          bulk_commit();                         // one group per block, empty or not: the wait above counts groups
         }
       }
     }
@@ -277,7 +293,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
   __syncthreads();
   const int ntiles = sh.ntiles;
 
-  if (warp < 4) {
+  if (warp < kMmaWarp) {
     // ================================================================== producers
     const int ptid = threadIdx.x;
     const int row_pieces = p.wbox * p.cch;      // 16-byte pieces per patch row; piece q = (col, chunk)
@@ -327,7 +343,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     cp_async_wait_all();                         // nothing of this thread is in flight when the CTA leaves
   } else {
     // ---- consumer preparation
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
       tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
       tmem_relinquish();
     } else {
@@ -342,7 +358,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = sh.tmem_base;
 
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
       // ================================================================== MMA issue
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
       const uint32_t desc_hi = (128u >> 4) | (1u << 14);
@@ -401,7 +417,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     }
     tc_fence_before();
     bar_sync(kBarConsumers, kConsumerThreads);
-    if (warp == 4) {
+    if (warp == kMmaWarp) {
       tc_fence_after();
       tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
     }
@@ -435,7 +451,7 @@ int sm_count() {
   return n;
 }
 
-constexpr int kSmemBudget = 200 * 1024;
+constexpr int kSmemBudget = 220 * 1024;
 
 // plane stride in 16-byte units, chosen so that the chunks of one pixel (written by neighbouring
 // producer threads) fall into different bank groups
@@ -463,6 +479,7 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->slots = 512 / p->n_pad;
   if (p->slots > kMaxSlots) p->slots = kMaxSlots;
   if (p->slots < 2) return false;
+  p->groups = p->slots < kGroups ? p->slots : kGroups;
   int cols = 32;
   while (cols < p->slots * p->n_pad) cols *= 2;
   p->tmem_cols = cols;
@@ -472,6 +489,7 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->nxt = dc_div_up(wo, p->tw);
   p->wbox = p->tw + g->k - 1;
   if (p->wbox * p->cch >= 4096) return false;
+  p->wbox_inv = ((1u << 20) + (uint32_t)p->wbox - 1) / (uint32_t)p->wbox;
   // rows per tile: bounded by the accumulator blocks, the image, shared memory, and a target of
   // about six tiles per CTA so that load, MMA and epilogue overlap
   const long long total_rows = (long long)n * ho * p->nxt;
@@ -500,7 +518,7 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->off_b = 0;
   p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
   p->off_out = p->off_bias + 128;
-  p->off_xch = p->off_out + kGroups * p->out_buf_bytes;
+  p->off_xch = p->off_out + kGroups * 2 * p->out_buf_bytes;
   p->off_a = (int)dc_round_up((size_t)p->off_xch + xch_bytes, 128);
   long long per_cta = total_rows / th / n_sm + 2;
   int stages = kMaxStages;

@@ -222,6 +222,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t *v) {
       : "r"(addr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld8(uint32_t addr, uint32_t *v) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(addr)
+               : "memory");
+}
+// 32 lanes x N consecutive fp32 columns, N in {8, 16, 24, 32}
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t addr, uint32_t *v) {
+  static_assert(N == 8 || N == 16 || N == 24 || N == 32, "column count");
+  if (N == 8) tmem_ld8(addr, v);
+  else if (N == 16) tmem_ld16(addr, v);
+  else if (N == 24) { tmem_ld16(addr, v); tmem_ld8(addr + 16, v + 16); }
+  else tmem_ld32(addr, v);
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory operand descriptors (K-major, no swizzle) are built inline: 14-bit start>>4,
