@@ -40,7 +40,10 @@ static inline int dc_out_extent(int h, int k, int s, int p) {
 // rounded up to 8): one instruction then produces, for every tap column at once, the partial sums
 // Z[m][s][o] = sum_{r,c} x[m + r * pitch][c] * W[o][c][r][s], and the epilogue adds the k column
 // groups with a row shift, y[m][o] = sum_s Z[m + s][s][o].  This cuts the number of tensor-core
-// instructions per output by k, which is what bounds small-channel convolutions.
+// instructions per output by k, which is what bounds small-channel convolutions.  With an odd
+// number of entries the zero padding entry sits in front of the last one (positions e-1 and e), so
+// that the activation side may pair the last entry with entry 0 read a second time -- a chunk that
+// lies at a lower address, as the operand descriptor needs, and that always holds staged data.
 // ----------------------------------------------------------------------------------------------
 struct KOrder {
   int k, stride, pad;
@@ -104,14 +107,20 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
 // entry index within a group -> (pc, ccg, r, s); returns false for the zero padding entry
 __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
                                                         int *r, int *s) {
-  if (e >= ko.e) return false;
   if (ko.fold) {
+    if (ko.e & 1) {
+      if (e == ko.e - 1 || e > ko.e) return false;
+      if (e == ko.e) e = ko.e - 1;
+    } else if (e >= ko.e) {
+      return false;
+    }
     *pc = 0;
     *ccg = e / ko.k;
     *r = e - *ccg * ko.k;
     *s = -1;               // the tap column is part of the row index, not of the entry
     return true;
   }
+  if (e >= ko.e) return false;
   if (ko.pcs == 1) {
     *pc = 0;
     *ccg = e / ko.taps;
@@ -136,7 +145,10 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 // (channel chunk cc in [0,cch), tap r, s) -> position of that chunk in the packed weights,
 // in units of chunk planes (n_pad * 8 elements each)
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
-  if (ko.fold) return cc * ko.k + r;
+  if (ko.fold) {
+    const int e = cc * ko.k + r;
+    return ((ko.e & 1) && e == ko.e - 1) ? e + 1 : e;
+  }
   int grp = cc / ko.cg, ccg = cc - grp * ko.cg;
   int e;
   if (ko.pcs == 1) {

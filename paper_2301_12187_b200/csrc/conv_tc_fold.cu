@@ -21,12 +21,12 @@
 // small dynamic instruction count: the CTA's tiles are decoded once into a table, loops are not
 // unrolled, activation / skip-input variants are compiled separately.  Behind the activation
 // stages the unit is the 128-row block: blocks go round-robin over a ring of accumulator slots in
-// tensor memory, one warp issues the MMAs, four epilogue groups of four warps take the blocks
-// in turn.  The valid outputs of a block are one contiguous range of the NHWC output when tiles
+// tensor memory, four warps issue the MMAs and three epilogue groups of four warps take the
+// blocks, both in turn.  The valid outputs of a block are one contiguous range of the NHWC output when tiles
 // span the image width, so each block leaves with one bulk copy.
 //
-// Roles (640 threads): warps 0-2 producers, warp 3 MMA issue (converged warp, elected lane) and
-// tensor-memory owner, warps 4-19 epilogue (four groups).  Waits are bounded (tc::mbar_wait).
+// Roles (608 threads): warps 0-2 producers, warps 3-6 MMA issue (converged warps, elected lane;
+// warp 3 owns the tensor memory), warps 7-18 epilogue (three groups).  Waits are bounded (tc::mbar_wait).
 #include "tc_ptx.cuh"
 
 namespace {
@@ -36,10 +36,10 @@ constexpr int kMaxStages = 8;
 constexpr int kMaxSlots = 6;
 constexpr int kProducerThreads = 96;
 constexpr int kMmaWarp = kProducerThreads / 32;
-constexpr int kGroups = 4;                       // epilogue groups of 4 warps
-constexpr int kFirstEpiWarp = kMmaWarp + 1;
-static_assert(kFirstEpiWarp % 4 == 0, "epilogue warp w reads tensor-memory lane quadrant w mod 4");
-constexpr int kConsumerThreads = (1 + 4 * kGroups) * 32;
+constexpr int kGroups = 3;                       // epilogue groups of 4 warps
+constexpr int kMmaWarps = 4;
+constexpr int kFirstEpiWarp = kMmaWarp + kMmaWarps;
+constexpr int kConsumerThreads = (kMmaWarps + 4 * kGroups) * 32;
 constexpr int kThreads = kProducerThreads + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barriers: 1..kGroups epilogue groups, 7 all consumers
 static_assert(kGroups < kBarConsumers, "named barrier ids");
@@ -58,7 +58,7 @@ struct FoldParams {
   int stages, slots, groups, act, bulk_out, out_buf_bytes, xch_buf_floats;
   int off_b, off_bias, off_out, off_xch, off_a, smem_bytes;
   int tmem_cols;
-  int npairs, odd;
+  int npairs;
   uint32_t cch_inv;            // ceil(65536 / cch): q / cch == (q * cch_inv) >> 16 for q < 4096
   uint32_t wbox_inv;           // ceil(2^20 / wbox): q / wbox == (q * wbox_inv) >> 20 for q < 4096
   uint32_t a_desc_lo[kMaxPairs];      // per instruction: (first chunk offset >> 4) | (distance >> 4) << 16
@@ -136,8 +136,14 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
     const Tile t = sh.tiles[ti];
 #pragma unroll 1
     for (int b = (int)next - t.c0; b < t.nblk; b += p.groups, next += p.groups) {
-      // the group passes or leaves together, so nobody is left alone at a named barrier
-      if (!bar_all(1 + grp, 128, mbar_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot))) return;
+      // One warp watches the accumulator's barrier, the others park at the group's named barrier
+      // (which costs no issue slots); the group passes or leaves together.
+      bool got = true;
+      if (q == (kFirstEpiWarp & 3)) {
+        got = mbar_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot);
+        tc_fence_before();
+      }
+      if (!bar_all(1 + grp, 128, got)) return;
       tc_fence_after();
       const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
       float *xw = xg + (mine & 1) * p.xch_buf_floats;
@@ -274,7 +280,6 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
   uint8_t *smem_out = smem + p.off_out;
   float *xch = reinterpret_cast<float *>(smem + p.off_xch);
   float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
-  uint8_t *smem_zero = smem_a + (size_t)p.stages * p.a_stage_bytes;   // always-zero plane + slack
 
   const int warp = threadIdx.x >> 5;
   volatile uint32_t *abort_flag = &sh.abort;
@@ -283,7 +288,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
   // first; the consumers (MMA + epilogue warps) finish their own preparation behind a second barrier.
   if (threadIdx.x == 0) {
     sh.abort = 0;
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], kProducerThreads); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], kProducerThreads); mbar_init(&sh.empty[s], kMmaWarps); }
     for (int a = 0; a < p.slots; ++a) { mbar_init(&sh.slot_full[a], 1); mbar_init(&sh.slot_empty[a], 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     prefetch_tensormap(&map_b);
@@ -346,61 +351,59 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     if (warp == kMmaWarp) {
       tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
       tmem_relinquish();
-    } else {
+    } else if (warp >= kFirstEpiWarp) {
       const int t = threadIdx.x - kFirstEpiWarp * 32;
       if (t < 32) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
-      uint4 *z = reinterpret_cast<uint4 *>(smem_zero);
-      for (int i = t; i < (p.mb * 2048 + 1024) / 16; i += 4 * kGroups * 32) z[i] = make_uint4(0u, 0u, 0u, 0u);
-      fence_proxy_async();
     }
     tc_fence_before();
     bar_sync(kBarConsumers, kConsumerThreads);
     tc_fence_after();
     const uint32_t tmem_base = sh.tmem_base;
 
-    if (warp == kMmaWarp) {
+    if (warp < kFirstEpiWarp) {
       // ================================================================== MMA issue
+      // Warp mw takes blocks c = mw mod kMmaWarps.  The warps sit on different schedulers, so the
+      // short issue sequences of several blocks progress side by side although each shares its
+      // scheduler with busy epilogue warps.  The warp stays converged; one elected lane issues.
+      const int mw = warp - kMmaWarp;
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
       const uint32_t desc_hi = (128u >> 4) | (1u << 14);
-      const uint32_t zero_addr = smem_u32(smem_zero);
-      const uint32_t b_base = smem_u32(smem_b);
-      const uint32_t b_lo0 = ((b_base >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
+      const uint32_t b_lo0 = ((smem_u32(smem_b) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
       const uint32_t b_step = 2u * (uint32_t)p.n_pad;
-      const uint32_t last = (uint32_t)(p.npairs - 1);
-      const uint32_t first_off = (p.a_desc_lo[last] & 0x3FFFu) << 4;
+      const uint32_t a_row0 = smem_u32(smem_a) >> 4, a_stage_rows = (uint32_t)p.a_stage_bytes >> 4;
       bool ok = true;
       int s = 0;                                 // stage and its phase, accumulator slot and its phase
-      uint32_t ph = 0, slot = 0, sph = 1;
+      uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+      int next = mw;                             // next block of this warp
 #pragma unroll 1
       for (int it = 0; it < ntiles && ok; ++it) {
-        const Tile t = sh.tiles[it];
+        const int c0 = sh.tiles[it].c0, nblk = sh.tiles[it].nblk;
         if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
         tc_fence_after();
-        const uint32_t a_base = smem_u32(smem_a + (size_t)s * p.a_stage_bytes);
-        // last pair of an odd entry count: its second chunk is the zero plane
-        const uint32_t pad_lo = (first_off >> 4) | (((zero_addr - a_base - first_off) >> 4) << 16);
 #pragma unroll 1
-        for (int b = 0; b < t.nblk; ++b) {
+        for (int b = next - c0; b < nblk; b += kMmaWarps, next += kMmaWarps) {
           if (!warp_wait(&sh.slot_empty[slot], sph, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
-          const uint32_t a_add = (a_base >> 4) + (uint32_t)(b * p.blk_rows);
+          const uint32_t a_add = a_row + (uint32_t)(b * p.blk_rows);
           // statically indexed so that the table entries are read straight from the constant bank
 #pragma unroll
           for (int j = 0; j < kMaxPairs; ++j) {
             if (j < p.npairs) {
-              uint32_t lo = p.a_desc_lo[j];
-              if (p.odd && (uint32_t)j == last) lo = pad_lo;
-              const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
+              const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(p.a_desc_lo[j] + a_add);
               const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
               if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
             }
           }
           if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
-          if (++slot == (uint32_t)p.slots) { slot = 0; sph ^= 1; }
+          slot += kMmaWarps;
+          while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
         }
-        if (ok && elect_one()) umma_commit(&sh.empty[s]);      // the stage may be refilled once these MMAs finish
-        if (++s == p.stages) { s = 0; ph ^= 1; }
+        // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
+        if (ok && elect_one()) umma_commit(&sh.empty[s]);
+        a_row += a_stage_rows;
+        if (++s == p.stages) { s = 0; ph ^= 1; a_row = a_row0; }
       }
     } else {
       switch (p.co8) {
@@ -474,7 +477,6 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->n_pad = ko.n_pad;
   p->blk_rows = 128 - (g->k - 1);
   p->npairs = ko.e_pad / 2;
-  p->odd = ko.e & 1;
   if (p->npairs > kMaxPairs) return false;
   p->slots = 512 / p->n_pad;
   if (p->slots > kMaxSlots) p->slots = kMaxSlots;
@@ -532,11 +534,10 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
     uint32_t off[2] = {0u, 16u};
     for (int q = 0; q < 2; ++q) {
       int pc, ccg, r, s;
-      if (dc_korder_decode(ko, 2 * j + q, &pc, &ccg, &r, &s))
-        off[q] = (uint32_t)(ccg * p->plane_stride + r * p->wbox * 16);
-      else if (q == 1)
-        off[1] = off[0] + 16;
+      // the padding entry reads entry 0 (offset 0) again; its weights are zero
+      off[q] = dc_korder_decode(ko, 2 * j + q, &pc, &ccg, &r, &s) ? (uint32_t)(ccg * p->plane_stride + r * p->wbox * 16) : 0u;
     }
+    if (off[1] <= off[0]) return false;
     p->a_desc_lo[j] = (off[0] >> 4) | (((off[1] - off[0]) >> 4) << 16);
   }
   return true;

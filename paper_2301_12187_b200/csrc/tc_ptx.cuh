@@ -62,7 +62,11 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parit
                                                    DcWsHeader *ws, uint32_t site) {
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
-    if (mbar_try(bar, parity, 20000u)) return true;
+    // a waiting warp shares its scheduler with working ones: the inner loop is probe + branch only,
+    // the abort flag and the clock are looked at once per batch of probes
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
     if (globaltimer_ns() - t0 > kWaitLimitNs) {
       *abort_flag = 1;
