@@ -226,17 +226,14 @@ def run_ours(args):
         return run_network(args)
     import torch
     import torch.distributed as dist
-    from paper_2301_12187_b200 import dc, inputs as I
+    from paper_2301_12187_b200 import dc, inputs as I, replicas as R
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = R.env_rank_world()
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    R.init_group("nccl", world, torch.device("cuda", local))
     dc.lib()
 
-    case = I.chain_case(WORKLOADS[args.workload], seed=rank)
+    case = I.chain_case(WORKLOADS[args.workload], seed=R.replica_seed(0, rank))
     n, h, w, c = case.x_shape
     layers = [dc.DeviceLayer(s) for s in case.layers]
     g, merge_ws_bytes = dc.merge_query(layers, case.residuals)
@@ -357,8 +354,7 @@ def run_ours(args):
         e2e_ms = h0.elapsed_time(h1) / e2e_steps
 
     times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    R.max_over_ranks(times, world)
     ms_total, e2e_ms = float(times[0]), float(times[1])
     clocks = sampler.stop(t_begin, t_end_clk) if rank == 0 else None
     if world > 1:
@@ -376,7 +372,7 @@ def run_ours(args):
         roof = {"bound": "tensor", "achieved": flops / conv_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = PROFILED_TRAFFIC.get(args.workload)
-    roof.update({"kernel": "k_conv_tc", "us_per_launch": conv_us, "peak_source": peak_src,
+    roof.update({"kernel": dc.conv_kernel_name(n, h, w, g, dc.BF16), "us_per_launch": conv_us, "peak_source": peak_src,
                  "algorithmic_bytes": abytes, "flops": flops, "tflops": flops / conv_s / 1e12,
                  "images_per_s_kernel_only": n / conv_s})
 
@@ -384,7 +380,7 @@ def run_ours(args):
     param_bytes = sum(int(s.weight.size) * 4 + 4 * int(s.c_out) * 4 for s in case.layers)
     out = {
         "metric": "merged-conv fwd TFLOP/s & images/s on 1 B200 vs roofline; merge latency us",
-        "value": world * n / (ms_step * 1e-3), "unit": "images/s", "n_gpus": world, "steps": args.steps,
+        "value": R.job_throughput(n, world, ms_step * 1e-3), "unit": "images/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": case.name, "batch_per_gpu": n, "input_nhwc": list(case.x_shape),
@@ -396,7 +392,7 @@ def run_ours(args):
         "gpu_launches": (launches_per_step if launches_per_step > 0 else 10) * args.steps,
         "launches_per_step": launches_per_step,
         "roofline": roof,
-        "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": "images/s",
+        "e2e": {"value": R.job_throughput(n, world, e2e_ms * 1e-3), "unit": "images/s",
                 "h2d_bytes_per_step": int(2 * n * h * w * c + param_bytes),
                 "d2h_bytes_per_step": int(2 * np.prod(yshape)), "ms_per_step": e2e_ms,
                 "api": "dc_chain_forward_host (pinned host buffers)"},
@@ -407,7 +403,8 @@ def run_ours(args):
     print(json.dumps(out))
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of k_conv_tc (profiles/); None until captured
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the conv forward kernel (profiles/);
+# None until captured, and again once the kernel has changed since
 PROFILED_TRAFFIC = {"cfg1": None, "cfg2": None, "cfg3": None}
 
 

@@ -168,6 +168,13 @@ dc_status dc_pack_weights(const float *w, const dc_geom *g, dc_dtype dtype, void
 size_t dc_conv_workspace_bytes(void);
 
 /*
+ * Host only, launches nothing: name of the kernel dc_conv_forward would run for this problem
+ * ("k_conv_tc_fold", "k_conv_tc", "k_conv_dense_bf16", "k_conv_dense_f32"), or NULL when the
+ * geometry is invalid.  For reports (which kernel a timing belongs to); the string is static.
+ */
+const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g, dc_dtype dtype);
+
+/*
  * Forward pass of one dense convolution (the merged layer f_{theta^_i} of Eq. 1, or an
  * unmerged 1x1 / stem / head layer):  y = act(conv(x) + bias + residual).
  * x: [n][h][w][c_in], y: [n][h_out][w_out][c_out], residual: same shape as y or NULL, all of

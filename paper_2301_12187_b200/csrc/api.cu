@@ -21,6 +21,15 @@ extern "C" const char *dc_status_string(dc_status s) {
 
 extern "C" size_t dc_conv_workspace_bytes(void) { return sizeof(DcWsHeader); }
 
+extern "C" const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g, dc_dtype dtype) {
+  if (dc_validate_geom(g) != DC_OK || g->groups != 1 || n <= 0 || h <= 0 || w <= 0) return nullptr;
+  if (dtype == DC_F32) return "k_conv_dense_f32";
+  if (dtype != DC_BF16) return nullptr;
+  if (dc_conv_fold_supported(n, h, w, g)) return "k_conv_tc_fold";
+  if (dc_conv_tc_supported(n, h, w, g)) return "k_conv_tc";
+  return "k_conv_dense_bf16";
+}
+
 extern "C" dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, const dc_geom *g,
                                           const void *w_packed, const float *bias, dc_act act,
                                           const void *residual, void *y, dc_dtype dtype, void *workspace,

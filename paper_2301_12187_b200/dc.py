@@ -63,6 +63,7 @@ EXPORTS = {
     "dc_merge_chain_static_capacity": (C.c_size_t, []),
     "dc_pack_weights": (C.c_int, [C.c_void_p, C.POINTER(Geom), C.c_int, C.c_void_p, C.c_void_p]),
     "dc_conv_workspace_bytes": (C.c_size_t, []),
+    "dc_conv_kernel_name": (C.c_char_p, [C.c_int, C.c_int, C.c_int, C.POINTER(Geom), C.c_int]),
     "dc_conv_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Geom), C.c_void_p,
                                   C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                   C.c_size_t, C.c_void_p]),
@@ -239,6 +240,11 @@ def pack_weights(w, g: Geom, dtype: int, w_packed, stream=None):
 
 def conv_workspace_bytes() -> int:
     return int(lib().dc_conv_workspace_bytes())
+
+
+def conv_kernel_name(n: int, h: int, w: int, g: Geom, dtype: int) -> Optional[str]:
+    r = lib().dc_conv_kernel_name(n, h, w, C.byref(g), dtype)
+    return r.decode() if r else None
 
 
 def conv_forward(x, g: Geom, w_packed, bias, act, residual, y, workspace, stream=None, algo=ALGO_AUTO):
