@@ -12,51 +12,60 @@
 // warp, a small shared-memory exchange across warp boundaries, and the last k-1 rows of each
 // 128-row block are recomputed by the next block (blocks advance by 128-(k-1) positions).
 //
-// Staging is the chunk-plane scheme of conv_tc.cu: the haloed input patch of a tile is loaded
-// once (16-byte cp.async, halo zero-filled) as planes of 8 channels at 16-byte pixel pitch, which
-// is the no-swizzle K-major operand layout, so tap row r is the same plane read r*pitch pixels
-// further on.  Weights arrive once per CTA by a 3-D TMA tile.
+// Staging.  The operand layout is the chunk-plane scheme of conv_tc.cu: per 8-channel chunk a
+// plane of all patch pixels at 16-byte pitch (the no-swizzle K-major layout), so tap row r is the
+// same plane read r*pitch pixels further on.  NHWC rows do not arrive in that layout, and an SM
+// pulls only ~12 bytes per cycle through per-thread 16-byte copies, so the input takes two hops:
+// whole pixel rows of the patch come in by bulk copies (one per row, tracked by an mbarrier) into
+// a raw ring, and the producer warps repack raw rows into chunk planes with 16-byte shared-memory
+// loads and stores, writing zeros for the halo that lies outside the image.  Weights arrive once
+// per CTA by a 3-D TMA tile.
 //
-// The kernel is bound by the number of instructions an SM issues, so every role is written for a
-// small dynamic instruction count: the CTA's tiles are decoded once into a table, loops are not
-// unrolled, activation / skip-input variants are compiled separately.  Behind the activation
-// stages the unit is the 128-row block: blocks go round-robin over a ring of accumulator slots in
-// tensor memory, four warps issue the MMAs and three epilogue groups of four warps take the
-// blocks, both in turn.  The valid outputs of a block are one contiguous range of the NHWC output when tiles
-// span the image width, so each block leaves with one bulk copy.
+// Work split.  Tiles are th output rows of one column strip of one image, on a fixed grid; CTAs
+// (one per SM) take contiguous runs of tiles and every role walks them with a few adds, no table.
+// Behind the activation stages the unit is the 128-row block: blocks go round-robin over a ring of
+// accumulator slots in tensor memory, the MMA warps and the epilogue groups take them in turn.
+// Each epilogue warp stages its 32 rows and sends them off with its own bulk copy (the valid
+// outputs of consecutive GEMM rows are contiguous in NHWC when tiles span the image width).
 //
 // Roles (608 threads): warps 0-2 producers, warps 3-6 MMA issue (converged warps, elected lane;
-// warp 3 owns the tensor memory), warps 7-18 epilogue (three groups).  Waits are bounded (tc::mbar_wait).
+// warp 3 owns the tensor memory), warps 7-18 epilogue (three groups of four).  The kernel is bound
+// by instruction issue and by the latency of the hand-offs between the roles, not by HBM or the
+// tensor pipe, so waits are cheap (tight probe loops, one probing warp per epilogue group, named
+// barriers elsewhere) and the per-block code is short.  All waits are bounded (tc::mbar_wait).
 #include "tc_ptx.cuh"
 
 namespace {
 using namespace tc;
 
-constexpr int kMaxStages = 8;
-constexpr int kMaxSlots = 6;
-constexpr int kProducerThreads = 96;
-constexpr int kMmaWarp = kProducerThreads / 32;
-constexpr int kGroups = 3;                       // epilogue groups of 4 warps
+constexpr int kMaxRaw = 4;                       // raw row buffers (bulk copies in flight)
+constexpr int kMaxStages = 4;                    // chunk-plane stages
+constexpr int kMaxSlots = 6;                     // accumulator slots in tensor memory
+constexpr int kProducerWarps = 3;
+constexpr int kProducerThreads = kProducerWarps * 32;
+constexpr int kMmaWarp = kProducerWarps;         // first MMA warp
 constexpr int kMmaWarps = 4;
 constexpr int kFirstEpiWarp = kMmaWarp + kMmaWarps;
-constexpr int kConsumerThreads = (kMmaWarps + 4 * kGroups) * 32;
+constexpr int kGroups = 3;                       // epilogue groups of 4 warps
+constexpr int kEpiWarps = 4 * kGroups;
+constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
 constexpr int kThreads = kProducerThreads + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barriers: 1..kGroups epilogue groups, 7 all consumers
 static_assert(kGroups < kBarConsumers, "named barrier ids");
-constexpr int kMaxTiles = 96;
-constexpr int kMaxPairs = 16;                   // tensor-core instructions per 128-row block
+constexpr int kMaxPairs = 16;                    // tensor-core instructions per 128-row block
 
 struct FoldParams {
   int n_img, h, w, ho, wo, c_in, c_out, co8;
   int k, pad, cch;
   int tw, th, nxt, wbox;       // tile size in outputs, x tiles per row, patch width (= GEMM row pitch)
+  int tiles_y;                 // tiles per column strip
+  int grid, tiles_per, tiles_rem;   // CTAs; CTA b takes tiles_per (+1 if b < tiles_rem) tiles
   int n_pad;                   // N of the instruction: k column groups of co8 channels, padded
   int blk_rows;                // output positions per 128-row block = 128 - (k-1)
-  int mb;                      // blocks per full tile
-  int total_units;             // output row segments, ordered (img, xt, y)
-  int plane_stride, a_stage_bytes, b_bytes;
-  int stages, slots, groups, act, bulk_out, out_buf_bytes, xch_buf_floats;
-  int off_b, off_bias, off_out, off_xch, off_a, smem_bytes;
+  int mb, mb_last;             // blocks of a full tile / of a strip's last (shorter) tile
+  int plane_stride, a_stage_bytes, b_bytes, raw_bytes;
+  int nraw, stages, slots, groups, act, bulk_out, out_buf_bytes, xch_buf_floats;
+  int off_b, off_bias, off_out, off_xch, off_raw, off_a, smem_bytes;
   int tmem_cols;
   int npairs;
   uint32_t cch_inv;            // ceil(65536 / cch): q / cch == (q * cch_inv) >> 16 for q < 4096
@@ -64,86 +73,100 @@ struct FoldParams {
   uint32_t a_desc_lo[kMaxPairs];      // per instruction: (first chunk offset >> 4) | (distance >> 4) << 16
 };
 
-// A tile = up to p.th output rows of one column strip of one image; c0 = index of its first
-// 128-row block in the CTA's block sequence.
-struct Tile {
-  int img, xt, y0, th, c0, nblk, rows, tw_valid;
-};
-
 struct Shared {
-  uint64_t full[kMaxStages], empty[kMaxStages], slot_full[kMaxSlots], slot_empty[kMaxSlots];
+  uint64_t raw_full[kMaxRaw], raw_empty[kMaxRaw];
+  uint64_t full[kMaxStages], empty[kMaxStages];
+  uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
+  uint64_t weights;
   uint32_t tmem_base;
   uint32_t abort;
-  int ntiles;
-  Tile tiles[kMaxTiles];
 };
 
-// The CTA's contiguous range of output row segments, cut into tiles that never cross an image or
-// column strip.  Written once by one thread; every role then walks the same table.
-__device__ __noinline__ void build_tiles(const FoldParams &p, Shared &sh, int begin, int end) {
-  int y0 = begin % p.ho;
-  const int q = begin / p.ho;
-  int xt = q % p.nxt, img = q / p.nxt;
-  int n = 0, c = 0;
-  for (int cur = begin; cur < end && n < kMaxTiles; ++n) {
-    int th = p.th;
-    if (th > p.ho - y0) th = p.ho - y0;
-    if (th > end - cur) th = end - cur;
-    Tile t;
-    t.img = img; t.xt = xt; t.y0 = y0; t.th = th; t.c0 = c;
-    t.rows = (th - 1) * p.wbox + p.tw;
-    t.nblk = (t.rows + p.blk_rows - 1) / p.blk_rows;
-    t.tw_valid = (p.wo - xt * p.tw < p.tw) ? p.wo - xt * p.tw : p.tw;
-    sh.tiles[n] = t;
-    c += t.nblk;
-    cur += th;
-    y0 += th;
-    if (y0 == p.ho) { y0 = 0; if (++xt == p.nxt) { xt = 0; ++img; } }
+// Position on the tile grid; every role keeps its own and steps it once per tile.
+struct Walk {
+  int img, xt, ty;
+  __device__ __forceinline__ void start(const FoldParams &p, int tile) {
+    const int strip = tile / p.tiles_y;
+    ty = tile - strip * p.tiles_y;
+    img = strip / p.nxt;
+    xt = strip - img * p.nxt;
   }
-  sh.ntiles = n;
-}
+  __device__ __forceinline__ void step(const FoldParams &p) {
+    if (++ty == p.tiles_y) {
+      ty = 0;
+      if (++xt == p.nxt) { xt = 0; ++img; }
+    }
+  }
+  __device__ __forceinline__ int rows_out(const FoldParams &p) const {   // output rows of this tile
+    const int left = p.ho - ty * p.th;
+    return left < p.th ? left : p.th;
+  }
+  __device__ __forceinline__ int nblk(const FoldParams &p) const { return ty == p.tiles_y - 1 ? p.mb_last : p.mb; }
+};
 
-// Epilogue of one group (4 warps = 128 threads, thread = GEMM row): blocks c = grp mod kGroups.
+// Patch of a tile in image coordinates: rows [r_lo, r_hi) and columns [c_lo, c_hi) of the patch lie
+// inside the image; the rest is zero padding.
+struct Patch {
+  int gx0, gy0, rows, r_lo, r_hi, c_lo, c_hi;
+  __device__ __forceinline__ void of(const FoldParams &p, const Walk &t) {
+    gx0 = t.xt * p.tw - p.pad;
+    gy0 = t.ty * p.th - p.pad;
+    rows = t.rows_out(p) + p.k - 1;
+    r_lo = gy0 < 0 ? -gy0 : 0;
+    r_hi = (p.h - gy0 < rows) ? p.h - gy0 : rows;
+    c_lo = gx0 < 0 ? -gx0 : 0;
+    c_hi = (p.w - gx0 < p.wbox) ? p.w - gx0 : p.wbox;
+  }
+};
+
+// Epilogue of one group (4 warps = 128 threads, thread = GEMM row): blocks c = grp mod groups.
 // ACT and RES are compile-time so the per-pixel code carries no runtime switches.  Per block the
-// group meets at two named barriers: after the cross-warp rows are in shared memory, and after the
-// block's pixels are staged for the bulk copy.  Exchange rows and staging buffer alternate between
-// two copies, so a block never waits for the previous block's readers.
+// group meets at two named barriers: when the accumulator is complete (one warp watches the
+// mbarrier) and when the cross-warp rows are in shared memory.  Exchange rows and staging buffers
+// alternate between two copies, so a block never waits for the previous block's readers.
 template <int CO8, int ACT, int RES>
 __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
                                               float *xch, uint8_t *smem_out, const __nv_bfloat16 *residual,
-                                              __nv_bfloat16 *y) {
+                                              __nv_bfloat16 *y, int tile0, int ntiles) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int grp = (warp - kFirstEpiWarp) >> 2;
+  const int ew = warp - kFirstEpiWarp;
+  const int grp = ew >> 2;
   const int q = warp & 3;                        // tensor-memory lane quadrant this warp may read
-  const bool elected = (threadIdx.x == (kFirstEpiWarp + 4 * grp) * 32);
+  const bool watcher = (q == (kFirstEpiWarp & 3));
+  // A waiter may trail its barrier by one phase at most, so a slot must not complete twice before
+  // its group has looked: no more groups than slots take part.
+  if (grp >= p.groups) return;
   const int km1 = p.k - 1;
   const int m = q * 32 + lane;
   const uint32_t tmem_row = sh.tmem_base + ((uint32_t)(q * 32) << 16);
   volatile uint32_t *abort_flag = &sh.abort;
-  uint8_t *obuf0 = smem_out + (size_t)grp * 2 * p.out_buf_bytes;
+  uint8_t *obuf0 = smem_out + (size_t)ew * 2 * p.out_buf_bytes;
   const int xch_q = (km1 * (km1 + 1) / 2) * 32;  // floats per quadrant: rows (s, lane < s), 32 channels each
   float *xg = xch + (size_t)grp * 2 * p.xch_buf_floats;
-  // accumulator slot and its phase for block c = grp, advanced by kGroups per block
+  // accumulator slot and its phase for block c = grp, advanced by the number of groups per block
   uint32_t slot = (uint32_t)grp, sph = 0;
   while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
-  uint32_t next = (uint32_t)grp, mine = 0;       // next block of this group, blocks it has done
-  // A waiter may trail its barrier by one phase at most, so a slot must not complete twice before
-  // its group has looked: no more groups than slots take part.
-  if (grp >= p.groups) return;
-  const int ntiles = sh.ntiles;
+  int next = grp, c0 = 0;                        // next block of this group; first block of the tile
+  uint32_t mine = 0;                             // blocks this group has done
+  Walk t;
+  t.start(p, tile0);
 #pragma unroll 1
   for (int ti = 0; ti < ntiles; ++ti) {
-    const Tile t = sh.tiles[ti];
+    const int nblk = t.nblk(p), th_t = t.rows_out(p);
+    const int tw_valid = (p.wo - t.xt * p.tw < p.tw) ? p.wo - t.xt * p.tw : p.tw;
+    const size_t tile_pix0 = ((size_t)t.img * p.ho + (size_t)(t.ty * p.th)) * p.wo + (size_t)(t.xt * p.tw);
 #pragma unroll 1
-    for (int b = (int)next - t.c0; b < t.nblk; b += p.groups, next += p.groups) {
-      // One warp watches the accumulator's barrier, the others park at the group's named barrier
-      // (which costs no issue slots); the group passes or leaves together.
+    for (int b = next - c0; b < nblk; b += p.groups, next += p.groups) {
       bool got = true;
-      if (q == (kFirstEpiWarp & 3)) {
+      if (watcher) {
         got = mbar_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot);
         tc_fence_before();
       }
-      if (!bar_all(1 + grp, 128, got)) return;
+      // the group passes or leaves together, so nobody is left alone at a named barrier
+      if (!bar_all(1 + grp, 128, got)) {
+        if (lane == 0) bulk_wait_all();
+        return;
+      }
       tc_fence_after();
       const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
       float *xw = xg + (mine & 1) * p.xch_buf_floats;
@@ -185,9 +208,7 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
       if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
       slot += (uint32_t)p.groups;
       while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
-      // the bulk copy that last read this staging buffer (two blocks ago) is done with it
-      if (p.bulk_out && elected) bulk_wait_read1();
-      bar_sync(1 + grp, 128);                    // exchange rows are visible, staging buffer is free
+      bar_sync(1 + grp, 128);                    // exchange rows are visible
       if (q < 3 && lane + km1 >= 32) {
 #pragma unroll 1
         for (int s = 32 - lane; s <= km1; ++s) {
@@ -199,28 +220,40 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
           }
         }
       }
-      const int pos0 = b * p.blk_rows;
-      const int pos = pos0 + m;
+      const int pos = b * p.blk_rows + m;
       const int yy = (int)(((uint32_t)pos * p.wbox_inv) >> 20), xx = pos - yy * p.wbox;
-      // first valid pixel of the block (the bulk copy starts there)
-      int fy = (int)(((uint32_t)pos0 * p.wbox_inv) >> 20), fx = pos0 - fy * p.wbox;
-      if (fx >= p.tw) { ++fy; fx = 0; }
-      if ((m < p.blk_rows) && (xx < t.tw_valid) && (yy < t.th)) {
-        const size_t pix = ((size_t)t.img * p.ho + (t.y0 + yy)) * p.wo + (t.xt * p.tw + xx);
-        uint8_t *sout = obuf + (size_t)((yy - fy) * p.tw + (xx - fx)) * p.c_out * 2;
-        __nv_bfloat16 *gout = y + pix * p.c_out;
+      const bool valid = (m < p.blk_rows) && (xx < tw_valid) && (yy < th_t);
+      const int off = yy * p.wo + xx;            // pixel offset from the tile's first output pixel
+      if (RES && valid) {
+        const __nv_bfloat16 *rp = residual + (tile_pix0 + (size_t)off) * p.c_out;
 #pragma unroll
         for (int ch = 0; ch < CO8; ch += 8) {
           if (ch < p.c_out) {
-            if (RES) {
-              const uint4 rv = *reinterpret_cast<const uint4 *>(residual + pix * p.c_out + ch);
-              const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+            const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
+            const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const float2 rf = __bfloat1622float2(rb[i]);
-                acc[ch + 2 * i] += rf.x; acc[ch + 2 * i + 1] += rf.y;
-              }
+            for (int i = 0; i < 4; ++i) {
+              const float2 rf = __bfloat1622float2(rb[i]);
+              acc[ch + 2 * i] += rf.x; acc[ch + 2 * i + 1] += rf.y;
             }
+          }
+        }
+      }
+      // In lane order the valid rows of a warp are consecutive output pixels (only halo columns
+      // and the tail of the block or tile drop out), so they leave as one contiguous range.
+      const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
+      uint8_t *dst;
+      if (p.bulk_out) {
+        if (lane == 0) bulk_wait_read1();        // the copy that last read this buffer (two blocks ago) is done
+        __syncwarp();
+        dst = obuf + (size_t)__popc(vmask & ((1u << lane) - 1u)) * p.c_out * 2;
+      } else {
+        dst = reinterpret_cast<uint8_t *>(y + (tile_pix0 + (size_t)off) * p.c_out);
+      }
+      if (valid) {
+#pragma unroll
+        for (int ch = 0; ch < CO8; ch += 8) {
+          if (ch < p.c_out) {
             uint4 ov;
             __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
 #pragma unroll
@@ -229,130 +262,178 @@ __device__ __forceinline__ void epilogue_role(const FoldParams &p, Shared &sh, D
               if (ACT) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
               ob[i] = __floats2bfloat162_rn(f0, f1);
             }
-            if (p.bulk_out) *reinterpret_cast<uint4 *>(sout + ch * 2) = ov;
-            else *reinterpret_cast<uint4 *>(gout + ch) = ov;
+            *reinterpret_cast<uint4 *>(dst + ch * 2) = ov;
           }
         }
       }
       if (p.bulk_out) {
         fence_proxy_async();                     // the staged pixels are read by the bulk copy engine
-        bar_sync(1 + grp, 128);
-        if (elected) {
-          // the block's valid pixels are one contiguous range of the output
-          int pos1 = pos0 + p.blk_rows - 1;
-          if (pos1 > t.rows - 1) pos1 = t.rows - 1;
-          int ly = (int)(((uint32_t)pos1 * p.wbox_inv) >> 20), lx = pos1 - ly * p.wbox;
-          if (lx >= p.tw) lx = p.tw - 1;
-          const int first = fy * p.tw + fx, last = ly * p.tw + lx;
-          if (last >= first && fy < t.th) {
-            const size_t pix0 = ((size_t)t.img * p.ho + t.y0) * p.wo + first;
-            bulk_store(y + pix0 * p.c_out, smem_u32(obuf), (uint32_t)((last - first + 1) * p.c_out * 2));
-          }
+        const int first = __ffs(vmask) - 1;
+        const int off_first = __shfl_sync(0xffffffffu, off, first < 0 ? 0 : first);
+        __syncwarp();
+        if (lane == 0) {
+          if (vmask)
+            bulk_store(y + (tile_pix0 + (size_t)off_first) * p.c_out, smem_u32(obuf),
+                       (uint32_t)(__popc(vmask) * p.c_out * 2));
           bulk_commit();                         // one group per block, empty or not: the wait above counts groups
         }
       }
     }
+    c0 += nblk;
+    t.step(p);
   }
-  if (p.bulk_out && elected) bulk_wait_all();
+  if (p.bulk_out && lane == 0) bulk_wait_all();
 }
 
 template <int CO8>
 __device__ __forceinline__ void epilogue_dispatch(const FoldParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
                                                   float *xch, uint8_t *smem_out, const __nv_bfloat16 *residual,
-                                                  __nv_bfloat16 *y) {
+                                                  __nv_bfloat16 *y, int tile0, int ntiles) {
   const int v = (p.act == DC_ACT_RELU6 ? 1 : 0) | (residual ? 2 : 0);
-  if (v == 0) epilogue_role<CO8, 0, 0>(p, sh, ws, bias_s, xch, smem_out, residual, y);
-  else if (v == 1) epilogue_role<CO8, 1, 0>(p, sh, ws, bias_s, xch, smem_out, residual, y);
-  else if (v == 2) epilogue_role<CO8, 0, 1>(p, sh, ws, bias_s, xch, smem_out, residual, y);
-  else epilogue_role<CO8, 1, 1>(p, sh, ws, bias_s, xch, smem_out, residual, y);
+  if (v == 0) epilogue_role<CO8, 0, 0>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles);
+  else if (v == 1) epilogue_role<CO8, 1, 0>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles);
+  else if (v == 2) epilogue_role<CO8, 0, 1>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles);
+  else epilogue_role<CO8, 1, 1>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles);
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ FoldParams p,
                const __nv_bfloat16 *__restrict__ x, const float *__restrict__ bias,
                const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
-  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw_base[];
   __shared__ __align__(8) Shared sh;
 
-  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~uintptr_t(1023));
   uint8_t *smem_b = smem + p.off_b;
   uint8_t *smem_a = smem + p.off_a;
+  uint8_t *smem_in = smem + p.off_raw;
   uint8_t *smem_out = smem + p.off_out;
   float *xch = reinterpret_cast<float *>(smem + p.off_xch);
   float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
 
-  const int warp = threadIdx.x >> 5;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile uint32_t *abort_flag = &sh.abort;
 
-  // ---- set-up.  Producers only need the barriers and the tile table, so they are released
-  // first; the consumers (MMA + epilogue warps) finish their own preparation behind a second barrier.
-  if (threadIdx.x == 0) {
-    sh.abort = 0;
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], kProducerThreads); mbar_init(&sh.empty[s], kMmaWarps); }
-    for (int a = 0; a < p.slots; ++a) { mbar_init(&sh.slot_full[a], 1); mbar_init(&sh.slot_empty[a], 4); }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tensormap(&map_b);
-    build_tiles(p, sh, (int)((long long)p.total_units * blockIdx.x / gridDim.x),
-                (int)((long long)p.total_units * (blockIdx.x + 1) / gridDim.x));
+  // this CTA's run of tiles
+  const int bid = (int)blockIdx.x;
+  const int ntiles = p.tiles_per + (bid < p.tiles_rem ? 1 : 0);
+  const int tile0 = bid * p.tiles_per + (bid < p.tiles_rem ? bid : p.tiles_rem);
+
+  // ---- set-up: the barriers are initialised by different threads side by side
+  {
+    const int t = (int)threadIdx.x;
+    bool did = false;
+    if (t < p.nraw) { mbar_init(&sh.raw_full[t], 1); mbar_init(&sh.raw_empty[t], kProducerWarps); did = true; }
+    else if (t >= 32 && t < 32 + p.stages) { mbar_init(&sh.full[t - 32], kProducerWarps); mbar_init(&sh.empty[t - 32], kMmaWarps); did = true; }
+    else if (t >= 64 && t < 64 + p.slots) { mbar_init(&sh.slot_full[t - 64], 1); mbar_init(&sh.slot_empty[t - 64], 4); did = true; }
+    else if (t == 95) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_b); did = true; }
+    if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  const int ntiles = sh.ntiles;
 
-  if (warp < kMmaWarp) {
+  if (warp < kProducerWarps) {
     // ================================================================== producers
-    const int ptid = threadIdx.x;
-    const int row_pieces = p.wbox * p.cch;      // 16-byte pieces per patch row; piece q = (col, chunk)
+    const int tid = (int)threadIdx.x;
     const int C2 = p.c_in * 2;
-    const uint32_t a_base0 = smem_u32(smem_a);
     const long long row_stride = (long long)p.w * C2;
-    const uint32_t drow_stride = (uint32_t)p.wbox * 16u;
-    int s = 0;
-    uint32_t ph = 0;
-#pragma unroll 1
-    for (int it = 0; it < ntiles; ++it) {
-      const Tile t = sh.tiles[it];
-      const int gx0 = t.xt * p.tw - p.pad;
-      const int gy0 = t.y0 - p.pad;
-      const int rows = t.th + p.k - 1;
-      const int r_lo = gy0 < 0 ? -gy0 : 0;                       // patch rows [r_lo, r_hi) lie inside the image
-      const int r_hi = (p.h - gy0 < rows) ? p.h - gy0 : rows;
-      // pieces of a pixel row are contiguous in memory: piece q sits 16*q bytes after the row start
-      const char *tile_base = reinterpret_cast<const char *>(x) + (size_t)t.img * p.h * row_stride +
-                              ((long long)gy0 * p.w + gx0) * C2;
-      if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
-      if (ptid == 0 && it == 0) {
-        // the weights ride on the first stage's barrier as transaction bytes and stay resident
-        mbar_expect_tx(&sh.full[0], (uint32_t)p.b_bytes);
-        tma_load_3d(smem_b, &map_b, &sh.full[0], 0, 0, 0);
+    const uint32_t raw_base = smem_u32(smem_in), a_base0 = smem_u32(smem_a);
+    const uint32_t raw_pitch = (uint32_t)(p.wbox * C2);
+    const int row_pieces = p.wbox * p.cch;      // 16-byte pieces per patch row; piece q = (col, chunk)
+    const uint32_t drow = (uint32_t)p.wbox * 16u;
+    bool ok = true;
+
+    // Warp 0 also fetches: tile j's in-image pixel rows go to raw buffer j mod nraw, one bulk copy
+    // per row issued by lane (row - r_lo), all reported to the buffer's barrier.
+    Walk wi;
+    wi.start(p, tile0);
+    int ir = 0;
+    uint32_t iph = 0;
+    auto fetch = [&]() {
+      Patch pt;
+      pt.of(p, wi);
+      if (!warp_wait(&sh.raw_empty[ir], iph ^ 1, abort_flag, ws, 0x50000u | ir)) { ok = false; return; }
+      const int nrows = pt.r_hi - pt.r_lo;
+      const uint32_t bytes_row = (uint32_t)((pt.c_hi - pt.c_lo) * C2);
+      if (lane == 0) mbar_arrive_expect_tx(&sh.raw_full[ir], (uint32_t)nrows * bytes_row);
+      __syncwarp();
+      if (lane < nrows) {
+        const int r = pt.r_lo + lane;
+        const char *src = reinterpret_cast<const char *>(x) +
+                          ((long long)wi.img * p.h + (pt.gy0 + r)) * row_stride + (long long)(pt.gx0 + pt.c_lo) * C2;
+        bulk_load(raw_base + (uint32_t)ir * (uint32_t)p.raw_bytes + (uint32_t)r * raw_pitch, src, bytes_row,
+                  &sh.raw_full[ir]);
       }
-      const uint32_t stage = a_base0 + (uint32_t)s * p.a_stage_bytes;
+      wi.step(p);
+      if (++ir == p.nraw) { ir = 0; iph ^= 1; }
+    };
+    if (warp == 0) {
+      if (lane == 0) {
+        mbar_arrive_expect_tx(&sh.weights, (uint32_t)p.b_bytes);
+        tma_load_3d(smem_b, &map_b, &sh.weights, 0, 0, 0);
+      }
+      __syncwarp();
+      for (int j = 0; j < p.nraw - 1 && j < ntiles && ok; ++j) fetch();
+    }
+
+    Walk wp;
+    wp.start(p, tile0);
+    int s = 0, pr = 0;
+    uint32_t ph = 0, pph = 0;
 #pragma unroll 1
-      for (int q = ptid; q < row_pieces; q += kProducerThreads) {
+    for (int it = 0; it < ntiles && ok; ++it) {
+      if (warp == 0 && it + p.nraw - 1 < ntiles) fetch();
+      if (!ok) break;
+      Patch pt;
+      pt.of(p, wp);
+      if (!mbar_wait(&sh.raw_full[pr], pph, abort_flag, ws, 0x60000u | pr)) break;
+      if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
+      const uint32_t stage = a_base0 + (uint32_t)s * (uint32_t)p.a_stage_bytes;
+      const uint32_t raw = raw_base + (uint32_t)pr * (uint32_t)p.raw_bytes;
+      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+      for (int q = tid; q < row_pieces; q += kProducerThreads) {
         const int col = (int)(((uint32_t)q * p.cch_inv) >> 16), cc = q - col * p.cch;
-        const int gx = gx0 + col;
-        const bool cv = (gx >= 0) && (gx < p.w);
+        const bool cv = (col >= pt.c_lo) && (col < pt.c_hi);
         uint32_t dst = stage + (uint32_t)(cc * p.plane_stride + col * 16);
-        const int lo = cv ? r_lo : rows, hi = cv ? r_hi : rows;    // rows [lo, hi) are real pixels
+        const int lo = cv ? pt.r_lo : pt.rows, hi = cv ? pt.r_hi : pt.rows;    // rows [lo, hi) are real pixels
         int r = 0;
 #pragma unroll 1
-        for (; r < lo; ++r, dst += drow_stride) cp_async16(dst, x, 0u);
-        const char *src = tile_base + (long long)q * 16 + (long long)r * row_stride;
-#pragma unroll 2
-        for (; r < hi; ++r, dst += drow_stride, src += row_stride) cp_async16_full(dst, src);
+        for (; r < lo; ++r, dst += drow) sts128(dst, zero);
+        uint32_t src = raw + (uint32_t)((col - pt.c_lo) * C2 + cc * 16) + (uint32_t)r * raw_pitch;
 #pragma unroll 1
-        for (; r < rows; ++r, dst += drow_stride) cp_async16(dst, x, 0u);
+        for (; r + 4 <= hi; r += 4, dst += 4 * drow, src += 4 * raw_pitch) {
+          const uint4 v0 = lds128(src), v1 = lds128(src + raw_pitch), v2 = lds128(src + 2 * raw_pitch),
+                      v3 = lds128(src + 3 * raw_pitch);
+          sts128(dst, v0); sts128(dst + drow, v1); sts128(dst + 2 * drow, v2); sts128(dst + 3 * drow, v3);
+        }
+#pragma unroll 1
+        for (; r < hi; ++r, dst += drow, src += raw_pitch) sts128(dst, lds128(src));
+#pragma unroll 1
+        for (; r < pt.rows; ++r, dst += drow) sts128(dst, zero);
       }
-      cp_async_arrive(&sh.full[s]);              // arrives by itself when this thread's copies have landed
+      fence_proxy_async();                       // the planes are read by the tensor core (async proxy)
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&sh.full[s]); mbar_arrive(&sh.raw_empty[pr]); }
+      wp.step(p);
       if (++s == p.stages) { s = 0; ph ^= 1; }
+      if (++pr == p.nraw) { pr = 0; pph ^= 1; }
     }
-    cp_async_wait_all();                         // nothing of this thread is in flight when the CTA leaves
   } else {
     // ---- consumer preparation
     if (warp == kMmaWarp) {
       tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
       tmem_relinquish();
     } else if (warp >= kFirstEpiWarp) {
-      const int t = threadIdx.x - kFirstEpiWarp * 32;
+      const int t = (int)threadIdx.x - kFirstEpiWarp * 32;
       if (t < 32) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
     }
     tc_fence_before();
@@ -371,14 +452,16 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
       const uint32_t b_lo0 = ((smem_u32(smem_b) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
       const uint32_t b_step = 2u * (uint32_t)p.n_pad;
       const uint32_t a_row0 = smem_u32(smem_a) >> 4, a_stage_rows = (uint32_t)p.a_stage_bytes >> 4;
-      bool ok = true;
+      bool ok = warp_wait(&sh.weights, 0, abort_flag, ws, 0x70000u);
       int s = 0;                                 // stage and its phase, accumulator slot and its phase
       uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
       while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
-      int next = mw;                             // next block of this warp
+      int next = mw, c0 = 0;                     // next block of this warp; first block of the tile
+      Walk t;
+      t.start(p, tile0);
 #pragma unroll 1
       for (int it = 0; it < ntiles && ok; ++it) {
-        const int c0 = sh.tiles[it].c0, nblk = sh.tiles[it].nblk;
+        const int nblk = t.nblk(p);
         if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
         tc_fence_after();
 #pragma unroll 1
@@ -402,15 +485,17 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
         }
         // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
         if (ok && elect_one()) umma_commit(&sh.empty[s]);
+        c0 += nblk;
+        t.step(p);
         a_row += a_stage_rows;
         if (++s == p.stages) { s = 0; ph ^= 1; a_row = a_row0; }
       }
     } else {
       switch (p.co8) {
-        case 8: epilogue_dispatch<8>(p, sh, ws, bias_s, xch, smem_out, residual, y); break;
-        case 16: epilogue_dispatch<16>(p, sh, ws, bias_s, xch, smem_out, residual, y); break;
-        case 24: epilogue_dispatch<24>(p, sh, ws, bias_s, xch, smem_out, residual, y); break;
-        default: epilogue_dispatch<32>(p, sh, ws, bias_s, xch, smem_out, residual, y); break;
+        case 8: epilogue_dispatch<8>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles); break;
+        case 16: epilogue_dispatch<16>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles); break;
+        case 24: epilogue_dispatch<24>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles); break;
+        default: epilogue_dispatch<32>(p, sh, ws, bias_s, xch, smem_out, residual, y, tile0, ntiles); break;
       }
     }
     // ---- consumer teardown
@@ -455,6 +540,7 @@ int sm_count() {
 }
 
 constexpr int kSmemBudget = 220 * 1024;
+constexpr int kStageLimit = 40 * 1024;
 
 // plane stride in 16-byte units, chosen so that the chunks of one pixel (written by neighbouring
 // producer threads) fall into different bank groups
@@ -492,43 +578,77 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->wbox = p->tw + g->k - 1;
   if (p->wbox * p->cch >= 4096) return false;
   p->wbox_inv = ((1u << 20) + (uint32_t)p->wbox - 1) / (uint32_t)p->wbox;
-  // rows per tile: bounded by the accumulator blocks, the image, shared memory, and a target of
-  // about six tiles per CTA so that load, MMA and epilogue overlap
-  const long long total_rows = (long long)n * ho * p->nxt;
-  if (total_rows >= (1ll << 31)) return false;
-  int th_target = (int)(total_rows / ((long long)n_sm * 6));
-  if (th_target < 1) th_target = 1;
-  int th = th_target;
-  if (th > ho) th = ho;
-  if (th > 16) th = 16;
-  while (th > 1 && (long long)p->cch * ((th + g->k - 1) * p->wbox + 8) * 16 > 40 * 1024) --th;
-  p->th = th;
-  const int rbox = th + g->k - 1;
-  p->mb = dc_div_up((th - 1) * p->wbox + p->tw, p->blk_rows);
-  p->plane_stride = padded_plane_units(rbox * p->wbox + 1, p->cch) * 16;
-  p->a_stage_bytes = (int)dc_round_up((size_t)p->cch * p->plane_stride, 128);
+  const long long strips = (long long)n * p->nxt;
+  if (strips * ho >= (1ll << 30)) return false;
+  const int C2 = g->c_in * 2;
+  // fixed part of shared memory: weights, bias, per-warp output staging, exchange rows
   p->b_bytes = ko.e_pad * p->n_pad * 16;
-  p->total_units = (int)total_rows;
-  // tiles of one CTA: its rows in chunks of th, plus one cut per image / column-strip boundary
-  if (total_rows / n_sm / th + total_rows / n_sm / ho + 4 > kMaxTiles) return false;
-  p->out_buf_bytes = (int)dc_round_up((size_t)p->blk_rows * g->c_out * 2, 128);
+  p->out_buf_bytes = (int)dc_round_up((size_t)32 * g->c_out * 2, 128);
   p->bulk_out = (p->tw == wo) ? 1 : 0;
   const int km1 = g->k - 1;
   p->xch_buf_floats = 4 * (km1 * (km1 + 1) / 2) * 32;
   const int xch_bytes = kGroups * 2 * p->xch_buf_floats * 4;
-  const int slack = p->mb * 2048 + 1024;
+  const int slack = 4096;      // a block's 128 GEMM rows may reach past the last plane; those rows are dropped
   p->off_b = 0;
   p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
   p->off_out = p->off_bias + 128;
-  p->off_xch = p->off_out + kGroups * 2 * p->out_buf_bytes;
-  p->off_a = (int)dc_round_up((size_t)p->off_xch + xch_bytes, 128);
-  long long per_cta = total_rows / th / n_sm + 2;
-  int stages = kMaxStages;
-  if (stages > per_cta) stages = (int)per_cta;
-  while (stages >= 2 && 1024ll + p->off_a + (long long)stages * p->a_stage_bytes + slack > kSmemBudget) --stages;
-  if (stages < 2) return false;
+  p->off_xch = p->off_out + kEpiWarps * 2 * p->out_buf_bytes;
+  p->off_raw = (int)dc_round_up((size_t)p->off_xch + xch_bytes, 128);
+  auto ring_bytes = [&](int th_c, int r, int s) {
+    const int rb = th_c + g->k - 1;
+    const long long stage = (long long)dc_round_up((size_t)p->cch * padded_plane_units(rb * p->wbox + 1, p->cch) * 16, 128);
+    const long long raw = (long long)dc_round_up((size_t)rb * p->wbox * C2, 128);
+    return 1024ll + p->off_raw + r * raw + s * stage + slack;
+  };
+  // Rows per tile.  A CTA's time is roughly (tiles it gets) x (blocks per tile + a fixed cost per
+  // tile + the patch rows it stages); the CTA with the most tiles sets the kernel's time, so the
+  // candidates are ranked by that product.  Bounds: patch rows fit a warp's lanes (one bulk copy
+  // per row and lane) and a stage fits its share of shared memory.
+  int th = 0;
+  double best = 0.0;
+  for (int cand = 1; cand <= 16 && cand <= ho; ++cand) {
+    const int rbox = cand + g->k - 1;
+    if (rbox > 32) break;
+    if ((long long)p->cch * (rbox * p->wbox + 8) * 16 > kStageLimit) break;
+    if (ring_bytes(cand, 2, 2) > kSmemBudget) break;
+    const long long tiles = strips * dc_div_up(ho, cand);
+    const long long per_max = (tiles + n_sm - 1) / n_sm;
+    const int mb = dc_div_up((cand - 1) * p->wbox + p->tw, p->blk_rows);
+    double cost = (double)per_max * (mb + 0.3 + 0.05 * rbox);
+    if (per_max < 3 && tiles >= 3ll * n_sm) cost *= 1.5;       // too few tiles to overlap the roles
+    if (th == 0 || cost < best) { th = cand; best = cost; }
+  }
+  if (th == 0) return false;
+  p->th = th;
+  p->tiles_y = dc_div_up(ho, th);
+  const long long total_tiles = strips * p->tiles_y;
+  const int grid = total_tiles < n_sm ? (int)total_tiles : n_sm;
+  p->grid = grid;
+  p->tiles_per = (int)(total_tiles / grid);
+  p->tiles_rem = (int)(total_tiles % grid);
+  const int rbox = th + g->k - 1;
+  p->mb = dc_div_up((th - 1) * p->wbox + p->tw, p->blk_rows);
+  const int th_last = ho - (p->tiles_y - 1) * th;
+  p->mb_last = dc_div_up((th_last - 1) * p->wbox + p->tw, p->blk_rows);
+  p->plane_stride = padded_plane_units(rbox * p->wbox + 1, p->cch) * 16;
+  p->a_stage_bytes = (int)dc_round_up((size_t)p->cch * p->plane_stride, 128);
+  p->raw_bytes = (int)dc_round_up((size_t)rbox * p->wbox * C2, 128);
+  // rings: as deep as the CTA's tile count and shared memory allow, the raw ring first
+  const long long per_cta = p->tiles_per + (p->tiles_rem ? 1 : 0);
+  int nraw = kMaxRaw < per_cta ? kMaxRaw : (int)per_cta, stages = kMaxStages < per_cta ? kMaxStages : (int)per_cta;
+  if (nraw < 2) nraw = 2;
+  if (stages < 2) stages = 2;
+  auto total = [&](int r, int s) { return ring_bytes(th, r, s); };
+  while (total(nraw, stages) > kSmemBudget && (nraw > 2 || stages > 2)) {
+    if (stages >= nraw && stages > 2) --stages;
+    else if (nraw > 2) --nraw;
+    else --stages;
+  }
+  if (total(nraw, stages) > kSmemBudget) return false;
+  p->nraw = nraw;
   p->stages = stages;
-  p->smem_bytes = 1024 + p->off_a + stages * p->a_stage_bytes + slack;
+  p->off_a = p->off_raw + nraw * p->raw_bytes;
+  p->smem_bytes = (int)total(nraw, stages);
   // chunk-pair table: entry e = (chunk cc, tap row r) -> byte offset of its 16-byte column in a stage
   for (int j = 0; j < p->npairs; ++j) {
     uint32_t off[2] = {0u, 16u};
@@ -576,8 +696,7 @@ dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom 
     DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_fold, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     attr_set = true;
   }
-  int grid = p.total_units < n_sm ? p.total_units : n_sm;
-  k_conv_tc_fold<<<grid, kThreads, p.smem_bytes, stream>>>(map_b, p, (const __nv_bfloat16 *)x, bias,
+  k_conv_tc_fold<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_b, p, (const __nv_bfloat16 *)x, bias,
                                                           (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                                           (DcWsHeader *)workspace);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
