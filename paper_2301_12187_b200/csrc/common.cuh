@@ -44,6 +44,14 @@ static inline int dc_out_extent(int h, int k, int s, int p) {
 // number of entries the zero padding entry sits in front of the last one (positions e-1 and e), so
 // that the activation side may pair the last entry with entry 0 read a second time -- a chunk that
 // lies at a lower address, as the operand descriptor needs, and that always holds staged data.
+//
+// "Pair" order (stride 1, k >= 3, few channels, cheap enough): a GEMM row is a PAIR of neighbouring
+// output pixels (2j, 2j+1) and the operand has 2 * co8 rows n = e * co8 + o, e = which pixel of the
+// pair.  The pair reads input columns 2j + dx, dx = 0..k, so the planes are split by column parity
+// as for stride 2 and an entry is (parity, chunk, tap row r, dx >> 1); the weight of entry dx for
+// pixel e is W[o][c][r][dx - e] (zero where dx - e is no tap).  This costs (k+1)/2k more tensor-core
+// work than plain order per output -- far less than it saves in instructions: half as many
+// accumulator rows, and no reduction in the epilogue as fold order needs.
 // ----------------------------------------------------------------------------------------------
 struct KOrder {
   int k, stride, pad;
@@ -57,6 +65,7 @@ struct KOrder {
   int e_pad;          // e rounded up to even
   int n_pad;          // operand rows rounded up to 16 (output channels, or k * co8 in fold order)
   int fold;           // 1: fold order
+  int pair;           // 1: pair order
   int co8;            // output channels rounded up to 8
 };
 
@@ -68,9 +77,27 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->n_pad = (int)dc_round_up((size_t)g->c_out, 16);
   ko->co8 = (int)dc_round_up((size_t)g->c_out, 8);
   ko->fold = 0;
+  ko->pair = 0;
   ko->pcs = (g->stride == 2) ? 2 : 1;
   if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch <= 8 && ko->co8 <= 32 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
+    // pair order when its tensor-core cost stays small: instructions of ~48 cycles (N <= 64) per
+    // 256 outputs; beyond ~5 cycles per output fold order (one instruction row per tap row) wins
+    {
+      const int e = ko->cch * g->k * (g->k + 1);
+      const int n_pad = (int)dc_round_up((size_t)(2 * ko->co8), 16);
+      if (((e + 1) / 2) * 48 <= 5 * 256 && (size_t)((e + 1) & ~1) * n_pad * 16 <= 96 * 1024) {
+        ko->pair = 1;
+        ko->pcs = 2;
+        ko->n_pad = n_pad;
+        ko->ns[0] = ko->ns[1] = (g->k + 1) / 2;   // dx values of each parity
+        ko->s0[0] = 0; ko->s0[1] = 1;
+        ko->cg = ko->cch; ko->ng = 1;
+        ko->e = e;
+        ko->e_pad = (e + 1) & ~1;
+        return;
+      }
+    }
     const int n_pad = (int)dc_round_up((size_t)(g->k * ko->co8), 16);
     if ((size_t)ko->cch * g->k * n_pad * 16 <= 64 * 1024) {
       ko->fold = 1;
@@ -107,6 +134,23 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
 // entry index within a group -> (pc, ccg, r, s); returns false for the zero padding entry
 __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
                                                         int *r, int *s) {
+  if (ko.pair) {
+    // (parity, chunk, tap row, dx >> 1); *s returns dx.  Odd counts are padded as in fold order.
+    if (ko.e & 1) {
+      if (e == ko.e - 1 || e > ko.e) return false;
+      if (e == ko.e) e = ko.e - 1;
+    } else if (e >= ko.e) {
+      return false;
+    }
+    const int nd = ko.ns[0];
+    const int dxh = e % nd, t = e / nd;
+    *r = t % ko.k;
+    const int pl = t / ko.k;
+    *pc = pl / ko.cch;
+    *ccg = pl - *pc * ko.cch;
+    *s = 2 * dxh + *pc;
+    return true;
+  }
   if (ko.fold) {
     if (ko.e & 1) {
       if (e == ko.e - 1 || e > ko.e) return false;
@@ -145,6 +189,11 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 // (channel chunk cc in [0,cch), tap r, s) -> position of that chunk in the packed weights,
 // in units of chunk planes (n_pad * 8 elements each)
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
+  if (ko.pair) {               // the copy for the first pixel of the pair: dx = s
+    const int pc = s & 1;
+    const int e = (((pc * ko.cch + cc) * ko.k + r) * ko.ns[0]) + (s >> 1);
+    return ((ko.e & 1) && e == ko.e - 1) ? e + 1 : e;
+  }
   if (ko.fold) {
     const int e = cc * ko.k + r;
     return ((ko.e & 1) && e == ko.e - 1) ? e + 1 : e;
@@ -164,7 +213,7 @@ __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc,
 
 // row of output channel o (and tap column s) inside a chunk plane of the packed weights
 __host__ __device__ static inline int dc_korder_row(const KOrder &ko, int s, int o) {
-  return ko.fold ? s * ko.co8 + o : o;
+  return ko.fold ? s * ko.co8 + o : o;   // pair order: the first pixel's rows are 0..co8-1
 }
 
 __device__ __forceinline__ float dc_act_apply(float v, int act) {
@@ -186,6 +235,10 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
                             const float *bias, dc_act act, const void *residual, void *y,
                             void *workspace, cudaStream_t stream);
 bool dc_conv_tc_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_launch_conv_pair(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y,
+                              void *workspace, cudaStream_t stream);
+bool dc_conv_pair_supported(int n, int h, int w, const dc_geom *g);
 dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                               const float *bias, dc_act act, const void *residual, void *y,
                               void *workspace, cudaStream_t stream);

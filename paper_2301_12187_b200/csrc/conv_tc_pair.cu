@@ -1,0 +1,653 @@
+// Dense stride-1 convolution with few channels as an implicit GEMM whose rows are PAIRS of
+// neighbouring output pixels (see KOrder, "pair" order).
+//
+// With 24..32 channels one tcgen05.mma of shape 128 x N x 16 costs ~48 cycles for any N <= 64 (it
+// is bound by fetching the 128 x 16 activation operand from shared memory), and one SM sees only a
+// few thousand output pixels of a layer, so what limits such a convolution is neither HBM nor the
+// tensor pipe but the number of accumulator rows that have to be walked through issue, tensor
+// memory, epilogue and store.  A GEMM row here produces two output pixels (2j, 2j+1):
+//     D[j][e][o] = sum_{dx = 0..k} sum_{r,c} x[2j + dx + r*pitch][c] * W[o][c][r][dx - e],  e = 0, 1
+// i.e. N = 2 * c_out and the reduction runs over k+1 input columns; input planes are split by
+// column parity (as for stride 2), so that "column 2j + dx of every pair j" is again one plane read
+// from a shifted start.  Per output this needs (k+1)/2k of the instructions of tap-by-tap issue and
+// half the accumulator rows, and the epilogue is a plain read-out: each thread owns 2 pixels x c_out
+// channels = one contiguous piece of the NHWC output, no reduction across lanes.
+//
+// Staging.  Chunk planes as in conv_tc.cu: per (column parity, 8-channel chunk) a plane of patch
+// pixels at 16-byte pitch (the no-swizzle K-major layout), tap row r = the same plane read r*pitch
+// further on.  NHWC rows do not arrive in that layout, and an SM pulls only ~12 bytes per cycle
+// through per-thread 16-byte copies, so the input takes two hops: whole pixel rows of the patch
+// come in by bulk copies (one per row, tracked by an mbarrier) into a raw ring, and the producer
+// warps repack raw rows into the planes with 16-byte shared-memory loads and stores, writing zeros
+// for the halo outside the image.  Weights arrive once per CTA by a 3-D TMA tile.
+//
+// Work split.  Tiles are th output rows of one column strip of one image, on a fixed grid; CTAs
+// (one per SM) take contiguous runs of tiles and every role walks them with a few adds, no table.
+// Behind the activation stages the unit is the 128-row block (256 outputs): blocks go round-robin
+// over a ring of accumulator slots in tensor memory; the MMA warps take them in turn, and so do
+// the epilogue warps, each on its own (one tensor-memory lane quadrant of every third block), with
+// its own staging buffer and bulk store.
+//
+// Roles (608 threads): warps 0-2 producers, warps 3-6 MMA issue (converged warps, elected lane;
+// warp 3 owns the tensor memory), warps 7-18 epilogue.  All waits are bounded (tc::mbar_wait).
+#include "tc_ptx.cuh"
+
+namespace {
+using namespace tc;
+
+constexpr int kMaxRaw = 4;                       // raw row buffers (bulk copies in flight)
+constexpr int kMaxStages = 4;                    // chunk-plane stages
+constexpr int kMaxSlots = 6;                     // accumulator slots in tensor memory
+constexpr int kProducerWarps = 3;
+constexpr int kProducerThreads = kProducerWarps * 32;
+constexpr int kMmaWarp = kProducerWarps;         // first MMA warp
+constexpr int kMmaWarps = 4;
+constexpr int kFirstEpiWarp = kMmaWarp + kMmaWarps;
+constexpr int kGroups = 3;                       // epilogue warps per tensor-memory lane quadrant
+constexpr int kEpiWarps = 4 * kGroups;
+constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
+constexpr int kThreads = kProducerThreads + kConsumerThreads;
+constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
+constexpr int kMaxPairs = 32;                    // tensor-core instructions per block
+
+struct PairParams {
+  int n_img, h, w, ho, wo, c_in, c_out, co8;
+  int k, pad, cch;
+  int tw, th, nxt;             // tile size in outputs, x tiles per row
+  int tw2, wbox2, wboxp;       // output pairs per tile row, plane row pitch in pairs, patch width in pixels
+  int tiles_y;                 // tiles per column strip
+  int grid, tiles_per, tiles_rem;   // CTAs; CTA b takes tiles_per (+1 if b < tiles_rem) tiles
+  int n_pad;                   // N of the instruction: 2 * co8, padded to 16
+  int mb, mb_last;             // blocks of a full tile / of a strip's last (shorter) tile
+  int plane_stride, a_stage_bytes, b_bytes, raw_bytes;
+  int nraw, stages, slots, groups, act, bulk_out, out_buf_bytes;
+  int off_b, off_bias, off_out, off_raw, off_a, smem_bytes;
+  int tmem_cols;
+  int npairs;
+  uint32_t cch_inv;            // ceil(65536 / cch): q / cch == (q * cch_inv) >> 16 for q < 4096
+  uint32_t wbox2_inv;          // ceil(2^20 / wbox2): q / wbox2 == (q * wbox2_inv) >> 20 for q < 4096
+  uint32_t a_desc_lo[kMaxPairs];      // per instruction: (first chunk offset >> 4) | (distance >> 4) << 16
+};
+
+struct Shared {
+  uint64_t raw_full[kMaxRaw], raw_empty[kMaxRaw];
+  uint64_t full[kMaxStages], empty[kMaxStages];
+  uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
+  uint64_t weights;
+  uint32_t tmem_base;
+  uint32_t abort;
+};
+
+// Position on the tile grid; every role keeps its own and steps it once per tile.
+struct Walk {
+  int img, xt, ty;
+  __device__ __forceinline__ void start(const PairParams &p, int tile) {
+    const int strip = tile / p.tiles_y;
+    ty = tile - strip * p.tiles_y;
+    img = strip / p.nxt;
+    xt = strip - img * p.nxt;
+  }
+  __device__ __forceinline__ void step(const PairParams &p) {
+    if (++ty == p.tiles_y) {
+      ty = 0;
+      if (++xt == p.nxt) { xt = 0; ++img; }
+    }
+  }
+  __device__ __forceinline__ int rows_out(const PairParams &p) const {   // output rows of this tile
+    const int left = p.ho - ty * p.th;
+    return left < p.th ? left : p.th;
+  }
+  __device__ __forceinline__ int nblk(const PairParams &p) const { return ty == p.tiles_y - 1 ? p.mb_last : p.mb; }
+};
+
+// Patch of a tile in image coordinates: rows [r_lo, r_hi) and columns [c_lo, c_hi) of the patch lie
+// inside the image; the rest is zero padding.
+struct Patch {
+  int gx0, gy0, rows, r_lo, r_hi, c_lo, c_hi;
+  __device__ __forceinline__ void of(const PairParams &p, const Walk &t) {
+    gx0 = t.xt * p.tw - p.pad;
+    gy0 = t.ty * p.th - p.pad;
+    rows = t.rows_out(p) + p.k - 1;
+    r_lo = gy0 < 0 ? -gy0 : 0;
+    r_hi = (p.h - gy0 < rows) ? p.h - gy0 : rows;
+    c_lo = gx0 < 0 ? -gx0 : 0;
+    c_hi = (p.w - gx0 < p.wboxp) ? p.w - gx0 : p.wboxp;
+  }
+};
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Epilogue of one warp: tensor-memory lane quadrant q of every block c = grp mod groups, where grp
+// counts the warps of the same quadrant.  Nothing is shared with other warps: the thread of GEMM
+// row m owns output pixels (2j, 2j+1) of pair m, adds bias and skip input, applies the activation,
+// converts to bf16 and stages them; the warp's valid pixels are consecutive in the NHWC output (only
+// halo pairs and the tail of the block or tile drop out), so they leave as one bulk copy.
+// ACT and RES are compile-time so the per-pixel code carries no runtime switches.
+template <int CO8, int ACT, int RES>
+__device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+                                              uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
+                                              int tile0, int ntiles) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ew = warp - kFirstEpiWarp;
+  const int grp = ew >> 2;
+  const int q = warp & 3;                        // tensor-memory lane quadrant this warp may read
+  // A waiter may trail its barrier by one phase at most, so a slot must not complete twice before
+  // its warp has looked: no more warps per quadrant than slots take part.
+  if (grp >= p.groups) return;
+  const int m = q * 32 + lane;
+  const uint32_t tmem_row = sh.tmem_base + ((uint32_t)(q * 32) << 16);
+  volatile uint32_t *abort_flag = &sh.abort;
+  uint8_t *obuf0 = smem_out + (size_t)ew * 2 * p.out_buf_bytes;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t slot = (uint32_t)grp, sph = 0;        // accumulator slot and its phase for block c = grp
+  while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+  int next = grp, c0 = 0;                        // next block of this warp; first block of the tile
+  uint32_t mine = 0;                             // blocks this warp has done
+  Walk t;
+  t.start(p, tile0);
+#pragma unroll 1
+  for (int ti = 0; ti < ntiles; ++ti) {
+    const int nblk = t.nblk(p), th_t = t.rows_out(p);
+    const int tw_valid = (p.wo - t.xt * p.tw < p.tw) ? p.wo - t.xt * p.tw : p.tw;
+    const size_t tile_pix0 = ((size_t)t.img * p.ho + (size_t)(t.ty * p.th)) * p.wo + (size_t)(t.xt * p.tw);
+#pragma unroll 1
+    for (int b = next - c0; b < nblk; b += p.groups, next += p.groups) {
+      if (!warp_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot)) {
+        if (lane == 0) bulk_wait_all();
+        return;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
+      uint32_t v0[CO8], v1[CO8];
+      tmem_ld_cols<CO8>(taddr, v0);
+      tmem_ld_cols<CO8>(taddr + (uint32_t)CO8, v1);
+      tmem_ld_wait();
+      // the accumulator slot is free again: one arrival per warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
+      slot += (uint32_t)p.groups;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+      uint8_t *obuf = obuf0 + (mine & 1) * p.out_buf_bytes;
+      ++mine;
+
+      const int pos = b * 128 + m;
+      const int yy = (int)(((uint32_t)pos * p.wbox2_inv) >> 20), jj = pos - yy * p.wbox2;
+      const int xx = 2 * jj;
+      const bool valid0 = (xx < tw_valid) && (yy < th_t);
+      const bool valid1 = valid0 && (xx + 1 < tw_valid);
+      const int off = yy * p.wo + xx;            // pixel offset from the tile's first output pixel
+      const uint32_t m0 = __ballot_sync(0xffffffffu, valid0), m1 = __ballot_sync(0xffffffffu, valid1);
+      uint8_t *dst;
+      if (p.bulk_out) {
+        if (lane == 0) bulk_wait_read1();        // the copy that last read this buffer (two blocks ago) is done
+        __syncwarp();
+        dst = obuf + (size_t)(__popc(m0 & lt) + __popc(m1 & lt)) * p.c_out * 2;
+      } else {
+        dst = reinterpret_cast<uint8_t *>(y + (tile_pix0 + (size_t)off) * p.c_out);
+      }
+      const __nv_bfloat16 *rp = RES ? residual + (tile_pix0 + (size_t)off) * p.c_out : nullptr;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint32_t *v = e ? v1 : v0;
+        if (e ? valid1 : valid0) {
+#pragma unroll
+          for (int ch = 0; ch < CO8; ch += 8) {
+            if (ch < p.c_out) {
+              float f[8];
+              const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
+              const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
+              f[0] = __uint_as_float(v[ch]) + b0.x; f[1] = __uint_as_float(v[ch + 1]) + b0.y;
+              f[2] = __uint_as_float(v[ch + 2]) + b0.z; f[3] = __uint_as_float(v[ch + 3]) + b0.w;
+              f[4] = __uint_as_float(v[ch + 4]) + b1.x; f[5] = __uint_as_float(v[ch + 5]) + b1.y;
+              f[6] = __uint_as_float(v[ch + 6]) + b1.z; f[7] = __uint_as_float(v[ch + 7]) + b1.w;
+              if (RES) {
+                const uint4 rv = *reinterpret_cast<const uint4 *>(rp + e * p.c_out + ch);
+                const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float2 rf = __bfloat1622float2(rb[i]);
+                  f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                }
+              }
+              uint4 ov;
+              __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float f0 = f[2 * i], f1 = f[2 * i + 1];
+                if (ACT) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
+                ob[i] = __floats2bfloat162_rn(f0, f1);
+              }
+              *reinterpret_cast<uint4 *>(dst + (e * p.c_out + ch) * 2) = ov;
+            }
+          }
+        }
+      }
+      if (p.bulk_out) {
+        fence_proxy_async();                     // the staged pixels are read by the bulk copy engine
+        const int first = __ffs(m0) - 1;
+        const int off_first = __shfl_sync(0xffffffffu, off, first < 0 ? 0 : first);
+        __syncwarp();
+        if (lane == 0) {
+          if (m0)
+            bulk_store(y + (tile_pix0 + (size_t)off_first) * p.c_out, smem_u32(obuf),
+                       (uint32_t)((__popc(m0) + __popc(m1)) * p.c_out * 2));
+          bulk_commit();                         // one group per block, empty or not: the wait above counts groups
+        }
+      }
+    }
+    c0 += nblk;
+    t.step(p);
+  }
+  if (p.bulk_out && lane == 0) bulk_wait_all();
+}
+
+template <int CO8>
+__device__ __forceinline__ void epilogue_dispatch(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+                                                  uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
+                                                  int tile0, int ntiles) {
+  const int v = (p.act == DC_ACT_RELU6 ? 1 : 0) | (residual ? 2 : 0);
+  if (v == 0) epilogue_role<CO8, 0, 0>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  else if (v == 1) epilogue_role<CO8, 1, 0>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  else if (v == 2) epilogue_role<CO8, 0, 1>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  else epilogue_role<CO8, 1, 1>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_conv_tc_pair(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ PairParams p,
+               const __nv_bfloat16 *__restrict__ x, const float *__restrict__ bias,
+               const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
+  extern __shared__ __align__(1024) uint8_t smem_raw_base[];
+  __shared__ __align__(8) Shared sh;
+
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~uintptr_t(1023));
+  uint8_t *smem_b = smem + p.off_b;
+  uint8_t *smem_a = smem + p.off_a;
+  uint8_t *smem_in = smem + p.off_raw;
+  uint8_t *smem_out = smem + p.off_out;
+  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile uint32_t *abort_flag = &sh.abort;
+
+  // this CTA's run of tiles
+  const int bid = (int)blockIdx.x;
+  const int ntiles = p.tiles_per + (bid < p.tiles_rem ? 1 : 0);
+  const int tile0 = bid * p.tiles_per + (bid < p.tiles_rem ? bid : p.tiles_rem);
+
+  // ---- set-up: the barriers are initialised by different threads side by side
+  {
+    const int t = (int)threadIdx.x;
+    bool did = false;
+    if (t < p.nraw) { mbar_init(&sh.raw_full[t], 1); mbar_init(&sh.raw_empty[t], kProducerWarps); did = true; }
+    else if (t >= 32 && t < 32 + p.stages) { mbar_init(&sh.full[t - 32], kProducerWarps); mbar_init(&sh.empty[t - 32], kMmaWarps); did = true; }
+    else if (t >= 64 && t < 64 + p.slots) { mbar_init(&sh.slot_full[t - 64], 1); mbar_init(&sh.slot_empty[t - 64], 4); did = true; }
+    else if (t == 95) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_b); did = true; }
+    if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp < kProducerWarps) {
+    // ================================================================== producers
+    const int tid = (int)threadIdx.x;
+    const int C2 = p.c_in * 2;
+    const long long row_stride = (long long)p.w * C2;
+    const uint32_t raw_base = smem_u32(smem_in), a_base0 = smem_u32(smem_a);
+    const uint32_t raw_pitch = (uint32_t)(p.wboxp * C2);
+    const int row_pieces = p.wboxp * p.cch;     // 16-byte pieces per patch row; piece q = (col, chunk)
+    const uint32_t drow = (uint32_t)p.wbox2 * 16u;
+    bool ok = true;
+
+    // Warp 0 also fetches: tile j's in-image pixel rows go to raw buffer j mod nraw, one bulk copy
+    // per row issued by lane (row - r_lo), all reported to the buffer's barrier.
+    Walk wi;
+    wi.start(p, tile0);
+    int ir = 0;
+    uint32_t iph = 0;
+    auto fetch = [&]() {
+      Patch pt;
+      pt.of(p, wi);
+      if (!warp_wait(&sh.raw_empty[ir], iph ^ 1, abort_flag, ws, 0x50000u | ir)) { ok = false; return; }
+      const int nrows = pt.r_hi - pt.r_lo;
+      const uint32_t bytes_row = (uint32_t)((pt.c_hi - pt.c_lo) * C2);
+      if (lane == 0) mbar_arrive_expect_tx(&sh.raw_full[ir], (uint32_t)nrows * bytes_row);
+      __syncwarp();
+      if (lane < nrows) {
+        const int r = pt.r_lo + lane;
+        const char *src = reinterpret_cast<const char *>(x) +
+                          ((long long)wi.img * p.h + (pt.gy0 + r)) * row_stride + (long long)(pt.gx0 + pt.c_lo) * C2;
+        bulk_load(raw_base + (uint32_t)ir * (uint32_t)p.raw_bytes + (uint32_t)r * raw_pitch, src, bytes_row,
+                  &sh.raw_full[ir]);
+      }
+      wi.step(p);
+      if (++ir == p.nraw) { ir = 0; iph ^= 1; }
+    };
+    if (warp == 0) {
+      if (lane == 0) {
+        mbar_arrive_expect_tx(&sh.weights, (uint32_t)p.b_bytes);
+        tma_load_3d(smem_b, &map_b, &sh.weights, 0, 0, 0);
+      }
+      __syncwarp();
+      for (int j = 0; j < p.nraw - 1 && j < ntiles && ok; ++j) fetch();
+    }
+
+    Walk wp;
+    wp.start(p, tile0);
+    int s = 0, pr = 0;
+    uint32_t ph = 0, pph = 0;
+#pragma unroll 1
+    for (int it = 0; it < ntiles && ok; ++it) {
+      if (warp == 0 && it + p.nraw - 1 < ntiles) fetch();
+      if (!ok) break;
+      Patch pt;
+      pt.of(p, wp);
+      if (!mbar_wait(&sh.raw_full[pr], pph, abort_flag, ws, 0x60000u | pr)) break;
+      if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
+      const uint32_t stage = a_base0 + (uint32_t)s * (uint32_t)p.a_stage_bytes;
+      const uint32_t raw = raw_base + (uint32_t)pr * (uint32_t)p.raw_bytes;
+      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+      for (int q = tid; q < row_pieces; q += kProducerThreads) {
+        const int col = (int)(((uint32_t)q * p.cch_inv) >> 16), cc = q - col * p.cch;
+        const bool cv = (col >= pt.c_lo) && (col < pt.c_hi);
+        // plane (column parity, chunk), pixel col >> 1 of the plane's row
+        uint32_t dst = stage + (uint32_t)(((col & 1) * p.cch + cc) * p.plane_stride + (col >> 1) * 16);
+        const int lo = cv ? pt.r_lo : pt.rows, hi = cv ? pt.r_hi : pt.rows;    // rows [lo, hi) are real pixels
+        int r = 0;
+#pragma unroll 1
+        for (; r < lo; ++r, dst += drow) sts128(dst, zero);
+        uint32_t src = raw + (uint32_t)((col - pt.c_lo) * C2 + cc * 16) + (uint32_t)r * raw_pitch;
+#pragma unroll 1
+        for (; r + 4 <= hi; r += 4, dst += 4 * drow, src += 4 * raw_pitch) {
+          const uint4 v0 = lds128(src), v1 = lds128(src + raw_pitch), v2 = lds128(src + 2 * raw_pitch),
+                      v3 = lds128(src + 3 * raw_pitch);
+          sts128(dst, v0); sts128(dst + drow, v1); sts128(dst + 2 * drow, v2); sts128(dst + 3 * drow, v3);
+        }
+#pragma unroll 1
+        for (; r < hi; ++r, dst += drow, src += raw_pitch) sts128(dst, lds128(src));
+#pragma unroll 1
+        for (; r < pt.rows; ++r, dst += drow) sts128(dst, zero);
+      }
+      fence_proxy_async();                       // the planes are read by the tensor core (async proxy)
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&sh.full[s]); mbar_arrive(&sh.raw_empty[pr]); }
+      wp.step(p);
+      if (++s == p.stages) { s = 0; ph ^= 1; }
+      if (++pr == p.nraw) { pr = 0; pph ^= 1; }
+    }
+  } else {
+    // ---- consumer preparation
+    if (warp == kMmaWarp) {
+      tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
+      tmem_relinquish();
+    } else if (warp >= kFirstEpiWarp) {
+      const int t = (int)threadIdx.x - kFirstEpiWarp * 32;
+      if (t < 32) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
+    }
+    tc_fence_before();
+    bar_sync(kBarConsumers, kConsumerThreads);
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp < kFirstEpiWarp) {
+      // ================================================================== MMA issue
+      // Warp mw takes blocks c = mw mod kMmaWarps.  The warps sit on different schedulers, so the
+      // issue sequences of several blocks progress side by side although each shares its scheduler
+      // with epilogue warps.  The warp stays converged; one elected lane issues.
+      const int mw = warp - kMmaWarp;
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
+      const uint32_t desc_hi = (128u >> 4) | (1u << 14);
+      const uint32_t b_lo0 = ((smem_u32(smem_b) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
+      const uint32_t b_step = 2u * (uint32_t)p.n_pad;
+      const uint32_t a_row0 = smem_u32(smem_a) >> 4, a_stage_rows = (uint32_t)p.a_stage_bytes >> 4;
+      bool ok = warp_wait(&sh.weights, 0, abort_flag, ws, 0x70000u);
+      int s = 0;                                 // stage and its phase, accumulator slot and its phase
+      uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+      int next = mw, c0 = 0;                     // next block of this warp; first block of the tile
+      Walk t;
+      t.start(p, tile0);
+#pragma unroll 1
+      for (int it = 0; it < ntiles && ok; ++it) {
+        const int nblk = t.nblk(p);
+        if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int b = next - c0; b < nblk; b += kMmaWarps, next += kMmaWarps) {
+          if (!warp_wait(&sh.slot_empty[slot], sph, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
+          const uint32_t a_add = a_row + (uint32_t)(b * 128);
+          uint32_t b_lo = b_lo0;
+#pragma unroll 2
+          for (int j = 0; j < p.npairs; ++j, b_lo += b_step) {
+            const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(p.a_desc_lo[j] + a_add);
+            const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)b_lo;
+            if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+          }
+          if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
+          slot += kMmaWarps;
+          while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+        }
+        // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
+        if (ok && elect_one()) umma_commit(&sh.empty[s]);
+        c0 += nblk;
+        t.step(p);
+        a_row += a_stage_rows;
+        if (++s == p.stages) { s = 0; ph ^= 1; a_row = a_row0; }
+      }
+    } else {
+      switch (p.co8) {
+        case 8: epilogue_dispatch<8>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        case 16: epilogue_dispatch<16>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        case 24: epilogue_dispatch<24>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        default: epilogue_dispatch<32>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+      }
+    }
+    // ---- consumer teardown
+    if (*abort_flag) {
+      const unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    bar_sync(kBarConsumers, kConsumerThreads);
+    if (warp == kMmaWarp) {
+      tc_fence_after();
+      tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+constexpr int kSmemBudget = 220 * 1024;
+constexpr int kStageLimit = 40 * 1024;
+
+// plane stride in 16-byte units: odd, so that the planes a warp writes side by side start in
+// different bank groups
+int padded_plane_units(int units) { return units | 1; }
+
+bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
+  KOrder ko;
+  dc_korder_init(&ko, g);
+  if (!ko.pair) return false;
+  const int ho = dc_out_extent(h, g->k, 1, g->pad), wo = dc_out_extent(w, g->k, 1, g->pad);
+  if (ho <= 0 || wo <= 0) return false;
+  if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;
+  p->n_img = n; p->h = h; p->w = w; p->ho = ho; p->wo = wo;
+  p->c_in = g->c_in; p->c_out = g->c_out; p->co8 = ko.co8;
+  p->k = g->k; p->pad = g->pad; p->cch = ko.cch;
+  p->n_pad = ko.n_pad;
+  p->npairs = ko.e_pad / 2;
+  if (p->npairs > kMaxPairs) return false;
+  p->slots = 512 / p->n_pad;
+  if (p->slots > kMaxSlots) p->slots = kMaxSlots;
+  if (p->slots < 2) return false;
+  p->groups = p->slots < kGroups ? p->slots : kGroups;
+  int cols = 32;
+  while (cols < p->slots * p->n_pad) cols *= 2;
+  p->tmem_cols = cols;
+  p->cch_inv = (65536u + (uint32_t)p->cch - 1) / (uint32_t)p->cch;
+  const int nxt = dc_div_up(wo, 128);
+  p->tw = dc_div_up(wo, nxt);
+  if (p->tw & 1) ++p->tw;                        // tiles start on an even output column
+  p->nxt = dc_div_up(wo, p->tw);
+  p->tw2 = p->tw / 2;
+  p->wbox2 = p->tw2 + (g->k >> 1);
+  p->wboxp = 2 * p->wbox2;
+  if (p->wboxp * p->cch >= 4096) return false;
+  p->wbox2_inv = ((1u << 20) + (uint32_t)p->wbox2 - 1) / (uint32_t)p->wbox2;
+  const long long strips = (long long)n * p->nxt;
+  if (strips * ho >= (1ll << 30)) return false;
+  const int C2 = g->c_in * 2;
+  // fixed part of shared memory: weights, bias, per-warp output staging
+  p->b_bytes = ko.e_pad * p->n_pad * 16;
+  p->out_buf_bytes = (int)dc_round_up((size_t)64 * g->c_out * 2, 128);
+  p->bulk_out = (p->nxt == 1) ? 1 : 0;
+  const int slack = 4096;      // a block's 128 GEMM rows may reach past the last plane; those rows are dropped
+  p->off_b = 0;
+  p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
+  p->off_out = p->off_bias + 128;
+  p->off_raw = p->off_out + kEpiWarps * 2 * p->out_buf_bytes;
+  auto stage_bytes = [&](int th_c) {
+    const int rb = th_c + g->k - 1;
+    return (long long)dc_round_up((size_t)2 * p->cch * padded_plane_units(rb * p->wbox2 + 1) * 16, 128);
+  };
+  auto ring_bytes = [&](int th_c, int r, int s) {
+    const int rb = th_c + g->k - 1;
+    const long long raw = (long long)dc_round_up((size_t)rb * p->wboxp * C2, 128);
+    return 1024ll + p->off_raw + r * raw + s * stage_bytes(th_c) + slack;
+  };
+  // Rows per tile.  A CTA's time is roughly (tiles it gets) x (blocks per tile + a fixed cost per
+  // tile + the patch rows it stages); the CTA with the most tiles sets the kernel's time, so the
+  // candidates are ranked by that product.  Bounds: patch rows fit a warp's lanes (one bulk copy
+  // per row and lane) and the rings fit shared memory.
+  int th = 0;
+  double best = 0.0;
+  for (int cand = 1; cand <= 16 && cand <= ho; ++cand) {
+    const int rbox = cand + g->k - 1;
+    if (rbox > 32) break;
+    if (stage_bytes(cand) > kStageLimit) break;
+    if (ring_bytes(cand, 2, 2) > kSmemBudget) break;
+    const long long tiles = strips * dc_div_up(ho, cand);
+    const long long per_max = (tiles + n_sm - 1) / n_sm;
+    const int mb = dc_div_up((cand - 1) * p->wbox2 + p->tw2, 128);
+    double cost = (double)per_max * (mb + 0.3 + 0.05 * rbox);
+    if (per_max < 3 && tiles >= 3ll * n_sm) cost *= 1.5;       // too few tiles to overlap the roles
+    if (th == 0 || cost < best) { th = cand; best = cost; }
+  }
+  if (th == 0) return false;
+  p->th = th;
+  p->tiles_y = dc_div_up(ho, th);
+  const long long total_tiles = strips * p->tiles_y;
+  const int grid = total_tiles < n_sm ? (int)total_tiles : n_sm;
+  p->grid = grid;
+  p->tiles_per = (int)(total_tiles / grid);
+  p->tiles_rem = (int)(total_tiles % grid);
+  const int rbox = th + g->k - 1;
+  p->mb = dc_div_up((th - 1) * p->wbox2 + p->tw2, 128);
+  const int th_last = ho - (p->tiles_y - 1) * th;
+  p->mb_last = dc_div_up((th_last - 1) * p->wbox2 + p->tw2, 128);
+  p->plane_stride = padded_plane_units(rbox * p->wbox2 + 1) * 16;
+  p->a_stage_bytes = (int)stage_bytes(th);
+  p->raw_bytes = (int)dc_round_up((size_t)rbox * p->wboxp * C2, 128);
+  // rings: as deep as the CTA's tile count and shared memory allow
+  const long long per_cta = p->tiles_per + (p->tiles_rem ? 1 : 0);
+  int nraw = kMaxRaw < per_cta ? kMaxRaw : (int)per_cta, stages = kMaxStages < per_cta ? kMaxStages : (int)per_cta;
+  if (nraw < 2) nraw = 2;
+  if (stages < 2) stages = 2;
+  while (ring_bytes(th, nraw, stages) > kSmemBudget && (nraw > 2 || stages > 2)) {
+    if (stages >= nraw && stages > 2) --stages;
+    else if (nraw > 2) --nraw;
+    else --stages;
+  }
+  if (ring_bytes(th, nraw, stages) > kSmemBudget) return false;
+  p->nraw = nraw;
+  p->stages = stages;
+  p->off_a = p->off_raw + nraw * p->raw_bytes;
+  p->smem_bytes = (int)ring_bytes(th, nraw, stages);
+  // chunk-pair table: entry = (parity, chunk, tap row r, dx >> 1) -> byte offset of its 16-byte column in a stage
+  for (int j = 0; j < p->npairs; ++j) {
+    uint32_t off[2] = {0u, 16u};
+    for (int q = 0; q < 2; ++q) {
+      int pc, cc, r, dx;
+      // the padding entry reads entry 0 (offset 0) again; its weights are zero
+      off[q] = dc_korder_decode(ko, 2 * j + q, &pc, &cc, &r, &dx)
+                   ? (uint32_t)((pc * p->cch + cc) * p->plane_stride + (r * p->wbox2 + (dx >> 1)) * 16) : 0u;
+    }
+    if (off[1] <= off[0]) return false;
+    p->a_desc_lo[j] = (off[0] >> 4) | (((off[1] - off[0]) >> 4) << 16);
+  }
+  return true;
+}
+
+}  // namespace
+
+bool dc_conv_pair_supported(int n, int h, int w, const dc_geom *g) {
+  PairParams p;
+  return pair_plan(n, h, w, g, 148, &p);
+}
+
+dc_status dc_launch_conv_pair(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y, void *workspace,
+                              cudaStream_t stream) {
+  PairParams p;
+  const int n_sm = sm_count();
+  if (!pair_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
+  p.act = (int)act;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return DC_ERR_CUDA;
+  CUtensorMap map_b;
+  {
+    const int e_pad = p.npairs * 2;
+    cuuint64_t gdim[3] = {8, (cuuint64_t)p.n_pad, (cuuint64_t)e_pad};
+    cuuint64_t gstr[2] = {16, (cuuint64_t)p.n_pad * 16};
+    cuuint32_t box[3] = {8, (cuuint32_t)p.n_pad, (cuuint32_t)e_pad};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w_packed), gdim, gstr, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    attr_set = true;
+  }
+  k_conv_tc_pair<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_b, p, (const __nv_bfloat16 *)x, bias,
+                                                            (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
+                                                            (DcWsHeader *)workspace);
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}

@@ -77,7 +77,8 @@ def test_packed_bytes():
     assert dc.packed_bytes(dc.geom(96, 96, 96, 3, 1, 1), dc.BF16) == 96 * 9 * 4
     # fold order: 3 chunks x 3 tap rows = 9 entries padded to 10; rows = 3 tap columns x 24 channels,
     # padded to 80; 16 bytes per (entry, row)
-    assert dc.packed_bytes(dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == 10 * 80 * 16
+    # pair order: 2 parities x 3 chunks x 3 rows x 2 column pairs = 36 entries, N = 2 x 24
+    assert dc.packed_bytes(dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == 36 * 48 * 16
     assert dc.packed_bytes(dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == 20 * 160 * 16
     # general order: 18 chunks x 9 taps in 3 groups of 6 chunks, 64 output channels
     assert dc.packed_bytes(dc.geom(144, 64, 1, 3, 1, 1), dc.BF16) == 3 * 54 * 64 * 16
@@ -86,9 +87,9 @@ def test_packed_bytes():
 
 
 def test_kernel_name_query_follows_the_dispatch_rules():
-    # small-channel stride-1 3x3 / 5x5: fold order; wide or strided: general tensor-core kernel;
+    # small-channel stride-1 3x3: pair order, 5x5: fold order; wide or strided: general tensor-core kernel;
     # channel counts that are no multiple of 8: CUDA cores
-    assert dc.conv_kernel_name(64, 56, 56, dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_fold"
+    assert dc.conv_kernel_name(64, 56, 56, dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_pair"
     assert dc.conv_kernel_name(128, 28, 28, dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_fold"
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(24, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 14, 14, dc.geom(96, 576, 1, 1, 1, 0), dc.BF16) == "k_conv_tc"
