@@ -52,7 +52,15 @@ static inline int dc_out_extent(int h, int k, int s, int p) {
 // pixel e is W[o][c][r][dx - e] (zero where dx - e is no tap).  This costs (k+1)/2k more tensor-core
 // work than plain order per output -- far less than it saves in instructions: half as many
 // accumulator rows, and no reduction in the epilogue as fold order needs.
+//
+// "Pair rows" (pair == 2) is the same GEMM fed straight from TMA tiles: a shared-memory row is the
+// 128-byte line of two neighbouring pixels (2 * c_in <= 64 channels, zero filled beyond), rows are
+// 128-byte swizzled, and the K index of a row is simply its 16-byte chunks: chunk q holds
+// elements 8q..8q+7 of (pixel 0 channels, pixel 1 channels).  An entry is (tap row r, pair shift t,
+// chunk q); the weight of element (pixel px, channel c) of shift t for output pixel e of the pair
+// is W[o][c][r][2t + px - e].  Nothing is repacked on the way in.
 // ----------------------------------------------------------------------------------------------
+#define DC_PAIR_ROWS 1
 struct KOrder {
   int k, stride, pad;
   int c_in, cch;      // input channels, chunks of 8 (rounded up)
@@ -65,7 +73,7 @@ struct KOrder {
   int e_pad;          // e rounded up to even
   int n_pad;          // operand rows rounded up to 16 (output channels, or k * co8 in fold order)
   int fold;           // 1: fold order
-  int pair;           // 1: pair order
+  int pair;           // 1: pair order on parity planes, 2: pair rows fed by TMA
   int co8;            // output channels rounded up to 8
 };
 
@@ -86,6 +94,17 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
     {
       const int e = ko->cch * g->k * (g->k + 1);
       const int n_pad = (int)dc_round_up((size_t)(2 * ko->co8), 16);
+      const int nt = (g->k + 1) / 2;
+      if (DC_PAIR_ROWS && g->k * nt * ko->cch <= 32 && ko->cch <= 4 &&
+          (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 96 * 1024) {
+        ko->pair = 2;
+        ko->n_pad = n_pad;
+        ko->ns[0] = nt; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
+        ko->cg = ko->cch; ko->ng = 1;
+        ko->e = g->k * nt * 2 * ko->cch;
+        ko->e_pad = ko->e;
+        return;
+      }
       if (((e + 1) / 2) * 48 <= 5 * 256 && (size_t)((e + 1) & ~1) * n_pad * 16 <= 96 * 1024) {
         ko->pair = 1;
         ko->pcs = 2;
@@ -134,6 +153,17 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
 // entry index within a group -> (pc, ccg, r, s); returns false for the zero padding entry
 __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
                                                         int *r, int *s) {
+  if (ko.pair == 2) {
+    // (tap row, pair shift, chunk of the pair row); *ccg returns the chunk, *s the shift
+    if (e >= ko.e) return false;
+    const int nq = 2 * ko.cch;
+    *ccg = e % nq;
+    const int u = e / nq;
+    *s = u % ko.ns[0];
+    *r = u / ko.ns[0];
+    *pc = 0;
+    return true;
+  }
   if (ko.pair) {
     // (parity, chunk, tap row, dx >> 1); *s returns dx.  Odd counts are padded as in fold order.
     if (ko.e & 1) {
@@ -189,6 +219,8 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 // (channel chunk cc in [0,cch), tap r, s) -> position of that chunk in the packed weights,
 // in units of chunk planes (n_pad * 8 elements each)
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
+  if (ko.pair == 2)            // the copy for the first pixel of the pair: dx = s, pixel s & 1 of shift s >> 1
+    return (r * ko.ns[0] + (s >> 1)) * 2 * ko.cch + (s & 1) * ko.cch + cc;
   if (ko.pair) {               // the copy for the first pixel of the pair: dx = s
     const int pc = s & 1;
     const int e = (((pc * ko.cch + cc) * ko.k + r) * ko.ns[0]) + (s >> 1);
@@ -239,6 +271,10 @@ dc_status dc_launch_conv_pair(const void *x, int n, int h, int w, const dc_geom 
                               const float *bias, dc_act act, const void *residual, void *y,
                               void *workspace, cudaStream_t stream);
 bool dc_conv_pair_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                                  const float *bias, dc_act act, const void *residual, void *y,
+                                  void *workspace, cudaStream_t stream);
+bool dc_conv_pairrows_supported(int n, int h, int w, const dc_geom *g);
 dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                               const float *bias, dc_act act, const void *residual, void *y,
                               void *workspace, cudaStream_t stream);

@@ -144,12 +144,11 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
   const int m = q * 32 + lane;
   const uint32_t tmem_row = sh.tmem_base + ((uint32_t)(q * 32) << 16);
   volatile uint32_t *abort_flag = &sh.abort;
-  uint8_t *obuf0 = smem_out + (size_t)ew * 2 * p.out_buf_bytes;
+  uint8_t *obuf = smem_out + (size_t)ew * p.out_buf_bytes;
   const uint32_t lt = (1u << lane) - 1u;
   uint32_t slot = (uint32_t)grp, sph = 0;        // accumulator slot and its phase for block c = grp
   while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
   int next = grp, c0 = 0;                        // next block of this warp; first block of the tile
-  uint32_t mine = 0;                             // blocks this warp has done
   Walk t;
   t.start(p, tile0);
 #pragma unroll 1
@@ -175,8 +174,6 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
       if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
       slot += (uint32_t)p.groups;
       while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
-      uint8_t *obuf = obuf0 + (mine & 1) * p.out_buf_bytes;
-      ++mine;
 
       const int pos = b * 128 + m;
       const int yy = (int)(((uint32_t)pos * p.wbox2_inv) >> 20), jj = pos - yy * p.wbox2;
@@ -187,7 +184,7 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
       const uint32_t m0 = __ballot_sync(0xffffffffu, valid0), m1 = __ballot_sync(0xffffffffu, valid1);
       uint8_t *dst;
       if (p.bulk_out) {
-        if (lane == 0) bulk_wait_read1();        // the copy that last read this buffer (two blocks ago) is done
+        if (lane == 0) bulk_wait_read0();        // the warp's previous copy (several blocks ago) has read the buffer
         __syncwarp();
         dst = obuf + (size_t)(__popc(m0 & lt) + __popc(m1 & lt)) * p.c_out * 2;
       } else {
@@ -239,7 +236,7 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
           if (m0)
             bulk_store(y + (tile_pix0 + (size_t)off_first) * p.c_out, smem_u32(obuf),
                        (uint32_t)((__popc(m0) + __popc(m1)) * p.c_out * 2));
-          bulk_commit();                         // one group per block, empty or not: the wait above counts groups
+          bulk_commit();
         }
       }
     }
@@ -502,7 +499,7 @@ int padded_plane_units(int units) { return units | 1; }
 bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   KOrder ko;
   dc_korder_init(&ko, g);
-  if (!ko.pair) return false;
+  if (ko.pair != 1) return false;
   const int ho = dc_out_extent(h, g->k, 1, g->pad), wo = dc_out_extent(w, g->k, 1, g->pad);
   if (ho <= 0 || wo <= 0) return false;
   if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;
@@ -540,7 +537,7 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   p->off_b = 0;
   p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
   p->off_out = p->off_bias + 128;
-  p->off_raw = p->off_out + kEpiWarps * 2 * p->out_buf_bytes;
+  p->off_raw = p->off_out + kEpiWarps * p->out_buf_bytes;
   auto stage_bytes = [&](int th_c) {
     const int rb = th_c + g->k - 1;
     return (long long)dc_round_up((size_t)2 * p->cch * padded_plane_units(rb * p->wbox2 + 1) * 16, 128);
@@ -564,7 +561,8 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
     const long long tiles = strips * dc_div_up(ho, cand);
     const long long per_max = (tiles + n_sm - 1) / n_sm;
     const int mb = dc_div_up((cand - 1) * p->wbox2 + p->tw2, 128);
-    double cost = (double)per_max * (mb + 0.3 + 0.05 * rbox);
+    // the first tile is fetched, repacked, multiplied and written out with nothing to overlap with
+    double cost = (double)per_max * (mb + 0.3 + 0.05 * rbox) + 0.25 * rbox;
     if (per_max < 3 && tiles >= 3ll * n_sm) cost *= 1.5;       // too few tiles to overlap the roles
     if (th == 0 || cost < best) { th = cand; best = cost; }
   }

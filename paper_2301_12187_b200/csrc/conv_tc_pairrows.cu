@@ -1,0 +1,543 @@
+// Dense stride-1 convolution with few channels (c_in <= 32) as an implicit GEMM over PAIR ROWS fed
+// straight from TMA tiles (see KOrder, pair == 2).
+//
+// A GEMM row is the 128-byte shared-memory line that holds two neighbouring input pixels, and it
+// produces the two output pixels that start there:
+//     D[j][e][o] = sum_{r} sum_{t} sum_{px,c} x[row y+r, pixel 2(j+t)+px][c] * W[o][c][r][2t + px - e]
+// (e = 0, 1; weights are zero where 2t + px - e is no tap).  So N = 2 * c_out, the K index of a row
+// is just its 16-byte chunks, tap row r and pair shift t move the operand's start address by whole
+// rows, and nothing has to be rearranged between HBM and the tensor core: one 4-D TMA tile per
+// patch (box = 128 bytes x pairs x rows x 1 image, 128-byte swizzle, zero fill outside the image)
+// is the A operand of every instruction of the tile.  The tensor map views an image row as W/2
+// pairs of 2*c_in channels; the box is 64 channels wide, so the tail of each line is zero filled.
+// When the padding is odd the patch starts one pixel further left (so that pairs stay aligned in
+// memory) and output pair j is (2j-1, 2j); the epilogue masks the pixel that falls off either end.
+//
+// Operand descriptors: K-major, 128-byte swizzle, 1024 bytes between 8-row groups.  Tap rows, pair
+// shifts (whole 128-byte lines) and the 32-byte K step inside a line are all added to the start
+// address, with the base-offset field left at 0: the tensor core applies the swizzle to the bits of
+// the shared-memory address itself, exactly as the TMA engine did when it wrote the tile (stages
+// are 1024-byte aligned), so any line of the tile can be row 0 of an operand.  A descriptor that
+// put the start's phase, (address >> 7) & 7, into the base-offset field read wrong chunks here.
+// Weights: no-swizzle K-major chunk planes, one 3-D TMA tile per CTA.
+//
+// Work split as in the other tensor-core kernels: tiles of th output rows on a fixed grid, CTAs
+// (one per SM) take contiguous runs of tiles; behind the stages the unit is the 128-row block (256
+// outputs): blocks go round-robin over accumulator slots in tensor memory, the MMA warps take them
+// in turn, and so do the epilogue warps, each on its own (one tensor-memory lane quadrant of every
+// third block) with its own staging buffer and bulk store.
+//
+// Roles (512 threads): warp 0 producer (one lane issues the TMA loads), warps 1-3 MMA issue
+// (converged warps, elected lane; warp 1 owns the tensor memory), warps 4-15 epilogue.  All waits
+// are bounded (tc::mbar_wait).
+#include "tc_ptx.cuh"
+
+namespace {
+using namespace tc;
+
+constexpr int kMaxStages = 6;                    // activation tiles in flight
+constexpr int kMaxSlots = 6;                     // accumulator slots in tensor memory
+constexpr int kMmaWarp = 1;                      // first MMA warp
+constexpr int kMmaWarps = 3;
+constexpr int kFirstEpiWarp = kMmaWarp + kMmaWarps;
+constexpr int kGroups = 3;                       // epilogue warps per tensor-memory lane quadrant
+constexpr int kEpiWarps = 4 * kGroups;
+constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
+constexpr int kThreads = 32 + kConsumerThreads;
+constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
+constexpr int kMaxMma = 32;                      // tensor-core instructions per block
+
+struct PairParams {
+  int n_img, h, w, ho, wo, c_in, c_out, co8;
+  int k, pad, cch;
+  int align;                   // pad & 1: output pair j is (2j - align, 2j - align + 1)
+  int tw, th, nxt;             // tile size in outputs, x tiles per row
+  int tw2, wbox2, rbox;        // output pairs per tile row, pair rows per patch row, patch rows
+  int tiles_y;                 // tiles per column strip
+  int grid, tiles_per, tiles_rem;   // CTAs; CTA b takes tiles_per (+1 if b < tiles_rem) tiles
+  int n_pad;                   // N of the instruction: 2 * co8, padded to 16
+  int mb, mb_last;             // blocks of a full tile / of a strip's last (shorter) tile
+  int a_stage_bytes, a_box_bytes, b_bytes;
+  int stages, slots, groups, act, bulk_out, out_buf_bytes;
+  int off_b, off_bias, off_out, off_a, smem_bytes;
+  int tmem_cols;
+  int nmma;
+  uint32_t wbox2_inv;          // ceil(2^20 / wbox2): q / wbox2 == (q * wbox2_inv) >> 20 for q < 4096
+  uint32_t a_lo[kMaxMma];      // per instruction: byte offset of its operand in a stage, >> 4
+};
+
+struct Shared {
+  uint64_t full[kMaxStages], empty[kMaxStages];
+  uint64_t slot_full[kMaxSlots], slot_empty[kMaxSlots];
+  uint64_t weights;
+  uint32_t tmem_base;
+  uint32_t abort;
+};
+
+// Position on the tile grid; every role keeps its own and steps it once per tile.
+struct Walk {
+  int img, xt, ty;
+  __device__ __forceinline__ void start(const PairParams &p, int tile) {
+    const int strip = tile / p.tiles_y;
+    ty = tile - strip * p.tiles_y;
+    img = strip / p.nxt;
+    xt = strip - img * p.nxt;
+  }
+  __device__ __forceinline__ void step(const PairParams &p) {
+    if (++ty == p.tiles_y) {
+      ty = 0;
+      if (++xt == p.nxt) { xt = 0; ++img; }
+    }
+  }
+  __device__ __forceinline__ int rows_out(const PairParams &p) const {   // output rows of this tile
+    const int left = p.ho - ty * p.th;
+    return left < p.th ? left : p.th;
+  }
+  __device__ __forceinline__ int nblk(const PairParams &p) const { return ty == p.tiles_y - 1 ? p.mb_last : p.mb; }
+};
+
+// Epilogue of one warp: tensor-memory lane quadrant q of every block c = grp mod groups, where grp
+// counts the warps of the same quadrant.  Nothing is shared with other warps: the thread of GEMM
+// row m owns the two output pixels of pair m, adds bias and skip input, applies the activation,
+// converts to bf16 and stages them; the warp's valid pixels are consecutive in the NHWC output (only
+// halo pairs and the tail of the block or tile drop out), so they leave as one bulk copy.
+// ACT and RES are compile-time so the per-pixel code carries no runtime switches.
+template <int CO8, int ACT, int RES>
+__device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+                                              uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
+                                              int tile0, int ntiles) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int ew = warp - kFirstEpiWarp;
+  const int grp = ew >> 2;
+  const int q = warp & 3;                        // tensor-memory lane quadrant this warp may read
+  // A waiter may trail its barrier by one phase at most, so a slot must not complete twice before
+  // its warp has looked: no more warps per quadrant than slots take part.
+  if (grp >= p.groups) return;
+  const int m = q * 32 + lane;
+  const uint32_t tmem_row = sh.tmem_base + ((uint32_t)(q * 32) << 16);
+  volatile uint32_t *abort_flag = &sh.abort;
+  uint8_t *obuf = smem_out + (size_t)ew * p.out_buf_bytes;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t slot = (uint32_t)grp, sph = 0;        // accumulator slot and its phase for block c = grp
+  while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+  int next = grp, c0 = 0;                        // next block of this warp; first block of the tile
+  Walk t;
+  t.start(p, tile0);
+#pragma unroll 1
+  for (int ti = 0; ti < ntiles; ++ti) {
+    const int nblk = t.nblk(p), th_t = t.rows_out(p);
+    const int tw_valid = (p.wo - t.xt * p.tw < p.tw) ? p.wo - t.xt * p.tw : p.tw;
+    const size_t tile_pix0 = ((size_t)t.img * p.ho + (size_t)(t.ty * p.th)) * p.wo + (size_t)(t.xt * p.tw);
+#pragma unroll 1
+    for (int b = next - c0; b < nblk; b += p.groups, next += p.groups) {
+      if (!warp_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot)) {
+        if (lane == 0) bulk_wait_all();
+        return;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
+      uint32_t v0[CO8], v1[CO8];
+      tmem_ld_cols<CO8>(taddr, v0);
+      tmem_ld_cols<CO8>(taddr + (uint32_t)CO8, v1);
+      tmem_ld_wait();
+      // the accumulator slot is free again: one arrival per warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
+      slot += (uint32_t)p.groups;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+
+      const int pos = b * 128 + m;
+      const int yy = (int)(((uint32_t)pos * p.wbox2_inv) >> 20), jj = pos - yy * p.wbox2;
+      const int xx = 2 * jj - p.align;           // first output column of the pair; -1 or >= tw_valid: no such pixel
+      const bool valid0 = (xx >= 0) && (xx < tw_valid) && (yy < th_t);
+      const bool valid1 = (xx + 1 < tw_valid) && (yy < th_t);
+      const int off = yy * p.wo + xx;            // pixel offset from the tile's first output pixel
+      const uint32_t m0 = __ballot_sync(0xffffffffu, valid0), m1 = __ballot_sync(0xffffffffu, valid1);
+      uint8_t *dst;
+      if (p.bulk_out) {
+        if (lane == 0) bulk_wait_read0();        // the warp's previous copy (several blocks ago) has read the buffer
+        __syncwarp();
+        dst = obuf + (size_t)(__popc(m0 & lt) + __popc(m1 & lt)) * p.c_out * 2;
+      } else {
+        dst = reinterpret_cast<uint8_t *>(y + (tile_pix0 + (size_t)off) * p.c_out);
+      }
+      const __nv_bfloat16 *rp = RES ? residual + (tile_pix0 + (size_t)off) * p.c_out : nullptr;
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint32_t *v = e ? v1 : v0;
+        if (e ? valid1 : valid0) {
+#pragma unroll
+          for (int ch = 0; ch < CO8; ch += 8) {
+            if (ch < p.c_out) {
+              float f[8];
+              const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
+              const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
+              f[0] = __uint_as_float(v[ch]) + b0.x; f[1] = __uint_as_float(v[ch + 1]) + b0.y;
+              f[2] = __uint_as_float(v[ch + 2]) + b0.z; f[3] = __uint_as_float(v[ch + 3]) + b0.w;
+              f[4] = __uint_as_float(v[ch + 4]) + b1.x; f[5] = __uint_as_float(v[ch + 5]) + b1.y;
+              f[6] = __uint_as_float(v[ch + 6]) + b1.z; f[7] = __uint_as_float(v[ch + 7]) + b1.w;
+              if (RES) {
+                const uint4 rv = *reinterpret_cast<const uint4 *>(rp + e * p.c_out + ch);
+                const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float2 rf = __bfloat1622float2(rb[i]);
+                  f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                }
+              }
+              uint4 ov;
+              __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float f0 = f[2 * i], f1 = f[2 * i + 1];
+                if (ACT) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
+                ob[i] = __floats2bfloat162_rn(f0, f1);
+              }
+              // in the staging buffer the warp's pixels are packed: the second follows the first only if there is one
+              *reinterpret_cast<uint4 *>(dst + ((e && (valid0 || !p.bulk_out) ? p.c_out : 0) + ch) * 2) = ov;
+            }
+          }
+        }
+      }
+      if (p.bulk_out) {
+        fence_proxy_async();                     // the staged pixels are read by the bulk copy engine
+        const int first = __ffs(m0 | m1) - 1;
+        const int off_first = __shfl_sync(0xffffffffu, valid0 ? off : off + 1, first < 0 ? 0 : first);
+        __syncwarp();
+        if (lane == 0) {
+          if (m0 | m1)
+            bulk_store(y + (tile_pix0 + (size_t)off_first) * p.c_out, smem_u32(obuf),
+                       (uint32_t)((__popc(m0) + __popc(m1)) * p.c_out * 2));
+          bulk_commit();
+        }
+      }
+    }
+    c0 += nblk;
+    t.step(p);
+  }
+  if (p.bulk_out && lane == 0) bulk_wait_all();
+}
+
+template <int CO8>
+__device__ __forceinline__ void epilogue_dispatch(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+                                                  uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
+                                                  int tile0, int ntiles) {
+  const int v = (p.act == DC_ACT_RELU6 ? 1 : 0) | (residual ? 2 : 0);
+  if (v == 0) epilogue_role<CO8, 0, 0>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  else if (v == 1) epilogue_role<CO8, 1, 0>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  else if (v == 2) epilogue_role<CO8, 0, 1>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  else epilogue_role<CO8, 1, 1>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                   const __grid_constant__ PairParams p, const float *__restrict__ bias,
+                   const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
+  extern __shared__ __align__(1024) uint8_t smem_raw_base[];
+  __shared__ __align__(8) Shared sh;
+
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~uintptr_t(1023));
+  uint8_t *smem_b = smem + p.off_b;
+  uint8_t *smem_a = smem + p.off_a;              // 1024-byte aligned stages (the swizzle pattern repeats every 1024 bytes)
+  uint8_t *smem_out = smem + p.off_out;
+  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile uint32_t *abort_flag = &sh.abort;
+
+  // this CTA's run of tiles
+  const int bid = (int)blockIdx.x;
+  const int ntiles = p.tiles_per + (bid < p.tiles_rem ? 1 : 0);
+  const int tile0 = bid * p.tiles_per + (bid < p.tiles_rem ? bid : p.tiles_rem);
+
+  // ---- set-up: the barriers are initialised by different threads side by side
+  {
+    const int t = (int)threadIdx.x;
+    bool did = false;
+    if (t < p.stages) { mbar_init(&sh.full[t], 1); mbar_init(&sh.empty[t], kMmaWarps); did = true; }
+    else if (t >= 32 && t < 32 + p.slots) { mbar_init(&sh.slot_full[t - 32], 1); mbar_init(&sh.slot_empty[t - 32], 4); did = true; }
+    else if (t == 64) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); did = true; }
+    if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    // ================================================================== producer
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&sh.weights, (uint32_t)p.b_bytes);
+      tma_load_3d(smem_b, &map_b, &sh.weights, 0, 0, 0);
+      const uint32_t a_base0 = smem_u32(smem_a);
+      Walk t;
+      t.start(p, tile0);
+      int s = 0;
+      uint32_t ph = 0;
+#pragma unroll 1
+      for (int it = 0; it < ntiles; ++it) {
+        if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
+        // the box always has rbox rows; rows and pairs outside the image arrive as zeros
+        mbar_arrive_expect_tx(&sh.full[s], (uint32_t)p.a_box_bytes);
+        tma_load_4d(a_base0 + (uint32_t)s * (uint32_t)p.a_stage_bytes, &map_a, &sh.full[s], 0,
+                    (t.xt * p.tw - p.pad - p.align) >> 1, t.ty * p.th - p.pad, t.img);
+        t.step(p);
+        if (++s == p.stages) { s = 0; ph ^= 1; }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- consumer preparation
+    if (warp == kMmaWarp) {
+      tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
+      tmem_relinquish();
+    } else if (warp >= kFirstEpiWarp) {
+      const int t = (int)threadIdx.x - kFirstEpiWarp * 32;
+      if (t < 32) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
+    }
+    tc_fence_before();
+    bar_sync(kBarConsumers, kConsumerThreads);
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp < kFirstEpiWarp) {
+      // ================================================================== MMA issue
+      // Warp mw takes blocks c = mw mod kMmaWarps.  The warps sit on different schedulers, so the
+      // issue sequences of several blocks progress side by side although each shares its scheduler
+      // with epilogue warps.  The warp stays converged; one elected lane issues.
+      const int mw = warp - kMmaWarp;
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
+      const uint32_t b_hi = (128u >> 4) | (1u << 14);            // no swizzle: 128 bytes between 8-row groups
+      const uint32_t a_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128-byte swizzle: 1024 bytes between 8-row groups
+      const uint32_t b_lo0 = ((smem_u32(smem_b) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
+      const uint32_t b_step = 2u * (uint32_t)p.n_pad;
+      const uint32_t a_row0 = smem_u32(smem_a) >> 4, a_stage_rows = (uint32_t)p.a_stage_bytes >> 4;
+      bool ok = warp_wait(&sh.weights, 0, abort_flag, ws, 0x70000u);
+      int s = 0;                                 // stage and its phase, accumulator slot and its phase
+      uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+      int next = mw, c0 = 0;                     // next block of this warp; first block of the tile
+      Walk t;
+      t.start(p, tile0);
+#pragma unroll 1
+      for (int it = 0; it < ntiles && ok; ++it) {
+        const int nblk = t.nblk(p);
+        if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int b = next - c0; b < nblk; b += kMmaWarps, next += kMmaWarps) {
+          if (!warp_wait(&sh.slot_empty[slot], sph, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
+          const uint32_t a_add = a_row + (uint32_t)(b * 1024);    // 128 rows of 128 bytes, in 16-byte units
+          uint32_t b_lo = b_lo0;
+#pragma unroll 2
+          for (int j = 0; j < p.nmma; ++j, b_lo += b_step) {
+            const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(p.a_lo[j] + a_add);
+            const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
+            if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+          }
+          if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
+          slot += kMmaWarps;
+          while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+        }
+        // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
+        if (ok && elect_one()) umma_commit(&sh.empty[s]);
+        c0 += nblk;
+        t.step(p);
+        a_row += a_stage_rows;
+        if (++s == p.stages) { s = 0; ph ^= 1; a_row = a_row0; }
+      }
+    } else {
+      switch (p.co8) {
+        case 8: epilogue_dispatch<8>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        case 16: epilogue_dispatch<16>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        case 24: epilogue_dispatch<24>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        default: epilogue_dispatch<32>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+      }
+    }
+    // ---- consumer teardown
+    if (*abort_flag) {
+      const unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    bar_sync(kBarConsumers, kConsumerThreads);
+    if (warp == kMmaWarp) {
+      tc_fence_after();
+      tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+constexpr int kSmemBudget = 220 * 1024;
+constexpr int kStageLimit = 48 * 1024;
+constexpr int kSlack = 17 * 1024;   // a block's 128 rows may reach past the last stage; those rows are dropped
+
+bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
+  KOrder ko;
+  dc_korder_init(&ko, g);
+  if (ko.pair != 2) return false;
+  if (w & 1) return false;                        // an image row must be a whole number of pixel pairs
+  const int ho = dc_out_extent(h, g->k, 1, g->pad), wo = dc_out_extent(w, g->k, 1, g->pad);
+  if (ho <= 0 || wo <= 0) return false;
+  if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;
+  p->n_img = n; p->h = h; p->w = w; p->ho = ho; p->wo = wo;
+  p->c_in = g->c_in; p->c_out = g->c_out; p->co8 = ko.co8;
+  p->k = g->k; p->pad = g->pad; p->cch = ko.cch;
+  p->align = g->pad & 1;
+  p->n_pad = ko.n_pad;
+  const int nt = (g->k + 1) / 2;
+  p->nmma = g->k * nt * ko.cch;
+  if (p->nmma > kMaxMma) return false;
+  p->slots = 512 / p->n_pad;
+  if (p->slots > kMaxSlots) p->slots = kMaxSlots;
+  if (p->slots < 2) return false;
+  p->groups = p->slots < kGroups ? p->slots : kGroups;
+  int cols = 32;
+  while (cols < p->slots * p->n_pad) cols *= 2;
+  p->tmem_cols = cols;
+  const int nxt = dc_div_up(wo, 128);
+  p->tw = dc_div_up(wo, nxt);
+  if (p->tw & 1) ++p->tw;                        // tiles start on an even output column
+  p->nxt = dc_div_up(wo, p->tw);
+  p->tw2 = (p->tw + p->align + 1) / 2;
+  p->wbox2 = p->tw2 + (g->k >> 1);
+  if (p->wbox2 > 256) return false;
+  p->wbox2_inv = ((1u << 20) + (uint32_t)p->wbox2 - 1) / (uint32_t)p->wbox2;
+  const long long strips = (long long)n * p->nxt;
+  if (strips * ho >= (1ll << 30)) return false;
+  // fixed part of shared memory: weights, bias, per-warp output staging
+  p->b_bytes = ko.e_pad * p->n_pad * 16;
+  p->out_buf_bytes = (int)dc_round_up((size_t)64 * g->c_out * 2, 128);
+  p->bulk_out = (p->nxt == 1) ? 1 : 0;
+  p->off_b = 0;
+  p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
+  p->off_out = p->off_bias + 128;
+  p->off_a = (int)dc_round_up((size_t)p->off_out + kEpiWarps * p->out_buf_bytes, 1024);
+  auto stage_bytes = [&](int th_c) { return (long long)dc_round_up((size_t)(th_c + g->k - 1) * p->wbox2 * 128, 1024); };
+  auto total_bytes = [&](int th_c, int s) { return 1024ll + p->off_a + s * stage_bytes(th_c) + kSlack; };
+  // Rows per tile.  A CTA's time is roughly (tiles it gets) x (blocks per tile + a fixed cost per
+  // tile + the patch rows it stages) plus the start-up of its first tile, which nothing overlaps;
+  // the CTA with the most tiles sets the kernel's time, so the candidates are ranked by that sum.
+  int th = 0;
+  double best = 0.0;
+  for (int cand = 1; cand <= 32 && cand <= ho; ++cand) {
+    const int rbox = cand + g->k - 1;
+    if (rbox > 256) break;
+    if (stage_bytes(cand) > kStageLimit) break;
+    if (total_bytes(cand, 2) > kSmemBudget) break;
+    if ((cand - 1) * p->wbox2 + p->tw2 + 128 >= 4096) break;
+    const long long tiles = strips * dc_div_up(ho, cand);
+    const long long per_max = (tiles + n_sm - 1) / n_sm;
+    const int mb = dc_div_up((cand - 1) * p->wbox2 + p->tw2, 128);
+    double cost = (double)per_max * (mb + 0.2 + 0.03 * rbox) + 0.15 * rbox;
+    if (per_max < 3 && tiles >= 3ll * n_sm) cost *= 1.5;       // too few tiles to overlap the roles
+    if (th == 0 || cost < best) { th = cand; best = cost; }
+  }
+  if (th == 0) return false;
+  p->th = th;
+  p->rbox = th + g->k - 1;
+  p->tiles_y = dc_div_up(ho, th);
+  const long long total_tiles = strips * p->tiles_y;
+  const int grid = total_tiles < n_sm ? (int)total_tiles : n_sm;
+  p->grid = grid;
+  p->tiles_per = (int)(total_tiles / grid);
+  p->tiles_rem = (int)(total_tiles % grid);
+  p->mb = dc_div_up((th - 1) * p->wbox2 + p->tw2, 128);
+  const int th_last = ho - (p->tiles_y - 1) * th;
+  p->mb_last = dc_div_up((th_last - 1) * p->wbox2 + p->tw2, 128);
+  p->a_stage_bytes = (int)stage_bytes(th);
+  p->a_box_bytes = p->rbox * p->wbox2 * 128;
+  const long long per_cta = p->tiles_per + (p->tiles_rem ? 1 : 0);
+  int stages = kMaxStages < per_cta ? kMaxStages : (int)per_cta;
+  if (stages < 2) stages = 2;
+  while (stages > 2 && total_bytes(th, stages) > kSmemBudget) --stages;
+  if (total_bytes(th, stages) > kSmemBudget) return false;
+  p->stages = stages;
+  p->smem_bytes = (int)total_bytes(th, stages);
+  // one instruction per (tap row r, pair shift t, 32-byte K step): where its operand starts in a stage
+  int j = 0;
+  for (int r = 0; r < g->k; ++r)
+    for (int t = 0; t < nt; ++t)
+      for (int sl = 0; sl < ko.cch; ++sl, ++j) {
+        const uint32_t off = (uint32_t)((r * p->wbox2 + t) * 128 + sl * 32);
+        p->a_lo[j] = (off >> 4) | (1u << 16);    // leading-dimension field: 1 (unused for swizzled K-major)
+      }
+  return true;
+}
+
+}  // namespace
+
+bool dc_conv_pairrows_supported(int n, int h, int w, const dc_geom *g) {
+  PairParams p;
+  return pair_plan(n, h, w, g, 148, &p);
+}
+
+dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                                  const float *bias, dc_act act, const void *residual, void *y, void *workspace,
+                                  cudaStream_t stream) {
+  PairParams p;
+  const int n_sm = sm_count();
+  if (!pair_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
+  p.act = (int)act;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return DC_ERR_CUDA;
+  CUtensorMap map_a, map_b;
+  {
+    // activations: an image row is w/2 lines of 2*c_in channels; the box is 64 channels (128 bytes) wide
+    const cuuint64_t C = (cuuint64_t)g->c_in;
+    cuuint64_t gdim[4] = {2 * C, (cuuint64_t)(w / 2), (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t gstr[3] = {4 * C, (cuuint64_t)w * C * 2, (cuuint64_t)h * w * C * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)p.wbox2, (cuuint32_t)p.rbox, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), gdim, gstr, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
+  }
+  {
+    const int e_pad = 2 * p.nmma;
+    cuuint64_t gdim[3] = {8, (cuuint64_t)p.n_pad, (cuuint64_t)e_pad};
+    cuuint64_t gstr[2] = {16, (cuuint64_t)p.n_pad * 16};
+    cuuint32_t box[3] = {8, (cuuint32_t)p.n_pad, (cuuint32_t)e_pad};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w_packed), gdim, gstr, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_pairrows, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    attr_set = true;
+  }
+  k_conv_tc_pairrows<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_a, map_b, p, bias, (const __nv_bfloat16 *)residual,
+                                                                (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}

@@ -209,6 +209,14 @@ __global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrde
         s = o / ko.co8;
         o -= s * ko.co8;
         if (s >= ko.k) o = c_out;          // padding rows
+      } else if (ko.pair == 2) {           // row = (pixel of the pair, output channel); ccg = chunk of the pair row, s = shift
+        const int elem = ccg * 8 + c8, ipx = elem / ko.c_in;
+        const int px = o / ko.co8;
+        o -= px * ko.co8;
+        s = 2 * s + ipx - px;
+        ccg = 0;
+        c8 = elem - ipx * ko.c_in;         // channel (grp is 0 and cg irrelevant once ccg = 0)
+        if (px >= 2 || s < 0 || s >= ko.k) o = c_out;
       } else if (ko.pair) {                // row = (pixel of the pair, output channel); s holds dx
         const int px = o / ko.co8;
         o -= px * ko.co8;
