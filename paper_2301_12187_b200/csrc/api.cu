@@ -26,7 +26,6 @@ extern "C" const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g
   if (dtype == DC_F32) return "k_conv_dense_f32";
   if (dtype != DC_BF16) return nullptr;
   if (dc_conv_pairrows_supported(n, h, w, g)) return "k_conv_tc_pairrows";
-  if (dc_conv_pair_supported(n, h, w, g)) return "k_conv_tc_pair";
   if (dc_conv_fold_supported(n, h, w, g)) return "k_conv_tc_fold";
   if (dc_conv_tc_supported(n, h, w, g)) return "k_conv_tc";
   return "k_conv_dense_bf16";
@@ -52,12 +51,9 @@ extern "C" dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, co
   cudaStream_t st = (cudaStream_t)stream;
   if (dtype == DC_BF16 && algo != DC_ALGO_SIMT && dc_conv_pairrows_supported(n, h, w, g))
     return dc_launch_conv_pairrows(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
-  const bool pair_ok = dtype == DC_BF16 && dc_conv_pair_supported(n, h, w, g);
-  const bool fold_ok = dtype == DC_BF16 && !pair_ok && dc_conv_fold_supported(n, h, w, g);
-  const bool tc_ok = dtype == DC_BF16 && !pair_ok && !fold_ok && dc_conv_tc_supported(n, h, w, g);
-  if (algo == DC_ALGO_TCGEN05 && !tc_ok && !fold_ok && !pair_ok) return DC_ERR_UNSUPPORTED;
-  if (pair_ok && algo != DC_ALGO_SIMT)
-    return dc_launch_conv_pair(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
+  const bool fold_ok = dtype == DC_BF16 && dc_conv_fold_supported(n, h, w, g);
+  const bool tc_ok = dtype == DC_BF16 && !fold_ok && dc_conv_tc_supported(n, h, w, g);
+  if (algo == DC_ALGO_TCGEN05 && !tc_ok && !fold_ok) return DC_ERR_UNSUPPORTED;
   if (fold_ok && algo != DC_ALGO_SIMT)
     return dc_launch_conv_fold(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   if (tc_ok && algo != DC_ALGO_SIMT)

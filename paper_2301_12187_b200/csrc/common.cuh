@@ -45,22 +45,18 @@ static inline int dc_out_extent(int h, int k, int s, int p) {
 // that the activation side may pair the last entry with entry 0 read a second time -- a chunk that
 // lies at a lower address, as the operand descriptor needs, and that always holds staged data.
 //
-// "Pair" order (stride 1, k >= 3, few channels, cheap enough): a GEMM row is a PAIR of neighbouring
-// output pixels (2j, 2j+1) and the operand has 2 * co8 rows n = e * co8 + o, e = which pixel of the
-// pair.  The pair reads input columns 2j + dx, dx = 0..k, so the planes are split by column parity
-// as for stride 2 and an entry is (parity, chunk, tap row r, dx >> 1); the weight of entry dx for
-// pixel e is W[o][c][r][dx - e] (zero where dx - e is no tap).  This costs (k+1)/2k more tensor-core
-// work than plain order per output -- far less than it saves in instructions: half as many
-// accumulator rows, and no reduction in the epilogue as fold order needs.
-//
-// "Pair rows" (pair == 2) is the same GEMM fed straight from TMA tiles: a shared-memory row is the
+// "Pair rows" order (stride 1, k >= 3, c_in <= 32, cheap enough): a GEMM row is a PAIR of
+// neighbouring output pixels and the operand has 2 * co8 rows n = e * co8 + o, e = which pixel of
+// the pair; the pair reads k+1 input columns, i.e. (k+1)/2 pairs of input pixels.  This costs
+// (k+1)/2k more tensor-core work than plain order per output -- far less than it saves: half as
+// many accumulator rows, and no reduction in the epilogue as fold order needs.  The GEMM is fed
+// straight from TMA tiles: a shared-memory row is the
 // 128-byte line of two neighbouring pixels (2 * c_in <= 64 channels, zero filled beyond), rows are
 // 128-byte swizzled, and the K index of a row is simply its 16-byte chunks: chunk q holds
 // elements 8q..8q+7 of (pixel 0 channels, pixel 1 channels).  An entry is (tap row r, pair shift t,
 // chunk q); the weight of element (pixel px, channel c) of shift t for output pixel e of the pair
 // is W[o][c][r][2t + px - e].  Nothing is repacked on the way in.
 // ----------------------------------------------------------------------------------------------
-#define DC_PAIR_ROWS 1
 struct KOrder {
   int k, stride, pad;
   int c_in, cch;      // input channels, chunks of 8 (rounded up)
@@ -73,7 +69,7 @@ struct KOrder {
   int e_pad;          // e rounded up to even
   int n_pad;          // operand rows rounded up to 16 (output channels, or k * co8 in fold order)
   int fold;           // 1: fold order
-  int pair;           // 1: pair order on parity planes, 2: pair rows fed by TMA
+  int pair;           // 2: pair rows
   int co8;            // output channels rounded up to 8
 };
 
@@ -89,13 +85,12 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->pcs = (g->stride == 2) ? 2 : 1;
   if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch <= 8 && ko->co8 <= 32 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
-    // pair order when its tensor-core cost stays small: instructions of ~48 cycles (N <= 64) per
-    // 256 outputs; beyond ~5 cycles per output fold order (one instruction row per tap row) wins
+    // pair rows when their tensor-core cost stays small (instructions of ~48 cycles per 256
+    // outputs); beyond that fold order (one instruction row per tap row) wins
     {
-      const int e = ko->cch * g->k * (g->k + 1);
       const int n_pad = (int)dc_round_up((size_t)(2 * ko->co8), 16);
       const int nt = (g->k + 1) / 2;
-      if (DC_PAIR_ROWS && g->k * nt * ko->cch <= 32 && ko->cch <= 4 &&
+      if (g->k * nt * ko->cch <= 32 && ko->cch <= 4 &&
           (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 96 * 1024) {
         ko->pair = 2;
         ko->n_pad = n_pad;
@@ -103,17 +98,6 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
         ko->cg = ko->cch; ko->ng = 1;
         ko->e = g->k * nt * 2 * ko->cch;
         ko->e_pad = ko->e;
-        return;
-      }
-      if (((e + 1) / 2) * 48 <= 5 * 256 && (size_t)((e + 1) & ~1) * n_pad * 16 <= 96 * 1024) {
-        ko->pair = 1;
-        ko->pcs = 2;
-        ko->n_pad = n_pad;
-        ko->ns[0] = ko->ns[1] = (g->k + 1) / 2;   // dx values of each parity
-        ko->s0[0] = 0; ko->s0[1] = 1;
-        ko->cg = ko->cch; ko->ng = 1;
-        ko->e = e;
-        ko->e_pad = (e + 1) & ~1;
         return;
       }
     }
@@ -164,23 +148,6 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
     *pc = 0;
     return true;
   }
-  if (ko.pair) {
-    // (parity, chunk, tap row, dx >> 1); *s returns dx.  Odd counts are padded as in fold order.
-    if (ko.e & 1) {
-      if (e == ko.e - 1 || e > ko.e) return false;
-      if (e == ko.e) e = ko.e - 1;
-    } else if (e >= ko.e) {
-      return false;
-    }
-    const int nd = ko.ns[0];
-    const int dxh = e % nd, t = e / nd;
-    *r = t % ko.k;
-    const int pl = t / ko.k;
-    *pc = pl / ko.cch;
-    *ccg = pl - *pc * ko.cch;
-    *s = 2 * dxh + *pc;
-    return true;
-  }
   if (ko.fold) {
     if (ko.e & 1) {
       if (e == ko.e - 1 || e > ko.e) return false;
@@ -221,11 +188,6 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
   if (ko.pair == 2)            // the copy for the first pixel of the pair: dx = s, pixel s & 1 of shift s >> 1
     return (r * ko.ns[0] + (s >> 1)) * 2 * ko.cch + (s & 1) * ko.cch + cc;
-  if (ko.pair) {               // the copy for the first pixel of the pair: dx = s
-    const int pc = s & 1;
-    const int e = (((pc * ko.cch + cc) * ko.k + r) * ko.ns[0]) + (s >> 1);
-    return ((ko.e & 1) && e == ko.e - 1) ? e + 1 : e;
-  }
   if (ko.fold) {
     const int e = cc * ko.k + r;
     return ((ko.e & 1) && e == ko.e - 1) ? e + 1 : e;
@@ -267,10 +229,6 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
                             const float *bias, dc_act act, const void *residual, void *y,
                             void *workspace, cudaStream_t stream);
 bool dc_conv_tc_supported(int n, int h, int w, const dc_geom *g);
-dc_status dc_launch_conv_pair(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
-                              const float *bias, dc_act act, const void *residual, void *y,
-                              void *workspace, cudaStream_t stream);
-bool dc_conv_pair_supported(int n, int h, int w, const dc_geom *g);
 dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                                   const float *bias, dc_act act, const void *residual, void *y,
                                   void *workspace, cudaStream_t stream);

@@ -46,6 +46,7 @@ constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
 constexpr int kThreads = 32 + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
 constexpr int kMaxMma = 32;                      // tensor-core instructions per block
+constexpr int kInFlight = 2;                     // activation tiles a CTA requests ahead of their use
 
 struct PairParams {
   int n_img, h, w, ho, wo, c_in, c_out, co8;
@@ -275,6 +276,15 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
 #pragma unroll 1
       for (int it = 0; it < ntiles; ++it) {
         if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
+        // At most kInFlight tiles are on their way: every CTA starts at the same moment, and if
+        // each asked for all its tiles at once the first tile (which the tensor core is waiting
+        // for) would arrive together with the last.
+        if (it >= kInFlight) {
+          int sw = s - kInFlight;
+          uint32_t pw = ph;
+          if (sw < 0) { sw += p.stages; pw ^= 1; }
+          if (!mbar_wait(&sh.full[sw], pw, abort_flag, ws, 0x80000u | sw)) break;
+        }
         // the box always has rbox rows; rows and pairs outside the image arrive as zeros
         mbar_arrive_expect_tx(&sh.full[s], (uint32_t)p.a_box_bytes);
         tma_load_4d(a_base0 + (uint32_t)s * (uint32_t)p.a_stage_bytes, &map_a, &sh.full[s], 0,

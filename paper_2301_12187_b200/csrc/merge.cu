@@ -217,11 +217,6 @@ __global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrde
         ccg = 0;
         c8 = elem - ipx * ko.c_in;         // channel (grp is 0 and cg irrelevant once ccg = 0)
         if (px >= 2 || s < 0 || s >= ko.k) o = c_out;
-      } else if (ko.pair) {                // row = (pixel of the pair, output channel); s holds dx
-        const int px = o / ko.co8;
-        o -= px * ko.co8;
-        s -= px;
-        if (px >= 2 || s < 0 || s >= ko.k) o = c_out;   // padding rows, or dx - px is no tap
       }
       int c = (grp * ko.cg + ccg) * 8 + c8;
       if (o < c_out && c < ko.c_in) v = w[(((size_t)o * ko.c_in + c) * ko.k + r) * ko.k + s];
