@@ -90,8 +90,8 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
     {
       const int n_pad = (int)dc_round_up((size_t)(2 * ko->co8), 16);
       const int nt = (g->k + 1) / 2;
-      if (g->k * nt * ko->cch <= 32 && ko->cch <= 4 &&
-          (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 96 * 1024) {
+      if (g->k * nt * ko->cch <= 64 && ko->cch <= 4 &&
+          (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 128 * 1024) {
         ko->pair = 2;
         ko->n_pad = n_pad;
         ko->ns[0] = nt; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;

@@ -19,7 +19,7 @@
 // whole pixel rows of the patch come in by bulk copies (one per row, tracked by an mbarrier) into
 // a raw ring, and the producer warps repack raw rows into chunk planes with 16-byte shared-memory
 // loads and stores, writing zeros for the halo that lies outside the image.  Weights arrive once
-// per CTA by a 3-D TMA tile.
+// per CTA by one bulk copy (they are packed in HBM exactly as the operand wants them).
 //
 // Work split.  Tiles are th output rows of one column strip of one image, on a fixed grid; CTAs
 // (one per SM) take contiguous runs of tiles and every role walks them with a few adds, no table.
@@ -306,8 +306,8 @@ __device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ FoldParams p,
-               const __nv_bfloat16 *__restrict__ x, const float *__restrict__ bias,
+k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__restrict__ x,
+               const void *__restrict__ w_packed, const float *__restrict__ bias,
                const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
   extern __shared__ __align__(1024) uint8_t smem_raw_base[];
   __shared__ __align__(8) Shared sh;
@@ -335,7 +335,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     if (t < p.nraw) { mbar_init(&sh.raw_full[t], 1); mbar_init(&sh.raw_empty[t], kProducerWarps); did = true; }
     else if (t >= 32 && t < 32 + p.stages) { mbar_init(&sh.full[t - 32], kProducerWarps); mbar_init(&sh.empty[t - 32], kMmaWarps); did = true; }
     else if (t >= 64 && t < 64 + p.slots) { mbar_init(&sh.slot_full[t - 64], 1); mbar_init(&sh.slot_empty[t - 64], 4); did = true; }
-    else if (t == 95) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_b); did = true; }
+    else if (t == 95) { mbar_init(&sh.weights, 1); sh.abort = 0; did = true; }
     if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -378,7 +378,7 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
     if (warp == 0) {
       if (lane == 0) {
         mbar_arrive_expect_tx(&sh.weights, (uint32_t)p.b_bytes);
-        tma_load_3d(smem_b, &map_b, &sh.weights, 0, 0, 0);
+        bulk_load(smem_u32(smem_b), w_packed, (uint32_t)p.b_bytes, &sh.weights);   // packed weights are the operand layout
       }
       __syncwarp();
       for (int j = 0; j < p.nraw - 1 && j < ntiles && ok; ++j) fetch();
@@ -513,22 +513,6 @@ k_conv_tc_fold(const __grid_constant__ CUtensorMap map_b, const __grid_constant_
 }
 
 // ------------------------------------------------------------------------------------------ host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void *ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -677,26 +661,12 @@ dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom 
   const int n_sm = sm_count();
   if (!fold_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
-  EncodeTiledFn encode = get_encode_fn();
-  if (!encode) return DC_ERR_CUDA;
-  CUtensorMap map_b;
-  {
-    const int e_pad = p.npairs * 2;
-    cuuint64_t gdim[3] = {8, (cuuint64_t)p.n_pad, (cuuint64_t)e_pad};
-    cuuint64_t gstr[2] = {16, (cuuint64_t)p.n_pad * 16};
-    cuuint32_t box[3] = {8, (cuuint32_t)p.n_pad, (cuuint32_t)e_pad};
-    cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w_packed), gdim, gstr, box, es,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
-  }
   static bool attr_set = false;
   if (!attr_set) {
     DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_fold, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     attr_set = true;
   }
-  k_conv_tc_fold<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_b, p, (const __nv_bfloat16 *)x, bias,
+  k_conv_tc_fold<<<p.grid, kThreads, p.smem_bytes, stream>>>(p, (const __nv_bfloat16 *)x, w_packed, bias,
                                                           (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                                           (DcWsHeader *)workspace);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;

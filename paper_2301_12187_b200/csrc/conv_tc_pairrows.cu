@@ -19,7 +19,7 @@
 // the shared-memory address itself, exactly as the TMA engine did when it wrote the tile (stages
 // are 1024-byte aligned), so any line of the tile can be row 0 of an operand.  A descriptor that
 // put the start's phase, (address >> 7) & 7, into the base-offset field read wrong chunks here.
-// Weights: no-swizzle K-major chunk planes, one 3-D TMA tile per CTA.
+// Weights: no-swizzle K-major chunk planes, exactly as packed in HBM, one bulk copy per CTA.
 //
 // Work split as in the other tensor-core kernels: tiles of th output rows on a fixed grid, CTAs
 // (one per SM) take contiguous runs of tiles; behind the stages the unit is the 128-row block (256
@@ -45,7 +45,7 @@ constexpr int kEpiWarps = 4 * kGroups;
 constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
 constexpr int kThreads = 32 + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
-constexpr int kMaxMma = 32;                      // tensor-core instructions per block
+constexpr int kMaxMma = 64;                      // tensor-core instructions per block
 constexpr int kInFlight = 2;                     // activation tiles a CTA requests ahead of their use
 
 struct PairParams {
@@ -232,8 +232,8 @@ __device__ __forceinline__ void epilogue_dispatch(const PairParams &p, Shared &s
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                   const __grid_constant__ PairParams p, const float *__restrict__ bias,
+k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ PairParams p,
+                   const void *__restrict__ w_packed, const float *__restrict__ bias,
                    const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
   extern __shared__ __align__(1024) uint8_t smem_raw_base[];
   __shared__ __align__(8) Shared sh;
@@ -258,7 +258,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
     bool did = false;
     if (t < p.stages) { mbar_init(&sh.full[t], 1); mbar_init(&sh.empty[t], kMmaWarps); did = true; }
     else if (t >= 32 && t < 32 + p.slots) { mbar_init(&sh.slot_full[t - 32], 1); mbar_init(&sh.slot_empty[t - 32], 4); did = true; }
-    else if (t == 64) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); did = true; }
+    else if (t == 64) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_a); did = true; }
     if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -267,7 +267,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
     // ================================================================== producer
     if (lane == 0) {
       mbar_arrive_expect_tx(&sh.weights, (uint32_t)p.b_bytes);
-      tma_load_3d(smem_b, &map_b, &sh.weights, 0, 0, 0);
+      bulk_load(smem_u32(smem_b), w_packed, (uint32_t)p.b_bytes, &sh.weights);   // packed weights are the operand layout
       const uint32_t a_base0 = smem_u32(smem_a);
       Walk t;
       t.start(p, tile0);
@@ -407,7 +407,7 @@ int sm_count() {
 
 constexpr int kSmemBudget = 220 * 1024;
 constexpr int kStageLimit = 48 * 1024;
-constexpr int kSlack = 17 * 1024;   // a block's 128 rows may reach past the last stage; those rows are dropped
+constexpr int kSlack = 17 * 1024;   // a block's 128 rows may reach this far past the last stage
 
 bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   KOrder ko;
@@ -448,10 +448,12 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   p->bulk_out = (p->nxt == 1) ? 1 : 0;
   p->off_b = 0;
   p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
-  p->off_out = p->off_bias + 128;
-  p->off_a = (int)dc_round_up((size_t)p->off_out + kEpiWarps * p->out_buf_bytes, 1024);
+  p->off_a = (int)dc_round_up((size_t)p->off_bias + 128, 1024);
+  // the output staging buffers follow the stages and double as the room a block's last rows may
+  // reach into past the last stage (what is read there only feeds rows that are dropped)
+  const long long tail_bytes = kEpiWarps * p->out_buf_bytes > kSlack ? kEpiWarps * p->out_buf_bytes : kSlack;
   auto stage_bytes = [&](int th_c) { return (long long)dc_round_up((size_t)(th_c + g->k - 1) * p->wbox2 * 128, 1024); };
-  auto total_bytes = [&](int th_c, int s) { return 1024ll + p->off_a + s * stage_bytes(th_c) + kSlack; };
+  auto total_bytes = [&](int th_c, int s) { return 1024ll + p->off_a + s * stage_bytes(th_c) + tail_bytes; };
   // Rows per tile.  A CTA's time is roughly (tiles it gets) x (blocks per tile + a fixed cost per
   // tile + the patch rows it stages) plus the start-up of its first tile, which nothing overlaps;
   // the CTA with the most tiles sets the kernel's time, so the candidates are ranked by that sum.
@@ -490,6 +492,7 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   while (stages > 2 && total_bytes(th, stages) > kSmemBudget) --stages;
   if (total_bytes(th, stages) > kSmemBudget) return false;
   p->stages = stages;
+  p->off_out = p->off_a + stages * p->a_stage_bytes;
   p->smem_bytes = (int)total_bytes(th, stages);
   // one instruction per (tap row r, pair shift t, 32-byte K step): where its operand starts in a stage
   int j = 0;
@@ -518,7 +521,7 @@ dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_g
   p.act = (int)act;
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) return DC_ERR_CUDA;
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a;
   {
     // activations: an image row is w/2 lines of 2*c_in channels; the box is 64 channels (128 bytes) wide
     const cuuint64_t C = (cuuint64_t)g->c_in;
@@ -531,23 +534,12 @@ dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_g
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
   }
-  {
-    const int e_pad = 2 * p.nmma;
-    cuuint64_t gdim[3] = {8, (cuuint64_t)p.n_pad, (cuuint64_t)e_pad};
-    cuuint64_t gstr[2] = {16, (cuuint64_t)p.n_pad * 16};
-    cuuint32_t box[3] = {8, (cuuint32_t)p.n_pad, (cuuint32_t)e_pad};
-    cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w_packed), gdim, gstr, box, es,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
-  }
   static bool attr_set = false;
   if (!attr_set) {
     DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_pairrows, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     attr_set = true;
   }
-  k_conv_tc_pairrows<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_a, map_b, p, bias, (const __nv_bfloat16 *)residual,
+  k_conv_tc_pairrows<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_a, p, w_packed, bias, (const __nv_bfloat16 *)residual,
                                                                 (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }

@@ -79,7 +79,10 @@ def test_packed_bytes():
     # padded to 80; 16 bytes per (entry, row)
     # pair order: 2 parities x 3 chunks x 3 rows x 2 column pairs = 36 entries, N = 2 x 24
     assert dc.packed_bytes(dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == 36 * 48 * 16
-    assert dc.packed_bytes(dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == 20 * 160 * 16
+    # pair rows, 5x5: 5 tap rows x 3 pair shifts x 8 chunks of the 64-channel line, N = 2 x 32
+    assert dc.packed_bytes(dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == 120 * 64 * 16
+    # fold order (c_in too wide for a 128-byte pixel pair): 5 chunks x 5 tap rows (+1 padding entry), N = 5 x 32
+    assert dc.packed_bytes(dc.geom(40, 32, 1, 5, 1, 2), dc.BF16) == 26 * 160 * 16
     # general order: 18 chunks x 9 taps in 3 groups of 6 chunks, 64 output channels
     assert dc.packed_bytes(dc.geom(144, 64, 1, 3, 1, 1), dc.BF16) == 3 * 54 * 64 * 16
     assert dc.packed_bytes(dc.geom(3, 32, 1, 3, 2, 1), dc.BF16) == 10 * 32 * 16
@@ -90,7 +93,8 @@ def test_kernel_name_query_follows_the_dispatch_rules():
     # small-channel stride-1 3x3: pair order, 5x5: fold order; wide or strided: general tensor-core kernel;
     # channel counts that are no multiple of 8: CUDA cores
     assert dc.conv_kernel_name(64, 56, 56, dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_pairrows"
-    assert dc.conv_kernel_name(128, 28, 28, dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_fold"
+    assert dc.conv_kernel_name(128, 28, 28, dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_pairrows"
+    assert dc.conv_kernel_name(128, 14, 14, dc.geom(40, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_fold"
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(24, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 14, 14, dc.geom(96, 576, 1, 1, 1, 0), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 224, 224, dc.geom(3, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_dense_bf16"
