@@ -20,8 +20,9 @@
 // (global reads of a warp are contiguous; the scatter into planes happens on the shared-memory
 // side; halo pixels are zero-filled).  A tiled TMA copy cannot produce this layout at speed: its
 // innermost box row would be 16 bytes, and one request per 16 bytes measured 27 us for a 19 MB
-// problem.  Weights: one 3-D TMA tile per (output-channel tile, channel group), resident for the
-// whole kernel when they fit.  Output: the epilogue converts to bf16 into a dense shared-memory
+// problem.  Weights: the packed layout in HBM is the operand layout, so a (channel group, output-
+// channel pass) tile is one contiguous bulk copy (cp.async.bulk; one per entry when the output
+// channels are cut into passes), resident for the whole kernel when it fits.  Output: the epilogue converts to bf16 into a dense shared-memory
 // tile and one bulk copy (cp.async.bulk shared -> global) writes it when the tile is contiguous
 // in global memory; otherwise 16-byte stores.
 //
@@ -88,7 +89,7 @@ __device__ __forceinline__ Tile decode_tile(const TcParams &p, int cur, int end)
 
 // ------------------------------------------------------------------------------------------ kernel
 __global__ void __launch_bounds__(kThreads, 1)
-k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcParams p,
+k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
           const __nv_bfloat16 *__restrict__ x, const float *__restrict__ bias,
           const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -113,7 +114,6 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
     for (int s = 0; s < p.stages; ++s) { mbar_init(&bar_full[s], kProducerThreads); mbar_init(&bar_empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&bar_accfull[a], 1); mbar_init(&bar_accempty[a], 128); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    prefetch_tensormap(&map_b);
   }
   if (warp == 4) {
     tmem_alloc(&tmem_base_s, (uint32_t)p.tmem_cols);
@@ -136,7 +136,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
   const int cta_end = (int)((long long)p.total_units * (blockIdx.x + 1) / gridDim.x);
 
   if (warp < 4) {
-    // ================================================================== producers (cp.async + TMA for weights)
+    // ================================================================== producers (cp.async, bulk copies for weights)
     const int ptid = threadIdx.x;
     const int row_pieces = p.wbox * p.pcs * p.cg;
     const int C2 = p.c_in * 2;
@@ -178,9 +178,23 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
           // a weight tile rides along on the same barrier as transaction bytes
           const bool load_b = !p.b_resident || !b_loaded;
           if (load_b) {
-            mbar_expect_tx(&bar_full[s], (uint32_t)p.b_stage_bytes);
-            tma_load_3d(smem_b + (size_t)(p.b_resident ? 0 : s) * p.b_stage_bytes, &map_b, &bar_full[s], 0,
-                        t.nt * p.n_tile, grp * p.e_pad);
+            // The packed weights are stored as the operand wants them ([entry][n_pad rows][8]): a
+            // group's tile is one contiguous bulk copy, or one per entry when the output channels
+            // are cut into passes.  (A tiled TMA load with this 16-byte inner box fetched 16 bytes
+            // per request and took microseconds.)
+            const uint32_t dst = smem_u32(smem_b + (size_t)(p.b_resident ? 0 : s) * p.b_stage_bytes);
+            const char *src = reinterpret_cast<const char *>(w_packed) + (size_t)grp * p.e_pad * p.ko.n_pad * 16;
+            if (p.n_tile == p.ko.n_pad) {
+              mbar_expect_tx(&bar_full[s], (uint32_t)p.b_stage_bytes);
+              bulk_load(dst, src, (uint32_t)p.b_stage_bytes, &bar_full[s]);
+            } else {
+              const int lo = t.nt * p.n_tile;
+              const int rows = (p.ko.n_pad - lo < p.n_tile) ? p.ko.n_pad - lo : p.n_tile;
+              mbar_expect_tx(&bar_full[s], (uint32_t)(p.e_pad * rows * 16));
+              for (int e = 0; e < p.e_pad; ++e)
+                bulk_load(dst + (uint32_t)(e * p.n_tile * 16), src + ((size_t)e * p.ko.n_pad + lo) * 16,
+                          (uint32_t)(rows * 16), &bar_full[s]);
+            }
             b_loaded = true;
           }
         }
@@ -354,22 +368,6 @@ k_conv_tc(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ TcP
 }
 
 // ------------------------------------------------------------------------------------------ host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void *ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
 int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -532,27 +530,13 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
   const int n_sm = sm_count();
   if (!tc_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
-  EncodeTiledFn encode = get_encode_fn();
-  if (!encode) return DC_ERR_CUDA;
-
-  CUtensorMap map_b;
-  {
-    cuuint64_t gdim[3] = {8, (cuuint64_t)p.ko.n_pad, (cuuint64_t)p.ng * p.e_pad};
-    cuuint64_t gstr[2] = {16, (cuuint64_t)p.ko.n_pad * 16};
-    cuuint32_t box[3] = {8, (cuuint32_t)p.n_tile, (cuuint32_t)p.e_pad};
-    cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(w_packed), gdim, gstr, box, es,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
-  }
   static bool attr_set = false;
   if (!attr_set) {
     DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     attr_set = true;
   }
   int grid = p.total_units < n_sm ? p.total_units : n_sm;
-  k_conv_tc<<<grid, kThreads, p.smem_bytes, stream>>>(map_b, p, (const __nv_bfloat16 *)x, bias,
+  k_conv_tc<<<grid, kThreads, p.smem_bytes, stream>>>(w_packed, p, (const __nv_bfloat16 *)x, bias,
                                                      (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                                      (DcWsHeader *)workspace);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
