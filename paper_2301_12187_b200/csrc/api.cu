@@ -28,6 +28,7 @@ extern "C" const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g
   if (dc_conv_pairrows_supported(n, h, w, g)) return "k_conv_tc_pairrows";
   if (dc_conv_fold_supported(n, h, w, g)) return "k_conv_tc_fold";
   if (dc_conv_tc_supported(n, h, w, g)) return "k_conv_tc";
+  if (dc_conv_smallcin_supported(n, h, w, g)) return "k_conv_smallcin_bf16";
   return "k_conv_dense_bf16";
 }
 

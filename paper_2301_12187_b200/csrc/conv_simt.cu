@@ -103,6 +103,115 @@ static inline int simt_blocks(long long total, int threads, int cap) {
   return (int)b;
 }
 
+// ----------------------------------------------------------------------------------------------
+// dense conv with very few input channels (the 3-channel stem), bf16, fp32 accumulate.
+// The reduction is only k*k*c_in long (27 for the stem), far too short and too ragged (6-byte
+// pixels) for the tensor-core staging, and the layer is bound by writing its output.  One CTA =
+// one output row segment of 128 pixels, one thread = one pixel x CO_T output channels:
+//   * the k input rows of the segment are staged in shared memory with coalesced loads (zeros
+//     outside the image), each thread then reads its k*k*c_in inputs from there;
+//   * weights sit in shared memory as fp32 [tap][c][o]; every thread of a warp reads the same
+//     address (a broadcast), four output channels per load;
+//   * a thread's CO_T channels are 2*CO_T contiguous bytes of the NHWC output: 16-byte stores.
+// ----------------------------------------------------------------------------------------------
+constexpr int kSmallCinMax = 4;
+constexpr int kSmallTile = 128;
+
+template <int CO_T>
+__global__ void __launch_bounds__(kSmallTile)
+k_conv_smallcin_bf16(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w,
+                     const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ residual,
+                     __nv_bfloat16 *__restrict__ y, int n, int h, int wd, int ho, int wo, dc_geom g, KOrder ko,
+                     int act, int xtiles) {
+  extern __shared__ __align__(16) unsigned char sm_raw[];
+  const int taps = g.k * g.k;
+  float *w_s = reinterpret_cast<float *>(sm_raw);                       // [taps][c_in][CO_T]
+  float *b_s = w_s + taps * g.c_in * CO_T;                              // [CO_T]
+  __nv_bfloat16 *x_s = reinterpret_cast<__nv_bfloat16 *>(b_s + CO_T);   // [k][span][c_in]
+  const int span = (kSmallTile - 1) * g.stride + g.k;                   // input pixels per staged row
+  const int tid = (int)threadIdx.x;
+  int bid = (int)blockIdx.x;
+  const int xt = bid % xtiles; bid /= xtiles;
+  const int Y = bid % ho, img = bid / ho;
+  const int X0 = xt * kSmallTile;
+  const int gx0 = X0 * g.stride - g.pad, gy0 = Y * g.stride - g.pad;
+  // stage the input rows (2-byte elements, contiguous in memory along a row)
+  const int row_elems = span * g.c_in;
+  for (int r = 0; r < g.k; ++r) {
+    const int gy = gy0 + r;
+    const __nv_bfloat16 *src = x + ((size_t)img * h + (gy < 0 ? 0 : gy)) * wd * g.c_in;
+    for (int e = tid; e < row_elems; e += kSmallTile) {
+      const int gx = gx0 + e / g.c_in;
+      const bool ok = gy >= 0 && gy < h && gx >= 0 && gx < wd;
+      x_s[r * row_elems + e] = ok ? src[(long long)gx0 * g.c_in + e] : __float2bfloat16_rn(0.f);
+    }
+  }
+  const int X = X0 + tid;
+  for (int o0 = 0; o0 < g.c_out; o0 += CO_T) {
+    __syncthreads();                              // x_s staged / previous pass done with w_s
+    for (int i = tid; i < taps * g.c_in * CO_T; i += kSmallTile) {
+      const int o = i % CO_T, c = (i / CO_T) % g.c_in, t = i / (CO_T * g.c_in);
+      const int u = t / g.k, v = t - u * g.k;
+      float wv = 0.f;
+      if (o0 + o < g.c_out) {
+        const int plane = dc_korder_encode(ko, c / 8, u, v);
+        wv = __bfloat162float(w[((size_t)plane * ko.n_pad + dc_korder_row(ko, v, o0 + o)) * 8 + (c & 7)]);
+      }
+      w_s[i] = wv;
+    }
+    if (tid < CO_T) b_s[tid] = (bias && o0 + tid < g.c_out) ? bias[o0 + tid] : 0.f;
+    __syncthreads();
+    if (X < wo) {
+      float acc[CO_T];
+#pragma unroll
+      for (int o = 0; o < CO_T; ++o) acc[o] = b_s[o];
+      const __nv_bfloat16 *xp = x_s + tid * g.stride * g.c_in;
+      const float *wp = w_s;
+      for (int u = 0; u < g.k; ++u, xp += row_elems - g.k * g.c_in) {
+        for (int vc = 0; vc < g.k * g.c_in; ++vc, ++xp, wp += CO_T) {
+          const float xv = __bfloat162float(*xp);
+#pragma unroll
+          for (int o = 0; o < CO_T; o += 4) {
+            const float4 w4 = *reinterpret_cast<const float4 *>(wp + o);
+            acc[o] = fmaf(xv, w4.x, acc[o]); acc[o + 1] = fmaf(xv, w4.y, acc[o + 1]);
+            acc[o + 2] = fmaf(xv, w4.z, acc[o + 2]); acc[o + 3] = fmaf(xv, w4.w, acc[o + 3]);
+          }
+        }
+      }
+      const size_t oi = (((size_t)img * ho + Y) * wo + X) * g.c_out + o0;
+#pragma unroll
+      for (int o = 0; o < CO_T; o += 8) {
+        if (o0 + o < g.c_out) {                   // c_out is a multiple of 8
+          if (residual) {
+            const uint4 rv = *reinterpret_cast<const uint4 *>(residual + oi + o);
+            const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 rf = __bfloat1622float2(rb[i]);
+              acc[o + 2 * i] += rf.x; acc[o + 2 * i + 1] += rf.y;
+            }
+          }
+          uint4 ov;
+          __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            ob[i] = __floats2bfloat162_rn(dc_act_apply(acc[o + 2 * i], act), dc_act_apply(acc[o + 2 * i + 1], act));
+          *reinterpret_cast<uint4 *>(y + oi + o) = ov;
+        }
+      }
+    }
+  }
+}
+
+static bool smallcin_ok(const dc_geom *g) {
+  return g->groups == 1 && g->c_in <= kSmallCinMax && g->c_out % 8 == 0 && g->k <= 5 && g->stride <= 2;
+}
+
+bool dc_conv_smallcin_supported(int n, int h, int w, const dc_geom *g) {
+  (void)n; (void)h; (void)w;
+  return smallcin_ok(g);
+}
+
 dc_status dc_launch_conv_simt(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                               const float *bias, dc_act act, const void *residual, void *y,
                               dc_dtype dtype, cudaStream_t stream) {
@@ -115,6 +224,16 @@ dc_status dc_launch_conv_simt(const void *x, int n, int h, int w, const dc_geom 
   } else {
     KOrder ko;
     dc_korder_init(&ko, g);
+    if (smallcin_ok(g) && (long long)n * ho * dc_div_up(wo, kSmallTile) < (1ll << 31)) {
+      constexpr int CO_T = 32;
+      const int xtiles = dc_div_up(wo, kSmallTile);
+      const int span = (kSmallTile - 1) * g->stride + g->k;
+      const size_t smem = (size_t)(g->k * g->k * g->c_in * CO_T + CO_T) * 4 + (size_t)g->k * span * g->c_in * 2;
+      k_conv_smallcin_bf16<CO_T><<<(unsigned)((long long)n * ho * xtiles), kSmallTile, smem, stream>>>(
+          (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_packed, bias, (const __nv_bfloat16 *)residual,
+          (__nv_bfloat16 *)y, n, h, w, ho, wo, *g, ko, (int)act, xtiles);
+      return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+    }
     long long total = (long long)n * ho * wo * g->c_out;
     k_conv_dense_bf16<<<simt_blocks(total, 128, 148 * 64), 128, 0, stream>>>(
         (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_packed, bias, (const __nv_bfloat16 *)residual,
