@@ -106,8 +106,8 @@ static inline int simt_blocks(long long total, int threads, int cap) {
 // ----------------------------------------------------------------------------------------------
 // dense conv with very few input channels (the 3-channel stem), bf16, fp32 accumulate.
 // The reduction is only k*k*c_in long (27 for the stem), far too short and too ragged (6-byte
-// pixels) for the tensor-core staging, and the layer is bound by writing its output.  One CTA =
-// one output row segment of 128 pixels, one thread = one pixel x CO_T output channels:
+// pixels) for the tensor-core staging, and the layer is bound by writing its output.  Persistent
+// CTAs walk output row segments of 128 pixels; one thread = one pixel x CO_T output channels:
 //   * the k input rows of the segment are staged in shared memory with coalesced loads (zeros
 //     outside the image), each thread then reads its k*k*c_in inputs from there;
 //   * weights sit in shared memory as fp32 [tap][c][o]; every thread of a warp reads the same
@@ -122,45 +122,49 @@ __global__ void __launch_bounds__(kSmallTile)
 k_conv_smallcin_bf16(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w,
                      const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ residual,
                      __nv_bfloat16 *__restrict__ y, int n, int h, int wd, int ho, int wo, dc_geom g, KOrder ko,
-                     int act, int xtiles) {
+                     int act, int xtiles, int o0) {
   extern __shared__ __align__(16) unsigned char sm_raw[];
   const int taps = g.k * g.k;
   float *w_s = reinterpret_cast<float *>(sm_raw);                       // [taps][c_in][CO_T]
   float *b_s = w_s + taps * g.c_in * CO_T;                              // [CO_T]
   __nv_bfloat16 *x_s = reinterpret_cast<__nv_bfloat16 *>(b_s + CO_T);   // [k][span][c_in]
   const int span = (kSmallTile - 1) * g.stride + g.k;                   // input pixels per staged row
-  const int tid = (int)threadIdx.x;
-  int bid = (int)blockIdx.x;
-  const int xt = bid % xtiles; bid /= xtiles;
-  const int Y = bid % ho, img = bid / ho;
-  const int X0 = xt * kSmallTile;
-  const int gx0 = X0 * g.stride - g.pad, gy0 = Y * g.stride - g.pad;
-  // stage the input rows (2-byte elements, contiguous in memory along a row)
   const int row_elems = span * g.c_in;
-  for (int r = 0; r < g.k; ++r) {
-    const int gy = gy0 + r;
-    const __nv_bfloat16 *src = x + ((size_t)img * h + (gy < 0 ? 0 : gy)) * wd * g.c_in;
-    for (int e = tid; e < row_elems; e += kSmallTile) {
-      const int gx = gx0 + e / g.c_in;
-      const bool ok = gy >= 0 && gy < h && gx >= 0 && gx < wd;
-      x_s[r * row_elems + e] = ok ? src[(long long)gx0 * g.c_in + e] : __float2bfloat16_rn(0.f);
+  const int tid = (int)threadIdx.x;
+  // weights and bias of this pass's CO_T output channels: once per CTA (CTAs are persistent)
+  for (int i = tid; i < taps * g.c_in * CO_T; i += kSmallTile) {
+    const int o = i % CO_T, c = (i / CO_T) % g.c_in, t = i / (CO_T * g.c_in);
+    const int u = t / g.k, v = t - u * g.k;
+    float wv = 0.f;
+    if (o0 + o < g.c_out) {
+      const int plane = dc_korder_encode(ko, c / 8, u, v);
+      wv = __bfloat162float(w[((size_t)plane * ko.n_pad + dc_korder_row(ko, v, o0 + o)) * 8 + (c & 7)]);
     }
+    w_s[i] = wv;
   }
-  const int X = X0 + tid;
-  for (int o0 = 0; o0 < g.c_out; o0 += CO_T) {
-    __syncthreads();                              // x_s staged / previous pass done with w_s
-    for (int i = tid; i < taps * g.c_in * CO_T; i += kSmallTile) {
-      const int o = i % CO_T, c = (i / CO_T) % g.c_in, t = i / (CO_T * g.c_in);
-      const int u = t / g.k, v = t - u * g.k;
-      float wv = 0.f;
-      if (o0 + o < g.c_out) {
-        const int plane = dc_korder_encode(ko, c / 8, u, v);
-        wv = __bfloat162float(w[((size_t)plane * ko.n_pad + dc_korder_row(ko, v, o0 + o)) * 8 + (c & 7)]);
+  if (tid < CO_T) b_s[tid] = (bias && o0 + tid < g.c_out) ? bias[o0 + tid] : 0.f;
+  const long long total = (long long)n * ho * xtiles;
+  for (long long tile = blockIdx.x; tile < total; tile += gridDim.x) {
+    const int xt = (int)(tile % xtiles);
+    const long long rowi = tile / xtiles;
+    const int Y = (int)(rowi % ho), img = (int)(rowi / ho);
+    const int X0 = xt * kSmallTile;
+    const int gx0 = X0 * g.stride - g.pad, gy0 = Y * g.stride - g.pad;
+    __syncthreads();                              // weights staged / previous tile done with x_s
+    // stage the k input rows of the segment: thread = pixel, contiguous along the row
+    for (int r = 0; r < g.k; ++r) {
+      const int gy = gy0 + r;
+      const bool rok = gy >= 0 && gy < h;
+      const __nv_bfloat16 *src = x + (((size_t)img * h + (rok ? gy : 0)) * wd) * g.c_in;
+      for (int px = tid; px < span; px += kSmallTile) {
+        const int gx = gx0 + px;
+        const bool ok = rok && gx >= 0 && gx < wd;
+        for (int c = 0; c < g.c_in; ++c)
+          x_s[r * row_elems + px * g.c_in + c] = ok ? src[(size_t)gx * g.c_in + c] : __float2bfloat16_rn(0.f);
       }
-      w_s[i] = wv;
     }
-    if (tid < CO_T) b_s[tid] = (bias && o0 + tid < g.c_out) ? bias[o0 + tid] : 0.f;
     __syncthreads();
+    const int X = X0 + tid;
     if (X < wo) {
       float acc[CO_T];
 #pragma unroll
@@ -224,14 +228,17 @@ dc_status dc_launch_conv_simt(const void *x, int n, int h, int w, const dc_geom 
   } else {
     KOrder ko;
     dc_korder_init(&ko, g);
-    if (smallcin_ok(g) && (long long)n * ho * dc_div_up(wo, kSmallTile) < (1ll << 31)) {
+    if (smallcin_ok(g)) {
       constexpr int CO_T = 32;
       const int xtiles = dc_div_up(wo, kSmallTile);
       const int span = (kSmallTile - 1) * g->stride + g->k;
       const size_t smem = (size_t)(g->k * g->k * g->c_in * CO_T + CO_T) * 4 + (size_t)g->k * span * g->c_in * 2;
-      k_conv_smallcin_bf16<CO_T><<<(unsigned)((long long)n * ho * xtiles), kSmallTile, smem, stream>>>(
-          (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_packed, bias, (const __nv_bfloat16 *)residual,
-          (__nv_bfloat16 *)y, n, h, w, ho, wo, *g, ko, (int)act, xtiles);
+      const long long tiles = (long long)n * ho * xtiles;
+      const int grid = (int)(tiles < 148 * 8 ? tiles : 148 * 8);      // persistent CTAs, 8 per SM
+      for (int o0 = 0; o0 < g->c_out; o0 += CO_T)                      // one pass per 32 output channels
+        k_conv_smallcin_bf16<CO_T><<<grid, kSmallTile, smem, stream>>>(
+            (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_packed, bias, (const __nv_bfloat16 *)residual,
+            (__nv_bfloat16 *)y, n, h, w, ho, wo, *g, ko, (int)act, xtiles, o0);
       return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
     }
     long long total = (long long)n * ho * wo * g->c_out;
