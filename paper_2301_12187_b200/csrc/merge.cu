@@ -43,52 +43,115 @@ struct Piece {
   const float *w;
   const float *b;
   int c_in, c_out, k, stride, diag;
+  int ident;   // 1: the piece stands for w + I (identity kernel of a skip addition: +1 on the centre
+               // tap of every (c, c) pair), added where the weights are read instead of by a launch
 };
+
+__device__ __forceinline__ float piece_dense_at(const Piece &p, int o, int i, int u, int v) {
+  float w = p.w[(((size_t)o * p.c_in + i) * p.k + u) * p.k + v];
+  const int ctr = (p.k - 1) / 2;
+  if (p.ident && o == i && u == ctr && v == ctr) w += 1.f;
+  return w;
+}
+__device__ __forceinline__ float piece_diag_at(const Piece &p, int c, int u, int v) {
+  float w = p.w[((size_t)c * p.k + u) * p.k + v];
+  const int ctr = (p.k - 1) / 2;
+  if (p.ident && u == ctr && v == ctr) w += 1.f;
+  return w;
+}
+
+// b'[o] = b2[o] + sum_c (sum_taps W2[o,c]) * b1[c]; one warp per output channel.  Runs in the
+// tail blocks of the composition kernels (block index `blk` counted from the first bias block).
+__device__ __forceinline__ void compose_bias_block(const Piece &first, const Piece &second, float *out, int blk) {
+  const int warp = (blk * (int)blockDim.x + (int)threadIdx.x) / 32, lane = threadIdx.x % 32;
+  if (warp >= second.c_out) return;
+  const int o = warp, t2 = second.k * second.k;
+  float acc = 0.f;
+  if (second.diag) {
+    if (lane == 0) {
+      float ws = second.ident ? 1.f : 0.f;
+      for (int t = 0; t < t2; ++t) ws += second.w[(size_t)o * t2 + t];
+      acc = ws * first.b[o];
+    }
+  } else {
+    for (int c = lane; c < second.c_in; c += 32) {
+      float ws = (second.ident && c == o) ? 1.f : 0.f;
+      for (int t = 0; t < t2; ++t) ws += second.w[((size_t)o * second.c_in + c) * t2 + t];
+      acc = fmaf(ws, first.b[c], acc);
+    }
+  }
+  for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+  if (lane == 0) out[o] = second.b[o] + acc;
+}
+static int bias_blocks(int c_out, int threads) { return dc_div_up(c_out * 32, threads); }
 
 // dense (second) o dense (first):  out[o][j] = sum_r A[o][r] * B[r][j] with
 //   r = (c, u2, v2),  j = (i, u', v'),  A = W2 as stored,
 //   B[r][j] = W1[c][i][u' - s1*u2][v' - s1*v2]  (0 when the tap falls outside W1).
-// 64x64 output tile, 16-deep slices, 256 threads, 4x4 outputs per thread.
-__global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece second, float *out, int kk) {
-  __shared__ float As[16][64 + 4];
-  __shared__ float Bs[16][64 + 4];
-  const int k1 = first.k, k2 = second.k, s1 = first.stride;
+// 64x64 output tile, 256 threads, 4x4 outputs per thread.  The reduction is staged in slices of up
+// to kDdSlice rows: the merges are small and latency-bound, so a slice's loads (dozens per
+// thread, all independent) are issued in one go and cost one round trip to L2, where 16-deep
+// slices cost one per 16 rows.  A thread gathers one column j of B, so (i, u', v') is decoded once.
+// Blocks [0, gx*gy) are the tiles (x fastest); the blocks after them compute the bias.
+constexpr int kDdSlice = 256;
+constexpr int kDdPitch = 64 + 4;
+__global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece second, float *out, float *b_out,
+                                                             int kk, int gx, int gy, int slice) {
+  extern __shared__ __align__(16) float dd_smem[];
+  float *As = dd_smem;                       // [slice][kDdPitch]
+  float *Bs = dd_smem + slice * kDdPitch;    // [slice][kDdPitch]
+  if ((int)blockIdx.x >= gx * gy) {
+    compose_bias_block(first, second, b_out, (int)blockIdx.x - gx * gy);
+    return;
+  }
+  const int ctr1 = (first.k - 1) / 2, ctr2 = (second.k - 1) / 2;
+  const int k1 = first.k, k2 = second.k, s1 = first.stride, t2sz = k2 * k2;
   const int c0 = first.c_in, c1 = first.c_out, c2 = second.c_out;
-  const int R = c1 * k2 * k2, J = c0 * kk * kk;
-  const int o0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+  const int R = c1 * t2sz, J = c0 * kk * kk;
+  const int o0 = ((int)blockIdx.x / gx) * 64, j0 = ((int)blockIdx.x % gx) * 64;
   const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+  // this thread's column of B and row phase of A
+  const int jj = t & 63, j = j0 + jj;
+  const int bi = j / (kk * kk), btp = j - bi * kk * kk, bup = btp / kk, bvp = btp - bup * kk;
+  const int arr = t & 15, arow = t >> 4;     // A: rows arow + 16q of the tile, slice row arr + 16p
   float acc[4][4] = {};
-  for (int r0 = 0; r0 < R; r0 += 16) {
+  for (int r0 = 0; r0 < R; r0 += slice) {
+    const int rows = R - r0 < slice ? R - r0 : slice;
+    // A[o][r]: consecutive threads read consecutive r of one output channel
+    for (int rr = arr; rr < rows; rr += 16) {
+      const int r = r0 + rr;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      int e = t + 256 * q;
-      int row = e / 16, rr = e % 16;
-      int o = o0 + row, r = r0 + rr;
-      As[rr][row] = (o < c2 && r < R) ? second.w[(size_t)o * R + r] : 0.f;
-    }
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      int e = t + 256 * q;
-      int rr = e / 64, jj = e % 64;
-      int r = r0 + rr, j = j0 + jj;
-      float v = 0.f;
-      if (r < R && j < J) {
-        int c = r / (k2 * k2), t2 = r - c * k2 * k2;
-        int u2 = t2 / k2, v2 = t2 - u2 * k2;
-        int i = j / (kk * kk), tp = j - i * kk * kk;
-        int up = tp / kk, vp = tp - up * kk;
-        int u1 = up - s1 * u2, v1 = vp - s1 * v2;
-        if (u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1)
-          v = first.w[(((size_t)c * c0 + i) * k1 + u1) * k1 + v1];
+      for (int q = 0; q < 4; ++q) {
+        const int row = arow + 16 * q, o = o0 + row;
+        float av = 0.f;
+        if (o < c2) {
+          av = second.w[(size_t)o * R + r];
+          if (second.ident && r == (o * k2 + ctr2) * k2 + ctr2) av += 1.f;
+        }
+        As[rr * kDdPitch + row] = av;
       }
-      Bs[rr][jj] = v;
+    }
+    // B[r][j]: consecutive threads read consecutive j (elements of W1 next to each other)
+    for (int rr = t >> 6; rr < rows; rr += 4) {
+      const int r = r0 + rr;
+      float v = 0.f;
+      if (j < J) {
+        const int c = r / t2sz, t2 = r - c * t2sz;
+        const int u2 = t2 / k2, v2 = t2 - u2 * k2;
+        const int u1 = bup - s1 * u2, v1 = bvp - s1 * v2;
+        if (u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1) {
+          v = first.w[(((size_t)c * c0 + bi) * k1 + u1) * k1 + v1];
+          if (first.ident && c == bi && u1 == ctr1 && v1 == ctr1) v += 1.f;
+        }
+      }
+      Bs[rr * kDdPitch + jj] = v;
     }
     __syncthreads();
-#pragma unroll
-    for (int rr = 0; rr < 16; ++rr) {
-      float a[4], b[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) { a[q] = As[rr][ty * 4 + q]; b[q] = Bs[rr][tx * 4 + q]; }
+#pragma unroll 4
+    for (int rr = 0; rr < rows; ++rr) {
+      const float4 a4 = *reinterpret_cast<const float4 *>(As + rr * kDdPitch + ty * 4);
+      const float4 b4 = *reinterpret_cast<const float4 *>(Bs + rr * kDdPitch + tx * 4);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
       for (int p = 0; p < 4; ++p)
 #pragma unroll
@@ -100,8 +163,8 @@ __global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece 
   for (int p = 0; p < 4; ++p)
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      int o = o0 + ty * 4 + p, j = j0 + tx * 4 + q;
-      if (o < c2 && j < J) out[(size_t)o * J + j] = acc[p][q];
+      int o = o0 + ty * 4 + p, jo = j0 + tx * 4 + q;
+      if (o < c2 && jo < J) out[(size_t)o * J + jo] = acc[p][q];
     }
 }
 
@@ -109,9 +172,14 @@ __global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece 
 //   second diag, first dense: out[o,i,u',v'] = sum_{u2,v2} W2[o,u2,v2] * W1[o,i,u1,v1]
 //   second dense, first diag: out[o,i,u',v'] = sum_{u2,v2} W2[o,i,u2,v2] * W1[i,u1,v1]
 //   both diag:                out[c,u',v']   = sum_{u2,v2} W2[c,u2,v2]   * W1[c,u1,v1]
-__global__ void k_compose_diag(Piece first, Piece second, float *out, int kk, int total) {
+// Blocks [0, nb) walk the elements; the blocks after them compute the bias.
+__global__ void k_compose_diag(Piece first, Piece second, float *out, float *b_out, int kk, int total, int nb) {
+  if ((int)blockIdx.x >= nb) {
+    compose_bias_block(first, second, b_out, (int)blockIdx.x - nb);
+    return;
+  }
   const int k1 = first.k, k2 = second.k, s1 = first.stride;
-  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += nb * blockDim.x) {
     int vp = idx % kk, up = (idx / kk) % kk, rest = idx / (kk * kk);
     int o, i;
     if (first.diag && second.diag) { o = rest; i = rest; }
@@ -123,59 +191,13 @@ __global__ void k_compose_diag(Piece first, Piece second, float *out, int kk, in
       for (int v2 = 0; v2 < k2; ++v2) {
         int v1 = vp - s1 * v2;
         if (v1 < 0 || v1 >= k1) continue;
-        float w2 = second.diag ? second.w[((size_t)o * k2 + u2) * k2 + v2]
-                               : second.w[(((size_t)o * second.c_in + i) * k2 + u2) * k2 + v2];
-        float w1 = first.diag ? first.w[((size_t)i * k1 + u1) * k1 + v1]
-                              : first.w[(((size_t)o * first.c_in + i) * k1 + u1) * k1 + v1];
+        float w2 = second.diag ? piece_diag_at(second, o, u2, v2) : piece_dense_at(second, o, i, u2, v2);
+        float w1 = first.diag ? piece_diag_at(first, i, u1, v1) : piece_dense_at(first, o, i, u1, v1);
         acc = fmaf(w2, w1, acc);
       }
     }
     out[idx] = acc;
   }
-}
-
-// b'[o] = b2[o] + sum_c (sum_taps W2[o,c]) * b1[c]; one warp per output channel.
-__global__ void k_compose_bias(Piece first, Piece second, float *out) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
-  if (warp >= second.c_out) return;
-  const int o = warp, t2 = second.k * second.k;
-  float acc = 0.f;
-  if (second.diag) {
-    if (lane == 0) {
-      float ws = 0.f;
-      for (int t = 0; t < t2; ++t) ws += second.w[(size_t)o * t2 + t];
-      acc = ws * first.b[o];
-    }
-  } else {
-    for (int c = lane; c < second.c_in; c += 32) {
-      float ws = 0.f;
-      for (int t = 0; t < t2; ++t) ws += second.w[((size_t)o * second.c_in + c) * t2 + t];
-      acc = fmaf(ws, first.b[c], acc);
-    }
-  }
-  for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
-  if (lane == 0) out[o] = second.b[o] + acc;
-}
-
-// identity kernel of a skip addition: +1 on the centre tap of every (c, c) pair
-__global__ void k_add_identity(float *w, int c, int k, int diag) {
-  int o = blockIdx.x * blockDim.x + threadIdx.x;
-  if (o >= c) return;
-  int ctr = (k - 1) / 2;
-  size_t idx = diag ? ((size_t)o * k + ctr) * k + ctr : (((size_t)o * c + o) * k + ctr) * k + ctr;
-  w[idx] += 1.f;
-}
-
-__global__ void k_lift_diag(const float *wd, float *w, int c, int k) {
-  int total = c * c * k * k;
-  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-    int t = idx % (k * k), i = (idx / (k * k)) % c, o = idx / (k * k * c);
-    w[idx] = (o == i) ? wd[(size_t)o * k * k + t] : 0.f;
-  }
-}
-
-__global__ void k_copy(const float *src, float *dst, int n) {
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) dst[i] = src[i];
 }
 
 // fp32 [o][i][u][v] -> fp32 [u][v][i][o]
@@ -222,6 +244,76 @@ __global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrde
       if (o < c_out && c < ko.c_in) v = w[(((size_t)o * ko.c_in + c) * ko.k + r) * ko.k + s];
     }
     out[idx] = __float2bfloat16_rn(v);
+  }
+}
+
+// Element (o, i, tap t) of the finished run as a dense kernel: a diagonal result is lifted, a
+// pending identity is added.
+__device__ __forceinline__ float merged_at(const Piece &p, int o, int i, int t) {
+  const int kk = p.k * p.k, ctr = ((p.k - 1) / 2) * (p.k + 1);
+  float w;
+  if (p.diag) w = (o == i) ? p.w[(size_t)o * kk + t] : 0.f;
+  else w = p.w[((size_t)o * p.c_in + i) * kk + t];
+  if (p.ident && o == i && t == ctr) w += 1.f;
+  return w;
+}
+
+// Last launch of a merge: writes the dense fp32 kernel (blocks [0, nb_w)), the bias (block nb_w)
+// and, when asked for, the packed copy for the forward kernels (blocks after that; mode 1: fp32
+// [u][v][i][o], mode 2: bf16 chunk planes in the K order of KOrder), all straight from the
+// accumulated piece.
+__global__ void k_deliver(Piece acc, float *w_merged, float *b_merged, void *packed, int mode, KOrder ko,
+                          int nb_w, int nb_p) {
+  const int c_out = acc.c_out, c_in = acc.c_in, kk = acc.k * acc.k;
+  int blk = (int)blockIdx.x;
+  if (blk < nb_w) {
+    const int total = c_out * c_in * kk;
+    for (int idx = blk * blockDim.x + threadIdx.x; idx < total; idx += nb_w * blockDim.x) {
+      const int t = idx % kk, i = (idx / kk) % c_in, o = idx / (kk * c_in);
+      w_merged[idx] = merged_at(acc, o, i, t);
+    }
+    return;
+  }
+  blk -= nb_w;
+  if (blk == 0) {
+    for (int o = threadIdx.x; o < c_out; o += blockDim.x) b_merged[o] = acc.b[o];
+    return;
+  }
+  blk -= 1;
+  if (mode == 1) {
+    float *out = reinterpret_cast<float *>(packed);
+    const int total = c_out * c_in * kk;
+    for (int idx = blk * blockDim.x + threadIdx.x; idx < total; idx += nb_p * blockDim.x) {
+      const int o = idx % c_out, i = (idx / c_out) % c_in, t = idx / (c_out * c_in);
+      out[idx] = merged_at(acc, o, i, t);
+    }
+  } else if (mode == 2) {
+    __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(packed);
+    const int total = ko.ng * ko.e_pad * ko.n_pad * 8;
+    for (int idx = blk * blockDim.x + threadIdx.x; idx < total; idx += nb_p * blockDim.x) {
+      int c8 = idx % 8, o = (idx / 8) % ko.n_pad, plane = idx / (8 * ko.n_pad);
+      int grp = plane / ko.e_pad, e = plane - grp * ko.e_pad;
+      int pc, ccg, r, sx;
+      float v = 0.f;
+      if (dc_korder_decode(ko, e, &pc, &ccg, &r, &sx)) {
+        if (ko.fold) {
+          sx = o / ko.co8;
+          o -= sx * ko.co8;
+          if (sx >= ko.k) o = c_out;
+        } else if (ko.pair == 2) {
+          const int elem = ccg * 8 + c8, ipx = elem / ko.c_in;
+          const int px = o / ko.co8;
+          o -= px * ko.co8;
+          sx = 2 * sx + ipx - px;
+          ccg = 0;
+          c8 = elem - ipx * ko.c_in;
+          if (px >= 2 || sx < 0 || sx >= ko.k) o = c_out;
+        }
+        const int c = (grp * ko.cg + ccg) * 8 + c8;
+        if (o < c_out && c < ko.c_in) v = merged_at(acc, o, c, r * ko.k + sx);
+      }
+      out[idx] = __float2bfloat16_rn(v);
+    }
   }
 }
 
@@ -318,18 +410,29 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
   out.k = first.k + (second.k - 1) * first.stride;
   out.stride = first.stride * second.stride;
   out.diag = first.diag && second.diag;
+  out.ident = 0;
   size_t elems = piece_elems(out.c_in, out.c_out, out.k, out.diag);
   float *w = bump.take(elems);
   float *b = bump.take(out.c_out);
   out.w = w; out.b = b;
   if (go) {
+    const int nbias = bias_blocks(out.c_out, 256);
     if (!first.diag && !second.diag) {
-      dim3 grid(dc_div_up(out.c_in * out.k * out.k, 64), dc_div_up(out.c_out, 64));
-      k_compose_dense_dense<<<grid, 256, 0, st>>>(first, second, w, out.k);
+      const int gx = dc_div_up(out.c_in * out.k * out.k, 64), gy = dc_div_up(out.c_out, 64);
+      const int R = first.c_out * second.k * second.k;
+      const int slice = R < kDdSlice ? (int)dc_round_up((size_t)R, 16) : kDdSlice;
+      const size_t smem = (size_t)2 * slice * kDdPitch * sizeof(float);
+      static bool attr_set = false;
+      if (!attr_set) {
+        cudaFuncSetAttribute(k_compose_dense_dense, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             2 * kDdSlice * kDdPitch * (int)sizeof(float));
+        attr_set = true;
+      }
+      k_compose_dense_dense<<<gx * gy + nbias, 256, smem, st>>>(first, second, w, b, out.k, gx, gy, slice);
     } else {
-      k_compose_diag<<<blocks_for(elems, 256), 256, 0, st>>>(first, second, w, out.k, (int)elems);
+      const int nb = blocks_for(elems, 256);
+      k_compose_diag<<<nb + nbias, 256, 0, st>>>(first, second, w, b, out.k, (int)elems, nb);
     }
-    k_compose_bias<<<dc_div_up(out.c_out * 32, 128), 128, 0, st>>>(first, second, b);
   }
   return out;
 }
@@ -362,7 +465,7 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
       t.w_out[j] = w; t.b_out[j] = b;
       t.c_out[j] = L.c_out; t.per_out[j] = (int)(elems / L.c_out);
       if (elems > max_total) max_total = elems;
-      folded[l0 + j] = Piece{w, b, L.c_in, L.c_out, L.k, L.stride, diag};
+      folded[l0 + j] = Piece{w, b, L.c_in, L.c_out, L.k, L.stride, diag, 0};
     }
     if (go) {
       int bx = blocks_for(max_total, 256);
@@ -384,9 +487,7 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
     } else {
       piece = folded[res[gi].first];
       for (int j = res[gi].first + 1; j <= res[gi].last; ++j) piece = compose(piece, folded[j], bump, go, st);
-      if (go)
-        k_add_identity<<<dc_div_up(piece.c_out, 128), 128, 0, st>>>(const_cast<float *>(piece.w), piece.c_out,
-                                                                   piece.k, piece.diag);
+      piece.ident = 1;          // f(x) + x: the identity kernel rides along as a flag
       i = res[gi].last + 1;
     }
     if (!have) { acc = piece; have = true; }
@@ -395,15 +496,19 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
   if (need) *need = bump.off + 256;
   if (!go) return DC_OK;
 
-  // 3. deliver: dense fp32 result, bias, optional packed copy
+  // 3. deliver: dense fp32 result, bias, optional packed copy, in one launch
   size_t elems = (size_t)mg.c_out * mg.c_in * mg.k * mg.k;
-  if (acc.diag) k_lift_diag<<<blocks_for(elems, 256), 256, 0, st>>>(acc.w, w_merged, mg.c_out, mg.k);
-  else k_copy<<<blocks_for(elems, 256), 256, 0, st>>>(acc.w, w_merged, (int)elems);
-  k_copy<<<1, 256, 0, st>>>(acc.b, b_merged, mg.c_out);
+  KOrder ko;
+  dc_korder_init(&ko, &mg);
+  int mode = 0;
+  size_t p_elems = 0;
   if (w_packed) {
-    dc_status ps = dc_pack_weights(w_merged, &mg, packed_dtype, w_packed, (dc_stream)st);
-    if (ps != DC_OK) return ps;
+    mode = packed_dtype == DC_F32 ? 1 : 2;
+    p_elems = mode == 1 ? elems : (size_t)ko.ng * ko.e_pad * ko.n_pad * 8;
+    if (!dc_aligned16(w_packed)) return DC_ERR_ALIGNMENT;
   }
+  const int nb_w = blocks_for(elems, 256), nb_p = mode ? blocks_for(p_elems, 256) : 0;
+  k_deliver<<<nb_w + 1 + nb_p, 256, 0, st>>>(acc, w_merged, b_merged, w_packed, mode, ko, nb_w, nb_p);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
 
