@@ -168,6 +168,70 @@ __global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece 
     }
 }
 
+// dense o dense for small results (the usual case: a merged kernel has a few thousand elements):
+// 8 x 32 output tile, one output per thread, so that even a 24 x 216 result spreads over 21 CTAs;
+// operands staged in shared memory a slice of up to kDdSmallSlice reduction rows at a time, all of
+// a slice's loads in flight together.  Same reduction order (c, u2, v2) as the large-tile kernel.
+// Blocks [0, gx*gy) are the tiles (x fastest); the blocks after them compute the bias.
+constexpr int kDdSmallSlice = 256;
+__global__ void __launch_bounds__(256) k_compose_dd_small(Piece first, Piece second, float *out, float *b_out,
+                                                          int kk, int gx, int gy) {
+  __shared__ float As[kDdSmallSlice][8];
+  __shared__ float Bs[kDdSmallSlice][32];
+  __shared__ unsigned char tap_u[64], tap_v[64];     // (u2, v2) of tap t2 of the second kernel
+  if ((int)blockIdx.x >= gx * gy) {
+    compose_bias_block(first, second, b_out, (int)blockIdx.x - gx * gy);
+    return;
+  }
+  const int ctr1 = (first.k - 1) / 2, ctr2 = (second.k - 1) / 2;
+  const int k1 = first.k, k2 = second.k, s1 = first.stride, t2sz = k2 * k2;
+  const int c0 = first.c_in, c1 = first.c_out, c2 = second.c_out;
+  const int R = c1 * t2sz, J = c0 * kk * kk;
+  const int o0 = ((int)blockIdx.x / gx) * 8, j0 = ((int)blockIdx.x % gx) * 32;
+  const int t = threadIdx.x, ol = t >> 5, jl = t & 31;
+  if (t < t2sz) { tap_u[t] = (unsigned char)(t / k2); tap_v[t] = (unsigned char)(t % k2); }
+  __syncthreads();
+  const int j = j0 + jl, o = o0 + ol;
+  const int bi = j / (kk * kk), btp = j - bi * kk * kk, bup = btp / kk, bvp = btp - bup * kk;
+  float acc = 0.f;
+  for (int r0 = 0; r0 < R; r0 += kDdSmallSlice) {
+    const int rows = R - r0 < kDdSmallSlice ? R - r0 : kDdSmallSlice;
+    // A[o][r]: a warp reads 32 consecutive r of one output channel
+    for (int rr = jl; rr < rows; rr += 32) {
+      float av = 0.f;
+      if (o < c2) {
+        const int r = r0 + rr;
+        av = second.w[(size_t)o * R + r];
+        if (second.ident && r == (o * k2 + ctr2) * k2 + ctr2) av += 1.f;
+      }
+      As[rr][ol] = av;
+    }
+    // B[r][j]: a warp reads one row r, 32 consecutive j; (c, t2) of the row advance by 8 rows a step
+    {
+      int r = r0 + ol;
+      int c = r / t2sz, t2 = r - c * t2sz;
+      for (int rr = ol; rr < rows; rr += 8) {
+        float v = 0.f;
+        if (j < J) {
+          const int u1 = bup - s1 * tap_u[t2], v1 = bvp - s1 * tap_v[t2];
+          if (u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1) {
+            v = first.w[(((size_t)c * c0 + bi) * k1 + u1) * k1 + v1];
+            if (first.ident && c == bi && u1 == ctr1 && v1 == ctr1) v += 1.f;
+          }
+        }
+        Bs[rr][jl] = v;
+        t2 += 8;
+        while (t2 >= t2sz) { t2 -= t2sz; ++c; }
+      }
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int rr = 0; rr < rows; ++rr) acc = fmaf(As[rr][ol], Bs[rr][jl], acc);
+    __syncthreads();
+  }
+  if (o < c2 && j < J) out[(size_t)o * J + j] = acc;
+}
+
 // Compositions in which at least one operand is diagonal: one thread per output element.
 //   second diag, first dense: out[o,i,u',v'] = sum_{u2,v2} W2[o,u2,v2] * W1[o,i,u1,v1]
 //   second dense, first diag: out[o,i,u',v'] = sum_{u2,v2} W2[o,i,u2,v2] * W1[i,u1,v1]
@@ -417,7 +481,10 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
   out.w = w; out.b = b;
   if (go) {
     const int nbias = bias_blocks(out.c_out, 256);
-    if (!first.diag && !second.diag) {
+    if (!first.diag && !second.diag && elems <= (size_t)80000 && second.k <= 7) {
+      const int gx = dc_div_up(out.c_in * out.k * out.k, 32), gy = dc_div_up(out.c_out, 8);
+      k_compose_dd_small<<<gx * gy + nbias, 256, 0, st>>>(first, second, w, b, out.k, gx, gy);
+    } else if (!first.diag && !second.diag) {
       const int gx = dc_div_up(out.c_in * out.k * out.k, 64), gy = dc_div_up(out.c_out, 64);
       const int R = first.c_out * second.k * second.k;
       const int slice = R < kDdSlice ? (int)dc_round_up((size_t)R, 16) : kDdSlice;
