@@ -481,7 +481,7 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
   out.w = w; out.b = b;
   if (go) {
     const int nbias = bias_blocks(out.c_out, 256);
-    if (!first.diag && !second.diag && elems <= (size_t)80000 && second.k <= 7) {
+    if (!first.diag && !second.diag && elems <= (size_t)200000 && second.k <= 7) {
       const int gx = dc_div_up(out.c_in * out.k * out.k, 32), gy = dc_div_up(out.c_out, 8);
       k_compose_dd_small<<<gx * gy + nbias, 256, 0, st>>>(first, second, w, b, out.k, gx, gy);
     } else if (!first.diag && !second.diag) {
