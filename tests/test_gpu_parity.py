@@ -192,6 +192,44 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     assert O.rel_l2(nchw(y), ref) <= TOL_BF16
 
 
+# One case per branch of the forward kernels: the expected kernel is asserted, so a change of the
+# dispatch rules cannot silently drop a kernel from the parity suite.
+@pytest.mark.parametrize("c_in,c_out,k,s,p,n,h,w,kernel", [
+    (24, 24, 3, 1, 1, 3, 30, 22, "k_conv_tc_pairrows"),     # odd padding: pairs (2j-1, 2j), masked ends
+    (32, 32, 5, 1, 2, 2, 28, 28, "k_conv_tc_pairrows"),     # 5x5, even padding, full 128-byte lines
+    (16, 8, 3, 1, 0, 1, 18, 40, "k_conv_tc_pairrows"),      # no padding, 16 of 64 channels of a line used
+    (8, 16, 3, 1, 1, 1, 6, 300, "k_conv_tc_pairrows"),      # three column strips: per-pixel stores, strip halos
+    (16, 16, 7, 1, 3, 1, 20, 20, "k_conv_tc_pairrows"),     # 7x7: 56 instructions per block
+    (24, 24, 3, 1, 1, 1, 9, 15, "k_conv_dense_bf16"),       # odd width: pair-order weights read by the CUDA-core kernel
+    (40, 32, 5, 1, 2, 2, 14, 14, "k_conv_tc_fold"),         # odd entry count (padding entry), 5 tap columns
+    (48, 24, 3, 1, 1, 2, 20, 20, "k_conv_tc_fold"),
+    (64, 32, 3, 1, 1, 1, 12, 70, "k_conv_tc_fold"),         # two column strips
+    (4, 16, 5, 1, 2, 1, 9, 200, "k_conv_smallcin_bf16"),    # two row segments per output row
+    (3, 40, 3, 2, 1, 2, 17, 33, "k_conv_smallcin_bf16"),    # two passes of 32 output channels, odd sizes
+    (24, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc"),
+])
+def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, w, kernel):
+    g = dc.geom(c_in, c_out, 1, k, s, p)
+    assert dc.conv_kernel_name(n, h, w, g, dc.BF16) == kernel
+    spec = I.make_layer(11, 0, c_in, c_out, k, s, p)
+    lay = dc.DeviceLayer(spec)
+    wf = torch.empty_like(lay.weight)
+    bf = torch.empty(c_out, device="cuda")
+    dc.fold_bn(lay, wf, bf)
+    packed = torch.empty(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
+    dc.pack_weights(wf, g, dc.BF16, packed)
+    x = I.make_input(12, (n, h, w, c_in), bf16=True)
+    ho, wo = O.out_extent(h, k, s, p), O.out_extent(w, k, s, p)
+    r = I.round_bf16(I.normal(13, 99, (n, ho, wo, c_out)))
+    Wf, bfo = O.fold_bn(spec)
+    lin = O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p)
+    # plain, and with skip input + ReLU6
+    y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bf, dc.ACT_IDENTITY)
+    assert O.rel_l2(nchw(y), lin) <= TOL_BF16
+    y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bf, dc.ACT_RELU6, residual=dev(r, torch.bfloat16))
+    assert O.rel_l2(nchw(y), O.relu6(lin + r.transpose(0, 3, 1, 2))) <= TOL_BF16
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("c,k,s,p,n,h,w", [(32, 3, 1, 1, 2, 12, 12), (96, 3, 2, 1, 1, 15, 17),
                                            (144, 3, 1, 1, 1, 9, 30), (20, 5, 1, 2, 1, 8, 8),
