@@ -126,7 +126,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   int best = 1;
   for (int d = 1; d <= 8 && d <= ko->cch; ++d) {
     if (ko->cch % d) continue;
-    if ((size_t)d * ko->taps * n_tile * 16 <= 64 * 1024) best = d;
+    if ((size_t)d * ko->taps * n_tile * 16 <= 96 * 1024) best = d;
   }
   ko->cg = best;
   ko->ng = ko->cch / best;
