@@ -56,6 +56,11 @@ static inline int dc_out_extent(int h, int k, int s, int p) {
 // elements 8q..8q+7 of (pixel 0 channels, pixel 1 channels).  An entry is (tap row r, pair shift t,
 // chunk q); the weight of element (pixel px, channel c) of shift t for output pixel e of the pair
 // is W[o][c][r][2t + px - e].  Nothing is repacked on the way in.
+//
+// Stride 2 (pair == 3) sits on the same lines with one output per GEMM row: output X reads the
+// input columns 2X - pad + s, i.e. pixel px = (s + a) & 1 of pair shift t = (s + a) >> 1 with
+// a = pad & 1 (the patch starts a pixels further left to keep pairs aligned); the operand has co8
+// rows and the weight of element (px, c) of shift t is W[o][c][r][2t + px - a].
 // ----------------------------------------------------------------------------------------------
 struct KOrder {
   int k, stride, pad;
@@ -69,7 +74,7 @@ struct KOrder {
   int e_pad;          // e rounded up to even
   int n_pad;          // operand rows rounded up to 16 (output channels, or k * co8 in fold order)
   int fold;           // 1: fold order
-  int pair;           // 2: pair rows
+  int pair;           // 2: pair rows (stride 1), 3: pair rows, stride 2
   int co8;            // output channels rounded up to 8
 };
 
@@ -83,6 +88,22 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->fold = 0;
   ko->pair = 0;
   ko->pcs = (g->stride == 2) ? 2 : 1;
+  if (g->groups == 1 && g->stride == 2 && g->k >= 3 && g->k <= 7 && ko->cch <= 4 && ko->co8 <= 32 &&
+      g->c_in % 8 == 0 && g->c_out % 8 == 0) {
+    const int a = g->pad & 1;
+    const int nt = ((g->k - 1 + a) >> 1) + 1;
+    const int n_pad = (int)dc_round_up((size_t)ko->co8, 16);
+    if (g->k * nt * ko->cch <= 64 && (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 128 * 1024) {
+      ko->pair = 3;
+      ko->pcs = 1;
+      ko->n_pad = n_pad;
+      ko->ns[0] = nt; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
+      ko->cg = ko->cch; ko->ng = 1;
+      ko->e = g->k * nt * 2 * ko->cch;
+      ko->e_pad = ko->e;
+      return;
+    }
+  }
   if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch <= 8 && ko->co8 <= 32 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
     // pair rows when their tensor-core cost stays small (instructions of ~48 cycles per 256
@@ -137,7 +158,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
 // entry index within a group -> (pc, ccg, r, s); returns false for the zero padding entry
 __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
                                                         int *r, int *s) {
-  if (ko.pair == 2) {
+  if (ko.pair >= 2) {
     // (tap row, pair shift, chunk of the pair row); *ccg returns the chunk, *s the shift
     if (e >= ko.e) return false;
     const int nq = 2 * ko.cch;
@@ -188,6 +209,10 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
   if (ko.pair == 2)            // the copy for the first pixel of the pair: dx = s, pixel s & 1 of shift s >> 1
     return (r * ko.ns[0] + (s >> 1)) * 2 * ko.cch + (s & 1) * ko.cch + cc;
+  if (ko.pair == 3) {          // tap s sits at patch column s + a of the output's pair
+    const int sa = s + (ko.pad & 1);
+    return (r * ko.ns[0] + (sa >> 1)) * 2 * ko.cch + (sa & 1) * ko.cch + cc;
+  }
   if (ko.fold) {
     const int e = cc * ko.k + r;
     return ((ko.e & 1) && e == ko.e - 1) ? e + 1 : e;

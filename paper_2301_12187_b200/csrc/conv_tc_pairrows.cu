@@ -13,6 +13,12 @@
 // When the padding is odd the patch starts one pixel further left (so that pairs stay aligned in
 // memory) and output pair j is (2j-1, 2j); the epilogue masks the pixel that falls off either end.
 //
+// Stride 2 (KOrder pair == 3) uses the same lines with ONE output per GEMM row: output X sits on
+// the pixel pair it reads first, D[X][o] = sum_r sum_t sum_{px,c} x[row 2Y+r, pixel 2(X+t)+px][c] *
+// W[o][c][r][2t+px-a].  Consecutive output rows need input rows two apart, so the tile is fetched as
+// two TMA boxes that take every second row (even and odd patch rows); tap row r then reads box
+// r & 1 from plane row r >> 1 on, and GEMM rows stay contiguous.
+//
 // Operand descriptors: K-major, 128-byte swizzle, 1024 bytes between 8-row groups.  Tap rows, pair
 // shifts (whole 128-byte lines) and the 32-byte K step inside a line are all added to the start
 // address, with the base-offset field left at 0: the tensor core applies the swizzle to the bits of
@@ -51,14 +57,15 @@ constexpr int kInFlight = 2;                     // activation tiles a CTA reque
 struct PairParams {
   int n_img, h, w, ho, wo, c_in, c_out, co8;
   int k, pad, cch;
-  int align;                   // pad & 1: output pair j is (2j - align, 2j - align + 1)
+  int stride;                  // 1: two outputs per GEMM row (a pair); 2: one output per GEMM row
+  int align;                   // pad & 1: output pair j is (2j - align, 2j - align + 1) (stride 1)
   int tw, th, nxt;             // tile size in outputs, x tiles per row
   int tw2, wbox2, rbox;        // output pairs per tile row, pair rows per patch row, patch rows
   int tiles_y;                 // tiles per column strip
   int grid, tiles_per, tiles_rem;   // CTAs; CTA b takes tiles_per (+1 if b < tiles_rem) tiles
   int n_pad;                   // N of the instruction: 2 * co8, padded to 16
   int mb, mb_last;             // blocks of a full tile / of a strip's last (shorter) tile
-  int a_stage_bytes, a_box_bytes, b_bytes;
+  int a_stage_bytes, a_box_bytes, a_plane_bytes, b_bytes;   // stride 2: a stage is two planes (even / odd rows)
   int stages, slots, groups, act, bulk_out, out_buf_bytes;
   int off_b, off_bias, off_out, off_a, smem_bytes;
   int tmem_cols;
@@ -139,7 +146,12 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
       const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
       uint32_t v0[CO8], v1[CO8];
       tmem_ld_cols<CO8>(taddr, v0);
-      tmem_ld_cols<CO8>(taddr + (uint32_t)CO8, v1);
+      if (p.stride == 1) {
+        tmem_ld_cols<CO8>(taddr + (uint32_t)CO8, v1);
+      } else {
+#pragma unroll
+        for (int i = 0; i < CO8; ++i) v1[i] = 0u;
+      }
       tmem_ld_wait();
       // the accumulator slot is free again: one arrival per warp
       tc_fence_before();
@@ -150,9 +162,10 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
 
       const int pos = b * 128 + m;
       const int yy = (int)(((uint32_t)pos * p.wbox2_inv) >> 20), jj = pos - yy * p.wbox2;
-      const int xx = 2 * jj - p.align;           // first output column of the pair; -1 or >= tw_valid: no such pixel
+      // first output column of the row; -1 or >= tw_valid: no such pixel
+      const int xx = p.stride == 1 ? 2 * jj - p.align : jj;
       const bool valid0 = (xx >= 0) && (xx < tw_valid) && (yy < th_t);
-      const bool valid1 = (xx + 1 < tw_valid) && (yy < th_t);
+      const bool valid1 = (p.stride == 1) && (xx + 1 < tw_valid) && (yy < th_t);
       const int off = yy * p.wo + xx;            // pixel offset from the tile's first output pixel
       const uint32_t m0 = __ballot_sync(0xffffffffu, valid0), m1 = __ballot_sync(0xffffffffu, valid1);
       uint8_t *dst;
@@ -286,9 +299,17 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
           if (!mbar_wait(&sh.full[sw], pw, abort_flag, ws, 0x80000u | sw)) break;
         }
         // the box always has rbox rows; rows and pairs outside the image arrive as zeros
-        mbar_arrive_expect_tx(&sh.full[s], (uint32_t)p.a_box_bytes);
-        tma_load_4d(a_base0 + (uint32_t)s * (uint32_t)p.a_stage_bytes, &map_a, &sh.full[s], 0,
-                    (t.xt * p.tw - p.pad - p.align) >> 1, t.ty * p.th - p.pad, t.img);
+        const uint32_t dst = a_base0 + (uint32_t)s * (uint32_t)p.a_stage_bytes;
+        if (p.stride == 1) {
+          mbar_arrive_expect_tx(&sh.full[s], (uint32_t)p.a_box_bytes);
+          tma_load_4d(dst, &map_a, &sh.full[s], 0, (t.xt * p.tw - p.pad - p.align) >> 1, t.ty * p.th - p.pad, t.img);
+        } else {
+          // even and odd patch rows as two boxes (the map steps two rows at a time)
+          const int px0 = t.xt * p.tw - ((p.pad + p.align) >> 1), py0 = 2 * t.ty * p.th - p.pad;
+          mbar_arrive_expect_tx(&sh.full[s], 2u * (uint32_t)p.a_box_bytes);
+          tma_load_4d(dst, &map_a, &sh.full[s], 0, px0, py0, t.img);
+          tma_load_4d(dst + (uint32_t)p.a_plane_bytes, &map_a, &sh.full[s], 0, px0, py0 + 1, t.img);
+        }
         t.step(p);
         if (++s == p.stages) { s = 0; ph ^= 1; }
       }
@@ -412,17 +433,19 @@ constexpr int kSlack = 17 * 1024;   // a block's 128 rows may reach this far pas
 bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   KOrder ko;
   dc_korder_init(&ko, g);
-  if (ko.pair != 2) return false;
+  if (ko.pair != 2 && ko.pair != 3) return false;
+  const int S = g->stride;
   if (w & 1) return false;                        // an image row must be a whole number of pixel pairs
-  const int ho = dc_out_extent(h, g->k, 1, g->pad), wo = dc_out_extent(w, g->k, 1, g->pad);
+  const int ho = dc_out_extent(h, g->k, S, g->pad), wo = dc_out_extent(w, g->k, S, g->pad);
   if (ho <= 0 || wo <= 0) return false;
   if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;
   p->n_img = n; p->h = h; p->w = w; p->ho = ho; p->wo = wo;
   p->c_in = g->c_in; p->c_out = g->c_out; p->co8 = ko.co8;
   p->k = g->k; p->pad = g->pad; p->cch = ko.cch;
+  p->stride = S;
   p->align = g->pad & 1;
   p->n_pad = ko.n_pad;
-  const int nt = (g->k + 1) / 2;
+  const int nt = ko.ns[0];
   p->nmma = g->k * nt * ko.cch;
   if (p->nmma > kMaxMma) return false;
   p->slots = 512 / p->n_pad;
@@ -434,17 +457,17 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   p->tmem_cols = cols;
   const int nxt = dc_div_up(wo, 128);
   p->tw = dc_div_up(wo, nxt);
-  if (p->tw & 1) ++p->tw;                        // tiles start on an even output column
+  if (S == 1 && (p->tw & 1)) ++p->tw;            // tiles start on an even output column
   p->nxt = dc_div_up(wo, p->tw);
-  p->tw2 = (p->tw + p->align + 1) / 2;
-  p->wbox2 = p->tw2 + (g->k >> 1);
+  p->tw2 = S == 1 ? (p->tw + p->align + 1) / 2 : p->tw;    // GEMM rows per tile row
+  p->wbox2 = p->tw2 + nt - 1;
   if (p->wbox2 > 256) return false;
   p->wbox2_inv = ((1u << 20) + (uint32_t)p->wbox2 - 1) / (uint32_t)p->wbox2;
   const long long strips = (long long)n * p->nxt;
   if (strips * ho >= (1ll << 30)) return false;
   // fixed part of shared memory: weights, bias, per-warp output staging
   p->b_bytes = ko.e_pad * p->n_pad * 16;
-  p->out_buf_bytes = (int)dc_round_up((size_t)64 * g->c_out * 2, 128);
+  p->out_buf_bytes = (int)dc_round_up((size_t)(S == 1 ? 64 : 32) * g->c_out * 2, 128);
   p->bulk_out = (p->nxt == 1) ? 1 : 0;
   p->off_b = 0;
   p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
@@ -452,7 +475,13 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   // the output staging buffers follow the stages and double as the room a block's last rows may
   // reach into past the last stage (what is read there only feeds rows that are dropped)
   const long long tail_bytes = kEpiWarps * p->out_buf_bytes > kSlack ? kEpiWarps * p->out_buf_bytes : kSlack;
-  auto stage_bytes = [&](int th_c) { return (long long)dc_round_up((size_t)(th_c + g->k - 1) * p->wbox2 * 128, 1024); };
+  // patch rows of a tile of th_c output rows; stride 2 holds them as two planes of every second row
+  auto patch_rows = [&](int th_c) { return S == 1 ? th_c + g->k - 1 : 2 * (th_c - 1) + g->k; };
+  auto plane_bytes = [&](int th_c) {
+    const int rows = S == 1 ? patch_rows(th_c) : (patch_rows(th_c) + 1) / 2;
+    return (long long)dc_round_up((size_t)rows * p->wbox2 * 128, 1024);
+  };
+  auto stage_bytes = [&](int th_c) { return S * plane_bytes(th_c); };
   auto total_bytes = [&](int th_c, int s) { return 1024ll + p->off_a + s * stage_bytes(th_c) + tail_bytes; };
   // Rows per tile.  A CTA's time is roughly (tiles it gets) x (blocks per tile + a fixed cost per
   // tile + the patch rows it stages) plus the start-up of its first tile, which nothing overlaps;
@@ -460,8 +489,8 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   int th = 0;
   double best = 0.0;
   for (int cand = 1; cand <= 32 && cand <= ho; ++cand) {
-    const int rbox = cand + g->k - 1;
-    if (rbox > 256) break;
+    const int rbox = patch_rows(cand);
+    if (rbox > 127) break;
     if (stage_bytes(cand) > kStageLimit) break;
     if (total_bytes(cand, 2) > kSmemBudget) break;
     if ((cand - 1) * p->wbox2 + p->tw2 + 128 >= 4096) break;
@@ -474,7 +503,7 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   }
   if (th == 0) return false;
   p->th = th;
-  p->rbox = th + g->k - 1;
+  p->rbox = S == 1 ? patch_rows(th) : (patch_rows(th) + 1) / 2;     // rows of one TMA box
   p->tiles_y = dc_div_up(ho, th);
   const long long total_tiles = strips * p->tiles_y;
   const int grid = total_tiles < n_sm ? (int)total_tiles : n_sm;
@@ -485,6 +514,7 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   const int th_last = ho - (p->tiles_y - 1) * th;
   p->mb_last = dc_div_up((th_last - 1) * p->wbox2 + p->tw2, 128);
   p->a_stage_bytes = (int)stage_bytes(th);
+  p->a_plane_bytes = (int)plane_bytes(th);
   p->a_box_bytes = p->rbox * p->wbox2 * 128;
   const long long per_cta = p->tiles_per + (p->tiles_rem ? 1 : 0);
   int stages = kMaxStages < per_cta ? kMaxStages : (int)per_cta;
@@ -499,7 +529,8 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   for (int r = 0; r < g->k; ++r)
     for (int t = 0; t < nt; ++t)
       for (int sl = 0; sl < ko.cch; ++sl, ++j) {
-        const uint32_t off = (uint32_t)((r * p->wbox2 + t) * 128 + sl * 32);
+        const uint32_t off = S == 1 ? (uint32_t)((r * p->wbox2 + t) * 128 + sl * 32)
+                                    : (uint32_t)((r & 1) * p->a_plane_bytes + ((r >> 1) * p->wbox2 + t) * 128 + sl * 32);
         p->a_lo[j] = (off >> 4) | (1u << 16);    // leading-dimension field: 1 (unused for swizzled K-major)
       }
   return true;
@@ -527,8 +558,9 @@ dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_g
     const cuuint64_t C = (cuuint64_t)g->c_in;
     cuuint64_t gdim[4] = {2 * C, (cuuint64_t)(w / 2), (cuuint64_t)h, (cuuint64_t)n};
     cuuint64_t gstr[3] = {4 * C, (cuuint64_t)w * C * 2, (cuuint64_t)h * w * C * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)p.wbox2, (cuuint32_t)p.rbox, 1};
-    cuuint32_t es[4] = {1, 1, 1, 1};
+    // stride 2: the box spans 2 * rbox rows and takes every second one
+    cuuint32_t box[4] = {64, (cuuint32_t)p.wbox2, (cuuint32_t)(p.stride * p.rbox), 1};
+    cuuint32_t es[4] = {1, 1, (cuuint32_t)p.stride, 1};
     CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), gdim, gstr, box, es,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

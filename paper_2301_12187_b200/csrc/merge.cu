@@ -303,6 +303,12 @@ __global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrde
         ccg = 0;
         c8 = elem - ipx * ko.c_in;         // channel (grp is 0 and cg irrelevant once ccg = 0)
         if (px >= 2 || s < 0 || s >= ko.k) o = c_out;
+      } else if (ko.pair == 3) {           // stride 2: row = output channel; tap column = 2 * shift + pixel - (pad & 1)
+        const int elem = ccg * 8 + c8, ipx = elem / ko.c_in;
+        s = 2 * s + ipx - (ko.pad & 1);
+        ccg = 0;
+        c8 = elem - ipx * ko.c_in;
+        if (s < 0 || s >= ko.k) o = c_out;
       }
       int c = (grp * ko.cg + ccg) * 8 + c8;
       if (o < c_out && c < ko.c_in) v = w[(((size_t)o * ko.c_in + c) * ko.k + r) * ko.k + s];
@@ -372,6 +378,12 @@ __global__ void k_deliver(Piece acc, float *w_merged, float *b_merged, void *pac
           ccg = 0;
           c8 = elem - ipx * ko.c_in;
           if (px >= 2 || sx < 0 || sx >= ko.k) o = c_out;
+        } else if (ko.pair == 3) {
+          const int elem = ccg * 8 + c8, ipx = elem / ko.c_in;
+          sx = 2 * sx + ipx - (ko.pad & 1);
+          ccg = 0;
+          c8 = elem - ipx * ko.c_in;
+          if (sx < 0 || sx >= ko.k) o = c_out;
         }
         const int c = (grp * ko.cg + ccg) * 8 + c8;
         if (o < c_out && c < ko.c_in) v = merged_at(acc, o, c, r * ko.k + sx);

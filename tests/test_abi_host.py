@@ -95,7 +95,8 @@ def test_kernel_name_query_follows_the_dispatch_rules():
     assert dc.conv_kernel_name(64, 56, 56, dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_pairrows"
     assert dc.conv_kernel_name(128, 28, 28, dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_pairrows"
     assert dc.conv_kernel_name(128, 14, 14, dc.geom(40, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_fold"
-    assert dc.conv_kernel_name(128, 56, 56, dc.geom(24, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_tc"
+    assert dc.conv_kernel_name(128, 56, 56, dc.geom(24, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_tc_pairrows"
+    assert dc.conv_kernel_name(128, 56, 56, dc.geom(96, 144, 1, 5, 2, 2), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 14, 14, dc.geom(96, 576, 1, 1, 1, 0), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 224, 224, dc.geom(3, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_smallcin_bf16"
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(20, 12, 1, 3, 1, 1), dc.BF16) == "k_conv_dense_bf16"

@@ -206,7 +206,10 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (64, 32, 3, 1, 1, 1, 12, 70, "k_conv_tc_fold"),         # two column strips
     (4, 16, 5, 1, 2, 1, 9, 200, "k_conv_smallcin_bf16"),    # two row segments per output row
     (3, 40, 3, 2, 1, 2, 17, 33, "k_conv_smallcin_bf16"),    # two passes of 32 output channels, odd sizes
-    (24, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc"),
+    (24, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc_pairrows"),     # stride 2: one output per line, even/odd row boxes
+    (32, 16, 5, 2, 2, 1, 30, 44, "k_conv_tc_pairrows"),     # stride 2, even padding, 5x5
+    (16, 24, 3, 2, 0, 2, 17, 36, "k_conv_tc_pairrows"),     # stride 2, no padding, odd height
+    (40, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc"),              # stride 2 on parity planes (more than 32 channels)
 ])
 def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, w, kernel):
     g = dc.geom(c_in, c_out, 1, k, s, p)
