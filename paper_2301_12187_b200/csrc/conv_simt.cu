@@ -327,6 +327,78 @@ __global__ void __launch_bounds__(256) k_dwconv_vec(const T *__restrict__ x, con
   }
 }
 
+// Register-tiled variant for the common shapes (k = 3 or 5, stride 1 or 2): a CTA works on one
+// output row, a thread on TX consecutive outputs x V channels, so the (TX-1)*S + K input vectors of
+// a tap row are loaded once and reused by all the outputs they reach, and the tap row's weights are
+// loaded once per TX outputs.  All index arithmetic is 32-bit and per row.
+template <typename T, int K, int S, int TX>
+__global__ void __launch_bounds__(128) k_dwconv_rows(const T *__restrict__ x, const float *__restrict__ w,
+                                                     const float *__restrict__ bias, T *__restrict__ y, int h, int wd,
+                                                     int c, int ho, int wo, int pad, int act) {
+  constexpr int V = DwVec<T>::V;
+  constexpr int NJ = (TX - 1) * S + K;
+  const int cv = c / V;
+  const int xtiles = (wo + TX - 1) / TX;
+  const int row = (int)blockIdx.x;               // img * ho + Y
+  const int img = row / ho, Y = row - img * ho;
+  const T *ximg = x + (size_t)img * h * wd * c;
+  T *yrow = y + (size_t)row * wo * c;
+  for (int item = (int)threadIdx.x; item < xtiles * cv; item += (int)blockDim.x) {
+    const int xt = item / cv, c0 = (item - xt * cv) * V;
+    const int X0 = xt * TX;
+    float acc[TX][V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) {
+      const float b = bias ? bias[c0 + q] : 0.f;
+#pragma unroll
+      for (int t = 0; t < TX; ++t) acc[t][q] = b;
+    }
+#pragma unroll
+    for (int r = 0; r < K; ++r) {
+      const int yy = Y * S + r - pad;
+      if (yy < 0 || yy >= h) continue;
+      float wr[K][V];
+#pragma unroll
+      for (int sx = 0; sx < K; ++sx) {
+        const float *wp = w + (size_t)(r * K + sx) * c + c0;
+#pragma unroll
+        for (int q = 0; q < V; q += 4) {
+          const float4 wv = *reinterpret_cast<const float4 *>(wp + q);
+          wr[sx][q] = wv.x; wr[sx][q + 1] = wv.y; wr[sx][q + 2] = wv.z; wr[sx][q + 3] = wv.w;
+        }
+      }
+      const T *xrow = ximg + (size_t)yy * wd * c + c0;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        const int xx = X0 * S + j - pad;
+        float xv[V];
+        if (xx >= 0 && xx < wd) {
+          DwVec<T>::load(xrow + (size_t)xx * c, xv);
+        } else {
+#pragma unroll
+          for (int q = 0; q < V; ++q) xv[q] = 0.f;
+        }
+#pragma unroll
+        for (int t = 0; t < TX; ++t) {
+          const int sx = j - t * S;                // tap column with which input j feeds output t
+          if (sx >= 0 && sx < K) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) acc[t][q] = fmaf(xv[q], wr[sx][q], acc[t][q]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < TX; ++t) {
+      if (X0 + t < wo) {
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[t][q] = dc_act_apply(acc[t][q], act);
+        DwVec<T>::store(yrow + (size_t)(X0 + t) * c + c0, acc[t]);
+      }
+    }
+  }
+}
+
 // any channel count: one thread = one output element
 template <typename T>
 __global__ void k_dwconv_scalar(const T *__restrict__ x, const float *__restrict__ w, const float *__restrict__ bias,
@@ -357,7 +429,20 @@ static dc_status launch_dw(const void *x, int n, int h, int w, int c, int k, int
                            const float *bias, dc_act act, void *y, cudaStream_t st) {
   const int ho = dc_out_extent(h, k, stride, pad), wo = dc_out_extent(w, k, stride, pad);
   constexpr int V = DwVec<T>::V;
-  if (c % V == 0) {
+  if (c % V == 0 && (k == 3 || k == 5) && (stride == 1 || stride == 2) && (long long)n * ho < (1ll << 31)) {
+    // stride 1: 4 outputs per thread share 6 (k = 3) input columns; stride 2 shares less, so 2 outputs
+    // keep the register count down.  Threads per CTA: the row's work items, in whole warps, up to 128.
+    const int rows = n * ho;
+    const T *xp = (const T *)x;
+    T *yp = (T *)y;
+    const int tx = stride == 1 ? 4 : 2;
+    int items = dc_div_up(wo, tx) * (c / V);
+    int threads = items >= 128 ? 128 : (int)dc_round_up((size_t)items, 32);
+    if (k == 3 && stride == 1) k_dwconv_rows<T, 3, 1, 4><<<rows, threads, 0, st>>>(xp, wp, bias, yp, h, w, c, ho, wo, pad, (int)act);
+    else if (k == 3) k_dwconv_rows<T, 3, 2, 2><<<rows, threads, 0, st>>>(xp, wp, bias, yp, h, w, c, ho, wo, pad, (int)act);
+    else if (stride == 1) k_dwconv_rows<T, 5, 1, 4><<<rows, threads, 0, st>>>(xp, wp, bias, yp, h, w, c, ho, wo, pad, (int)act);
+    else k_dwconv_rows<T, 5, 2, 2><<<rows, threads, 0, st>>>(xp, wp, bias, yp, h, w, c, ho, wo, pad, (int)act);
+  } else if (c % V == 0) {
     long long total = (long long)n * ho * wo * (c / V);
     k_dwconv_vec<T><<<simt_blocks(total, 256, 148 * 32), 256, 0, st>>>((const T *)x, wp, bias, (T *)y, n, h, w, c, ho,
                                                                       wo, k, stride, pad, (int)act);
