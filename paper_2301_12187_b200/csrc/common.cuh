@@ -88,7 +88,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->fold = 0;
   ko->pair = 0;
   ko->pcs = (g->stride == 2) ? 2 : 1;
-  if (g->groups == 1 && g->stride == 2 && g->k >= 3 && g->k <= 7 && ko->cch <= 4 && ko->co8 <= 32 &&
+  if (g->groups == 1 && g->stride == 2 && g->k >= 3 && g->k <= 7 && ko->cch <= 4 && ko->co8 <= 128 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
     const int a = g->pad & 1;
     const int nt = ((g->k - 1 + a) >> 1) + 1;
@@ -104,24 +104,26 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
       return;
     }
   }
+  // pair rows (stride 1, 1x1 included) when their tensor-core cost stays small; beyond that fold
+  // order (one instruction row per tap row) wins for narrow outputs
+  // (1x1 layers with many output channels are bound by writing their output, which the general
+  // kernel's staged bulk stores do better than this kernel's per-thread stores for wide outputs)
+  if (g->groups == 1 && g->stride == 1 && g->k <= 7 && ko->cch <= 4 && ko->co8 <= (g->k == 1 ? 32 : 128) &&
+      g->c_in % 8 == 0 && g->c_out % 8 == 0) {
+    const int n_pad = (int)dc_round_up((size_t)(2 * ko->co8), 16);
+    const int nt = (g->k + 1) / 2;
+    if (g->k * nt * ko->cch <= 64 && (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 128 * 1024) {
+      ko->pair = 2;
+      ko->n_pad = n_pad;
+      ko->ns[0] = nt; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
+      ko->cg = ko->cch; ko->ng = 1;
+      ko->e = g->k * nt * 2 * ko->cch;
+      ko->e_pad = ko->e;
+      return;
+    }
+  }
   if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch <= 8 && ko->co8 <= 32 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
-    // pair rows when their tensor-core cost stays small (instructions of ~48 cycles per 256
-    // outputs); beyond that fold order (one instruction row per tap row) wins
-    {
-      const int n_pad = (int)dc_round_up((size_t)(2 * ko->co8), 16);
-      const int nt = (g->k + 1) / 2;
-      if (g->k * nt * ko->cch <= 64 && ko->cch <= 4 &&
-          (size_t)g->k * nt * 2 * ko->cch * n_pad * 16 <= 128 * 1024) {
-        ko->pair = 2;
-        ko->n_pad = n_pad;
-        ko->ns[0] = nt; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
-        ko->cg = ko->cch; ko->ng = 1;
-        ko->e = g->k * nt * 2 * ko->cch;
-        ko->e_pad = ko->e;
-        return;
-      }
-    }
     const int n_pad = (int)dc_round_up((size_t)(g->k * ko->co8), 16);
     if ((size_t)ko->cch * g->k * n_pad * 16 <= 64 * 1024) {
       ko->fold = 1;

@@ -64,7 +64,7 @@ struct FoldParams {
   int blk_rows;                // output positions per 128-row block = 128 - (k-1)
   int mb, mb_last;             // blocks of a full tile / of a strip's last (shorter) tile
   int plane_stride, a_stage_bytes, b_bytes, raw_bytes;
-  int nraw, stages, slots, groups, act, bulk_out, out_buf_bytes, xch_buf_floats;
+  int nraw, stages, slots, groups, mma_warps, act, bulk_out, out_buf_bytes, xch_buf_floats;
   int off_b, off_bias, off_out, off_xch, off_raw, off_a, smem_bytes;
   int tmem_cols;
   int npairs;
@@ -443,7 +443,7 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
 
     if (warp < kFirstEpiWarp) {
       // ================================================================== MMA issue
-      // Warp mw takes blocks c = mw mod kMmaWarps.  The warps sit on different schedulers, so the
+      // Warp mw takes blocks c = mw mod mma_warps.  The warps sit on different schedulers, so the
       // short issue sequences of several blocks progress side by side although each shares its
       // scheduler with busy epilogue warps.  The warp stays converged; one elected lane issues.
       const int mw = warp - kMmaWarp;
@@ -456,7 +456,9 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
       int s = 0;                                 // stage and its phase, accumulator slot and its phase
       uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
       while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
-      int next = mw, c0 = 0;                     // next block of this warp; first block of the tile
+      // next block of this warp (warps beyond mma_warps take none, they only hand the stages back);
+      // first block of the tile
+      int next = mw < p.mma_warps ? mw : 0x40000000, c0 = 0;
       Walk t;
       t.start(p, tile0);
 #pragma unroll 1
@@ -465,7 +467,7 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
         if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
         tc_fence_after();
 #pragma unroll 1
-        for (int b = next - c0; b < nblk; b += kMmaWarps, next += kMmaWarps) {
+        for (int b = next - c0; b < nblk; b += p.mma_warps, next += p.mma_warps) {
           if (!warp_wait(&sh.slot_empty[slot], sph, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
@@ -480,7 +482,7 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
             }
           }
           if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
-          slot += kMmaWarps;
+          slot += (uint32_t)p.mma_warps;
           while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
         }
         // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
@@ -551,7 +553,13 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
   p->slots = 512 / p->n_pad;
   if (p->slots > kMaxSlots) p->slots = kMaxSlots;
   if (p->slots < 2) return false;
+  // A waiter can trail its mbarrier by one phase at most, so every slot must have exactly one
+  // MMA warp issuing into it and one epilogue group draining it: the slot count is a multiple of
+  // the number of groups and of the number of MMA warps that take blocks.
   p->groups = p->slots < kGroups ? p->slots : kGroups;
+  p->slots = p->slots / p->groups * p->groups;
+  p->mma_warps = kMmaWarps;
+  while (p->slots % p->mma_warps) --p->mma_warps;
   int cols = 32;
   while (cols < p->slots * p->n_pad) cols *= 2;
   p->tmem_cols = cols;

@@ -66,7 +66,7 @@ struct PairParams {
   int n_pad;                   // N of the instruction: 2 * co8, padded to 16
   int mb, mb_last;             // blocks of a full tile / of a strip's last (shorter) tile
   int a_stage_bytes, a_box_bytes, a_plane_bytes, b_bytes;   // stride 2: a stage is two planes (even / odd rows)
-  int stages, slots, groups, act, bulk_out, out_buf_bytes;
+  int stages, slots, groups, mma_warps, act, bulk_out, out_buf_bytes;
   int off_b, off_bias, off_out, off_a, smem_bytes;
   int tmem_cols;
   int nmma;
@@ -233,6 +233,98 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
   if (p.bulk_out && lane == 0) bulk_wait_all();
 }
 
+// The same for more than 32 output channels: the channels are walked 8 at a time in a run-time
+// loop (any c_out that is a multiple of 8), and a thread stores its pixels' channels straight to
+// global memory (2 * c_out contiguous bytes per pixel; no staging buffer of that size per warp).
+__device__ __noinline__ void epilogue_wide(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+                                           const __nv_bfloat16 *residual, __nv_bfloat16 *y, int tile0, int ntiles) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int grp = (warp - kFirstEpiWarp) >> 2;
+  const int q = warp & 3;
+  if (grp >= p.groups) return;
+  const int m = q * 32 + lane;
+  const uint32_t tmem_row = sh.tmem_base + ((uint32_t)(q * 32) << 16);
+  volatile uint32_t *abort_flag = &sh.abort;
+  uint32_t slot = (uint32_t)grp, sph = 0;
+  while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+  int next = grp, c0 = 0;
+  Walk t;
+  t.start(p, tile0);
+#pragma unroll 1
+  for (int ti = 0; ti < ntiles; ++ti) {
+    const int nblk = t.nblk(p), th_t = t.rows_out(p);
+    const int tw_valid = (p.wo - t.xt * p.tw < p.tw) ? p.wo - t.xt * p.tw : p.tw;
+    const size_t tile_pix0 = ((size_t)t.img * p.ho + (size_t)(t.ty * p.th)) * p.wo + (size_t)(t.xt * p.tw);
+#pragma unroll 1
+    for (int b = next - c0; b < nblk; b += p.groups, next += p.groups) {
+      if (!warp_wait(&sh.slot_full[slot], sph, abort_flag, ws, 0x40000u | slot)) return;
+      tc_fence_after();
+      const uint32_t taddr = tmem_row + slot * (uint32_t)p.n_pad;
+      const int pos = b * 128 + m;
+      const int yy = (int)(((uint32_t)pos * p.wbox2_inv) >> 20), jj = pos - yy * p.wbox2;
+      const int xx = p.stride == 1 ? 2 * jj - p.align : jj;
+      const bool valid0 = (xx >= 0) && (xx < tw_valid) && (yy < th_t);
+      const bool valid1 = (p.stride == 1) && (xx + 1 < tw_valid) && (yy < th_t);
+      const size_t pix = tile_pix0 + (size_t)(yy * p.wo + xx);
+      __nv_bfloat16 *dst = y + pix * p.c_out;
+      const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out : nullptr;
+#pragma unroll 1
+      for (int ch = 0; ch < p.c_out; ch += 8) {
+        uint32_t v0[8], v1[8];
+        tmem_ld8(taddr + (uint32_t)ch, v0);
+        if (p.stride == 1) {
+          tmem_ld8(taddr + (uint32_t)(p.co8 + ch), v1);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v1[i] = 0u;
+        }
+        tmem_ld_wait();
+        if (ch + 8 >= p.c_out) {
+          // all of the accumulator has been read: the slot is free again, one arrival per warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
+        }
+        const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
+        const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const uint32_t *v = e ? v1 : v0;
+          if (e ? valid1 : valid0) {
+            float f[8];
+            f[0] = __uint_as_float(v[0]) + b0.x; f[1] = __uint_as_float(v[1]) + b0.y;
+            f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
+            f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
+            f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
+            if (rp) {
+              const uint4 rv = *reinterpret_cast<const uint4 *>(rp + e * p.c_out + ch);
+              const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 rf = __bfloat1622float2(rb[i]);
+                f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+              }
+            }
+            uint4 ov;
+            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float f0 = f[2 * i], f1 = f[2 * i + 1];
+              if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
+              ob[i] = __floats2bfloat162_rn(f0, f1);
+            }
+            *reinterpret_cast<uint4 *>(dst + e * p.c_out + ch) = ov;
+          }
+        }
+      }
+      slot += (uint32_t)p.groups;
+      while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
+    }
+    c0 += nblk;
+    t.step(p);
+  }
+}
+
 template <int CO8>
 __device__ __forceinline__ void epilogue_dispatch(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
                                                   uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
@@ -322,7 +414,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
       tmem_relinquish();
     } else if (warp >= kFirstEpiWarp) {
       const int t = (int)threadIdx.x - kFirstEpiWarp * 32;
-      if (t < 32) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
+      if (t < p.co8) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
     }
     tc_fence_before();
     bar_sync(kBarConsumers, kConsumerThreads);
@@ -331,7 +423,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
 
     if (warp < kFirstEpiWarp) {
       // ================================================================== MMA issue
-      // Warp mw takes blocks c = mw mod kMmaWarps.  The warps sit on different schedulers, so the
+      // Warp mw takes blocks c = mw mod mma_warps.  The warps sit on different schedulers, so the
       // issue sequences of several blocks progress side by side although each shares its scheduler
       // with epilogue warps.  The warp stays converged; one elected lane issues.
       const int mw = warp - kMmaWarp;
@@ -345,7 +437,9 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
       int s = 0;                                 // stage and its phase, accumulator slot and its phase
       uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
       while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
-      int next = mw, c0 = 0;                     // next block of this warp; first block of the tile
+      // next block of this warp (warps beyond mma_warps take none, they only hand the stages back);
+      // first block of the tile
+      int next = mw < p.mma_warps ? mw : 0x40000000, c0 = 0;
       Walk t;
       t.start(p, tile0);
 #pragma unroll 1
@@ -354,7 +448,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (!warp_wait(&sh.full[s], ph, abort_flag, ws, 0x30000u | s)) break;
         tc_fence_after();
 #pragma unroll 1
-        for (int b = next - c0; b < nblk; b += kMmaWarps, next += kMmaWarps) {
+        for (int b = next - c0; b < nblk; b += p.mma_warps, next += p.mma_warps) {
           if (!warp_wait(&sh.slot_empty[slot], sph, abort_flag, ws, 0x20000u | slot)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
@@ -367,7 +461,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
             if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
           }
           if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
-          slot += kMmaWarps;
+          slot += (uint32_t)p.mma_warps;
           while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
         }
         // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
@@ -378,7 +472,8 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (++s == p.stages) { s = 0; ph ^= 1; a_row = a_row0; }
       }
     } else {
-      switch (p.co8) {
+      if (p.co8 > 32) epilogue_wide(p, sh, ws, bias_s, residual, y, tile0, ntiles);
+      else switch (p.co8) {
         case 8: epilogue_dispatch<8>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
         case 16: epilogue_dispatch<16>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
         case 24: epilogue_dispatch<24>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
@@ -451,7 +546,13 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   p->slots = 512 / p->n_pad;
   if (p->slots > kMaxSlots) p->slots = kMaxSlots;
   if (p->slots < 2) return false;
+  // A waiter can trail its mbarrier by one phase at most, so every slot must have exactly one
+  // MMA warp issuing into it and one epilogue group draining it: the slot count is a multiple of
+  // the number of groups and of the number of MMA warps that take blocks.
   p->groups = p->slots < kGroups ? p->slots : kGroups;
+  p->slots = p->slots / p->groups * p->groups;
+  p->mma_warps = kMmaWarps;
+  while (p->slots % p->mma_warps) --p->mma_warps;
   int cols = 32;
   while (cols < p->slots * p->n_pad) cols *= 2;
   p->tmem_cols = cols;
@@ -467,11 +568,11 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   if (strips * ho >= (1ll << 30)) return false;
   // fixed part of shared memory: weights, bias, per-warp output staging
   p->b_bytes = ko.e_pad * p->n_pad * 16;
-  p->out_buf_bytes = (int)dc_round_up((size_t)(S == 1 ? 64 : 32) * g->c_out * 2, 128);
-  p->bulk_out = (p->nxt == 1) ? 1 : 0;
+  p->bulk_out = (p->nxt == 1 && ko.co8 <= 32) ? 1 : 0;     // wider outputs are stored straight from registers
+  p->out_buf_bytes = p->bulk_out ? (int)dc_round_up((size_t)(S == 1 ? 64 : 32) * g->c_out * 2, 128) : 0;
   p->off_b = 0;
   p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
-  p->off_a = (int)dc_round_up((size_t)p->off_bias + 128, 1024);
+  p->off_a = (int)dc_round_up((size_t)p->off_bias + 1024, 1024);
   // the output staging buffers follow the stages and double as the room a block's last rows may
   // reach into past the last stage (what is read there only feeds rows that are dropped)
   const long long tail_bytes = kEpiWarps * p->out_buf_bytes > kSlack ? kEpiWarps * p->out_buf_bytes : kSlack;

@@ -210,6 +210,10 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (32, 16, 5, 2, 2, 1, 30, 44, "k_conv_tc_pairrows"),     # stride 2, even padding, 5x5
     (16, 24, 3, 2, 0, 2, 17, 36, "k_conv_tc_pairrows"),     # stride 2, no padding, odd height
     (40, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc"),              # stride 2 on parity planes (more than 32 channels)
+    (32, 16, 1, 1, 0, 2, 20, 24, "k_conv_tc_pairrows"),     # 1x1: one instruction per 32-byte K step
+    (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with a wide output: general kernel
+    (16, 128, 3, 1, 1, 1, 12, 16, "k_conv_tc_pairrows"),    # N = 256: two accumulator slots, run-time channel loop
+    (32, 64, 3, 2, 1, 1, 28, 28, "k_conv_tc_pairrows"),     # stride 2, 64 output channels
 ])
 def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, w, kernel):
     g = dc.geom(c_in, c_out, 1, k, s, p)
