@@ -241,6 +241,31 @@ __device__ __forceinline__ float dc_act_apply(float v, int act) {
   return act == DC_ACT_RELU6 ? fminf(fmaxf(v, 0.f), 6.f) : v;
 }
 
+// Programmatic dependent launch.  A kernel launched through dc_launch_pdl may be scheduled while the
+// previous kernel of the stream is still running (its launch latency and start-up then overlap that
+// kernel's end); it must call dc_pdl_enter() before it reads or writes global memory: that waits
+// until the previous kernel has finished and its writes are visible, and lets the next kernel of
+// the stream be scheduled in turn.  Launched in the ordinary way, the call returns at once.
+__device__ __forceinline__ void dc_pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t dc_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                        Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Workspace header written by kernels with bounded waits.
 struct DcWsHeader {
   unsigned int status;      // 0 or DC_ERR_TIMEOUT

@@ -366,11 +366,7 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
     else if (t == 64) { mbar_init(&sh.weights, 1); sh.abort = 0; prefetch_tensormap(&map_a); did = true; }
     if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // Programmatic dependent launch: the next kernel in the stream may be brought up while this one
-  // runs, and this one was possibly brought up while its predecessor ran; nothing here has touched
-  // global memory yet, everything after the wait may.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  dc_pdl_enter();                                // nothing above touched global memory; everything below may
   __syncthreads();
 
   if (warp == 0) {
@@ -677,20 +673,9 @@ dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_g
     DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_pairrows, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
     attr_set = true;
   }
-  // launched so that its start-up (scheduling, barrier set-up) may overlap the previous kernel's end; the
-  // kernel itself waits for that kernel's memory before it reads or writes anything
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(p.grid);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = (size_t)p.smem_bytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, k_conv_tc_pairrows, map_a, p, w_packed, bias, (const __nv_bfloat16 *)residual,
-                                      (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  cudaError_t le = dc_launch_pdl(k_conv_tc_pairrows, dim3(p.grid), dim3(kThreads), (size_t)p.smem_bytes, stream, map_a, p,
+                                 w_packed, bias, (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
+                                 (DcWsHeader *)workspace);
   if (le != cudaSuccess) return DC_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
