@@ -26,6 +26,7 @@ extern "C" const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g
   if (dtype == DC_F32) return "k_conv_dense_f32";
   if (dtype != DC_BF16) return nullptr;
   if (dc_conv_pairrows_supported(n, h, w, g)) return "k_conv_tc_pairrows";
+  if (dc_conv_rows_supported(n, h, w, g)) return "k_conv_tc_rows";
   if (dc_conv_fold_supported(n, h, w, g)) return "k_conv_tc_fold";
   if (dc_conv_tc_supported(n, h, w, g)) return "k_conv_tc";
   if (dc_conv_smallcin_supported(n, h, w, g)) return "k_conv_smallcin_bf16";
@@ -52,6 +53,8 @@ extern "C" dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, co
   cudaStream_t st = (cudaStream_t)stream;
   if (dtype == DC_BF16 && algo != DC_ALGO_SIMT && dc_conv_pairrows_supported(n, h, w, g))
     return dc_launch_conv_pairrows(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
+  if (dtype == DC_BF16 && algo != DC_ALGO_SIMT && dc_conv_rows_supported(n, h, w, g))
+    return dc_launch_conv_rows(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   const bool fold_ok = dtype == DC_BF16 && dc_conv_fold_supported(n, h, w, g);
   const bool tc_ok = dtype == DC_BF16 && !fold_ok && dc_conv_tc_supported(n, h, w, g);
   if (algo == DC_ALGO_TCGEN05 && !tc_ok && !fold_ok) return DC_ERR_UNSUPPORTED;

@@ -75,6 +75,8 @@ struct KOrder {
   int n_pad;          // operand rows rounded up to 16 (output channels, or k * co8 in fold order)
   int fold;           // 1: fold order
   int pair;           // 2: pair rows (stride 1), 3: pair rows, stride 2
+  int rows;           // 1: rows order (planes of 64 channels, passes of n_tile output channels)
+  int n_tile, nnt;    // rows order: output channels per pass, passes (n_pad = nnt * n_tile)
   int co8;            // output channels rounded up to 8
 };
 
@@ -87,6 +89,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   ko->co8 = (int)dc_round_up((size_t)g->c_out, 8);
   ko->fold = 0;
   ko->pair = 0;
+  ko->rows = 0; ko->n_tile = 0; ko->nnt = 1;
   ko->pcs = (g->stride == 2) ? 2 : 1;
   if (g->groups == 1 && g->stride == 2 && g->k >= 3 && g->k <= 7 && ko->cch <= 4 && ko->co8 <= 128 &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
@@ -135,6 +138,23 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
       return;
     }
   }
+  // rows order: stride 1, k >= 3, more channels than a pixel pair's line holds.  Chunk planes are
+  // ordered (plane g of 64 channels, tap row r, tap column s, 16-channel step, half): the planes of
+  // one (g, r) step are contiguous, which is the unit the kernel streams.
+  if (g->groups == 1 && g->stride == 1 && g->k >= 3 && g->k <= 7 && ko->cch >= 5 &&
+      g->c_in % 8 == 0 && g->c_out % 8 == 0) {
+    const int n16 = (int)dc_round_up((size_t)g->c_out, 16);
+    ko->rows = 1;
+    ko->nnt = dc_div_up(n16, 128);
+    ko->n_tile = (int)dc_round_up((size_t)dc_div_up(n16, ko->nnt), 16);
+    ko->n_pad = ko->nnt * ko->n_tile;
+    ko->ns[0] = g->k; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
+    ko->cg = ko->cch; ko->ng = 1;
+    const int steps = dc_div_up(g->c_in, 16);            // 16-channel steps over all planes
+    ko->e = g->k * g->k * steps * 2;
+    ko->e_pad = ko->e;
+    return;
+  }
   if (ko->pcs == 1) {
     ko->ns[0] = g->k; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;
   } else {
@@ -160,6 +180,21 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
 // entry index within a group -> (pc, ccg, r, s); returns false for the zero padding entry
 __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e, int *pc, int *ccg,
                                                         int *r, int *s) {
+  if (ko.rows) {
+    // plane g holds k * k * nsl(g) * 2 chunk planes, nsl = 4 except for a partial last plane
+    if (e >= ko.e) return false;
+    const int per_full = ko.k * ko.k * 8;
+    const int gpl = e / per_full, rem = e - gpl * per_full;
+    const int left = ko.c_in - 64 * gpl;
+    const int nsl = left >= 64 ? 4 : (left + 15) / 16;
+    const int half = rem & 1, q = rem >> 1;
+    const int sl = q % nsl, tap = q / nsl;
+    *r = tap / ko.k;
+    *s = tap - *r * ko.k;
+    *ccg = gpl * 8 + sl * 2 + half;
+    *pc = 0;
+    return true;
+  }
   if (ko.pair >= 2) {
     // (tap row, pair shift, chunk of the pair row); *ccg returns the chunk, *s the shift
     if (e >= ko.e) return false;
@@ -209,6 +244,11 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
 // (channel chunk cc in [0,cch), tap r, s) -> position of that chunk in the packed weights,
 // in units of chunk planes (n_pad * 8 elements each)
 __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc, int r, int s) {
+  if (ko.rows) {
+    const int gpl = cc >> 3, left = ko.c_in - 64 * gpl;
+    const int nsl = left >= 64 ? 4 : (left + 15) / 16;
+    return gpl * ko.k * ko.k * 8 + ((r * ko.k + s) * nsl + ((cc & 7) >> 1)) * 2 + (cc & 1);
+  }
   if (ko.pair == 2)            // the copy for the first pixel of the pair: dx = s, pixel s & 1 of shift s >> 1
     return (r * ko.ns[0] + (s >> 1)) * 2 * ko.cch + (s & 1) * ko.cch + cc;
   if (ko.pair == 3) {          // tap s sits at patch column s + a of the output's pair
@@ -285,6 +325,10 @@ dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_g
                                   const float *bias, dc_act act, const void *residual, void *y,
                                   void *workspace, cudaStream_t stream);
 bool dc_conv_pairrows_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_launch_conv_rows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y,
+                              void *workspace, cudaStream_t stream);
+bool dc_conv_rows_supported(int n, int h, int w, const dc_geom *g);
 dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                               const float *bias, dc_act act, const void *residual, void *y,
                               void *workspace, cudaStream_t stream);

@@ -396,7 +396,7 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   if (g->stride == 2 && (w % 2 || g->k == 1)) return false;
   KOrder ko;
   dc_korder_init(&ko, g);
-  if (ko.e_pad > 256 || ko.fold || ko.pair) return false;    // fold- and pair-order weights belong to their own kernels
+  if (ko.e_pad > 256 || ko.fold || ko.pair || ko.rows) return false;    // fold- and pair-order weights belong to their own kernels
   const int ho = dc_out_extent(h, g->k, g->stride, g->pad), wo = dc_out_extent(w, g->k, g->stride, g->pad);
   if (ho <= 0 || wo <= 0) return false;
   if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;

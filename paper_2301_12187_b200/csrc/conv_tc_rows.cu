@@ -1,0 +1,447 @@
+// Dense stride-1 convolution with many input channels as an implicit GEMM over PIXEL ROWS fed
+// straight from TMA tiles (see KOrder, "rows" order).
+//
+// A shared-memory line (128 bytes) holds 64 channels of one pixel; the input channels are cut into
+// planes of 64 (the last one zero filled by the TMA unit), and a GEMM row is a pixel of the haloed
+// patch.  Tap (r, s) of plane g is the plane's tile read (r * patch width + s) lines further on, so
+// one 4-D TMA load per (tile, plane) -- box 64 channels x patch width x patch rows x images, 128-byte
+// swizzle, zero fill outside the image -- feeds every instruction of that plane.  Small feature
+// maps are tiled several images at a time (the box's image extent), so that the 128 rows of a
+// block are not mostly halo and the weights, which are far larger than the activations in these
+// layers, are streamed once per group of images instead of once per image.
+//
+// The reduction runs over (plane g, tap row r) steps.  Each step needs k * nsl(g) * 2 chunk planes
+// of weights ([n_tile rows][8] bf16, no swizzle), which stream through their own ring: a layer such
+// as 160 -> 960, 3x3 has 2.8 MB of weights, 40x the activations of an image.  Output channels go in
+// passes of n_tile <= 128; accumulators (blocks of 128 rows x n_tile columns) live in tensor memory,
+// two sets when they fit so that the epilogue of one work item overlaps the MMAs of the next.
+//
+// Roles (352 threads): warp 0 producer (one lane issues TMA / bulk loads in consumption order),
+// warps 1-2 MMA issue (blocks alternate between them), warps 3-10 epilogue (two per tensor-memory
+// lane quadrant, blocks alternate).  A work item is (tile, output-channel pass); CTAs (one per SM)
+// take contiguous runs of items.  All waits are bounded (tc::mbar_wait).
+#include "tc_ptx.cuh"
+
+namespace {
+using namespace tc;
+
+constexpr int kMaxA = 3;                         // activation plane stages
+constexpr int kMaxB = 4;                         // weight stages
+constexpr int kMmaWarp = 1;
+constexpr int kMmaWarps = 2;
+constexpr int kFirstEpiWarp = kMmaWarp + kMmaWarps;
+constexpr int kEpiWarps = 8;
+constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
+constexpr int kThreads = 32 + kConsumerThreads;
+constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
+constexpr int kMaxBlocks = 2;                    // 128-row blocks per tile
+
+struct RowsParams {
+  int n_img, h, w, ho, wo, c_in, c_out;
+  int k, pad, planes;          // planes of 64 input channels
+  int tw, th, nxt, wbox, rbox, ni;   // tile: outputs per row, rows, strips per row, patch width / rows, images
+  int tiles_y, img_groups;
+  int grid, items_per, items_rem;    // CTAs; CTA b takes items_per (+1 if b < items_rem) work items
+  int n_tile, nnt, n_pad;      // output channels per pass, passes, nnt * n_tile
+  int mb;                      // blocks per tile
+  int lines_img;               // rbox * wbox: GEMM rows per image of a tile
+  int a_stage_bytes, a_box_bytes, b_stage_bytes;
+  int sa, sb, nacc, act;
+  int off_bias, off_b, off_a, smem_bytes;
+  int tmem_cols;
+};
+
+struct Shared {
+  uint64_t a_full[kMaxA], a_empty[kMaxA];
+  uint64_t b_full[kMaxB], b_empty[kMaxB];
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  uint32_t abort;
+};
+
+// 16-channel K steps of plane g
+__device__ __forceinline__ int plane_steps(const RowsParams &p, int g) {
+  const int left = p.c_in - 64 * g;
+  return left >= 64 ? 4 : (left + 15) >> 4;
+}
+
+// work item -> (pass, image group, column strip, row tile); items are ordered (tile, pass)
+struct Item {
+  int nt, img0, xt, ty;
+  __device__ __forceinline__ void of(const RowsParams &p, int item) {
+    const int tile = item / p.nnt;
+    nt = item - tile * p.nnt;
+    const int strip = tile / p.tiles_y;
+    ty = tile - strip * p.tiles_y;
+    const int ig = strip / p.nxt;
+    xt = strip - ig * p.nxt;
+    img0 = ig * p.ni;
+  }
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ RowsParams p,
+               const void *__restrict__ w_packed, const float *__restrict__ bias,
+               const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y, DcWsHeader *ws) {
+  extern __shared__ __align__(1024) uint8_t smem_raw_base[];
+  __shared__ __align__(8) Shared sh;
+
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~uintptr_t(1023));
+  uint8_t *smem_b = smem + p.off_b;
+  uint8_t *smem_a = smem + p.off_a;              // 1024-byte aligned stages (the swizzle pattern repeats every 1024 bytes)
+  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile uint32_t *abort_flag = &sh.abort;
+
+  const int bid = (int)blockIdx.x;
+  const int nitems = p.items_per + (bid < p.items_rem ? 1 : 0);
+  const int item0 = bid * p.items_per + (bid < p.items_rem ? bid : p.items_rem);
+
+  {
+    const int t = (int)threadIdx.x;
+    bool did = false;
+    if (t < p.sa) { mbar_init(&sh.a_full[t], 1); mbar_init(&sh.a_empty[t], kMmaWarps); did = true; }
+    else if (t >= 32 && t < 32 + p.sb) { mbar_init(&sh.b_full[t - 32], 1); mbar_init(&sh.b_empty[t - 32], kMmaWarps); did = true; }
+    else if (t >= 64 && t < 66) { mbar_init(&sh.acc_full[t - 64], kMmaWarps); mbar_init(&sh.acc_empty[t - 64], kEpiWarps); did = true; }
+    else if (t == 96) { sh.abort = 0; prefetch_tensormap(&map_a); did = true; }
+    if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == 0) {
+    // ================================================================== producer
+    if (lane == 0) {
+      const uint32_t a_base0 = smem_u32(smem_a), b_base0 = smem_u32(smem_b);
+      const char *wsrc = reinterpret_cast<const char *>(w_packed);
+      int sa = 0, sb = 0;
+      uint32_t pa = 0, pb = 0;
+      bool ok = true;
+#pragma unroll 1
+      for (int it = 0; it < nitems && ok; ++it) {
+        Item q;
+        q.of(p, item0 + it);
+#pragma unroll 1
+        for (int g = 0; g < p.planes && ok; ++g) {
+          if (!mbar_wait(&sh.a_empty[sa], pa ^ 1, abort_flag, ws, 0x10000u | sa)) { ok = false; break; }
+          // channels past c_in, pixels outside the image and images past the batch arrive as zeros
+          mbar_arrive_expect_tx(&sh.a_full[sa], (uint32_t)p.a_box_bytes);
+          tma_load_4d(a_base0 + (uint32_t)sa * (uint32_t)p.a_stage_bytes, &map_a, &sh.a_full[sa], 64 * g,
+                      q.xt * p.tw - p.pad, q.ty * p.th - p.pad, q.img0);
+          if (++sa == p.sa) { sa = 0; pa ^= 1; }
+          const int nsl = plane_steps(p, g);
+          const int nplanes = p.k * nsl * 2;     // chunk planes of one (g, r) step
+#pragma unroll 1
+          for (int r = 0; r < p.k; ++r) {
+            if (!mbar_wait(&sh.b_empty[sb], pb ^ 1, abort_flag, ws, 0x20000u | sb)) { ok = false; break; }
+            const uint32_t dst = b_base0 + (uint32_t)sb * (uint32_t)p.b_stage_bytes;
+            const size_t plane0 = (size_t)g * p.k * p.k * 8 + (size_t)r * nplanes;
+            mbar_arrive_expect_tx(&sh.b_full[sb], (uint32_t)(nplanes * p.n_tile * 16));
+            if (p.nnt == 1) {
+              bulk_load(dst, wsrc + plane0 * p.n_pad * 16, (uint32_t)(nplanes * p.n_tile * 16), &sh.b_full[sb]);
+            } else {
+              for (int pl = 0; pl < nplanes; ++pl)
+                bulk_load(dst + (uint32_t)(pl * p.n_tile * 16),
+                          wsrc + ((plane0 + pl) * p.n_pad + (size_t)q.nt * p.n_tile) * 16, (uint32_t)(p.n_tile * 16),
+                          &sh.b_full[sb]);
+            }
+            if (++sb == p.sb) { sb = 0; pb ^= 1; }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- consumer preparation
+    if (warp == kMmaWarp) {
+      tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
+      tmem_relinquish();
+    } else if (warp >= kFirstEpiWarp) {
+      for (int t = (int)threadIdx.x - kFirstEpiWarp * 32; t < p.n_pad; t += kEpiWarps * 32)
+        bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
+    }
+    tc_fence_before();
+    bar_sync(kBarConsumers, kConsumerThreads);
+    tc_fence_after();
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp < kFirstEpiWarp) {
+      // ================================================================== MMA issue
+      const int mw = warp - kMmaWarp;
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) | (8u << 24);
+      const uint32_t b_hi = (128u >> 4) | (1u << 14);                 // no swizzle: 128 bytes between 8-row groups
+      const uint32_t a_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128-byte swizzle: 1024 bytes between 8-row groups
+      const uint32_t a_row0 = smem_u32(smem_a) >> 4, b_row0 = smem_u32(smem_b) >> 4;
+      int sa = 0, sb = 0;
+      uint32_t pa = 0, pb = 0;
+      uint32_t acc_ph[2] = {1u, 1u};             // parity this warp waits for on acc_empty (first use passes)
+      bool ok = true;
+#pragma unroll 1
+      for (int it = 0; it < nitems && ok; ++it) {
+        const int set = p.nacc == 2 ? (it & 1) : 0;
+        if (!warp_wait(&sh.acc_empty[set], acc_ph[set], abort_flag, ws, 0x30000u | set)) break;
+        acc_ph[set] ^= 1u;
+        tc_fence_after();
+        bool first = true;
+#pragma unroll 1
+        for (int g = 0; g < p.planes && ok; ++g) {
+          if (!warp_wait(&sh.a_full[sa], pa, abort_flag, ws, 0x40000u | sa)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_stage = a_row0 + (uint32_t)sa * ((uint32_t)p.a_stage_bytes >> 4);
+          const int nsl = plane_steps(p, g);
+#pragma unroll 1
+          for (int r = 0; r < p.k; ++r) {
+            if (!warp_wait(&sh.b_full[sb], pb, abort_flag, ws, 0x50000u | sb)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t b_stage = b_row0 + (uint32_t)sb * ((uint32_t)p.b_stage_bytes >> 4);
+#pragma unroll 1
+            for (int b = mw; b < p.mb; b += kMmaWarps) {
+              const uint32_t d = tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile);
+              const uint32_t a_blk = a_stage + (uint32_t)(b * 1024 + r * p.wbox * 8);
+#pragma unroll 1
+              for (int s = 0; s < p.k; ++s) {
+#pragma unroll 1
+                for (int sl = 0; sl < nsl; ++sl) {
+                  const uint32_t a_lo = ((a_blk + (uint32_t)(s * 8 + sl * 2)) & 0x3FFFu) | (1u << 16);
+                  const uint32_t b_lo = ((b_stage + (uint32_t)((s * nsl + sl) * 2 * p.n_tile)) & 0x3FFFu) |
+                                        ((uint32_t)p.n_tile << 16);
+                  const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)a_lo;
+                  const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
+                  const uint32_t accum = (first && s == 0 && sl == 0) ? 0u : 1u;
+                  if (elect_one()) umma_bf16(d, ad, bd, idesc, accum);
+                }
+              }
+            }
+            first = false;
+            if (elect_one()) umma_commit(&sh.b_empty[sb]);      // this warp is done with the weight stage
+            if (++sb == p.sb) { sb = 0; pb ^= 1; }
+          }
+          if (ok && elect_one()) umma_commit(&sh.a_empty[sa]);  // ... and with the plane
+          if (++sa == p.sa) { sa = 0; pa ^= 1; }
+        }
+        if (ok && elect_one()) umma_commit(&sh.acc_full[set]);  // this warp's blocks of the item are complete
+      }
+    } else {
+      // ================================================================== epilogue
+      // Two warps per tensor-memory lane quadrant; blocks alternate between them.  A thread owns a
+      // GEMM row = one pixel of the patch; valid ones store their n_tile channels 16 bytes at a time.
+      const int ew = warp - kFirstEpiWarp;
+      const int q = warp & 3, par = ew >> 2;
+      const uint32_t tmem_row = tmem_base + ((uint32_t)(q * 32) << 16);
+      uint32_t acc_ph[2] = {0u, 0u};
+#pragma unroll 1
+      for (int it = 0; it < nitems; ++it) {
+        const int set = p.nacc == 2 ? (it & 1) : 0;
+        Item iq;
+        iq.of(p, item0 + it);
+        if (!warp_wait(&sh.acc_full[set], acc_ph[set], abort_flag, ws, 0x60000u | set)) break;
+        acc_ph[set] ^= 1u;
+        tc_fence_after();
+        const int x0 = iq.xt * p.tw, y0 = iq.ty * p.th;
+        const int tw_valid = p.wo - x0 < p.tw ? p.wo - x0 : p.tw;
+        const int th_valid = p.ho - y0 < p.th ? p.ho - y0 : p.th;
+        const int ch0 = iq.nt * p.n_tile;
+        const int nch = p.c_out - ch0 < p.n_tile ? p.c_out - ch0 : p.n_tile;   // multiple of 8
+#pragma unroll 1
+        for (int b = par; b < p.mb; b += 2) {
+          const int pos = b * 128 + q * 32 + lane;
+          const int il = pos / p.lines_img, rem = pos - il * p.lines_img;
+          const int yy = rem / p.wbox, xx = rem - yy * p.wbox;
+          const bool valid = il < p.ni && iq.img0 + il < p.n_img && yy < th_valid && xx < tw_valid;
+          const size_t pix = ((size_t)(iq.img0 + il) * p.ho + (size_t)(y0 + yy)) * p.wo + (size_t)(x0 + xx);
+          __nv_bfloat16 *dst = y + pix * p.c_out + ch0;
+          const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out + ch0 : nullptr;
+          const uint32_t taddr = tmem_row + (uint32_t)((set * p.mb + b) * p.n_tile);
+#pragma unroll 1
+          for (int ch = 0; ch < nch; ch += 8) {
+            uint32_t v[8];
+            tmem_ld8(taddr + (uint32_t)ch, v);
+            tmem_ld_wait();
+            if (valid) {
+              const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch);
+              const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch + 4);
+              float f[8];
+              f[0] = __uint_as_float(v[0]) + b0.x; f[1] = __uint_as_float(v[1]) + b0.y;
+              f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
+              f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
+              f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
+              if (rp) {
+                const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
+                const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float2 rf = __bfloat1622float2(rb[i]);
+                  f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                }
+              }
+              uint4 ov;
+              __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float f0 = f[2 * i], f1 = f[2 * i + 1];
+                if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
+                ob[i] = __floats2bfloat162_rn(f0, f1);
+              }
+              *reinterpret_cast<uint4 *>(dst + ch) = ov;
+            }
+          }
+        }
+        // this warp has read what it needs of the accumulator set
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.acc_empty[set]);
+      }
+    }
+    // ---- consumer teardown
+    if (*abort_flag) {
+      const unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    bar_sync(kBarConsumers, kConsumerThreads);
+    if (warp == kMmaWarp) {
+      tc_fence_after();
+      tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+constexpr int kSmemBudget = 220 * 1024;
+constexpr int kMaxLines = 128 * kMaxBlocks;      // GEMM rows of a tile
+constexpr int kSlack = 1024;
+
+bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
+  KOrder ko;
+  dc_korder_init(&ko, g);
+  if (!ko.rows) return false;
+  const int ho = dc_out_extent(h, g->k, 1, g->pad), wo = dc_out_extent(w, g->k, 1, g->pad);
+  if (ho <= 0 || wo <= 0) return false;
+  if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;
+  p->n_img = n; p->h = h; p->w = w; p->ho = ho; p->wo = wo;
+  p->c_in = g->c_in; p->c_out = g->c_out;
+  p->k = g->k; p->pad = g->pad;
+  p->planes = dc_div_up(g->c_in, 64);
+  p->n_tile = ko.n_tile; p->nnt = ko.nnt; p->n_pad = ko.n_pad;
+  // tile: as many rows as fit kMaxLines GEMM rows; whole small images several at a time
+  p->nxt = 1;
+  while (dc_div_up(wo, p->nxt) + g->k - 1 > kMaxLines / g->k) ++p->nxt;   // at least one output row per tile
+  p->tw = dc_div_up(wo, p->nxt);
+  p->nxt = dc_div_up(wo, p->tw);
+  p->wbox = p->tw + g->k - 1;
+  int th = kMaxLines / p->wbox - (g->k - 1);
+  if (th < 1) return false;
+  if (th > ho) th = ho;
+  p->th = th;
+  p->rbox = th + g->k - 1;
+  p->lines_img = p->rbox * p->wbox;
+  p->ni = 1;
+  if (th == ho && p->nxt == 1) {
+    p->ni = kMaxLines / p->lines_img;
+    if (p->ni > n) p->ni = n;
+    if (p->ni > 8) p->ni = 8;
+    if (p->ni < 1) p->ni = 1;
+  }
+  if (p->wbox > 256 || p->rbox > 256) return false;
+  p->tiles_y = dc_div_up(ho, th);
+  p->img_groups = dc_div_up(n, p->ni);
+  const int last = (p->ni - 1) * p->lines_img + (th - 1) * p->wbox + p->tw;    // GEMM rows up to the last valid one
+  p->mb = dc_div_up(last, 128);
+  if (p->mb > kMaxBlocks) return false;
+  p->nacc = (2 * p->mb * p->n_tile <= 512) ? 2 : 1;
+  if (p->nacc * p->mb * p->n_tile > 512) return false;
+  int cols = 32;
+  while (cols < p->nacc * p->mb * p->n_tile) cols *= 2;
+  p->tmem_cols = cols;
+  const long long items = (long long)p->img_groups * p->nxt * p->tiles_y * p->nnt;
+  if (items >= (1ll << 30)) return false;
+  p->grid = items < n_sm ? (int)items : n_sm;
+  p->items_per = (int)(items / p->grid);
+  p->items_rem = (int)(items % p->grid);
+  p->a_box_bytes = p->ni * p->lines_img * 128;
+  p->a_stage_bytes = (int)dc_round_up((size_t)p->a_box_bytes, 1024);
+  p->b_stage_bytes = (int)dc_round_up((size_t)g->k * 4 * 2 * p->n_tile * 16, 1024);
+  // Layout: bias, activation stages, weight stages.  A block's 128 GEMM rows plus the tap shift may
+  // reach up to ~200 lines (25 KB) past its stage; behind the last activation stage that lands in
+  // the weight stages, which are larger (what is read there only feeds rows that are dropped).
+  p->off_bias = 0;
+  p->off_a = (int)dc_round_up((size_t)p->n_pad * 4, 1024);
+  // rings: weights first (they are the larger stream), then activation planes
+  int sa = 2, sb = 2;
+  auto total = [&](int a, int b) {
+    const long long wbytes = (long long)b * p->b_stage_bytes;
+    const long long tail = wbytes >= 26 * 1024 ? kSlack : 26 * 1024 - wbytes + kSlack;   // room for the overrun
+    return 1024ll + p->off_a + wbytes + (long long)a * p->a_stage_bytes + tail;
+  };
+  if (total(sa, sb) > kSmemBudget) return false;
+  while (sb < kMaxB && total(sa, sb + 1) <= kSmemBudget) ++sb;
+  while (sa < kMaxA && total(sa + 1, sb) <= kSmemBudget) ++sa;
+  p->sa = sa; p->sb = sb;
+  p->off_b = p->off_a + sa * p->a_stage_bytes;
+  p->smem_bytes = (int)total(sa, sb);
+  return true;
+}
+
+}  // namespace
+
+bool dc_conv_rows_supported(int n, int h, int w, const dc_geom *g) {
+  RowsParams p;
+  return rows_plan(n, h, w, g, 148, &p);
+}
+
+dc_status dc_launch_conv_rows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y, void *workspace,
+                              cudaStream_t stream) {
+  RowsParams p;
+  const int n_sm = sm_count();
+  if (!rows_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
+  p.act = (int)act;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return DC_ERR_CUDA;
+  CUtensorMap map_a;
+  {
+    const cuuint64_t C = (cuuint64_t)g->c_in;
+    cuuint64_t gdim[4] = {C, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t gstr[3] = {2 * C, (cuuint64_t)w * C * 2, (cuuint64_t)h * w * C * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)p.wbox, (cuuint32_t)p.rbox, (cuuint32_t)p.ni};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), gdim, gstr, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_rows, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+    attr_set = true;
+  }
+  k_conv_tc_rows<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_a, p, w_packed, bias, (const __nv_bfloat16 *)residual,
+                                                            (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
