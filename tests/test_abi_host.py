@@ -90,14 +90,16 @@ def test_packed_bytes():
 
 
 def test_kernel_name_query_follows_the_dispatch_rules():
-    # small-channel stride-1 3x3: pair order, 5x5: fold order; wide or strided: general tensor-core kernel;
+    # few input channels: pair rows; many channels and >= 48 outputs, stride 1: rows; 40-64 channels, few outputs: fold; wide or strided: general tensor-core kernel;
     # channel counts that are no multiple of 8: CUDA cores
     assert dc.conv_kernel_name(64, 56, 56, dc.geom(24, 24, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_pairrows"
     assert dc.conv_kernel_name(128, 28, 28, dc.geom(32, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_pairrows"
     assert dc.conv_kernel_name(128, 14, 14, dc.geom(40, 32, 1, 5, 1, 2), dc.BF16) == "k_conv_tc_fold"
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(24, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_tc_pairrows"
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(96, 144, 1, 5, 2, 2), dc.BF16) == "k_conv_tc"
-    assert dc.conv_kernel_name(128, 14, 14, dc.geom(96, 576, 1, 1, 1, 0), dc.BF16) == "k_conv_tc"
+    assert dc.conv_kernel_name(128, 14, 14, dc.geom(96, 576, 1, 1, 1, 0), dc.BF16) == "k_conv_tc_rows"
+    assert dc.conv_kernel_name(128, 7, 7, dc.geom(160, 960, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_rows"
+    assert dc.conv_kernel_name(128, 28, 28, dc.geom(144, 32, 1, 3, 1, 1), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 224, 224, dc.geom(3, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_smallcin_bf16"
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(20, 12, 1, 3, 1, 1), dc.BF16) == "k_conv_dense_bf16"
     assert dc.conv_kernel_name(2, 16, 16, dc.geom(16, 24, 1, 3, 1, 1), dc.F32) == "k_conv_dense_f32"

@@ -214,6 +214,11 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with a wide output: general kernel
     (16, 128, 3, 1, 1, 1, 12, 16, "k_conv_tc_pairrows"),    # N = 256: two accumulator slots, run-time channel loop
     (32, 64, 3, 2, 1, 1, 28, 28, "k_conv_tc_pairrows"),     # stride 2, 64 output channels
+    (160, 200, 3, 1, 1, 5, 7, 7, "k_conv_tc_rows"),         # three planes (the last half full), two passes, three images per tile
+    (96, 64, 1, 1, 0, 7, 7, 7, "k_conv_tc_rows"),           # 1x1: five images per tile, the last group partial
+    (64, 48, 5, 1, 2, 1, 20, 70, "k_conv_tc_rows"),         # 5x5, two column strips, row tiles
+    (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
+    (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc"),             # many channels, few outputs: general kernel
 ])
 def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, w, kernel):
     g = dc.geom(c_in, c_out, 1, k, s, p)
