@@ -16,7 +16,7 @@
 // passes of n_tile <= 128; accumulators (blocks of 128 rows x n_tile columns) live in tensor memory,
 // two sets when they fit so that the epilogue of one work item overlaps the MMAs of the next.
 //
-// Roles (352 threads): warp 0 producer (one lane issues TMA / bulk loads in consumption order),
+// Roles (352 threads): warp 0 producer (issues TMA / bulk loads in consumption order),
 // warps 1-2 MMA issue (blocks alternate between them), warps 3-10 epilogue (two per tensor-memory
 // lane quadrant, blocks alternate).  A work item is (tile, output-channel pass); CTAs (one per SM)
 // take contiguous runs of items.  All waits are bounded (tc::mbar_wait).
@@ -111,7 +111,9 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     // ================================================================== producer
-    if (lane == 0) {
+    // The whole warp walks the loop (every lane observes the barriers itself); lane 0 announces the
+    // bytes and issues the activation tile, the weight planes of a step are issued one per lane.
+    {
       const uint32_t a_base0 = smem_u32(smem_a), b_base0 = smem_u32(smem_b);
       const char *wsrc = reinterpret_cast<const char *>(w_packed);
       int sa = 0, sb = 0;
@@ -123,24 +125,29 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         q.of(p, item0 + it);
 #pragma unroll 1
         for (int g = 0; g < p.planes && ok; ++g) {
-          if (!mbar_wait(&sh.a_empty[sa], pa ^ 1, abort_flag, ws, 0x10000u | sa)) { ok = false; break; }
-          // channels past c_in, pixels outside the image and images past the batch arrive as zeros
-          mbar_arrive_expect_tx(&sh.a_full[sa], (uint32_t)p.a_box_bytes);
-          tma_load_4d(a_base0 + (uint32_t)sa * (uint32_t)p.a_stage_bytes, &map_a, &sh.a_full[sa], 64 * g,
-                      q.xt * p.tw - p.pad, q.ty * p.th - p.pad, q.img0);
+          if (!warp_wait(&sh.a_empty[sa], pa ^ 1, abort_flag, ws, 0x10000u | sa)) { ok = false; break; }
+          if (lane == 0) {
+            // channels past c_in, pixels outside the image and images past the batch arrive as zeros
+            mbar_arrive_expect_tx(&sh.a_full[sa], (uint32_t)p.a_box_bytes);
+            tma_load_4d(a_base0 + (uint32_t)sa * (uint32_t)p.a_stage_bytes, &map_a, &sh.a_full[sa], 64 * g,
+                        q.xt * p.tw - p.pad, q.ty * p.th - p.pad, q.img0);
+          }
           if (++sa == p.sa) { sa = 0; pa ^= 1; }
           const int nsl = plane_steps(p, g);
           const int nplanes = p.k * nsl * 2;     // chunk planes of one (g, r) step
 #pragma unroll 1
           for (int r = 0; r < p.k; ++r) {
-            if (!mbar_wait(&sh.b_empty[sb], pb ^ 1, abort_flag, ws, 0x20000u | sb)) { ok = false; break; }
+            if (!warp_wait(&sh.b_empty[sb], pb ^ 1, abort_flag, ws, 0x20000u | sb)) { ok = false; break; }
             const uint32_t dst = b_base0 + (uint32_t)sb * (uint32_t)p.b_stage_bytes;
             const size_t plane0 = (size_t)g * p.k * p.k * 8 + (size_t)r * nplanes;
-            mbar_arrive_expect_tx(&sh.b_full[sb], (uint32_t)(nplanes * p.n_tile * 16));
+            if (lane == 0) mbar_arrive_expect_tx(&sh.b_full[sb], (uint32_t)(nplanes * p.n_tile * 16));
+            __syncwarp();
             if (p.nnt == 1) {
-              bulk_load(dst, wsrc + plane0 * p.n_pad * 16, (uint32_t)(nplanes * p.n_tile * 16), &sh.b_full[sb]);
+              if (lane == 0)
+                bulk_load(dst, wsrc + plane0 * p.n_pad * 16, (uint32_t)(nplanes * p.n_tile * 16), &sh.b_full[sb]);
             } else {
-              for (int pl = 0; pl < nplanes; ++pl)
+              // a pass takes n_tile of the n_pad rows of every plane
+              for (int pl = lane; pl < nplanes; pl += 32)
                 bulk_load(dst + (uint32_t)(pl * p.n_tile * 16),
                           wsrc + ((plane0 + pl) * p.n_pad + (size_t)q.nt * p.n_tile) * 16, (uint32_t)(p.n_tile * 16),
                           &sh.b_full[sb]);
