@@ -405,7 +405,7 @@ def run_ours(args):
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the conv forward kernel (profiles/);
 # None until captured, and again once the kernel has changed since
-PROFILED_TRAFFIC = {"cfg1": 9741568, "cfg2": None, "cfg3": None}   # cfg1: profiles/k_conv_tc_pairrows_cfg1.md
+PROFILED_TRAFFIC = {"cfg1": 9743104, "cfg2": None, "cfg3": None}   # cfg1: profiles/k_conv_tc_pairrows_cfg1.md
 
 
 # --------------------------------------------------------------------------------------------- oracle
