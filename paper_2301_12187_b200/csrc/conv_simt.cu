@@ -116,6 +116,7 @@ static inline int simt_blocks(long long total, int threads, int cap) {
 // ----------------------------------------------------------------------------------------------
 constexpr int kSmallCinMax = 4;
 constexpr int kSmallTile = 128;
+constexpr int kSmallRows = 2;                    // output rows per thread
 
 template <int CO_T>
 __global__ void __launch_bounds__(kSmallTile)
@@ -127,7 +128,7 @@ k_conv_smallcin_bf16(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *_
   const int taps = g.k * g.k;
   float *w_s = reinterpret_cast<float *>(sm_raw);                       // [taps][c_in][CO_T]
   float *b_s = w_s + taps * g.c_in * CO_T;                              // [CO_T]
-  __nv_bfloat16 *x_s = reinterpret_cast<__nv_bfloat16 *>(b_s + CO_T);   // [k][span][c_in]
+  __nv_bfloat16 *x_s = reinterpret_cast<__nv_bfloat16 *>(b_s + CO_T);   // [(rows-1)*stride + k][span][c_in]
   const int span = (kSmallTile - 1) * g.stride + g.k;                   // input pixels per staged row
   const int row_elems = span * g.c_in;
   const int tid = (int)threadIdx.x;
@@ -143,16 +144,20 @@ k_conv_smallcin_bf16(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *_
     w_s[i] = wv;
   }
   if (tid < CO_T) b_s[tid] = (bias && o0 + tid < g.c_out) ? bias[o0 + tid] : 0.f;
-  const long long total = (long long)n * ho * xtiles;
+  // a tile = kSmallRows output rows x 128 pixels; a thread computes its pixel in each of the rows,
+  // so every weight vector it reads from shared memory feeds kSmallRows x 4 FMAs
+  const int ypairs = (ho + kSmallRows - 1) / kSmallRows;
+  const int srows = (kSmallRows - 1) * g.stride + g.k;                  // staged input rows
+  const long long total = (long long)n * ypairs * xtiles;
   for (long long tile = blockIdx.x; tile < total; tile += gridDim.x) {
     const int xt = (int)(tile % xtiles);
     const long long rowi = tile / xtiles;
-    const int Y = (int)(rowi % ho), img = (int)(rowi / ho);
+    const int Y0 = (int)(rowi % ypairs) * kSmallRows, img = (int)(rowi / ypairs);
     const int X0 = xt * kSmallTile;
-    const int gx0 = X0 * g.stride - g.pad, gy0 = Y * g.stride - g.pad;
+    const int gx0 = X0 * g.stride - g.pad, gy0 = Y0 * g.stride - g.pad;
     __syncthreads();                              // weights staged / previous tile done with x_s
-    // stage the k input rows of the segment: thread = pixel, contiguous along the row
-    for (int r = 0; r < g.k; ++r) {
+    // stage the input rows of the tile: thread = pixel, contiguous along the row
+    for (int r = 0; r < srows; ++r) {
       const int gy = gy0 + r;
       const bool rok = gy >= 0 && gy < h;
       const __nv_bfloat16 *src = x + (((size_t)img * h + (rok ? gy : 0)) * wd) * g.c_in;
@@ -166,41 +171,51 @@ k_conv_smallcin_bf16(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *_
     __syncthreads();
     const int X = X0 + tid;
     if (X < wo) {
-      float acc[CO_T];
+      float acc[kSmallRows][CO_T];
 #pragma unroll
-      for (int o = 0; o < CO_T; ++o) acc[o] = b_s[o];
+      for (int j = 0; j < kSmallRows; ++j)
+#pragma unroll
+        for (int o = 0; o < CO_T; ++o) acc[j][o] = b_s[o];
       const __nv_bfloat16 *xp = x_s + tid * g.stride * g.c_in;
       const float *wp = w_s;
       for (int u = 0; u < g.k; ++u, xp += row_elems - g.k * g.c_in) {
         for (int vc = 0; vc < g.k * g.c_in; ++vc, ++xp, wp += CO_T) {
-          const float xv = __bfloat162float(*xp);
+          float xv[kSmallRows];
+#pragma unroll
+          for (int j = 0; j < kSmallRows; ++j) xv[j] = __bfloat162float(xp[j * g.stride * row_elems]);
 #pragma unroll
           for (int o = 0; o < CO_T; o += 4) {
             const float4 w4 = *reinterpret_cast<const float4 *>(wp + o);
-            acc[o] = fmaf(xv, w4.x, acc[o]); acc[o + 1] = fmaf(xv, w4.y, acc[o + 1]);
-            acc[o + 2] = fmaf(xv, w4.z, acc[o + 2]); acc[o + 3] = fmaf(xv, w4.w, acc[o + 3]);
+#pragma unroll
+            for (int j = 0; j < kSmallRows; ++j) {
+              acc[j][o] = fmaf(xv[j], w4.x, acc[j][o]); acc[j][o + 1] = fmaf(xv[j], w4.y, acc[j][o + 1]);
+              acc[j][o + 2] = fmaf(xv[j], w4.z, acc[j][o + 2]); acc[j][o + 3] = fmaf(xv[j], w4.w, acc[j][o + 3]);
+            }
           }
         }
       }
-      const size_t oi = (((size_t)img * ho + Y) * wo + X) * g.c_out + o0;
 #pragma unroll
-      for (int o = 0; o < CO_T; o += 8) {
-        if (o0 + o < g.c_out) {                   // c_out is a multiple of 8
-          if (residual) {
-            const uint4 rv = *reinterpret_cast<const uint4 *>(residual + oi + o);
-            const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+      for (int j = 0; j < kSmallRows; ++j) {
+        const size_t oi = (((size_t)img * ho + (Y0 + j)) * wo + X) * g.c_out + o0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float2 rf = __bfloat1622float2(rb[i]);
-              acc[o + 2 * i] += rf.x; acc[o + 2 * i + 1] += rf.y;
+        for (int o = 0; o < CO_T; o += 8) {
+          if (Y0 + j < ho && o0 + o < g.c_out) {  // c_out is a multiple of 8
+            if (residual) {
+              const uint4 rv = *reinterpret_cast<const uint4 *>(residual + oi + o);
+              const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 rf = __bfloat1622float2(rb[i]);
+                acc[j][o + 2 * i] += rf.x; acc[j][o + 2 * i + 1] += rf.y;
+              }
             }
-          }
-          uint4 ov;
-          __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+            uint4 ov;
+            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            ob[i] = __floats2bfloat162_rn(dc_act_apply(acc[o + 2 * i], act), dc_act_apply(acc[o + 2 * i + 1], act));
-          *reinterpret_cast<uint4 *>(y + oi + o) = ov;
+            for (int i = 0; i < 4; ++i)
+              ob[i] = __floats2bfloat162_rn(dc_act_apply(acc[j][o + 2 * i], act), dc_act_apply(acc[j][o + 2 * i + 1], act));
+            *reinterpret_cast<uint4 *>(y + oi + o) = ov;
+          }
         }
       }
     }
@@ -232,8 +247,9 @@ dc_status dc_launch_conv_simt(const void *x, int n, int h, int w, const dc_geom 
       constexpr int CO_T = 32;
       const int xtiles = dc_div_up(wo, kSmallTile);
       const int span = (kSmallTile - 1) * g->stride + g->k;
-      const size_t smem = (size_t)(g->k * g->k * g->c_in * CO_T + CO_T) * 4 + (size_t)g->k * span * g->c_in * 2;
-      const long long tiles = (long long)n * ho * xtiles;
+      const size_t smem = (size_t)(g->k * g->k * g->c_in * CO_T + CO_T) * 4 +
+                          (size_t)((kSmallRows - 1) * g->stride + g->k) * span * g->c_in * 2;
+      const long long tiles = (long long)n * dc_div_up(ho, kSmallRows) * xtiles;
       const int grid = (int)(tiles < 148 * 8 ? tiles : 148 * 8);      // persistent CTAs, 8 per SM
       for (int o0 = 0; o0 < g->c_out; o0 += CO_T)                      // one pass per 32 output channels
         k_conv_smallcin_bf16<CO_T><<<grid, kSmallTile, smem, stream>>>(
