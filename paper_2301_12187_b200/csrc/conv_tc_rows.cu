@@ -204,18 +204,23 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
             for (int b = mw; b < p.mb; b += kMmaWarps) {
               const uint32_t d = tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile);
-              const uint32_t a_blk = a_stage + (uint32_t)(b * 1024 + r * p.wbox * 8);
+              // descriptors advance by adds only: +8 (one line) per tap column, +2 (32 bytes) per K step on
+              // the activation side, two chunk planes per instruction on the weight side
+              uint32_t a_lo = ((a_stage + (uint32_t)(b * 1024 + r * p.wbox * 8)) & 0x3FFFu) | (1u << 16);
+              uint32_t b_lo = (b_stage & 0x3FFFu) | ((uint32_t)p.n_tile << 16);
+              const uint32_t b_inc = 2u * (uint32_t)p.n_tile;
+              uint32_t accum = first ? 0u : 1u;
 #pragma unroll 1
-              for (int s = 0; s < p.k; ++s) {
-#pragma unroll 1
-                for (int sl = 0; sl < nsl; ++sl) {
-                  const uint32_t a_lo = ((a_blk + (uint32_t)(s * 8 + sl * 2)) & 0x3FFFu) | (1u << 16);
-                  const uint32_t b_lo = ((b_stage + (uint32_t)((s * nsl + sl) * 2 * p.n_tile)) & 0x3FFFu) |
-                                        ((uint32_t)p.n_tile << 16);
-                  const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)a_lo;
-                  const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-                  const uint32_t accum = (first && s == 0 && sl == 0) ? 0u : 1u;
-                  if (elect_one()) umma_bf16(d, ad, bd, idesc, accum);
+              for (int s = 0; s < p.k; ++s, a_lo += 8u) {
+#pragma unroll
+                for (int sl = 0; sl < 4; ++sl) {
+                  if (sl < nsl) {
+                    const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + 2u * sl);
+                    const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
+                    if (elect_one()) umma_bf16(d, ad, bd, idesc, accum);
+                    accum = 1u;
+                    b_lo += b_inc;
+                  }
                 }
               }
             }
