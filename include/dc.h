@@ -240,6 +240,19 @@ dc_status dc_chain_forward_host(const dc_layer *layers, int n_layers, const dc_r
                                 void *y_host, dc_dtype dtype, void *workspace,
                                 size_t workspace_bytes, dc_stream stream);
 
+/*
+ * The same without the final synchronisation: everything (copies in, merge, forward, copy out) is
+ * queued on `stream` and the call returns.  The host buffers, the layers' host arrays and the
+ * workspace must stay untouched until the stream has passed this point (y_host is valid after the
+ * caller has synchronised the stream or an event recorded behind the call).  With pinned host
+ * buffers and one workspace per stream, calls on different streams overlap their copies in both
+ * directions with each other's kernels: Sec. 5's deployment setting of a stream of input batches.
+ */
+dc_status dc_chain_forward_host_async(const dc_layer *layers, int n_layers, const dc_residual *res,
+                                int n_res, const void *x_host, int n, int h, int w, dc_act act,
+                                void *y_host, dc_dtype dtype, void *workspace,
+                                size_t workspace_bytes, dc_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -196,10 +196,10 @@ extern "C" dc_status dc_chain_host_workspace_bytes(const dc_layer *layers, int n
   return DC_OK;
 }
 
-extern "C" dc_status dc_chain_forward_host(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
-                                           const void *x_host, int n, int h, int w, dc_act act, void *y_host,
-                                           dc_dtype dtype, void *workspace, size_t workspace_bytes,
-                                           dc_stream stream) {
+extern "C" dc_status dc_chain_forward_host_async(const dc_layer *layers, int n_layers, const dc_residual *res,
+                                                 int n_res, const void *x_host, int n, int h, int w, dc_act act,
+                                                 void *y_host, dc_dtype dtype, void *workspace,
+                                                 size_t workspace_bytes, dc_stream stream) {
   HostPlan hp;
   dc_status s = host_plan(layers, n_layers, res, n_res, n, h, w, dtype, &hp);
   if (s != DC_OK) return s;
@@ -239,6 +239,16 @@ extern "C" dc_status dc_chain_forward_host(const dc_layer *layers, int n_layers,
                       stream);
   if (s != DC_OK) return s;
   DC_CUDA_OK(cudaMemcpyAsync(y_host, dy, hp.y_bytes, cudaMemcpyDeviceToHost, st));
-  DC_CUDA_OK(cudaStreamSynchronize(st));
+  return DC_OK;
+}
+
+extern "C" dc_status dc_chain_forward_host(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                                           const void *x_host, int n, int h, int w, dc_act act, void *y_host,
+                                           dc_dtype dtype, void *workspace, size_t workspace_bytes,
+                                           dc_stream stream) {
+  dc_status s = dc_chain_forward_host_async(layers, n_layers, res, n_res, x_host, n, h, w, act, y_host, dtype,
+                                            workspace, workspace_bytes, stream);
+  if (s != DC_OK) return s;
+  DC_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
   return DC_OK;
 }

@@ -82,6 +82,9 @@ EXPORTS = {
     "dc_chain_forward_host": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                         C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p,
                                         C.c_size_t, C.c_void_p]),
+    "dc_chain_forward_host_async": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
+                                        C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p,
+                                        C.c_size_t, C.c_void_p]),
 }
 
 _lib = None
@@ -315,3 +318,14 @@ def chain_forward_host(host_layers, n_layers, residuals, x_host, act, y_host, wo
                                        _ptr(y_host), dtype_code(x_host.dtype), _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _stream(stream)),
            "dc_chain_forward_host")
+
+
+def chain_forward_host_async(host_layers, n_layers, residuals, x_host, act, y_host, workspace, stream=None):
+    """As chain_forward_host, but only queues the work on `stream`: keep every buffer alive and untouched
+    until that stream has been synchronised."""
+    res, n_res = _res_array(residuals)
+    n, h, w, _ = x_host.shape
+    _check(lib().dc_chain_forward_host_async(host_layers, n_layers, res, n_res, _ptr(x_host), n, h, w, act,
+                                       _ptr(y_host), dtype_code(x_host.dtype), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)),
+           "dc_chain_forward_host_async")

@@ -348,6 +348,33 @@ def test_host_entry_point_matches_device_path(dc):
     assert O.rel_l2(yh.float().numpy().transpose(0, 3, 1, 2), ref) <= TOL_BF16
 
 
+def test_async_host_entry_point_overlaps_streams_and_matches_the_oracle(dc):
+    # three batches in flight on three streams, each with its own workspace and pinned buffers
+    arrs, outs, streams, cases = [], [], [], []
+    for slot in range(3):
+        case = I.chain_case(1, seed=20 + slot, batch=3)
+        arr, keep = dc.host_layer_array(case.layers)
+        n, h, w, c = case.x_shape
+        nbytes = dc.chain_host_workspace_bytes(arr, len(case.layers), case.residuals, n, h, w, dc.BF16)
+        ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+        xh = torch.from_numpy(case.x()).to(torch.bfloat16).pin_memory()
+        yh = torch.zeros((n, h, w, 24), dtype=torch.bfloat16).pin_memory()
+        st = torch.cuda.Stream()
+        arrs.append((arr, keep, ws, xh))
+        outs.append(yh); streams.append(st); cases.append(case)
+    torch.cuda.synchronize()
+    for slot in range(3):
+        arr, keep, ws, xh = arrs[slot]
+        dc.chain_forward_host_async(arr, len(cases[slot].layers), cases[slot].residuals, xh, dc.ACT_IDENTITY,
+                                    outs[slot], ws, streams[slot])
+    for slot in range(3):
+        streams[slot].synchronize()
+        assert dc.workspace_status(arrs[slot][2], streams[slot]) == dc.OK
+        case = cases[slot]
+        ref = O.chain_forward_reordered(case.x().transpose(0, 3, 1, 2), case.layers, case.residuals)
+        assert O.rel_l2(outs[slot].float().numpy().transpose(0, 3, 1, 2), ref) <= TOL_BF16
+
+
 def test_empty_and_degenerate_inputs_are_rejected_or_handled(dc):
     g = dc.geom(8, 8, 1, 3, 1, 1)
     packed = torch.zeros(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
