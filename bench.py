@@ -339,7 +339,7 @@ def run_ours(args):
         # memory, merges, runs the forward and copies the output back.  Steps rotate over three
         # streams, each with its own workspace and pinned buffers, so the copies of one step overlap
         # the work of its neighbours; a slot is reused only after its previous step has finished.
-        arr, keep = dc.host_layer_array(case.layers)
+        arr, keep = dc.host_layer_array(case.layers, pinned=True)
         ws_bytes = dc.chain_host_workspace_bytes(arr, len(case.layers), case.residuals, n, h, w, dc.BF16)
         n_slots = 3
         e_ws = [torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_slots)]

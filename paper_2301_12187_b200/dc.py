@@ -282,8 +282,10 @@ def workspace_status(workspace, stream=None) -> int:
     return int(lib().dc_workspace_status(_ptr(workspace), _stream(stream)))
 
 
-def host_layer_array(specs) -> Tuple["C.Array", list]:
-    """dc_layer array whose pointers are HOST pointers (numpy float32), for chain_forward_host."""
+def host_layer_array(specs, pinned: bool = False) -> Tuple["C.Array", list]:
+    """dc_layer array whose pointers are HOST pointers (float32), for chain_forward_host.  With
+    pinned=True the arrays live in page-locked memory, so their copies to the device are queued
+    instead of being staged by the calling thread."""
     import numpy as np
     keep = []
     arr = (Layer * len(specs))()
@@ -292,6 +294,11 @@ def host_layer_array(specs) -> Tuple["C.Array", list]:
         if a is None:
             return None
         a = np.ascontiguousarray(a, dtype=np.float32)
+        if pinned:
+            import torch
+            t = torch.from_numpy(a.copy()).pin_memory()
+            keep.append(t)
+            return t.data_ptr()
         keep.append(a)
         return a.ctypes.data
 
