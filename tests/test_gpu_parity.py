@@ -219,6 +219,7 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (64, 48, 5, 1, 2, 1, 20, 70, "k_conv_tc_rows"),         # 5x5, two column strips, row tiles
     (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
     (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc"),             # many channels, few outputs: general kernel
+    (192, 32, 1, 1, 0, 2, 28, 28, "k_conv_tc_rows"),        # 1x1 projection to 32 channels
 ])
 def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, w, kernel):
     g = dc.geom(c_in, c_out, 1, k, s, p)
