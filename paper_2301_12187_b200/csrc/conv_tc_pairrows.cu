@@ -52,7 +52,7 @@ constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
 constexpr int kThreads = 32 + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
 constexpr int kMaxMma = 64;                      // tensor-core instructions per block
-constexpr int kInFlight = 2;                     // activation tiles a CTA requests ahead of their use
+constexpr int kInFlight = 3;                     // activation tiles a CTA requests ahead of their use
 
 struct PairParams {
   int n_img, h, w, ho, wo, c_in, c_out, co8;
@@ -379,14 +379,15 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
       t.start(p, tile0);
       int s = 0;
       uint32_t ph = 0;
+      const int inflight = p.stages < kInFlight ? p.stages : kInFlight;   // never more than there are stages
 #pragma unroll 1
       for (int it = 0; it < ntiles; ++it) {
         if (!mbar_wait(&sh.empty[s], ph ^ 1, abort_flag, ws, 0x10000u | s)) break;
         // At most kInFlight tiles are on their way: every CTA starts at the same moment, and if
         // each asked for all its tiles at once the first tile (which the tensor core is waiting
         // for) would arrive together with the last.
-        if (it >= kInFlight) {
-          int sw = s - kInFlight;
+        if (it >= inflight) {
+          int sw = s - inflight;
           uint32_t pw = ph;
           if (sw < 0) { sw += p.stages; pw ^= 1; }
           if (!mbar_wait(&sh.full[sw], pw, abort_flag, ws, 0x80000u | sw)) break;
