@@ -169,7 +169,7 @@ size_t dc_conv_workspace_bytes(void);
 
 /*
  * Host only, launches nothing: name of the kernel dc_conv_forward would run for this problem
- * ("k_conv_tc_pairrows", "k_conv_tc_rows", "k_conv_tc_fold", "k_conv_tc", "k_conv_smallcin_bf16",
+ * ("k_conv_tc_pairrows", "k_conv_tc_rows", "k_conv_tc_fold", "k_conv_tc", "k_conv_stem_tc", "k_conv_smallcin_bf16",
  * "k_conv_dense_bf16", "k_conv_dense_f32"), or NULL when the
  * geometry is invalid.  For reports (which kernel a timing belongs to); the string is static.
  */

@@ -29,6 +29,7 @@ extern "C" const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g
   if (dc_conv_rows_supported(n, h, w, g)) return "k_conv_tc_rows";
   if (dc_conv_fold_supported(n, h, w, g)) return "k_conv_tc_fold";
   if (dc_conv_tc_supported(n, h, w, g)) return "k_conv_tc";
+  if (dc_conv_stem_supported(n, h, w, g)) return "k_conv_stem_tc";
   if (dc_conv_smallcin_supported(n, h, w, g)) return "k_conv_smallcin_bf16";
   return "k_conv_dense_bf16";
 }
@@ -57,11 +58,14 @@ extern "C" dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, co
     return dc_launch_conv_rows(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   const bool fold_ok = dtype == DC_BF16 && dc_conv_fold_supported(n, h, w, g);
   const bool tc_ok = dtype == DC_BF16 && !fold_ok && dc_conv_tc_supported(n, h, w, g);
-  if (algo == DC_ALGO_TCGEN05 && !tc_ok && !fold_ok) return DC_ERR_UNSUPPORTED;
+  const bool stem_ok = dtype == DC_BF16 && !fold_ok && !tc_ok && dc_conv_stem_supported(n, h, w, g);
+  if (algo == DC_ALGO_TCGEN05 && !tc_ok && !fold_ok && !stem_ok) return DC_ERR_UNSUPPORTED;
   if (fold_ok && algo != DC_ALGO_SIMT)
     return dc_launch_conv_fold(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   if (tc_ok && algo != DC_ALGO_SIMT)
     return dc_launch_conv_tc(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
+  if (stem_ok && algo != DC_ALGO_SIMT)
+    return dc_launch_conv_stem(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   return dc_launch_conv_simt(x, n, h, w, g, w_packed, bias, act, residual, y, dtype, st);
 }
 

@@ -334,4 +334,8 @@ dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom 
                               void *workspace, cudaStream_t stream);
 bool dc_conv_fold_supported(int n, int h, int w, const dc_geom *g);
 bool dc_conv_smallcin_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_launch_conv_stem(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                              const float *bias, dc_act act, const void *residual, void *y,
+                              void *workspace, cudaStream_t stream);
+bool dc_conv_stem_supported(int n, int h, int w, const dc_geom *g);
 dc_status dc_validate_geom(const dc_geom *g);

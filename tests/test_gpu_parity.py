@@ -204,8 +204,12 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (40, 32, 5, 1, 2, 2, 14, 14, "k_conv_tc_fold"),         # odd entry count (padding entry), 5 tap columns
     (48, 24, 3, 1, 1, 2, 20, 20, "k_conv_tc_fold"),
     (64, 32, 3, 1, 1, 1, 12, 70, "k_conv_tc_fold"),         # two column strips
-    (4, 16, 5, 1, 2, 1, 9, 200, "k_conv_smallcin_bf16"),    # two row segments per output row
-    (3, 40, 3, 2, 1, 2, 17, 33, "k_conv_smallcin_bf16"),    # two passes of 32 output channels, odd sizes
+    (4, 16, 5, 1, 2, 1, 9, 200, "k_conv_stem_tc"),          # two row segments per output row, 26 chunk planes
+    (3, 40, 3, 2, 1, 2, 17, 33, "k_conv_stem_tc"),          # 40 output channels (48 operand rows), odd sizes
+    (3, 32, 3, 2, 1, 3, 40, 300, "k_conv_stem_tc"),         # the stem's geometry, ragged second segment
+    (1, 8, 3, 1, 1, 2, 20, 20, "k_conv_stem_tc"),           # one input channel
+    (3, 24, 5, 2, 2, 2, 21, 304, "k_conv_stem_tc"),         # 16-byte row chunks with a shifted second segment
+    (3, 264, 3, 2, 1, 1, 20, 20, "k_conv_smallcin_bf16"),   # too many outputs for one accumulator: CUDA cores
     (24, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc_pairrows"),     # stride 2: one output per line, even/odd row boxes
     (32, 16, 5, 2, 2, 1, 30, 44, "k_conv_tc_pairrows"),     # stride 2, even padding, 5x5
     (16, 24, 3, 2, 0, 2, 17, 36, "k_conv_tc_pairrows"),     # stride 2, no padding, odd height
