@@ -128,6 +128,23 @@ dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const dc_residual
                          void *workspace, size_t workspace_bytes, dc_stream stream);
 
 /*
+ * How dc_merge_chain walks a run.  DC_MERGE_STEPS: fold every layer, then compose the pieces
+ * pairwise (one launch per step).  DC_MERGE_AUTO (what dc_merge_chain uses): as above, except
+ * that every inverted-residual block inside the run -- dense 1x1 with stride 1, depthwise k x k,
+ * dense 1x1 with stride 1, either a whole skip group or outside any -- is merged in one launch
+ * straight from the raw layers (BN folded on the fly, the 6x wider intermediate kernel never
+ * written): W'[o,i,t] = sum_c W3~[o,c] D~[c,t] W1~[c,i], which is Eq. 1 applied twice.  Both
+ * forms evaluate the same formula in fp32; they differ in rounding order only.
+ */
+typedef enum { DC_MERGE_AUTO = 0, DC_MERGE_STEPS = 1 } dc_merge_algo;
+
+/* As dc_merge_chain with the walk chosen by the caller (same workspace size for both). */
+dc_status dc_merge_chain_algo(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                              float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
+                              void *workspace, size_t workspace_bytes, dc_stream stream,
+                              dc_merge_algo algo);
+
+/*
  * dc_merge_chain for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this entry point exists for integration, it computes exactly what dc_merge_chain computes.)
  *

@@ -394,6 +394,103 @@ __global__ void k_deliver(Piece acc, float *w_merged, float *b_merged, void *pac
 }
 
 // ----------------------------------------------------------------------------------------------
+// An inverted-residual block in one step: dense 1x1 (stride 1) -> depthwise k x k -> dense 1x1.
+//
+//   W'[o][i][t] = sum_c W3~[o][c] * D~[c][t] * W1~[c][i],   ~ = BN folded (scale g = gamma / sqrt(var + eps))
+//   b'[o]       = b3~[o] + sum_c W3~[o][c] * (b2~[c] + (sum_t D~[c][t]) * b1~[c])
+//
+// which is what folding the three layers and composing them pairwise gives (Eq. 1 applied twice),
+// without the folded copies and the 6x wider intermediate kernel ever going through global memory:
+// each step of the pairwise walk waits for the one before, and for kernels of a few thousand
+// elements those waits are the whole cost.  One CTA per output channel o; the raw layer weights are
+// read once per CTA (they sit in L2), `chunk` hidden channels at a time.
+// ----------------------------------------------------------------------------------------------
+struct RawLayer {
+  const float *w, *b, *gamma, *beta, *mean, *var;
+  float eps;
+};
+struct BlockArgs {
+  RawLayer l1, l2, l3;
+  int c0, c1, c2, k;      // input, hidden, output channels; depthwise kernel size
+  int chunk;              // hidden channels staged per pass
+  float *w_out, *b_out;   // [c2][c0][k][k], [c2]
+};
+constexpr int kBlockThreads = 256;
+constexpr int kBlockMaxPerThread = 8;       // outputs per thread: c0 * k * k <= 2048
+
+__device__ __forceinline__ float raw_scale(const RawLayer &L, int o) {
+  return L.gamma ? L.gamma[o] / sqrtf(L.var[o] + L.eps) : 1.f;
+}
+__device__ __forceinline__ float raw_bias(const RawLayer &L, int o, float g) {
+  const float b = L.b ? L.b[o] : 0.f;
+  return L.gamma ? fmaf(b - L.mean[o], g, L.beta[o]) : b;
+}
+
+__global__ void __launch_bounds__(kBlockThreads) k_merge_block(const __grid_constant__ BlockArgs a) {
+  extern __shared__ __align__(16) float blk_smem[];
+  const int c0 = a.c0, c1 = a.c1, kk = a.k * a.k, J = c0 * kk, CH = a.chunk;
+  float *Ms = blk_smem;                 // [CH][c0]  raw W1 rows
+  float *Ds = Ms + CH * c0;             // [CH][kk]  raw D rows, then W3~[o][c] * D~[c][t] * g1[c]
+  float *sc = Ds + CH * kk;             // [CH]      W3~[o][c] * g2[c] * g1[c]
+  __shared__ float bias_part[kBlockThreads / 32];
+  const int o = blockIdx.x, tid = threadIdx.x;
+  const float g3 = raw_scale(a.l3, o);
+  float acc[kBlockMaxPerThread];
+  int oi[kBlockMaxPerThread], ot[kBlockMaxPerThread];
+#pragma unroll
+  for (int q = 0; q < kBlockMaxPerThread; ++q) {
+    const int j = tid + q * kBlockThreads;
+    acc[q] = 0.f;
+    oi[q] = j / kk;
+    ot[q] = j - oi[q] * kk;
+  }
+  float bsum = 0.f;
+  for (int cb = 0; cb < c1; cb += CH) {
+    const int rows = c1 - cb < CH ? c1 - cb : CH;
+    // all loads of the pass go out together: W1 rows, D rows, and the per-channel scalars
+    for (int e = tid; e < rows * c0; e += kBlockThreads) Ms[e] = a.l1.w[(size_t)cb * c0 + e];
+    for (int e = tid; e < rows * kk; e += kBlockThreads) Ds[e] = a.l2.w[(size_t)cb * kk + e];
+    for (int cl = tid; cl < rows; cl += kBlockThreads) {
+      const int c = cb + cl;
+      const float g1 = raw_scale(a.l1, c), g2 = raw_scale(a.l2, c);
+      const float w3 = g3 * a.l3.w[(size_t)o * c1 + c];
+      float dsum = 0.f;
+      for (int t = 0; t < kk; ++t) dsum += g2 * a.l2.w[(size_t)c * kk + t];
+      bsum = fmaf(w3, fmaf(dsum, raw_bias(a.l1, c, g1), raw_bias(a.l2, c, g2)), bsum);
+      sc[cl] = (w3 * g2) * g1;
+    }
+    __syncthreads();
+    for (int e = tid; e < rows * kk; e += kBlockThreads) Ds[e] *= sc[e / kk];
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < kBlockMaxPerThread; ++q) {
+      if (tid + q * kBlockThreads < J) {
+        const float *m = Ms + oi[q], *d = Ds + ot[q];
+        float s = acc[q];
+#pragma unroll 4
+        for (int cl = 0; cl < rows; ++cl) s = fmaf(d[cl * kk], m[cl * c0], s);
+        acc[q] = s;
+      }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int q = 0; q < kBlockMaxPerThread; ++q) {
+    const int j = tid + q * kBlockThreads;
+    if (j < J) a.w_out[(size_t)o * J + j] = acc[q];
+  }
+  // bias: the per-thread terms meet through warp shuffles and one shared-memory hop
+  for (int d = 16; d > 0; d >>= 1) bsum += __shfl_xor_sync(0xffffffffu, bsum, d);
+  if ((tid & 31) == 0) bias_part[tid >> 5] = bsum;
+  __syncthreads();
+  if (tid == 0) {
+    float b = 0.f;
+    for (int w = 0; w < kBlockThreads / 32; ++w) b += bias_part[w];
+    a.b_out[o] = raw_bias(a.l3, o, g3) + b;
+  }
+}
+
+// ----------------------------------------------------------------------------------------------
 // host: validation and geometry
 // ----------------------------------------------------------------------------------------------
 
@@ -516,51 +613,114 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
   return out;
 }
 
+// Index of the skip group that contains layer idx, or -1.
+static int group_of(const dc_residual *res, int n_res, int idx) {
+  for (int i = 0; i < n_res; ++i)
+    if (res[i].first <= idx && idx <= res[i].last) return i;
+  return -1;
+}
+
+// Hidden channels k_merge_block stages per pass for this block (0: the block does not qualify).
+static int block_chunk(const dc_layer *L, int n, const dc_residual *res, int n_res, int i) {
+  if (i + 2 >= n) return 0;
+  const dc_layer &e = L[i], &d = L[i + 1], &p = L[i + 2];
+  if (e.groups != 1 || e.k != 1 || e.stride != 1 || e.pad != 0) return 0;
+  if (d.groups == 1 || d.groups != d.c_in) return 0;
+  if (p.groups != 1 || p.k != 1 || p.stride != 1 || p.pad != 0) return 0;
+  if (e.c_in * d.k * d.k > kBlockThreads * kBlockMaxPerThread) return 0;
+  const int g0 = group_of(res, n_res, i), g1 = group_of(res, n_res, i + 1), g2 = group_of(res, n_res, i + 2);
+  const bool whole = g0 >= 0 && g0 == g1 && g1 == g2 && res[g0].first == i && res[g0].last == i + 2;
+  if (!whole && (g0 >= 0 || g1 >= 0 || g2 >= 0)) return 0;
+  const int per = e.c_in + d.k * d.k + 1;
+  int ch = (200 * 1024 / 4) / per;
+  if (ch > e.c_out) ch = e.c_out;
+  return ch >= 32 || ch == e.c_out ? ch : 0;
+}
+
+static RawLayer raw_of(const dc_layer &L) {
+  return RawLayer{L.weight, L.bias, L.bn_gamma, L.bn_beta, L.bn_mean, L.bn_var, L.bn_eps};
+}
+
 // One walk drives both the size query (go == false: nothing is dereferenced or launched) and the
 // launches (go == true: the caller has already checked workspace_bytes against the query).
 static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *res, int n_res,
                             float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
-                            void *workspace, cudaStream_t st, bool go, dc_geom *merged, size_t *need) {
+                            void *workspace, cudaStream_t st, bool go, dc_geom *merged, size_t *need,
+                            dc_merge_algo algo = DC_MERGE_AUTO) {
   dc_geom mg;
   dc_status s = check_chain(layers, n, res, n_res, &mg);
   if (s != DC_OK) return s;
   if (merged) *merged = mg;
   Bump bump{go ? (char *)workspace : nullptr, 0};
 
-  // 1. fold every layer
+  // 0. inverted-residual blocks (1x1, depthwise, 1x1) are merged in one step from the raw layers
+  std::vector<int> chunk_at(n, 0), covered(n, 0);
+  if (algo != DC_MERGE_STEPS)
+    for (int i = 0; i + 2 < n;) {
+      const int ch = block_chunk(layers, n, res, n_res, i);
+      if (ch > 0) { chunk_at[i] = ch; covered[i] = covered[i + 1] = covered[i + 2] = 1; i += 3; }
+      else ++i;
+    }
+
+  // 1. fold every other layer
   std::vector<Piece> folded(n);
-  for (int l0 = 0; l0 < n; l0 += DC_FOLD_MAX) {
+  {
     FoldTable t;
-    int cnt = n - l0 < DC_FOLD_MAX ? n - l0 : DC_FOLD_MAX;
-    t.n = cnt;
+    int cnt = 0;
     size_t max_total = 1;
-    for (int j = 0; j < cnt; ++j) {
-      const dc_layer &L = layers[l0 + j];
+    auto flush = [&]() {
+      if (cnt == 0) return;
+      t.n = cnt;
+      if (go) {
+        int bx = blocks_for(max_total, 256);
+        dim3 grid(bx > 64 ? 64 : bx, cnt);
+        k_fold_bn<<<grid, 256, 0, st>>>(t);
+      }
+      cnt = 0;
+      max_total = 1;
+    };
+    for (int l = 0; l < n; ++l) {
+      if (covered[l]) continue;
+      const dc_layer &L = layers[l];
       int diag = L.groups != 1;
       size_t elems = piece_elems(L.c_in, L.c_out, L.k, diag);
       float *w = bump.take(elems), *b = bump.take(L.c_out);
-      t.w[j] = L.weight; t.b[j] = L.bias; t.gamma[j] = L.bn_gamma; t.beta[j] = L.bn_beta;
-      t.mean[j] = L.bn_mean; t.var[j] = L.bn_var; t.eps[j] = L.bn_eps;
-      t.w_out[j] = w; t.b_out[j] = b;
-      t.c_out[j] = L.c_out; t.per_out[j] = (int)(elems / L.c_out);
+      t.w[cnt] = L.weight; t.b[cnt] = L.bias; t.gamma[cnt] = L.bn_gamma; t.beta[cnt] = L.bn_beta;
+      t.mean[cnt] = L.bn_mean; t.var[cnt] = L.bn_var; t.eps[cnt] = L.bn_eps;
+      t.w_out[cnt] = w; t.b_out[cnt] = b;
+      t.c_out[cnt] = L.c_out; t.per_out[cnt] = (int)(elems / L.c_out);
       if (elems > max_total) max_total = elems;
-      folded[l0 + j] = Piece{w, b, L.c_in, L.c_out, L.k, L.stride, diag, 0};
+      folded[l] = Piece{w, b, L.c_in, L.c_out, L.k, L.stride, diag, 0};
+      if (++cnt == DC_FOLD_MAX) flush();
     }
-    if (go) {
-      int bx = blocks_for(max_total, 256);
-      dim3 grid(bx > 64 ? 64 : bx, cnt);
-      k_fold_bn<<<grid, 256, 0, st>>>(t);
-    }
+    flush();
   }
 
-  // 2. compose: skip groups first (with their identity tap), then left to right
+  // 2. compose: blocks and skip groups first (with their identity tap), then left to right
   Piece acc{};
   bool have = false;
   int i = 0;
   while (i < n) {
     Piece piece;
     int gi = find_group(res, n_res, i);
-    if (gi < 0) {
+    if (chunk_at[i] > 0) {
+      const dc_layer &e = layers[i], &d = layers[i + 1], &p = layers[i + 2];
+      piece = Piece{nullptr, nullptr, e.c_in, p.c_out, d.k, d.stride, 0, gi >= 0 ? 1 : 0};
+      float *w = bump.take(piece_elems(piece.c_in, piece.c_out, piece.k, 0));
+      float *b = bump.take(piece.c_out);
+      piece.w = w; piece.b = b;
+      if (go) {
+        BlockArgs a{raw_of(e), raw_of(d), raw_of(p), e.c_in, e.c_out, p.c_out, d.k, chunk_at[i], w, b};
+        const size_t smem = (size_t)chunk_at[i] * (e.c_in + d.k * d.k + 1) * sizeof(float);
+        static bool attr_set = false;
+        if (!attr_set) {
+          cudaFuncSetAttribute(k_merge_block, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+          attr_set = true;
+        }
+        k_merge_block<<<p.c_out, kBlockThreads, smem, st>>>(a);
+      }
+      i += 3;
+    } else if (gi < 0) {
       piece = folded[i];
       ++i;
     } else {
@@ -591,6 +751,20 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
 
+// Workspace bytes that cover either launch form.
+static dc_status merge_need(const dc_layer *layers, int n, const dc_residual *res, int n_res, dc_geom *merged,
+                            size_t *need) {
+  size_t a = 0, b = 0;
+  dc_status s = merge_walk(layers, n, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr, false, merged,
+                           &a, DC_MERGE_AUTO);
+  if (s != DC_OK) return s;
+  s = merge_walk(layers, n, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr, false, nullptr, &b,
+                 DC_MERGE_STEPS);
+  if (s != DC_OK) return s;
+  if (need) *need = a > b ? a : b;
+  return DC_OK;
+}
+
 // ----------------------------------------------------------------------------------------------
 // exported
 // ----------------------------------------------------------------------------------------------
@@ -614,18 +788,18 @@ extern "C" dc_status dc_fold_bn(const dc_layer *layer, float *w_out, float *b_ou
 
 extern "C" dc_status dc_merge_query(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
                                     dc_geom *merged, size_t *workspace_bytes) {
-  return merge_walk(layers, n_layers, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr, false,
-                    merged, workspace_bytes);
+  return merge_need(layers, n_layers, res, n_res, merged, workspace_bytes);
 }
 
-extern "C" dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
-                                    float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
-                                    void *workspace, size_t workspace_bytes, dc_stream stream) {
+extern "C" dc_status dc_merge_chain_algo(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                                         float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
+                                         void *workspace, size_t workspace_bytes, dc_stream stream,
+                                         dc_merge_algo algo) {
   if (!w_merged || !b_merged) return DC_ERR_INVALID_ARG;
   if (packed_dtype != DC_F32 && packed_dtype != DC_BF16) return DC_ERR_INVALID_ARG;
+  if (algo != DC_MERGE_AUTO && algo != DC_MERGE_STEPS) return DC_ERR_INVALID_ARG;
   size_t need = 0;
-  dc_status s = merge_walk(layers, n_layers, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr,
-                           false, nullptr, &need);
+  dc_status s = merge_need(layers, n_layers, res, n_res, nullptr, &need);
   if (s != DC_OK) return s;
   if (!workspace || workspace_bytes < need) return DC_ERR_WORKSPACE;
   if (!dc_aligned16(w_merged) || !dc_aligned16(b_merged) || !dc_aligned16(workspace) ||
@@ -634,7 +808,14 @@ extern "C" dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const 
   for (int i = 0; i < n_layers; ++i)
     if (!dc_aligned16(layers[i].weight)) return DC_ERR_ALIGNMENT;
   return merge_walk(layers, n_layers, res, n_res, w_merged, b_merged, w_packed, packed_dtype, workspace,
-                    (cudaStream_t)stream, true, nullptr, nullptr);
+                    (cudaStream_t)stream, true, nullptr, nullptr, algo);
+}
+
+extern "C" dc_status dc_merge_chain(const dc_layer *layers, int n_layers, const dc_residual *res, int n_res,
+                                    float *w_merged, float *b_merged, void *w_packed, dc_dtype packed_dtype,
+                                    void *workspace, size_t workspace_bytes, dc_stream stream) {
+  return dc_merge_chain_algo(layers, n_layers, res, n_res, w_merged, b_merged, w_packed, packed_dtype, workspace,
+                             workspace_bytes, stream, DC_MERGE_AUTO);
 }
 
 extern "C" dc_status dc_packed_bytes(const dc_geom *g, dc_dtype dtype, size_t *bytes) {
@@ -695,8 +876,7 @@ extern "C" dc_status dc_merge_chain_static(const dc_layer *layers, int n_layers,
   if (!w_merged || !b_merged) return DC_ERR_INVALID_ARG;
   if (packed_dtype != DC_F32 && packed_dtype != DC_BF16) return DC_ERR_INVALID_ARG;
   size_t need = 0;
-  dc_status s = merge_walk(layers, n_layers, res, n_res, nullptr, nullptr, nullptr, DC_F32, nullptr, nullptr,
-                           false, nullptr, &need);
+  dc_status s = merge_need(layers, n_layers, res, n_res, nullptr, &need);
   if (s != DC_OK) return s;
   if (need > (size_t)DC_STATIC_SCRATCH_BYTES) return DC_ERR_WORKSPACE;   // run too large for the built-in scratch
   if (!dc_aligned16(w_merged) || !dc_aligned16(b_merged) || (w_packed && !dc_aligned16(w_packed)))

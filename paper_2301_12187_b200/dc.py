@@ -18,6 +18,7 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_UNSUPPORTED, ERR_NOT_MERGEABLE, ERR_WORKSPAC
 F32, BF16 = 0, 1
 ACT_IDENTITY, ACT_RELU6 = 0, 1
 ALGO_AUTO, ALGO_TCGEN05, ALGO_SIMT = 0, 1, 2
+MERGE_AUTO, MERGE_STEPS = 0, 1
 
 _FP = C.POINTER(C.c_float)
 
@@ -58,6 +59,8 @@ EXPORTS = {
     "dc_packed_bytes": (C.c_int, [C.POINTER(Geom), C.c_int, C.POINTER(C.c_size_t)]),
     "dc_merge_chain": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "dc_merge_chain_algo": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p, C.c_int]),
     "dc_merge_chain_static": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "dc_merge_chain_static_capacity": (C.c_size_t, []),
@@ -213,12 +216,13 @@ def packed_bytes(g: Geom, dtype: int) -> int:
     return int(nbytes.value)
 
 
-def merge_chain(layers, residuals, w_merged, b_merged, w_packed, packed_dtype, workspace, stream=None):
+def merge_chain(layers, residuals, w_merged, b_merged, w_packed, packed_dtype, workspace, stream=None,
+                algo=MERGE_AUTO):
     arr = layer_array(layers)
     res, n_res = _res_array(residuals)
-    _check(lib().dc_merge_chain(arr, len(layers), res, n_res, _ptr(w_merged), _ptr(b_merged),
-                                _ptr(w_packed), packed_dtype, _ptr(workspace),
-                                workspace.numel() * workspace.element_size(), _stream(stream)),
+    _check(lib().dc_merge_chain_algo(arr, len(layers), res, n_res, _ptr(w_merged), _ptr(b_merged),
+                                     _ptr(w_packed), packed_dtype, _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream), algo),
            "dc_merge_chain")
 
 

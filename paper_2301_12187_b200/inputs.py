@@ -95,14 +95,14 @@ class LayerSpec:
     role: str = ""
 
 
-_KIND_W, _KIND_G, _KIND_B, _KIND_M, _KIND_V = range(5)
+_KIND_W, _KIND_G, _KIND_B, _KIND_M, _KIND_V, _KIND_BIAS = range(6)
 _X_TENSOR_ID = 1 << 20
 
 
 def make_layer(seed, index, c_in, c_out, k, stride, pad, depthwise=False, act=None, name="",
-               block=-1, role="", with_bn=True) -> LayerSpec:
+               block=-1, role="", with_bn=True, with_bias=False) -> LayerSpec:
     """Weights N(0, 1/fan_in) (variance), fan_in = (c_in/groups) k^2; BN gamma, var ~ U[0.5,1.5),
-    beta, running mean ~ N(0, 0.1^2); no conv bias."""
+    beta, running mean ~ N(0, 0.1^2); no conv bias unless asked for (then N(0, 0.1^2))."""
     groups = c_in if depthwise else 1
     if depthwise:
         assert c_in == c_out
@@ -116,7 +116,8 @@ def make_layer(seed, index, c_in, c_out, k, stride, pad, depthwise=False, act=No
               normal(seed, tid + _KIND_B, (c_out,), std=0.1),
               normal(seed, tid + _KIND_M, (c_out,), std=0.1),
               uniform(seed, tid + _KIND_V, (c_out,), 0.5, 1.5))
-    return LayerSpec(c_in, c_out, groups, k, stride, pad, w, None, bn, 1e-5, act, name, block, role)
+    bias = normal(seed, tid + _KIND_BIAS, (c_out,), std=0.1) if with_bias else None
+    return LayerSpec(c_in, c_out, groups, k, stride, pad, w, bias, bn, 1e-5, act, name, block, role)
 
 
 def make_input(seed, shape_nhwc, bf16=False):

@@ -36,7 +36,7 @@ def new_ws(dc, nbytes=None):
     return torch.zeros(max(nbytes or 0, dc.conv_workspace_bytes()), dtype=torch.uint8, device="cuda")
 
 
-def run_merge(dc, specs, residuals, packed_dtype=None):
+def run_merge(dc, specs, residuals, packed_dtype=None, algo=0):
     layers = [dc.DeviceLayer(s) for s in specs]
     g, ws_bytes = dc.merge_query(layers, residuals)
     wm = torch.empty((g.c_out, g.c_in, g.k, g.k), dtype=torch.float32, device="cuda")
@@ -45,7 +45,8 @@ def run_merge(dc, specs, residuals, packed_dtype=None):
     packed = None
     if packed_dtype is not None:
         packed = torch.empty(dc.packed_bytes(g, packed_dtype), dtype=torch.uint8, device="cuda")
-    dc.merge_chain(layers, residuals, wm, bm, packed, packed_dtype if packed_dtype is not None else dc.F32, ws)
+    dc.merge_chain(layers, residuals, wm, bm, packed, packed_dtype if packed_dtype is not None else dc.F32, ws,
+                   algo=algo)
     torch.cuda.synchronize()
     return g, wm, bm, packed
 
@@ -115,6 +116,74 @@ def test_merge_chain_weights(dc, name):
     assert (g.k, g.stride, g.pad, g.c_in, g.c_out) == (k, s, p, W.shape[1], W.shape[0])
     assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W
     assert O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+
+
+def wide_chain(name, s=5):
+    """Runs with more arithmetic than `small_chain`: two skip blocks in a row at three widths, a
+    dense 3x3 o 3x3 o 3x3 run (7x7 result) and a stride-2 run with a 5x5 depthwise layer."""
+    mk = I.make_layer
+    if name in ("two_blocks_32", "two_blocks_64", "two_blocks_48"):
+        c = int(name.rsplit("_", 1)[1])
+        L = []
+        for b in range(2):
+            L += [mk(s, 3 * b, c, 6 * c, 1, 1, 0), mk(s, 3 * b + 1, 6 * c, 6 * c, 3, 1, 1, depthwise=True),
+                  mk(s, 3 * b + 2, 6 * c, c, 1, 1, 0)]
+        return L, [(0, 2), (3, 5)]
+    if name == "dense_7x7":
+        return [mk(s, 0, 16, 24, 3, 1, 1), mk(s, 1, 24, 24, 3, 1, 1), mk(s, 2, 24, 16, 3, 1, 1)], [(1, 1)]
+    if name == "s2_dw5":
+        return [mk(s, 0, 40, 240, 1, 1, 0), mk(s, 1, 240, 240, 5, 2, 2, depthwise=True), mk(s, 2, 240, 48, 1, 1, 0)], []
+    raise KeyError(name)
+
+
+WIDE = ["two_blocks_32", "two_blocks_64", "two_blocks_48", "dense_7x7", "s2_dw5"]
+
+
+@pytest.mark.parametrize("algo", ["steps", "auto"])
+@pytest.mark.parametrize("name", CHAINS + WIDE)
+def test_merge_chain_both_walks(dc, name, algo):
+    """The pairwise walk and the walk that merges inverted-residual blocks in one step, each
+    against the oracle's formula (weights, bias, and the bf16 packed copy through the fp32 result)."""
+    specs, res = small_chain(name) if name in CHAINS else wide_chain(name)
+    code = dc.MERGE_STEPS if algo == "steps" else dc.MERGE_AUTO
+    g, wm, bm, packed = run_merge(dc, specs, res, packed_dtype=dc.BF16, algo=code)
+    W, b, k, s, p = O.merge_formula(specs, res)
+    assert (g.k, g.stride, g.pad) == (k, s, p)
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W
+    assert O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    # the packed copy must be what dc_pack_weights makes of the delivered fp32 kernel, bit for bit
+    again = torch.empty_like(packed)
+    dc.pack_weights(wm, g, dc.BF16, again)
+    torch.cuda.synchronize()
+    assert torch.equal(packed, again)
+
+
+@pytest.mark.parametrize("case", ["no_bn", "bias_no_bn", "wide_hidden", "block_inside_run"])
+def test_block_step_edge_cases(dc, case):
+    """Blocks without BN, with plain biases, with a hidden width that is staged in several passes,
+    and a block in the middle of a longer run (neighbours composed pairwise around it)."""
+    mk = I.make_layer
+    if case == "no_bn":
+        specs = [mk(11, 0, 8, 48, 1, 1, 0, with_bn=False), mk(11, 1, 48, 48, 3, 1, 1, depthwise=True, with_bn=False),
+                 mk(11, 2, 48, 8, 1, 1, 0, with_bn=False)]
+        res = [(0, 2)]
+    elif case == "bias_no_bn":
+        specs = [mk(12, 0, 16, 96, 1, 1, 0, with_bn=False, with_bias=True),
+                 mk(12, 1, 96, 96, 5, 2, 2, depthwise=True), mk(12, 2, 96, 24, 1, 1, 0, with_bias=True)]
+        res = []
+    elif case == "wide_hidden":
+        specs = [mk(13, 0, 160, 960, 1, 1, 0), mk(13, 1, 960, 960, 3, 1, 1, depthwise=True), mk(13, 2, 960, 160, 1, 1, 0)]
+        res = [(0, 2)]
+    else:
+        specs = [mk(14, 0, 16, 8, 3, 1, 1), mk(14, 1, 8, 48, 1, 1, 0), mk(14, 2, 48, 48, 3, 1, 1, depthwise=True),
+                 mk(14, 3, 48, 8, 1, 1, 0), mk(14, 4, 8, 24, 1, 1, 0)]
+        res = [(1, 3)]
+    g, wm, bm, _ = run_merge(dc, specs, res)
+    W, b, *_ = O.merge_formula(specs, res)
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W
+    assert O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    g2, wm2, bm2, _ = run_merge(dc, specs, res, algo=dc.MERGE_STEPS)
+    assert O.rel_l2(wm2.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm2.cpu().numpy(), b) <= TOL_W
 
 
 @pytest.mark.parametrize("name", CHAINS)
