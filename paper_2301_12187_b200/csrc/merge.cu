@@ -117,34 +117,55 @@ __global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece 
   float acc[4][4] = {};
   for (int r0 = 0; r0 < R; r0 += slice) {
     const int rows = R - r0 < slice ? R - r0 : slice;
+    // Operand loads are issued in batches with no branch between them (an element outside the
+    // operand reads element 0 and is zeroed afterwards): a load behind a branch would wait for the
+    // one before it, and a slice would cost dozens of round trips to L2 instead of a few.
     // A[o][r]: consecutive threads read consecutive r of one output channel
-    for (int rr = arr; rr < rows; rr += 16) {
-      const int r = r0 + rr;
+    for (int rb = arr; rb < rows; rb += 64) {
+      float av[4][4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int row = arow + 16 * q, o = o0 + row;
-        float av = 0.f;
-        if (o < c2) {
-          av = second.w[(size_t)o * R + r];
-          if (second.ident && r == (o * k2 + ctr2) * k2 + ctr2) av += 1.f;
+      for (int u = 0; u < 4; ++u) {
+        const int rr = rb + 16 * u, r = r0 + (rr < rows ? rr : rows - 1);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int o = o0 + arow + 16 * q;
+          const bool ok = o < c2 && rr < rows;
+          const float x = second.w[ok ? (size_t)o * R + r : 0];
+          av[u][q] = ok ? ((second.ident && r == (o * k2 + ctr2) * k2 + ctr2) ? x + 1.f : x) : 0.f;
         }
-        As[rr * kDdPitch + row] = av;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int rr = rb + 16 * u;
+        if (rr < rows) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) As[rr * kDdPitch + arow + 16 * q] = av[u][q];
+        }
       }
     }
     // B[r][j]: consecutive threads read consecutive j (elements of W1 next to each other)
-    for (int rr = t >> 6; rr < rows; rr += 4) {
-      const int r = r0 + rr;
-      float v = 0.f;
-      if (j < J) {
-        const int c = r / t2sz, t2 = r - c * t2sz;
-        const int u2 = t2 / k2, v2 = t2 - u2 * k2;
-        const int u1 = bup - s1 * u2, v1 = bvp - s1 * v2;
-        if (u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1) {
-          v = first.w[(((size_t)c * c0 + bi) * k1 + u1) * k1 + v1];
-          if (first.ident && c == bi && u1 == ctr1 && v1 == ctr1) v += 1.f;
+    for (int rb = t >> 6; rb < rows; rb += 32) {
+      float bv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int rr = rb + 4 * u, r = r0 + (rr < rows ? rr : rows - 1);
+        int c = r, u2 = 0, v2 = 0;
+        if (t2sz != 1) {
+          c = r / t2sz;
+          const int t2 = r - c * t2sz;
+          u2 = t2 / k2;
+          v2 = t2 - u2 * k2;
         }
+        const int u1 = bup - s1 * u2, v1 = bvp - s1 * v2;
+        const bool ok = j < J && u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1;
+        const float x = first.w[ok ? (((size_t)c * c0 + bi) * k1 + u1) * k1 + v1 : 0];
+        bv[u] = ok ? ((first.ident && c == bi && u1 == ctr1 && v1 == ctr1) ? x + 1.f : x) : 0.f;
       }
-      Bs[rr * kDdPitch + jj] = v;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int rr = rb + 4 * u;
+        if (rr < rows) Bs[rr * kDdPitch + jj] = bv[u];
+      }
     }
     __syncthreads();
 #pragma unroll 4
@@ -196,33 +217,37 @@ __global__ void __launch_bounds__(256) k_compose_dd_small(Piece first, Piece sec
   float acc = 0.f;
   for (int r0 = 0; r0 < R; r0 += kDdSmallSlice) {
     const int rows = R - r0 < kDdSmallSlice ? R - r0 : kDdSmallSlice;
+    // Operand loads go out in batches with no branch between them (see k_compose_dense_dense).
     // A[o][r]: a warp reads 32 consecutive r of one output channel
-    for (int rr = jl; rr < rows; rr += 32) {
-      float av = 0.f;
-      if (o < c2) {
-        const int r = r0 + rr;
-        av = second.w[(size_t)o * R + r];
-        if (second.ident && r == (o * k2 + ctr2) * k2 + ctr2) av += 1.f;
-      }
-      As[rr][ol] = av;
-    }
-    // B[r][j]: a warp reads one row r, 32 consecutive j; (c, t2) of the row advance by 8 rows a step
     {
-      int r = r0 + ol;
-      int c = r / t2sz, t2 = r - c * t2sz;
-      for (int rr = ol; rr < rows; rr += 8) {
-        float v = 0.f;
-        if (j < J) {
-          const int u1 = bup - s1 * tap_u[t2], v1 = bvp - s1 * tap_v[t2];
-          if (u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1) {
-            v = first.w[(((size_t)c * c0 + bi) * k1 + u1) * k1 + v1];
-            if (first.ident && c == bi && u1 == ctr1 && v1 == ctr1) v += 1.f;
-          }
-        }
-        Bs[rr][jl] = v;
-        t2 += 8;
-        while (t2 >= t2sz) { t2 -= t2sz; ++c; }
+      float av[kDdSmallSlice / 32];
+#pragma unroll
+      for (int u = 0; u < kDdSmallSlice / 32; ++u) {
+        const int rr = jl + 32 * u, r = r0 + (rr < rows ? rr : rows - 1);
+        const bool ok = o < c2 && rr < rows;
+        const float x = second.w[ok ? (size_t)o * R + r : 0];
+        av[u] = ok ? ((second.ident && r == (o * k2 + ctr2) * k2 + ctr2) ? x + 1.f : x) : 0.f;
       }
+#pragma unroll
+      for (int u = 0; u < kDdSmallSlice / 32; ++u)
+        if (jl + 32 * u < rows) As[jl + 32 * u][ol] = av[u];
+    }
+    // B[r][j]: a warp reads one row r, 32 consecutive j
+    for (int rb = ol; rb < rows; rb += 64) {
+      float bv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int rr = rb + 8 * u, r = r0 + (rr < rows ? rr : rows - 1);
+        int c = r, t2 = 0;
+        if (t2sz != 1) { c = r / t2sz; t2 = r - c * t2sz; }
+        const int u1 = bup - s1 * tap_u[t2], v1 = bvp - s1 * tap_v[t2];
+        const bool ok = j < J && u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1;
+        const float x = first.w[ok ? (((size_t)c * c0 + bi) * k1 + u1) * k1 + v1 : 0];
+        bv[u] = ok ? ((first.ident && c == bi && u1 == ctr1 && v1 == ctr1) ? x + 1.f : x) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (rb + 8 * u < rows) Bs[rb + 8 * u][jl] = bv[u];
     }
     __syncthreads();
 #pragma unroll 8

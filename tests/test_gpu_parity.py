@@ -158,7 +158,7 @@ def test_merge_chain_both_walks(dc, name, algo):
     assert torch.equal(packed, again)
 
 
-@pytest.mark.parametrize("case", ["no_bn", "bias_no_bn", "wide_hidden", "block_inside_run"])
+@pytest.mark.parametrize("case", ["no_bn", "bias_no_bn", "wide_hidden", "block_inside_run", "fold_order", "rows_order"])
 def test_block_step_edge_cases(dc, case):
     """Blocks without BN, with plain biases, with a hidden width that is staged in several passes,
     and a block in the middle of a longer run (neighbours composed pairwise around it)."""
@@ -174,14 +174,24 @@ def test_block_step_edge_cases(dc, case):
     elif case == "wide_hidden":
         specs = [mk(13, 0, 160, 960, 1, 1, 0), mk(13, 1, 960, 960, 3, 1, 1, depthwise=True), mk(13, 2, 960, 160, 1, 1, 0)]
         res = [(0, 2)]
+    elif case == "fold_order":      # 40-64 input channels, narrow output: packed copy in the fold order
+        specs = [mk(15, 0, 48, 288, 1, 1, 0), mk(15, 1, 288, 288, 3, 1, 1, depthwise=True), mk(15, 2, 288, 24, 1, 1, 0)]
+        res = []
+    elif case == "rows_order":      # wide input and output: packed copy in 64-channel planes
+        specs = [mk(16, 0, 64, 384, 1, 1, 0), mk(16, 1, 384, 384, 3, 1, 1, depthwise=True), mk(16, 2, 384, 64, 1, 1, 0)]
+        res = [(0, 2)]
     else:
         specs = [mk(14, 0, 16, 8, 3, 1, 1), mk(14, 1, 8, 48, 1, 1, 0), mk(14, 2, 48, 48, 3, 1, 1, depthwise=True),
                  mk(14, 3, 48, 8, 1, 1, 0), mk(14, 4, 8, 24, 1, 1, 0)]
         res = [(1, 3)]
-    g, wm, bm, _ = run_merge(dc, specs, res)
+    g, wm, bm, packed = run_merge(dc, specs, res, packed_dtype=dc.BF16)
     W, b, *_ = O.merge_formula(specs, res)
     assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W
     assert O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    again = torch.empty_like(packed)
+    dc.pack_weights(wm, g, dc.BF16, again)
+    torch.cuda.synchronize()
+    assert torch.equal(packed, again)
     g2, wm2, bm2, _ = run_merge(dc, specs, res, algo=dc.MERGE_STEPS)
     assert O.rel_l2(wm2.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm2.cpu().numpy(), b) <= TOL_W
 
