@@ -257,15 +257,76 @@ __global__ void __launch_bounds__(256) k_compose_dd_small(Piece first, Piece sec
   if (o < c2 && j < J) out[(size_t)o * J + j] = acc;
 }
 
+// dense k x k (second) after a dense 1x1 with stride 1 (first): every tap sum has one term,
+//   out[o][i][t] = sum_c W2[o][c][t] * W1[c][i],
+// so the general gather would multiply k*k - 1 zeros per product.  blockIdx.y = o; the CTA stages
+// W2[o] ([c1][k*k], at most kAfter1x1MaxFloats) in shared memory, a thread owns one (i, t) and
+// walks c.  Blocks with blockIdx.y == c_out compute the bias.
+constexpr int kAfter1x1MaxFloats = 11264;
+__global__ void __launch_bounds__(256) k_compose_after_1x1(Piece first, Piece second, float *out, float *b_out) {
+  __shared__ float Ws[kAfter1x1MaxFloats];
+  const int c0 = first.c_in, c1 = first.c_out, c2 = second.c_out, kk = second.k * second.k, J = c0 * kk;
+  if ((int)blockIdx.y >= c2) {
+    compose_bias_block(first, second, b_out, (int)blockIdx.x);
+    return;
+  }
+  const int o = blockIdx.y, ctr = ((second.k - 1) / 2) * (second.k + 1);
+  for (int e = threadIdx.x; e < c1 * kk; e += blockDim.x) {
+    float w = second.w[(size_t)o * c1 * kk + e];
+    if (second.ident && e == o * kk + ctr) w += 1.f;
+    Ws[e] = w;
+  }
+  __syncthreads();
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= J) return;
+  const int i = j / kk, t = j - i * kk;
+  const float *w1 = first.w + i, *w2 = Ws + t;
+  float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+  int c = 0;
+  for (; c + 4 <= c1; c += 4) {
+    const float b0 = w1[(size_t)(c + 0) * c0], b1 = w1[(size_t)(c + 1) * c0];
+    const float b2 = w1[(size_t)(c + 2) * c0], b3 = w1[(size_t)(c + 3) * c0];
+    acc0 = fmaf(w2[(c + 0) * kk], b0, acc0);
+    acc1 = fmaf(w2[(c + 1) * kk], b1, acc1);
+    acc2 = fmaf(w2[(c + 2) * kk], b2, acc2);
+    acc3 = fmaf(w2[(c + 3) * kk], b3, acc3);
+  }
+  for (; c < c1; ++c) acc0 = fmaf(w2[c * kk], w1[(size_t)c * c0], acc0);
+  float acc = (acc0 + acc1) + (acc2 + acc3);
+  if (first.ident && i < c1) acc += w2[i * kk];      // first + I: the c == i term once more
+  out[(size_t)o * J + j] = acc;
+}
+
 // Compositions in which at least one operand is diagonal: one thread per output element.
 //   second diag, first dense: out[o,i,u',v'] = sum_{u2,v2} W2[o,u2,v2] * W1[o,i,u1,v1]
 //   second dense, first diag: out[o,i,u',v'] = sum_{u2,v2} W2[o,i,u2,v2] * W1[i,u1,v1]
 //   both diag:                out[c,u',v']   = sum_{u2,v2} W2[c,u2,v2]   * W1[c,u1,v1]
 // Blocks [0, nb) walk the elements; the blocks after them compute the bias.
+// Depthwise K2 x K2 after a dense 1x1 with stride 1 (expand -> depthwise): the tap sums have one
+// term, out[o][i][t] = W2[o][t] * W1[o][i].
+template <int K2>
+__device__ __forceinline__ void compose_diag_after_1x1(const Piece &first, const Piece &second, float *out, int total,
+                                                       int nb) {
+  constexpr int KK = K2 * K2, CTR = (K2 / 2) * (K2 + 1);
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += nb * blockDim.x) {
+    const int t = idx % KK, rest = idx / KK;
+    const int o = rest / first.c_in, i = rest - o * first.c_in;
+    float w2 = second.w[(size_t)o * KK + t];
+    if (second.ident && t == CTR) w2 += 1.f;
+    float w1 = first.w[rest];
+    if (first.ident && o == i) w1 += 1.f;
+    out[idx] = fmaf(w2, w1, 0.f);
+  }
+}
+
 __global__ void k_compose_diag(Piece first, Piece second, float *out, float *b_out, int kk, int total, int nb) {
   if ((int)blockIdx.x >= nb) {
     compose_bias_block(first, second, b_out, (int)blockIdx.x - nb);
     return;
+  }
+  if (second.diag && !first.diag && first.k == 1 && first.stride == 1) {
+    if (second.k == 3) { compose_diag_after_1x1<3>(first, second, out, total, nb); return; }
+    if (second.k == 5) { compose_diag_after_1x1<5>(first, second, out, total, nb); return; }
   }
   const int k1 = first.k, k2 = second.k, s1 = first.stride;
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += nb * blockDim.x) {
@@ -615,13 +676,21 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
   out.w = w; out.b = b;
   if (go) {
     const int nbias = bias_blocks(out.c_out, 256);
-    if (!first.diag && !second.diag && elems <= (size_t)200000 && second.k <= 7) {
+    if (!first.diag && !second.diag && first.k == 1 && first.stride == 1 && second.k > 1 &&
+        first.c_out * second.k * second.k <= kAfter1x1MaxFloats) {
+      dim3 grid(dc_div_up(out.c_in * out.k * out.k, 256), out.c_out + 1);
+      if ((int)grid.x < nbias) grid.x = nbias;
+      k_compose_after_1x1<<<grid, 256, 0, st>>>(first, second, w, b);
+    } else if (!first.diag && !second.diag && elems <= (size_t)200000 && second.k <= 7) {
       const int gx = dc_div_up(out.c_in * out.k * out.k, 32), gy = dc_div_up(out.c_out, 8);
       k_compose_dd_small<<<gx * gy + nbias, 256, 0, st>>>(first, second, w, b, out.k, gx, gy);
     } else if (!first.diag && !second.diag) {
       const int gx = dc_div_up(out.c_in * out.k * out.k, 64), gy = dc_div_up(out.c_out, 64);
       const int R = first.c_out * second.k * second.k;
-      const int slice = R < kDdSlice ? (int)dc_round_up((size_t)R, 16) : kDdSlice;
+      // few tiles: one deep slice per round trip; many tiles (more than two per SM): shallow slices,
+      // so that several CTAs share an SM and one's loads overlap another's arithmetic
+      const int slice_max = gx * gy > 2 * 148 ? 64 : kDdSlice;
+      const int slice = R < slice_max ? (int)dc_round_up((size_t)R, 16) : slice_max;
       const size_t smem = (size_t)2 * slice * kDdPitch * sizeof(float);
       static bool attr_set = false;
       if (!attr_set) {
@@ -653,6 +722,8 @@ static int block_chunk(const dc_layer *L, int n, const dc_residual *res, int n_r
   if (d.groups == 1 || d.groups != d.c_in) return 0;
   if (p.groups != 1 || p.k != 1 || p.stride != 1 || p.pad != 0) return 0;
   if (e.c_in * d.k * d.k > kBlockThreads * kBlockMaxPerThread) return 0;
+  // wide blocks are faster step by step: their compositions fill the GPU, one CTA per output channel does not
+  if ((long)e.c_out * e.c_in * d.k * d.k > 150000) return 0;
   const int g0 = group_of(res, n_res, i), g1 = group_of(res, n_res, i + 1), g2 = group_of(res, n_res, i + 2);
   const bool whole = g0 >= 0 && g0 == g1 && g1 == g2 && res[g0].first == i && res[g0].last == i + 2;
   if (!whole && (g0 >= 0 || g1 >= 0 || g2 >= 0)) return 0;

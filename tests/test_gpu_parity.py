@@ -158,7 +158,8 @@ def test_merge_chain_both_walks(dc, name, algo):
     assert torch.equal(packed, again)
 
 
-@pytest.mark.parametrize("case", ["no_bn", "bias_no_bn", "wide_hidden", "block_inside_run", "fold_order", "rows_order"])
+@pytest.mark.parametrize("case", ["no_bn", "bias_no_bn", "wide_hidden", "block_inside_run", "fold_order", "rows_order",
+                                  "block_after_1x1", "skip_1x1_then_3x3"])
 def test_block_step_edge_cases(dc, case):
     """Blocks without BN, with plain biases, with a hidden width that is staged in several passes,
     and a block in the middle of a longer run (neighbours composed pairwise around it)."""
@@ -174,6 +175,13 @@ def test_block_step_edge_cases(dc, case):
     elif case == "wide_hidden":
         specs = [mk(13, 0, 160, 960, 1, 1, 0), mk(13, 1, 960, 960, 3, 1, 1, depthwise=True), mk(13, 2, 960, 160, 1, 1, 0)]
         res = [(0, 2)]
+    elif case == "block_after_1x1":  # a k x k piece composed after a 1x1 layer: one term per tap sum
+        specs = [mk(17, 0, 40, 16, 1, 1, 0), mk(17, 1, 16, 96, 1, 1, 0), mk(17, 2, 96, 96, 3, 1, 1, depthwise=True),
+                 mk(17, 3, 96, 16, 1, 1, 0)]
+        res = [(1, 3)]
+    elif case == "skip_1x1_then_3x3":  # (W1 + I) under a dense 3x3
+        specs = [mk(18, 0, 24, 24, 1, 1, 0), mk(18, 1, 24, 40, 3, 1, 1)]
+        res = [(0, 0)]
     elif case == "fold_order":      # 40-64 input channels, narrow output: packed copy in the fold order
         specs = [mk(15, 0, 48, 288, 1, 1, 0), mk(15, 1, 288, 288, 3, 1, 1, depthwise=True), mk(15, 2, 288, 24, 1, 1, 0)]
         res = []
