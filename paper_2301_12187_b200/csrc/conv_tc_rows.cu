@@ -264,38 +264,52 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __nv_bfloat16 *dst = y + pix * p.c_out + ch0;
           const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out + ch0 : nullptr;
           const uint32_t taddr = tmem_row + (uint32_t)((set * p.mb + b) * p.n_tile);
+          // eight channels of this thread's pixel: bias, skip input, activation, one 16-byte store
+          auto store8 = [&](const uint32_t *v, int ch) {
+            const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch);
+            const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch + 4);
+            float f[8];
+            f[0] = __uint_as_float(v[0]) + b0.x; f[1] = __uint_as_float(v[1]) + b0.y;
+            f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
+            f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
+            f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
+            if (rp) {
+              const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
+              const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float2 rf = __bfloat1622float2(rb[i]);
+                f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+              }
+            }
+            uint4 ov;
+            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float f0 = f[2 * i], f1 = f[2 * i + 1];
+              if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
+              ob[i] = __floats2bfloat162_rn(f0, f1);
+            }
+            *reinterpret_cast<uint4 *>(dst + ch) = ov;
+          };
+          // 32 accumulator columns per read while they last (one wait, four stores back to back), then 8
+          int ch = 0;
 #pragma unroll 1
-          for (int ch = 0; ch < nch; ch += 8) {
+          for (; ch + 32 <= nch; ch += 32) {
+            uint32_t v[32];
+            tmem_ld32(taddr + (uint32_t)ch, v);
+            tmem_ld_wait();
+            if (valid) {
+#pragma unroll
+              for (int g8 = 0; g8 < 4; ++g8) store8(v + 8 * g8, ch + 8 * g8);
+            }
+          }
+#pragma unroll 1
+          for (; ch < nch; ch += 8) {
             uint32_t v[8];
             tmem_ld8(taddr + (uint32_t)ch, v);
             tmem_ld_wait();
-            if (valid) {
-              const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch);
-              const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch + 4);
-              float f[8];
-              f[0] = __uint_as_float(v[0]) + b0.x; f[1] = __uint_as_float(v[1]) + b0.y;
-              f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
-              f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
-              f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
-              if (rp) {
-                const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
-                const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float2 rf = __bfloat1622float2(rb[i]);
-                  f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
-                }
-              }
-              uint4 ov;
-              __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                float f0 = f[2 * i], f1 = f[2 * i + 1];
-                if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
-                ob[i] = __floats2bfloat162_rn(f0, f1);
-              }
-              *reinterpret_cast<uint4 *>(dst + ch) = ov;
-            }
+            if (valid) store8(v, ch);
           }
         }
         // this warp has read what it needs of the accumulator set

@@ -302,7 +302,9 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (16, 24, 3, 2, 0, 2, 17, 36, "k_conv_tc_pairrows"),     # stride 2, no padding, odd height
     (40, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc"),              # stride 2 on parity planes (more than 32 channels)
     (32, 16, 1, 1, 0, 2, 20, 24, "k_conv_tc_pairrows"),     # 1x1: one instruction per 32-byte K step
-    (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with a wide output: general kernel
+    (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc_rows"),         # 1x1 expansion from few channels: one half-filled plane
+    (16, 96, 1, 1, 0, 1, 40, 112, "k_conv_tc_rows"),        # 1x1 expansion from 16 channels, row tiles
+    (32, 40, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with 40 outputs: general kernel
     (16, 128, 3, 1, 1, 1, 12, 16, "k_conv_tc_pairrows"),    # N = 256: two accumulator slots, run-time channel loop
     (32, 64, 3, 2, 1, 1, 28, 28, "k_conv_tc_pairrows"),     # stride 2, 64 output channels
     (160, 200, 3, 1, 1, 5, 7, 7, "k_conv_tc_rows"),         # three planes (the last half full), two passes, three images per tile
