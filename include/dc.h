@@ -270,6 +270,42 @@ dc_status dc_chain_forward_host_async(const dc_layer *layers, int n_layers, cons
                                 void *y_host, dc_dtype dtype, void *workspace,
                                 size_t workspace_bytes, dc_stream stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * The selector's two dynamic programmes (Sec. 4.3).  Host only: every pointer is host memory, no
+ * device call is made.  Boundaries are 0..L for a network of L layers; tables are row-major
+ * (L+1) x (L+1) and only entries [i][j] with i < j are read.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Latency of a span that cannot be merged into one convolution; sums that contain it stay at it. */
+#define DC_DP_INF (1ll << 60)
+
+/*
+ * Algorithm 1 (Eq. 6a, 6b): T_opt[k][l] = min over S in {k+1..l-1} of the summed latency
+ * T[s_{i-1}][s_i] of the pieces (k, s_1], ..., (s_n, l], with T_opt[k][k] = 0.
+ * T: integer latencies (any unit), DC_DP_INF where layers i+1..j do not merge.
+ * T_opt: out, (L+1) x (L+1).  split: out, (L+1) x (L+1) ints; split[k][l] = m is the last boundary
+ * of the optimal pattern of (k, l] (m == k: one merged layer), so that
+ * S_opt[k][l] = S_opt[k][m] + {m}; ties take the smallest m.  Entries with k >= l are set to 0 / k.
+ * DC_ERR_INVALID_ARG for NULL pointers, L <= 0 or a negative latency.
+ */
+dc_status dc_dp_optimal_latency(const long long *T, int L, long long *T_opt, int *split);
+
+/* Host only: writes S_opt[k][l] (increasing) into S (room for L ints) and its size into n_S, from
+ * the split table of dc_dp_optimal_latency. */
+dc_status dc_dp_pattern(const int *split, int L, int k, int l, int *S, int *n_S);
+
+/*
+ * Algorithm 2 (Eq. 5, 7, 8): the activations to keep (A) and the boundaries that stay after merging
+ * (S, A a subset of S) that maximise the summed importance I[a_{j-1}][a_j] of the blocks of A under
+ * "summed latency of the pieces of S < T0" (strict).  I: doubles, -infinity excludes a block.
+ * A, S: out, increasing, room for L ints each; objective: out, D[L][T0]; feasible: out, 0 when no
+ * pattern meets the budget (T0 <= T_opt[0][L]) or every pattern contains an excluded block -- A and
+ * S are then empty.  Ties take the smallest k.  Memory: (L+1)(T0+1) doubles and ints on the host
+ * heap; DC_ERR_WORKSPACE if that cannot be allocated, DC_ERR_INVALID_ARG for bad arguments.
+ */
+dc_status dc_dp_select(const long long *T, const double *I, int L, long long T0, int *A, int *n_A,
+                       int *S, int *n_S, double *objective, int *feasible);
+
 #ifdef __cplusplus
 }
 #endif

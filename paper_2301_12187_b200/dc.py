@@ -61,6 +61,11 @@ EXPORTS = {
                                  C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
     "dc_merge_chain_algo": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p, C.c_int]),
+    "dc_dp_optimal_latency": (C.c_int, [C.POINTER(C.c_longlong), C.c_int, C.POINTER(C.c_longlong), C.POINTER(C.c_int)]),
+    "dc_dp_pattern": (C.c_int, [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]),
+    "dc_dp_select": (C.c_int, [C.POINTER(C.c_longlong), C.POINTER(C.c_double), C.c_int, C.c_longlong,
+                               C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
+                               C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "dc_merge_chain_static": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "dc_merge_chain_static_capacity": (C.c_size_t, []),
@@ -238,6 +243,54 @@ def merge_chain_static(layers, residuals, w_merged, b_merged, w_packed, packed_d
 
 def merge_chain_static_capacity() -> int:
     return int(lib().dc_merge_chain_static_capacity())
+
+
+DP_INF = 1 << 60
+
+
+def _ll_table(T, L):
+    flat = (C.c_longlong * ((L + 1) * (L + 1)))()
+    for i in range(L + 1):
+        for j in range(L + 1):
+            flat[i * (L + 1) + j] = int(T[i][j]) if j > i else 0
+    return flat
+
+
+def dp_optimal_latency(T, L: int):
+    """Algorithm 1 on host tables (lists or arrays indexed [i][j]): returns (T_opt, split) as lists
+    of lists; split[k][l] is the last boundary of the optimal pattern of (k, l]."""
+    W = L + 1
+    t_opt = (C.c_longlong * (W * W))()
+    split = (C.c_int * (W * W))()
+    _check(lib().dc_dp_optimal_latency(_ll_table(T, L), L, t_opt, split), "dc_dp_optimal_latency")
+    return ([[int(t_opt[i * W + j]) for j in range(W)] for i in range(W)],
+            [[int(split[i * W + j]) for j in range(W)] for i in range(W)])
+
+
+def dp_pattern(split, L: int, k: int, l: int):
+    """S_opt[k][l] (increasing list) from the split table of dp_optimal_latency."""
+    W = L + 1
+    flat = (C.c_int * (W * W))(*[int(split[i][j]) for i in range(W) for j in range(W)])
+    out = (C.c_int * max(L, 1))()
+    n = C.c_int(0)
+    _check(lib().dc_dp_pattern(flat, L, k, l, out, C.byref(n)), "dc_dp_pattern")
+    return [int(out[i]) for i in range(n.value)]
+
+
+def dp_select(T, I, L: int, T0: int):
+    """Algorithm 2 on host tables: returns (A, S, objective, feasible)."""
+    W = L + 1
+    imp = (C.c_double * (W * W))()
+    for i in range(W):
+        for j in range(W):
+            imp[i * W + j] = float(I[i][j]) if j > i else 0.0
+    a = (C.c_int * max(L, 1))()
+    s = (C.c_int * max(L, 1))()
+    na, ns, ok = C.c_int(0), C.c_int(0), C.c_int(0)
+    obj = C.c_double(0.0)
+    _check(lib().dc_dp_select(_ll_table(T, L), imp, L, int(T0), a, C.byref(na), s, C.byref(ns), C.byref(obj),
+                              C.byref(ok)), "dc_dp_select")
+    return [int(a[i]) for i in range(na.value)], [int(s[i]) for i in range(ns.value)], obj.value, bool(ok.value)
 
 
 def pack_weights(w, g: Geom, dtype: int, w_packed, stream=None):

@@ -314,3 +314,21 @@ def plan_spans(net: Network, seed: int = 0, n_remove: int = 17, max_k3: int = 3)
         ops.append(op)
         produced_by[idx[-1]] = len(ops) - 1
     return acts, ops
+
+
+def random_dp_tables(rng, L, inf, unmergeable=0.2, neg_inf=0.0):
+    """Seeded latency / importance tables for the selector's dynamic programmes: T[i][j] small
+    positive integers growing with the span (`inf` for a share of the spans longer than one layer),
+    I[i][j] = 0 for single layers and negative for longer blocks (-infinity for a share of them).
+    `rng` is a random.Random."""
+    T = [[0] * (L + 1) for _ in range(L + 1)]
+    I = [[0.0] * (L + 1) for _ in range(L + 1)]
+    for i in range(L + 1):
+        for j in range(i + 1, L + 1):
+            T[i][j] = rng.randint(1, 9) + (j - i - 1) * rng.randint(0, 3)
+            if j - i > 1 and rng.random() < unmergeable:
+                T[i][j] = inf
+            I[i][j] = 0.0 if j - i == 1 else -rng.random() * (j - i)
+            if j - i > 1 and rng.random() < neg_inf:
+                I[i][j] = float("-inf")
+    return T, I

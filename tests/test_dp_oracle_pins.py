@@ -7,20 +7,11 @@ import random
 import pytest
 
 from oracle import dp_oracle as P
+from paper_2301_12187_b200 import inputs as I_
 
 
 def random_tables(rng, L, unmergeable=0.2, neg_inf=0.0):
-    T = [[0] * (L + 1) for _ in range(L + 1)]
-    I = [[0.0] * (L + 1) for _ in range(L + 1)]
-    for i in range(L + 1):
-        for j in range(i + 1, L + 1):
-            T[i][j] = rng.randint(1, 9) + (j - i - 1) * rng.randint(0, 3)
-            if j - i > 1 and rng.random() < unmergeable:
-                T[i][j] = P.INF
-            I[i][j] = 0.0 if j - i == 1 else -rng.random() * (j - i)
-            if j - i > 1 and rng.random() < neg_inf:
-                I[i][j] = -math.inf
-    return T, I
+    return I_.random_dp_tables(rng, L, P.INF, unmergeable, neg_inf)
 
 
 @pytest.mark.parametrize("seed", range(6))
