@@ -1,0 +1,140 @@
+"""Latency table T[i][j] of a network on this GPU and the latency-optimal merge pattern.
+
+T[i][j] (Sec. 4.1) is the measured forward time of the one convolution that layers i+1..j merge
+into when the activations between them are identities: the span is merged with dc_merge_chain and
+its dc_conv_forward (dc_dwconv_forward for a lone depthwise layer) is timed with CUDA events.
+Spans that cannot be merged carry dc.DP_INF.  Algorithm 1 (dc_dp_optimal_latency) then gives, for
+every span, the pattern that merges only where merging is faster.
+
+Host logic only: which spans are valid, buffers, timing loops.  All arithmetic runs in the library.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Tuple
+
+from . import dc
+
+
+def _out_extent(h, k, s, p):
+    return (h + 2 * p - k) // s + 1
+
+
+def span_residuals(net, i: int, j: int, max_k: int = 7) -> Optional[List[Tuple[int, int]]]:
+    """Skip groups (relative to the span) if layers i..j-1 (0-based; boundaries i and j) may be
+    merged into one convolution, else None.  Rules: a skip block lies wholly inside the span or does
+    not touch it -- a single layer is always a valid span, its block's addition stays outside --
+    (App. E.1); no layer with k > 1 after a stride-2 layer of the span (App. B.2); merged kernel
+    size at most max_k (a limit of this harness, not of the method)."""
+    L = net.layers
+    if j - i == 1:
+        return []
+    res = []
+    for blk in net.blocks:
+        if not blk["residual"]:
+            continue
+        f, l = blk["first"], blk["last"]
+        inside = i <= f and l < j
+        disjoint = l < i or f >= j
+        if inside:
+            res.append((f - i, l - i))
+        elif not disjoint:
+            return None
+    k, s, seen_s2 = 1, 1, False
+    for a in range(i, j):
+        if seen_s2 and L[a].k > 1:
+            return None
+        k += (L[a].k - 1) * s
+        s *= L[a].stride
+        seen_s2 = seen_s2 or L[a].stride > 1
+    if k > max_k:
+        return None
+    return res
+
+
+def boundary_shapes(net):
+    """NHWC shape of the feature map at every boundary 0..L."""
+    n, h, w, c = net.x_shape
+    shapes = [(n, h, w, c)]
+    for lay in net.layers:
+        h, w = _out_extent(h, lay.k, lay.stride, lay.pad), _out_extent(w, lay.k, lay.stride, lay.pad)
+        shapes.append((n, h, w, lay.c_out))
+    return shapes
+
+
+def measure_latency_table(net, unit_us: float = 1.0, reps: int = 10, max_span: int = 9, max_k: int = 7):
+    """Returns (T, us): T[i][j] = ceil(latency / unit_us) as Python ints (dc.DP_INF where the span
+    is not mergeable or longer than max_span layers), us[i][j] the measured microseconds (None where
+    not measured).  bf16, this process's current CUDA device.  Each span's forward is captured `reps`
+    times in one CUDA graph and the graph's time divided by reps (inputs stay in L2 for small maps:
+    the table ranks merge patterns of one network against each other, it is not a roofline figure)."""
+    import math
+    import torch
+
+    nL = len(net.layers)
+    shapes = boundary_shapes(net)
+    devs = [dc.DeviceLayer(s) for s in net.layers]
+    T = [[0] * (nL + 1) for _ in range(nL + 1)]
+    us = [[None] * (nL + 1) for _ in range(nL + 1)]
+    conv_ws = torch.zeros(dc.conv_workspace_bytes(), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.Stream()
+    for i in range(nL):
+        x = torch.zeros(shapes[i], dtype=torch.bfloat16, device="cuda")
+        for j in range(i + 1, nL + 1):
+            T[i][j] = dc.DP_INF
+            if j - i > max_span:
+                continue
+            res = span_residuals(net, i, j, max_k)
+            if res is None:
+                continue
+            layers = devs[i:j]
+            try:
+                g, ws_bytes = dc.merge_query(layers, res)
+            except dc.DcError:
+                continue
+            y = torch.empty(shapes[j], dtype=torch.bfloat16, device="cuda")
+            lone_dw = j - i == 1 and net.layers[i].groups != 1
+            with torch.cuda.stream(stream):
+                if lone_dw:
+                    lay = net.layers[i]
+                    wf = torch.empty_like(devs[i].weight)
+                    bf = torch.empty(lay.c_out, device="cuda")
+                    dc.fold_bn(devs[i], wf, bf)
+                    gd = dc.geom(lay.c_in, lay.c_out, lay.groups, lay.k, lay.stride, lay.pad)
+                    packed = torch.empty(dc.packed_bytes(gd, dc.F32), dtype=torch.uint8, device="cuda")
+                    dc.pack_weights(wf, gd, dc.F32, packed)
+
+                    def run():
+                        dc.dwconv_forward(x, lay.k, lay.stride, lay.pad, packed, bf, dc.ACT_IDENTITY, y)
+                else:
+                    wm = torch.empty((g.c_out, g.c_in, g.k, g.k), dtype=torch.float32, device="cuda")
+                    bm = torch.empty((g.c_out,), dtype=torch.float32, device="cuda")
+                    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+                    packed = torch.empty(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
+                    dc.merge_chain(layers, res, wm, bm, packed, dc.BF16, ws)
+
+                    def run():
+                        dc.conv_forward(x, g, packed, bm, dc.ACT_IDENTITY, None, y, conv_ws)
+                run()
+                stream.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=stream):
+                    for _ in range(reps):
+                        run()
+                graph.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                graph.replay()
+                e1.record(stream)
+                stream.synchronize()
+            if dc.workspace_status(conv_ws) != dc.OK:
+                raise RuntimeError("device-side wait timed out while timing span (%d, %d)" % (i, j))
+            t_us = e0.elapsed_time(e1) * 1e3 / reps
+            us[i][j] = t_us
+            T[i][j] = max(1, int(math.ceil(t_us / unit_us)))
+    return T, us
+
+
+def optimal_pattern(T, L: int):
+    """Algorithm 1 on a measured table: (T_opt[0][L], S_opt[0][L], T_opt, split)."""
+    t_opt, split = dc.dp_optimal_latency(T, L)
+    return t_opt[0][L], dc.dp_pattern(split, L, 0, L), t_opt, split
