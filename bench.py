@@ -155,6 +155,13 @@ def run_network(args):
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     net = I.mobilenet_v2(seed=0, batch=128)
     acts, plan = I.plan_spans(net, seed=0)
+    plan_name = "every valid span merged"
+    if args.plan == "latency":
+        # the same kept activations, cut by Algorithm 1 over the latency table measured on this GPU
+        from paper_2301_12187_b200 import latency as LT
+        T, _ = LT.measure_latency_table(net, unit_us=0.1, reps=10, max_span=9)
+        plan, _, _ = LT.latency_optimal_plan(net, acts, T)
+        plan_name = "latency-optimal pattern (Algorithm 1 over the measured table)"
     cn = CompressedNetwork(net, acts, plan)
     x = torch.from_numpy(I.make_input(0, net.x_shape, bf16=True)).to("cuda", dtype=torch.bfloat16)
     stream = torch.cuda.Stream()
@@ -212,7 +219,7 @@ def run_network(args):
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": "cfg4_mbv2_full_batch128", "launch_groups": len(cn.ops),
-                   "merged_spans": sum(1 for op in cn.ops if op.merged), "plan_seed": 0,
+                   "merged_spans": sum(1 for op in cn.ops if op.merged), "plan_seed": 0, "plan": plan_name,
                    "step": "all dc_merge_chain calls + forward graph", "l2": "activation maps (0.1-0.6 GB each) exceed L2"},
         "forward_ms": ms_fwd, "forward_images_per_s": 128 / (ms_fwd * 1e-3), "merge_latency_us": ms_merge * 1e3,
         "roofline": {"bound": "hbm", "achieved": roof_s / (ms_fwd * 1e-3), "peak": 1.0, "unit": "fraction of summed per-group roofline time",
@@ -489,6 +496,8 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--plan", default="spans", choices=["spans", "latency"],
+                    help="cfg4 only: merge every valid span, or cut by Algorithm 1 over the measured latency table")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

@@ -301,7 +301,14 @@ def plan_spans(net: Network, seed: int = 0, n_remove: int = 17, max_k3: int = 3)
         prev_forced_after = cut_after
     close()
 
-    # ops, with the explicit skip additions wired to the op that produced the block input
+    return acts, ops_from_spans(net, acts, spans)
+
+
+def ops_from_spans(net: Network, acts, spans) -> List[PlanOp]:
+    """PlanOps for a list of spans (consecutive layer indices, folded skip groups relative to the
+    span), with the skip additions that stay explicit wired to the op that produced the block
+    input."""
+    L = net.layers
     ops: List[PlanOp] = []
     produced_by = {}                   # layer index -> op index whose output is that layer's output
     for idx, res in spans:
@@ -313,7 +320,31 @@ def plan_spans(net: Network, seed: int = 0, n_remove: int = 17, max_k3: int = 3)
             op.add_from = produced_by.get(blk["first"] - 1, -1)
         ops.append(op)
         produced_by[idx[-1]] = len(ops) - 1
-    return acts, ops
+    return ops
+
+
+def removed_activations(net: Network, seed: int = 0, n_remove: int = 17):
+    """acts[l] after the seeded choice of plan_spans: the first n_remove ReLU6 positions (head
+    excluded) in the order of a seeded hash become identities."""
+    L = net.layers
+    cand = [i for i in range(len(L) - 1) if L[i].act == "relu6"]
+    keys = _stream(seed, (1 << 21) + 7, 0, len(cand))
+    order = [cand[j] for j in np.argsort(keys, kind="stable")]
+    removed = set(order[:n_remove])
+    return [None if (i in removed) else L[i].act for i in range(len(L))]
+
+
+def plan_from_boundaries(net: Network, acts, boundaries, span_residuals) -> List[PlanOp]:
+    """PlanOps for the pieces (b_0, b_1], (b_1, b_2], ... of `boundaries` (0 = b_0 < ... < b_n = L):
+    the merge pattern S of Sec. 4 with the kept activations `acts`.  span_residuals(i, j) gives the
+    folded skip groups of a piece (or None if the piece cannot be merged: an error here)."""
+    spans = []
+    for a, c in zip(boundaries[:-1], boundaries[1:]):
+        res = span_residuals(a, c)
+        if res is None or any(acts[i] is not None for i in range(a, c - 1)):
+            raise ValueError("piece (%d, %d] cannot be merged" % (a, c))
+        spans.append((list(range(a, c)), list(res)))
+    return ops_from_spans(net, acts, spans)
 
 
 def random_dp_tables(rng, L, inf, unmergeable=0.2, neg_inf=0.0):

@@ -138,3 +138,21 @@ def optimal_pattern(T, L: int):
     """Algorithm 1 on a measured table: (T_opt[0][L], S_opt[0][L], T_opt, split)."""
     t_opt, split = dc.dp_optimal_latency(T, L)
     return t_opt[0][L], dc.dp_pattern(split, L, 0, L), t_opt, split
+
+
+def latency_optimal_plan(net, acts, T):
+    """Merge pattern for a network whose kept activations are fixed (`acts[l]` is None where layer
+    l's activation is an identity): spans that would swallow a kept activation become unmergeable,
+    Algorithm 1 picks the fastest pattern among the rest, and the pieces become plan ops.  Returns
+    (ops, boundaries, T_opt[0][L])."""
+    from . import inputs as I
+    L = len(net.layers)
+    Tm = [row[:] for row in T]
+    for i in range(L + 1):
+        for j in range(i + 2, L + 1):
+            if any(acts[a] is not None for a in range(i, j - 1)):
+                Tm[i][j] = dc.DP_INF
+    total, S, _, _ = optimal_pattern(Tm, L)
+    bounds = [0] + S + [L]
+    ops = I.plan_from_boundaries(net, acts, bounds, lambda a, c: span_residuals(net, a, c))
+    return ops, bounds, total

@@ -56,3 +56,67 @@ def test_measured_table_and_optimal_pattern():
     # a merged inverted-residual block replaces three launches over 6x wider maps: it must be in the table
     blk = [b for b in net.blocks if b["residual"]][0]
     assert T[blk["first"]][blk["last"] + 1] < dc.DP_INF
+
+
+@pytest.mark.gpu
+def test_latency_planned_network_matches_the_oracle():
+    """The network cut by Algorithm 1 over the measured table (kept activations fixed by the seed):
+    every piece is a valid merge, the plan is no slower by the table than merging every valid span,
+    and the forward pass matches the oracle's network end to end."""
+    import numpy as np
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from oracle import dc_oracle as O
+    from paper_2301_12187_b200 import dc
+    from paper_2301_12187_b200.network import CompressedNetwork
+    dc.lib()
+    net = I.mobilenet_v2(seed=0, batch=4, res=64)
+    L = len(net.layers)
+    acts = I.removed_activations(net, seed=0)
+    T, _ = LT.measure_latency_table(net, unit_us=0.1, reps=5, max_span=6)
+    ops, bounds, total = LT.latency_optimal_plan(net, acts, T)
+    assert bounds[0] == 0 and bounds[-1] == L and bounds == sorted(set(bounds))
+    assert sorted(i for op in ops for i in op.layers) == list(range(L))
+    # every kept activation ends a piece
+    assert all((i + 1) in bounds for i in range(L - 1) if acts[i] is not None)
+    # by the table, no slower than the plan that merges every valid span
+    _, greedy = I.plan_spans(net, seed=0)
+    t_greedy = sum(T[op.layers[0]][op.layers[-1] + 1] for op in greedy)
+    assert total <= t_greedy
+
+    cn = CompressedNetwork(net, acts, ops)
+    cn.merge()
+    x_np = I.make_input(0, net.x_shape, bf16=True)
+    x = torch.from_numpy(x_np).to("cuda", dtype=torch.bfloat16)
+    y = cn.forward(x)
+    torch.cuda.synchronize()
+    assert cn.status() == dc.OK
+
+    def nchw(t):
+        return t.float().cpu().numpy().astype(np.float64).transpose(0, 3, 1, 2)
+
+    cur, outs = nchw(x[:1]), []
+    for op in cn.ops:
+        specs = [net.layers[i] for i in op.layers]
+        if op.kind == "block":
+            nxt = cur
+            for s in specs:
+                Wf, bf = O.fold_bn(s)
+                nxt = O.conv_direct(nxt, Wf, bf, s.k, s.stride, s.pad, s.groups)
+                if s.act == "relu6":
+                    nxt = O.relu6(nxt)
+            if net.blocks[specs[0].block]["residual"]:
+                nxt = nxt + cur
+        else:
+            po = cn.plan_ops[op.plan_index[0]]
+            nxt = O.chain_forward_reordered(cur, specs, po.residuals)
+            if op.add_from == -1:
+                nxt = nxt + nchw(x[:1])
+            elif op.add_from >= 0:
+                nxt = nxt + outs[op.add_from]
+            if po.act == "relu6":
+                nxt = O.relu6(nxt)
+        cur = nxt
+        outs.append(cur)
+    assert O.rel_l2(nchw(y[:1]), cur) <= 2e-2
