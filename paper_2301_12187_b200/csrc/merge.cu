@@ -414,12 +414,74 @@ __device__ __forceinline__ float merged_at(const Piece &p, int o, int i, int t) 
   return w;
 }
 
+// The bf16 packed copy with one thread per 16-byte chunk (8 input channels of one operand row),
+// for large kernels (a thread walks eight elements, so small ones are faster element by element): the
+// entry and row are decoded once per chunk, the eight weights are fetched by eight independent
+// loads (an element that is padding reads element 0 and is then zeroed, so that no load sits behind
+// a branch) and the chunk is written by one store.
+__device__ __forceinline__ void deliver_packed_bf16_chunks(const Piece &acc, __nv_bfloat16 *out, const KOrder &ko,
+                                                           int start, int stride) {
+  const int c_out = acc.c_out, kk = acc.k * acc.k, ctr = ((acc.k - 1) / 2) * (acc.k + 1);
+  const int total8 = ko.ng * ko.e_pad * ko.n_pad;
+  for (int idx8 = start; idx8 < total8; idx8 += stride) {
+    const int plane = idx8 / ko.n_pad, o_row = idx8 - plane * ko.n_pad;
+    const int grp = plane / ko.e_pad, e = plane - grp * ko.e_pad;
+    int pc, ccg0, r, s0;
+    bool live = dc_korder_decode(ko, e, &pc, &ccg0, &r, &s0);
+    int o = o_row, px = 0;
+    if (live) {
+      if (ko.fold) {
+        s0 = o / ko.co8;
+        o -= s0 * ko.co8;
+        if (s0 >= ko.k) live = false;
+      } else if (ko.pair == 2) {
+        px = o / ko.co8;
+        o -= px * ko.co8;
+        if (px >= 2) live = false;
+      }
+    }
+    live = live && o < c_out;
+    int ch[8], tap[8];
+    bool ok[8];
+#pragma unroll
+    for (int c8 = 0; c8 < 8; ++c8) {
+      int sx = s0, c;
+      if (ko.pair >= 2) {
+        const int elem = ccg0 * 8 + c8, ipx = elem / ko.c_in;
+        sx = 2 * s0 + ipx - (ko.pair == 2 ? px : (ko.pad & 1));
+        c = grp * ko.cg * 8 + elem - ipx * ko.c_in;
+      } else {
+        c = (grp * ko.cg + ccg0) * 8 + c8;
+      }
+      ok[c8] = live && sx >= 0 && sx < ko.k && c >= 0 && c < ko.c_in;
+      ch[c8] = c;
+      tap[c8] = r * ko.k + sx;
+    }
+    float w[8];
+#pragma unroll
+    for (int c8 = 0; c8 < 8; ++c8) {
+      size_t off = 0;
+      if (ok[c8]) off = acc.diag ? (size_t)o * kk + tap[c8] : ((size_t)o * acc.c_in + ch[c8]) * kk + tap[c8];
+      w[c8] = acc.w[off];
+    }
+    __align__(16) __nv_bfloat16 v8[8];
+#pragma unroll
+    for (int c8 = 0; c8 < 8; ++c8) {
+      float v = w[c8];
+      if (acc.diag && o != ch[c8]) v = 0.f;
+      if (acc.ident && o == ch[c8] && tap[c8] == ctr) v += 1.f;
+      v8[c8] = __float2bfloat16_rn(ok[c8] ? v : 0.f);
+    }
+    *reinterpret_cast<uint4 *>(out + (size_t)idx8 * 8) = *reinterpret_cast<const uint4 *>(v8);
+  }
+}
+
 // Last launch of a merge: writes the dense fp32 kernel (blocks [0, nb_w)), the bias (block nb_w)
 // and, when asked for, the packed copy for the forward kernels (blocks after that; mode 1: fp32
 // [u][v][i][o], mode 2: bf16 chunk planes in the K order of KOrder), all straight from the
 // accumulated piece.
 __global__ void k_deliver(Piece acc, float *w_merged, float *b_merged, void *packed, int mode, KOrder ko,
-                          int nb_w, int nb_p) {
+                          int nb_w, int nb_p, int chunked) {
   const int c_out = acc.c_out, c_in = acc.c_in, kk = acc.k * acc.k;
   int blk = (int)blockIdx.x;
   if (blk < nb_w) {
@@ -443,6 +505,9 @@ __global__ void k_deliver(Piece acc, float *w_merged, float *b_merged, void *pac
       const int o = idx % c_out, i = (idx / c_out) % c_in, t = idx / (c_out * c_in);
       out[idx] = merged_at(acc, o, i, t);
     }
+  } else if (mode == 2 && chunked) {
+    deliver_packed_bf16_chunks(acc, reinterpret_cast<__nv_bfloat16 *>(packed), ko, blk * blockDim.x + threadIdx.x,
+                               nb_p * blockDim.x);
   } else if (mode == 2) {
     __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(packed);
     const int total = ko.ng * ko.e_pad * ko.n_pad * 8;
@@ -842,8 +907,9 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
     p_elems = mode == 1 ? elems : (size_t)ko.ng * ko.e_pad * ko.n_pad * 8;
     if (!dc_aligned16(w_packed)) return DC_ERR_ALIGNMENT;
   }
-  const int nb_w = blocks_for(elems, 256), nb_p = mode ? blocks_for(p_elems, 256) : 0;
-  k_deliver<<<nb_w + 1 + nb_p, 256, 0, st>>>(acc, w_merged, b_merged, w_packed, mode, ko, nb_w, nb_p);
+  const int chunked = mode == 2 && p_elems >= (size_t)262144;
+  const int nb_w = blocks_for(elems, 256), nb_p = mode ? blocks_for(chunked ? p_elems / 8 : p_elems, 256) : 0;
+  k_deliver<<<nb_w + 1 + nb_p, 256, 0, st>>>(acc, w_merged, b_merged, w_packed, mode, ko, nb_w, nb_p, chunked);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
 

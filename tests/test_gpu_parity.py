@@ -204,6 +204,22 @@ def test_block_step_edge_cases(dc, case):
     assert O.rel_l2(wm2.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm2.cpu().numpy(), b) <= TOL_W
 
 
+@pytest.mark.parametrize("stride", [1, 2])
+def test_large_packed_copy_is_written_chunk_by_chunk(dc, stride):
+    """Merged kernels whose packed copy has 262 144 elements or more are packed one 16-byte chunk per
+    thread (rows order for stride 1, general order for stride 2): same bits as dc_pack_weights."""
+    mk = I.make_layer
+    specs = [mk(21, 0, 192, 192, 1, 1, 0), mk(21, 1, 192, 192, 3, stride, 1)]
+    g, wm, bm, packed = run_merge(dc, specs, [], packed_dtype=dc.BF16)
+    assert packed.numel() // 2 >= 262144
+    W, b, *_ = O.merge_formula(specs, [])
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    again = torch.empty_like(packed)
+    dc.pack_weights(wm, g, dc.BF16, again)
+    torch.cuda.synchronize()
+    assert torch.equal(packed, again)
+
+
 @pytest.mark.parametrize("name", CHAINS)
 def test_merged_conv_fp32_equals_sequential_chain(dc, name):
     specs, res = small_chain(name, rng_seed=1)
