@@ -577,8 +577,17 @@ __device__ __forceinline__ float raw_bias(const RawLayer &L, int o, float g) {
   return L.gamma ? fmaf(b - L.mean[o], g, L.beta[o]) : b;
 }
 
-__global__ void __launch_bounds__(kBlockThreads) k_merge_block(const __grid_constant__ BlockArgs a) {
+// Up to kBlockBatch blocks of one run go out in one launch (blockIdx.y picks the block): they depend
+// on the raw layers only, not on one another.
+constexpr int kBlockBatch = 4;
+struct BlockBatch {
+  BlockArgs blk[kBlockBatch];
+};
+
+__global__ void __launch_bounds__(kBlockThreads) k_merge_block(const __grid_constant__ BlockBatch batch) {
   extern __shared__ __align__(16) float blk_smem[];
+  const BlockArgs &a = batch.blk[blockIdx.y];
+  if ((int)blockIdx.x >= a.c2) return;
   const int c0 = a.c0, c1 = a.c1, kk = a.k * a.k, J = c0 * kk, CH = a.chunk;
   float *Ms = blk_smem;                 // [CH][c0]  raw W1 rows
   float *Ds = Ms + CH * c0;             // [CH][kk]  raw D rows, then W3~[o][c] * D~[c][t] * g1[c]
@@ -858,6 +867,19 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
   }
 
   // 2. compose: blocks and skip groups first (with their identity tap), then left to right
+  BlockBatch batch;
+  int n_batch = 0, batch_grid = 0;
+  size_t batch_smem = 0;
+  auto flush_blocks = [&]() {
+    if (n_batch == 0) return;
+    static bool attr_set = false;
+    if (!attr_set) {
+      cudaFuncSetAttribute(k_merge_block, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      attr_set = true;
+    }
+    k_merge_block<<<dim3(batch_grid, n_batch), kBlockThreads, batch_smem, st>>>(batch);
+    n_batch = 0; batch_grid = 0; batch_smem = 0;
+  };
   Piece acc{};
   bool have = false;
   int i = 0;
@@ -871,14 +893,13 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
       float *b = bump.take(piece.c_out);
       piece.w = w; piece.b = b;
       if (go) {
-        BlockArgs a{raw_of(e), raw_of(d), raw_of(p), e.c_in, e.c_out, p.c_out, d.k, chunk_at[i], w, b};
+        batch.blk[n_batch] = BlockArgs{raw_of(e), raw_of(d), raw_of(p), e.c_in, e.c_out, p.c_out, d.k, chunk_at[i], w, b};
         const size_t smem = (size_t)chunk_at[i] * (e.c_in + d.k * d.k + 1) * sizeof(float);
-        static bool attr_set = false;
-        if (!attr_set) {
-          cudaFuncSetAttribute(k_merge_block, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-          attr_set = true;
-        }
-        k_merge_block<<<p.c_out, kBlockThreads, smem, st>>>(a);
+        if (smem > batch_smem) batch_smem = smem;
+        if (p.c_out > batch_grid) batch_grid = p.c_out;
+        // the blocks read raw layers only: hold the launch until the batch is full or a composition
+        // needs one of its pieces
+        if (++n_batch == kBlockBatch) flush_blocks();
       }
       i += 3;
     } else if (gi < 0) {
@@ -886,15 +907,20 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
       ++i;
     } else {
       piece = folded[res[gi].first];
+      if (go) flush_blocks();
       for (int j = res[gi].first + 1; j <= res[gi].last; ++j) piece = compose(piece, folded[j], bump, go, st);
       piece.ident = 1;          // f(x) + x: the identity kernel rides along as a flag
       i = res[gi].last + 1;
     }
     if (!have) { acc = piece; have = true; }
-    else acc = compose(acc, piece, bump, go, st);
+    else {
+      if (go) flush_blocks();
+      acc = compose(acc, piece, bump, go, st);
+    }
   }
   if (need) *need = bump.off + 256;
   if (!go) return DC_OK;
+  flush_blocks();
 
   // 3. deliver: dense fp32 result, bias, optional packed copy, in one launch
   size_t elems = (size_t)mg.c_out * mg.c_in * mg.k * mg.k;
