@@ -21,9 +21,9 @@ def _out_extent(h, k, s, p):
 
 def span_residuals(net, i: int, j: int, max_k: int = 7) -> Optional[List[Tuple[int, int]]]:
     """Skip groups (relative to the span) if layers i..j-1 (0-based; boundaries i and j) may be
-    merged into one convolution, else None.  Rules: a skip block lies wholly inside the span or does
-    not touch it -- a single layer is always a valid span, its block's addition stays outside --
-    (App. E.1); no layer with k > 1 after a stride-2 layer of the span (App. B.2); merged kernel
+    merged into one convolution, else None.  Rules: a skip block lies wholly inside the span (it is
+    folded as an identity kernel, App. E.1), does not touch it, or contains the whole span (the
+    block's addition then stays an explicit step after its last layer); no layer with k > 1 after a stride-2 layer of the span (App. B.2); merged kernel
     size at most max_k (a limit of this harness, not of the method)."""
     L = net.layers
     if j - i == 1:
@@ -35,9 +35,10 @@ def span_residuals(net, i: int, j: int, max_k: int = 7) -> Optional[List[Tuple[i
         f, l = blk["first"], blk["last"]
         inside = i <= f and l < j
         disjoint = l < i or f >= j
+        within = f <= i and j - 1 <= l
         if inside:
             res.append((f - i, l - i))
-        elif not disjoint:
+        elif not disjoint and not within:
             return None
     k, s, seen_s2 = 1, 1, False
     for a in range(i, j):

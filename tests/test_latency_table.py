@@ -16,7 +16,8 @@ def test_span_rules_on_mobilenet_v2():
     assert len(blocks) == 10
     f, l = blocks[0]["first"], blocks[0]["last"]
     assert LT.span_residuals(net, f, l + 1) == [(0, l - f)]              # the whole skip block: one group
-    assert LT.span_residuals(net, f + 1, l + 1) is None                   # cuts through the skip
+    assert LT.span_residuals(net, f + 1, l + 1) == []                     # inside the block: its addition stays explicit
+    assert LT.span_residuals(net, f + 1, l + 2) is None                   # leaves the block through its end
     assert LT.span_residuals(net, f - 1, l) is None
     assert LT.span_residuals(net, f - 1, l + 1) == [(1, l - f + 1)]       # a neighbour plus the whole block
     # stem (stride 2) followed by the first depthwise 3x3: a k > 1 layer after a stride-2 layer
@@ -120,3 +121,26 @@ def test_latency_planned_network_matches_the_oracle():
         cur = nxt
         outs.append(cur)
     assert O.rel_l2(nchw(y[:1]), cur) <= 2e-2
+
+
+def test_plan_from_boundaries_builds_the_same_ops_as_the_span_planner():
+    """Host logic: the ops built from explicit boundaries equal the span planner's when given its
+    own cuts, a piece that swallows a kept activation or cuts through a skip block is refused, and
+    explicit skip additions point at the op that produced the block input."""
+    net = I.mobilenet_v2(seed=0, batch=2, res=32)
+    L = len(net.layers)
+    acts, ops = I.plan_spans(net, seed=0)
+    assert acts == I.removed_activations(net, seed=0)
+    bounds = [0] + [op.layers[-1] + 1 for op in ops]
+    again = I.plan_from_boundaries(net, acts, bounds, lambda a, c: LT.span_residuals(net, a, c))
+    assert [(o.layers, o.residuals, o.act, o.add_from) for o in again] == \
+           [(o.layers, o.residuals, o.act, o.add_from) for o in ops]
+    # all single layers: every residual block's addition stays explicit and is wired backwards
+    singles = I.plan_from_boundaries(net, acts, list(range(L + 1)), lambda a, c: LT.span_residuals(net, a, c))
+    n_res = sum(1 for b in net.blocks if b["residual"])
+    assert sum(1 for o in singles if o.add_from >= -1) == n_res
+    assert all(o.add_from < i for i, o in enumerate(singles))
+    kept = next(i for i in range(L - 1) if acts[i] is not None)
+    with pytest.raises(ValueError):
+        I.plan_from_boundaries(net, acts, [0, kept, kept + 2] + list(range(kept + 3, L + 1)),
+                               lambda a, c: LT.span_residuals(net, a, c) if c - a > 1 else [])
