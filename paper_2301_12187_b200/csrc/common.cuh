@@ -146,7 +146,10 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
     const int n16 = (int)dc_round_up((size_t)g->c_out, 16);
     ko->rows = 1;
-    ko->nnt = dc_div_up(n16, 128);
+    // output channels per pass: at most 128, fewer for 5x5 and 7x7 kernels, whose weight stage of one
+    // (plane, tap row) step (k * 8 chunk planes of n_tile rows) must fit the shared-memory ring twice
+    const int n_tile_max = g->k <= 4 ? 128 : (g->k <= 5 ? 112 : 80);
+    ko->nnt = dc_div_up(n16, n_tile_max);
     ko->n_tile = (int)dc_round_up((size_t)dc_div_up(n16, ko->nnt), 16);
     ko->n_pad = ko->nnt * ko->n_tile;
     ko->ns[0] = g->k; ko->ns[1] = 0; ko->s0[0] = 0; ko->s0[1] = 0;

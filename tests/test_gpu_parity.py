@@ -204,6 +204,24 @@ def test_block_step_edge_cases(dc, case):
     assert O.rel_l2(wm2.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm2.cpu().numpy(), b) <= TOL_W
 
 
+@pytest.mark.parametrize("c,n,h,w", [(64, 2, 28, 28), (128, 2, 14, 14), (256, 1, 14, 14)])
+def test_vgg_style_dense_merge(dc, c, n, h, w):
+    """Two dense 3x3 layers (VGG-style, c -> c -> c) merged into one 5x5 layer: merged weights against
+    the formula, and the bf16 forward of the merged layer (tensor-bound for these widths) against the
+    sequential chain."""
+    mk = I.make_layer
+    specs = [mk(31, 0, c, c, 3, 1, 1), mk(31, 1, c, c, 3, 1, 1)]
+    g, wm, bm, packed = run_merge(dc, specs, [], packed_dtype=dc.BF16)
+    assert (g.k, g.stride, g.pad) == (5, 1, 2)
+    W, b, *_ = O.merge_formula(specs, [])
+    assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    assert dc.conv_kernel_name(n, h, w, g, dc.BF16) == "k_conv_tc_rows"
+    x = I.make_input(32, (n, h, w, c), bf16=True)
+    y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bm, dc.ACT_IDENTITY)
+    ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, [])
+    assert O.rel_l2(nchw(y), ref) <= TOL_BF16
+
+
 @pytest.mark.parametrize("stride", [1, 2])
 def test_large_packed_copy_is_written_chunk_by_chunk(dc, stride):
     """Merged kernels whose packed copy has 262 144 elements or more are packed one 16-byte chunk per
@@ -327,6 +345,8 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (96, 64, 1, 1, 0, 7, 7, 7, "k_conv_tc_rows"),           # 1x1: five images per tile, the last group partial
     (64, 48, 5, 1, 2, 1, 20, 70, "k_conv_tc_rows"),         # 5x5, two column strips, row tiles
     (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
+    (128, 128, 5, 1, 2, 2, 14, 14, "k_conv_tc_rows"),       # 5x5 with 128 outputs: two passes of 64 (weight stage limit)
+    (96, 96, 7, 1, 3, 1, 14, 14, "k_conv_tc_rows"),         # 7x7: passes of at most 80 output channels
     (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc"),             # many channels, few outputs: general kernel
     (192, 32, 1, 1, 0, 2, 28, 28, "k_conv_tc_rows"),        # 1x1 projection to 32 channels
 ])
