@@ -23,8 +23,9 @@ def span_residuals(net, i: int, j: int, max_k: int = 7) -> Optional[List[Tuple[i
     """Skip groups (relative to the span) if layers i..j-1 (0-based; boundaries i and j) may be
     merged into one convolution, else None.  Rules: a skip block lies wholly inside the span (it is
     folded as an identity kernel, App. E.1), does not touch it, or contains the whole span (the
-    block's addition then stays an explicit step after its last layer); no layer with k > 1 after a stride-2 layer of the span (App. B.2); merged kernel
-    size at most max_k (a limit of this harness, not of the method)."""
+    block's addition then stays an explicit step after its last layer); no layer with k > 1 after a
+    stride-2 layer of the span (App. B.2); merged kernel size at most max_k (a limit of this
+    harness, not of the method)."""
     L = net.layers
     if j - i == 1:
         return []
