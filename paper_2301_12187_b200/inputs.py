@@ -363,3 +363,21 @@ def random_dp_tables(rng, L, inf, unmergeable=0.2, neg_inf=0.0):
             if j - i > 1 and rng.random() < neg_inf:
                 I[i][j] = float("-inf")
     return T, I
+
+
+def random_dp_tables_ext(rng, L, inf, unmergeable=0.2, p_identity=0.4):
+    """Tables for the extended selector (App. B): T as random_dp_tables; I[i][j][a][b] the importance
+    of block (i, j] with end indicators (a, b) (single layers near 0, longer blocks more negative, a
+    kept non-linearity at an end slightly better); sigma_id[p] for p = 0..L says whether the original
+    activation at boundary p is an identity (each inner boundary with probability p_identity; the
+    network input counts as one, the last activation does not)."""
+    T, _ = random_dp_tables(rng, L, inf, unmergeable, 0.0)
+    I = [[[[0.0, 0.0], [0.0, 0.0]] for _ in range(L + 1)] for _ in range(L + 1)]
+    for i in range(L + 1):
+        for j in range(i + 1, L + 1):
+            base = -rng.random() * (j - i - 0.5)
+            for a in range(2):
+                for b in range(2):
+                    I[i][j][a][b] = base + 0.3 * rng.random() * (a + b) - 0.1 * rng.random()
+    sigma_id = [True] + [rng.random() < p_identity for _ in range(L - 1)] + [False]
+    return T, I, sigma_id
