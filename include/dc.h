@@ -306,6 +306,46 @@ dc_status dc_dp_pattern(const int *split, int L, int k, int l, int *S, int *n_S)
 dc_status dc_dp_select(const long long *T, const double *I, int L, long long T0, int *A, int *n_A,
                        int *S, int *n_S, double *objective, int *feasible);
 
+/*
+ * Extended selector (App. B).  A block (i, j] now carries the indicators d_i, d_j of a non-linear
+ * activation at its two ends, and its importance is I[i][j][d_i][d_j], stored as doubles at
+ * ((i * (L+1) + j) * 2 + d_i) * 2 + d_j.  sigma_id[p], p = 0..L (0 or 1), says whether the original
+ * activation at boundary p is an identity (p = 0: the network input).  Before either programme runs,
+ * the blocks that App. B excludes count as -infinity: d = 0 at an end whose original activation is
+ * non-linear, and d_j = 0 when both ends are identities in the original network (App. B.2).
+ *
+ * Algorithm 3: I_opt[k][l][a][b] = best summed importance of a chain of blocks from boundary k to
+ * boundary l with d_k = a, d_l = b and d = 0 at every inner boundary of the chain.  split (ints, same
+ * indexing) holds the chain's last inner boundary m (m == k: the single block), so that
+ * B_opt[k][l][a][b] = B_opt[k][m][a][0] + {m}; ties take the smallest m.  The listing's update is
+ * read with the maximiser m where it prints m', and its m' = k term as the single block
+ * I[k][l][a][b].  DC_ERR_INVALID_ARG for NULL pointers, L <= 0 or a flag other than 0 / 1.
+ */
+dc_status dc_dp_optimal_importance(const double *I, const unsigned char *sigma_id, int L, double *I_opt, int *split);
+
+/* Host only: writes B_opt[k][l][a][b] (increasing) into B (room for L ints) and its size into n_B,
+ * from the split table of dc_dp_optimal_importance. */
+dc_status dc_dp_importance_pattern(const int *split, int L, int k, int l, int a, int b, int *B, int *n_B);
+
+/* App. B.3, in place: every block's importance (j > i) loses alpha times the mean of the n_deltas
+ * accuracy changes measured on the size-one blocks.  DC_ERR_INVALID_ARG for NULL or n_deltas <= 0. */
+dc_status dc_dp_normalize_importance(double *I, int L, const double *deltas, int n_deltas, double alpha);
+
+/*
+ * Algorithm 4 (the extended surrogate problem of App. B): boundaries B of the importance blocks,
+ * the kept non-linear activations A (a subset of B and of S), the boundaries S that stay after
+ * merging, and the indicators of the network's two ends, maximising the summed
+ * I[b'][b][1_A(b')][1_A(b)] over the blocks of B under "summed latency of the pieces of S < T0".
+ * The state is D[l][t][a] with a = d_l; S and B carry that index like A, and the result is read at
+ * a_last = argmax_a D[L][T0][a] (where the listing prints A).  A, S, B: out, increasing, room for L
+ * ints each; d_first, d_last: out, d_0 and d_L; objective, feasible as for dc_dp_select.  Ties take
+ * the smallest k, then alpha = 0, then a = 0.  Memory: 2 (L+1)(T0+1) doubles and ints on the host
+ * heap (DC_ERR_WORKSPACE if that fails).
+ */
+dc_status dc_dp_select_ext(const long long *T, const double *I, const unsigned char *sigma_id, int L, long long T0,
+                           int *A, int *n_A, int *S, int *n_S, int *B, int *n_B, int *d_first, int *d_last,
+                           double *objective, int *feasible);
+
 #ifdef __cplusplus
 }
 #endif

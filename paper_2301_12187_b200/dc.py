@@ -66,6 +66,15 @@ EXPORTS = {
     "dc_dp_select": (C.c_int, [C.POINTER(C.c_longlong), C.POINTER(C.c_double), C.c_int, C.c_longlong,
                                C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
                                C.POINTER(C.c_double), C.POINTER(C.c_int)]),
+    "dc_dp_optimal_importance": (C.c_int, [C.POINTER(C.c_double), C.POINTER(C.c_ubyte), C.c_int, C.POINTER(C.c_double),
+                                          C.POINTER(C.c_int)]),
+    "dc_dp_importance_pattern": (C.c_int, [C.POINTER(C.c_int), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                          C.POINTER(C.c_int), C.POINTER(C.c_int)]),
+    "dc_dp_normalize_importance": (C.c_int, [C.POINTER(C.c_double), C.c_int, C.POINTER(C.c_double), C.c_int, C.c_double]),
+    "dc_dp_select_ext": (C.c_int, [C.POINTER(C.c_longlong), C.POINTER(C.c_double), C.POINTER(C.c_ubyte), C.c_int,
+                                  C.c_longlong, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                  C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                  C.POINTER(C.c_int), C.POINTER(C.c_double), C.POINTER(C.c_int)]),
     "dc_merge_chain_static": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "dc_merge_chain_static_capacity": (C.c_size_t, []),
@@ -291,6 +300,67 @@ def dp_select(T, I, L: int, T0: int):
     _check(lib().dc_dp_select(_ll_table(T, L), imp, L, int(T0), a, C.byref(na), s, C.byref(ns), C.byref(obj),
                               C.byref(ok)), "dc_dp_select")
     return [int(a[i]) for i in range(na.value)], [int(s[i]) for i in range(ns.value)], obj.value, bool(ok.value)
+
+
+def _imp4(I, L):
+    W = L + 1
+    flat = (C.c_double * (W * W * 4))()
+    for i in range(W):
+        for j in range(i + 1, W):
+            for a in range(2):
+                for b in range(2):
+                    flat[((i * W + j) * 2 + a) * 2 + b] = float(I[i][j][a][b])
+    return flat
+
+
+def _flags(sigma_id, L):
+    return (C.c_ubyte * (L + 1))(*[1 if x else 0 for x in sigma_id])
+
+
+def dp_optimal_importance(I, sigma_id, L: int):
+    """Algorithm 3 on host tables I[i][j][a][b]: returns (I_opt, split) as nested lists [k][l][a][b]."""
+    W = L + 1
+    out = (C.c_double * (W * W * 4))()
+    split = (C.c_int * (W * W * 4))()
+    _check(lib().dc_dp_optimal_importance(_imp4(I, L), _flags(sigma_id, L), L, out, split), "dc_dp_optimal_importance")
+    nest = lambda f: [[[[f[((i * W + j) * 2 + a) * 2 + b] for b in range(2)] for a in range(2)] for j in range(W)]
+                      for i in range(W)]
+    return nest(out), nest(split)
+
+
+def dp_importance_pattern(split, L: int, k: int, l: int, a: int, b: int):
+    """B_opt[k][l][a][b] (increasing list) from the split table of dp_optimal_importance."""
+    W = L + 1
+    flat = (C.c_int * (W * W * 4))(*[int(split[i][j][x][y]) for i in range(W) for j in range(W) for x in range(2)
+                                     for y in range(2)])
+    out = (C.c_int * max(L, 1))()
+    n = C.c_int(0)
+    _check(lib().dc_dp_importance_pattern(flat, L, k, l, a, b, out, C.byref(n)), "dc_dp_importance_pattern")
+    return [int(out[i]) for i in range(n.value)]
+
+
+def dp_normalize_importance(I, L: int, deltas, alpha: float):
+    """App. B.3 on a host table: returns the shifted copy as nested lists."""
+    W = L + 1
+    flat = _imp4(I, L)
+    d = (C.c_double * len(deltas))(*[float(x) for x in deltas])
+    _check(lib().dc_dp_normalize_importance(flat, L, d, len(deltas), float(alpha)), "dc_dp_normalize_importance")
+    return [[[[flat[((i * W + j) * 2 + a) * 2 + b] for b in range(2)] for a in range(2)] for j in range(W)]
+            for i in range(W)]
+
+
+def dp_select_ext(T, I, sigma_id, L: int, T0: int):
+    """Algorithm 4 on host tables: returns (A, S, B, d_first, d_last, objective, feasible)."""
+    a = (C.c_int * max(L, 1))()
+    s = (C.c_int * max(L, 1))()
+    b = (C.c_int * max(L, 1))()
+    na, ns, nb, d0, dl, ok = (C.c_int(0) for _ in range(6))
+    obj = C.c_double(0.0)
+    _check(lib().dc_dp_select_ext(_ll_table(T, L), _imp4(I, L), _flags(sigma_id, L), L, int(T0), a, C.byref(na), s,
+                                  C.byref(ns), b, C.byref(nb), C.byref(d0), C.byref(dl), C.byref(obj), C.byref(ok)),
+           "dc_dp_select_ext")
+    return ([int(a[i]) for i in range(na.value)], [int(s[i]) for i in range(ns.value)],
+            [int(b[i]) for i in range(nb.value)], d0.value, dl.value, obj.value, bool(ok.value))
 
 
 def pack_weights(w, g: Geom, dtype: int, w_packed, stream=None):
