@@ -2,12 +2,15 @@
 
 Tolerances (rel-L2 = ||a-b||/||b||, b the oracle): merged weights and bias 1e-5 (fp32 FMA merge);
 conv outputs 1e-4 in fp32 and 2e-2 in bf16 (bf16 rounding of the merged weights, of the input and
-of the output; fp32 accumulation)."""
+of the output; fp32 accumulation).  Every output is also held to the element-wise bound of
+parity_util (a localised fault cannot hide under a whole-tensor norm), and every buffer the library
+writes sits between sentinel bands that must come back untouched."""
 import numpy as np
 import pytest
 
 from oracle import dc_oracle as O
 from paper_2301_12187_b200 import inputs as I
+from parity_util import Guarded, assert_close
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -39,25 +42,34 @@ def new_ws(dc, nbytes=None):
 def run_merge(dc, specs, residuals, packed_dtype=None, algo=0):
     layers = [dc.DeviceLayer(s) for s in specs]
     g, ws_bytes = dc.merge_query(layers, residuals)
-    wm = torch.empty((g.c_out, g.c_in, g.k, g.k), dtype=torch.float32, device="cuda")
-    bm = torch.empty((g.c_out,), dtype=torch.float32, device="cuda")
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    bufs = [Guarded(torch, (g.c_out, g.c_in, g.k, g.k), torch.float32, fill=float("nan")),
+            Guarded(torch, (g.c_out,), torch.float32, fill=float("nan")),
+            Guarded(torch, (ws_bytes,), torch.uint8)]
+    wm, bm, ws = (b.t for b in bufs)
     packed = None
     if packed_dtype is not None:
-        packed = torch.empty(dc.packed_bytes(g, packed_dtype), dtype=torch.uint8, device="cuda")
+        bufs.append(Guarded(torch, (dc.packed_bytes(g, packed_dtype),), torch.uint8))
+        packed = bufs[-1].t
     dc.merge_chain(layers, residuals, wm, bm, packed, packed_dtype if packed_dtype is not None else dc.F32, ws,
                    algo=algo)
     torch.cuda.synchronize()
+    for b, name in zip(bufs, ("merged weights", "merged bias", "merge workspace", "packed weights")):
+        b.check(name)
+    assert not torch.isnan(wm).any() and not torch.isnan(bm).any()
     return g, wm, bm, packed
 
 
 def run_conv(dc, x, g, packed, bias, act, residual=None, algo=0):
     n, h, w, _ = x.shape
     ho, wo = O.out_extent(h, g.k, g.stride, g.pad), O.out_extent(w, g.k, g.stride, g.pad)
-    y = torch.full((n, ho, wo, g.c_out), float("nan"), dtype=x.dtype, device="cuda")
-    ws = new_ws(dc)
+    gy = Guarded(torch, (n, ho, wo, g.c_out), x.dtype, fill=float("nan"))
+    gws = Guarded(torch, (dc.conv_workspace_bytes(),), torch.uint8, fill=0)
+    y, ws = gy.t, gws.t
     dc.conv_forward(x, g, packed, bias, act, residual, y, ws, algo=algo)
     assert dc.workspace_status(ws) == dc.OK
+    gy.check("conv output")
+    gws.check("conv workspace")
+    assert not torch.isnan(y.float()).any(), "an output element was never written"
     return y
 
 
@@ -204,7 +216,7 @@ def test_block_step_edge_cases(dc, case):
     assert O.rel_l2(wm2.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm2.cpu().numpy(), b) <= TOL_W
 
 
-@pytest.mark.parametrize("c,n,h,w", [(64, 2, 28, 28), (128, 2, 14, 14), (256, 1, 14, 14)])
+@pytest.mark.parametrize("c,n,h,w", [(64, 2, 28, 28), (128, 2, 14, 14), (256, 1, 14, 14), (512, 1, 14, 14)])
 def test_vgg_style_dense_merge(dc, c, n, h, w):
     """Two dense 3x3 layers (VGG-style, c -> c -> c) merged into one 5x5 layer: merged weights against
     the formula, and the bf16 forward of the merged layer (tensor-bound for these widths) against the
@@ -219,7 +231,46 @@ def test_vgg_style_dense_merge(dc, c, n, h, w):
     x = I.make_input(32, (n, h, w, c), bf16=True)
     y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bm, dc.ACT_IDENTITY)
     ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, [])
-    assert O.rel_l2(nchw(y), ref) <= TOL_BF16
+    assert_close(nchw(y), ref, TOL_BF16)
+
+
+def width14_chain(name, s=41):
+    """Spans with the channel counts of MobileNetV2 at width 1.4 (Fig. 4: 48, 24, 32, 144, ...)."""
+    mk = I.make_layer
+    if name == "first_block":      # depthwise 48 + projection to 24 (t = 1 block after the 48-channel stem)
+        return [mk(s, 0, 48, 48, 3, 1, 1, depthwise=True), mk(s, 1, 48, 24, 1, 1, 0)], []
+    if name == "block_s2":         # 24 -> 144 -> 32, stride 2
+        return [mk(s, 0, 24, 144, 1, 1, 0), mk(s, 1, 144, 144, 3, 2, 1, depthwise=True), mk(s, 2, 144, 32, 1, 1, 0)], []
+    if name == "block_res_32":     # 32 -> 192 -> 32 with its skip folded
+        return [mk(s, 0, 32, 192, 1, 1, 0), mk(s, 1, 192, 192, 3, 1, 1, depthwise=True), mk(s, 2, 192, 32, 1, 1, 0)], [(0, 2)]
+    if name == "block_res_88":     # 88 -> 528 -> 88 (64 x 1.4 rounded to 8)
+        return [mk(s, 0, 88, 528, 1, 1, 0), mk(s, 1, 528, 528, 3, 1, 1, depthwise=True), mk(s, 2, 528, 88, 1, 1, 0)], [(0, 2)]
+    if name == "cross_block_48":   # two 48-channel blocks merged across their boundary: 5x5, 48 -> 48
+        L = []
+        for b in range(2):
+            L += [mk(s, 3 * b, 48, 288, 1, 1, 0), mk(s, 3 * b + 1, 288, 288, 3, 1, 1, depthwise=True),
+                  mk(s, 3 * b + 2, 288, 48, 1, 1, 0)]
+        return L, [(0, 2), (3, 5)]
+    if name == "project_expand":   # projection of one block and expansion of the next: 144 -> 32 -> 192
+        return [mk(s, 0, 144, 32, 1, 1, 0), mk(s, 1, 32, 192, 1, 1, 0)], []
+    raise KeyError(name)
+
+
+@pytest.mark.parametrize("name,n,h,w", [("first_block", 2, 28, 28), ("block_s2", 2, 28, 28), ("block_res_32", 2, 28, 28),
+                                        ("block_res_88", 2, 14, 14), ("cross_block_48", 2, 14, 14),
+                                        ("project_expand", 1, 14, 14)])
+def test_width_1p4_spans(dc, name, n, h, w):
+    """Merge and bf16 forward of spans at MobileNetV2-1.4 widths, both walks of the merge."""
+    specs, res = width14_chain(name)
+    W, b, k, s, p = O.merge_formula(specs, res)
+    for algo in (dc.MERGE_AUTO, dc.MERGE_STEPS):
+        g, wm, bm, packed = run_merge(dc, specs, res, packed_dtype=dc.BF16, algo=algo)
+        assert (g.k, g.stride, g.pad) == (k, s, p)
+        assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
+    x = I.make_input(42, (n, h, w, specs[0].c_in), bf16=True)
+    y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bm, dc.ACT_RELU6)
+    ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, res, final_act="relu6")
+    assert_close(nchw(y), ref, TOL_BF16, what=name)
 
 
 @pytest.mark.parametrize("stride", [1, 2])
@@ -246,7 +297,7 @@ def test_merged_conv_fp32_equals_sequential_chain(dc, name):
     y = run_conv(dc, dev(x), g, packed, bm, dc.ACT_IDENTITY)
     ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, res)
     assert y.shape[1:3] == ref.shape[2:]
-    assert O.rel_l2(nchw(y), ref) <= TOL_F32
+    assert_close(nchw(y), ref, TOL_F32, bf16=False)
 
 
 def test_config0_tiny_fp32(dc):
@@ -258,7 +309,7 @@ def test_config0_tiny_fp32(dc):
     x = case.x()
     y = run_conv(dc, dev(x), g, packed, bm, dc.ACT_IDENTITY)
     ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), case.layers, case.residuals)
-    assert O.rel_l2(nchw(y), ref) <= TOL_F32
+    assert_close(nchw(y), ref, TOL_F32, bf16=False)
     # the chain with its original per-layer padding agrees inside and differs on the border ring
     orig = O.chain_forward_original(x.transpose(0, 3, 1, 2), case.layers, case.residuals)
     assert O.rel_l2(nchw(y)[:, :, 1:-1, 1:-1], orig[:, :, 1:-1, 1:-1]) <= TOL_F32
@@ -284,7 +335,7 @@ def test_merged_conv_bf16_equals_sequential_chain(dc, name, n, h, w, algo):
         ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), specs, res,
                                         final_act="relu6" if act else None)
         assert not torch.isnan(y.float()).any()
-        assert O.rel_l2(nchw(y), ref) <= TOL_BF16
+        assert_close(nchw(y), ref, TOL_BF16)
 
 
 @pytest.mark.parametrize("algo", ["simt", "auto"])
@@ -310,7 +361,7 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
                  algo=dc.ALGO_SIMT if algo == "simt" else dc.ALGO_AUTO)
     Wf, bfo = O.fold_bn(spec)
     ref = O.relu6(O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p) + r.transpose(0, 3, 1, 2))
-    assert O.rel_l2(nchw(y), ref) <= TOL_BF16
+    assert_close(nchw(y), ref, TOL_BF16)
 
 
 # One case per branch of the forward kernels: the expected kernel is asserted, so a change of the
@@ -367,9 +418,9 @@ def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, 
     lin = O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p)
     # plain, and with skip input + ReLU6
     y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bf, dc.ACT_IDENTITY)
-    assert O.rel_l2(nchw(y), lin) <= TOL_BF16
+    assert_close(nchw(y), lin, TOL_BF16)
     y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bf, dc.ACT_RELU6, residual=dev(r, torch.bfloat16))
-    assert O.rel_l2(nchw(y), O.relu6(lin + r.transpose(0, 3, 1, 2))) <= TOL_BF16
+    assert_close(nchw(y), O.relu6(lin + r.transpose(0, 3, 1, 2)), TOL_BF16)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -388,11 +439,14 @@ def test_dwconv(dc, dtype, c, k, s, p, n, h, w):
     tdt = torch.float32 if dtype == "f32" else torch.bfloat16
     x = I.make_input(9, (n, h, w, c), bf16=(dtype == "bf16"))
     ho, wo = O.out_extent(h, k, s, p), O.out_extent(w, k, s, p)
-    y = torch.empty((n, ho, wo, c), dtype=tdt, device="cuda")
+    gy = Guarded(torch, (n, ho, wo, c), tdt, fill=float("nan"))
+    y = gy.t
     dc.dwconv_forward(dev(x, tdt), k, s, p, packed, bf, dc.ACT_RELU6, y)
+    torch.cuda.synchronize()
+    gy.check("depthwise output")
     Wf, bfo = O.fold_bn(spec)
     ref = O.relu6(O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p, groups=c))
-    assert O.rel_l2(nchw(y), ref) <= (TOL_F32 if dtype == "f32" else TOL_BF16)
+    assert_close(nchw(y), ref, TOL_F32 if dtype == "f32" else TOL_BF16, bf16=(dtype == "bf16"))
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -428,10 +482,14 @@ def test_block_forward(dc, dtype, c_in, c_out, t, s, n, h, w):
     x = I.make_input(11, (n, h, w, c_in), bf16=(dtype == "bf16"))
     ho = O.out_extent(h, 3, s, 1)
     wo = O.out_extent(w, 3, s, 1)
-    y = torch.empty((n, ho, wo, c_out), dtype=tdt, device="cuda")
-    ws = new_ws(dc, dc.block_workspace_bytes(n, h, w, blk, code))
+    gy = Guarded(torch, (n, ho, wo, c_out), tdt, fill=float("nan"))
+    gws = Guarded(torch, (max(dc.block_workspace_bytes(n, h, w, blk, code), dc.conv_workspace_bytes()),), torch.uint8,
+                  fill=0)
+    y, ws = gy.t, gws.t
     dc.block_forward(dev(x, tdt), blk, y, ws)
     assert dc.workspace_status(ws) == dc.OK
+    gy.check("block output")
+    gws.check("block workspace")
     cur = x.transpose(0, 3, 1, 2).astype(np.float64)
     skip = cur
     for spec in specs:
@@ -442,26 +500,30 @@ def test_block_forward(dc, dtype, c_in, c_out, t, s, n, h, w):
     if res:
         cur = cur + skip
     # bf16: three roundings of the intermediate maps on the GPU side -> 3x the single-layer budget
-    assert O.rel_l2(nchw(y), cur) <= (TOL_F32 if dtype == "f32" else 3 * TOL_BF16)
+    if dtype == "f32":
+        assert_close(nchw(y), cur, TOL_F32, bf16=False)
+    else:
+        assert_close(nchw(y), cur, 3 * TOL_BF16, scale=3.0)
 
 
 @pytest.mark.parametrize("idx", [1, 2, 3])
-def test_full_size_configs_on_sampled_images(dc, idx):
-    """The batch-64/128 workloads in the launch configuration the benchmark times; the oracle
-    runs the sequential chain on the first two and the last image."""
+def test_full_size_configs_on_every_image(dc, idx):
+    """The batch-64/128 workloads in the launch configuration the benchmark times, every image
+    against the oracle's sequential chain (each CTA owns a run of tiles somewhere in the batch, so a
+    sample of images would leave most CTAs unchecked)."""
     case = I.chain_case(idx)
     g, wm, bm, packed = run_merge(dc, case.layers, case.residuals, packed_dtype=dc.BF16)
     W, b, k, s, p = O.merge_formula(case.layers, case.residuals)
     assert O.rel_l2(wm.cpu().numpy(), W) <= TOL_W and O.rel_l2(bm.cpu().numpy(), b) <= TOL_W
     x = case.x()
     y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bm, dc.ACT_IDENTITY)
-    assert not torch.isnan(y.float()).any()
-    sel = [0, 1, x.shape[0] - 1]
-    ref = O.chain_forward_reordered(x[sel].transpose(0, 3, 1, 2), case.layers, case.residuals)
-    assert O.rel_l2(nchw(y[sel]), ref) <= TOL_BF16
-    # every image: the output is finite and has the scale of the sampled ones
-    norms = y.float().pow(2).mean(dim=(1, 2, 3)).sqrt().cpu().numpy()
-    assert np.all(np.isfinite(norms)) and norms.min() > 0.5 * norms[sel].min() and norms.max() < 2 * norms[sel].max()
+    ref = O.chain_forward_reordered(x.transpose(0, 3, 1, 2), case.layers, case.residuals)
+    r, worst, max_abs = assert_close(nchw(y), ref, TOL_BF16, what=case.name)
+    print("%s: rel-L2 %.3e, worst element at %.2f of its bound, max abs error %.3e" % (case.name, r, worst, max_abs))
+    # per image as well: no single image may carry the whole error budget
+    yn = nchw(y)
+    for i in range(x.shape[0]):
+        assert O.rel_l2(yn[i], ref[i]) <= TOL_BF16, (case.name, i)
 
 
 def test_host_entry_point_matches_device_path(dc):
@@ -475,7 +537,7 @@ def test_host_entry_point_matches_device_path(dc):
     dc.chain_forward_host(arr, len(case.layers), case.residuals, xh, dc.ACT_IDENTITY, yh, ws)
     assert dc.workspace_status(ws) == dc.OK
     ref = O.chain_forward_reordered(case.x().transpose(0, 3, 1, 2), case.layers, case.residuals)
-    assert O.rel_l2(yh.float().numpy().transpose(0, 3, 1, 2), ref) <= TOL_BF16
+    assert_close(yh.float().numpy().transpose(0, 3, 1, 2), ref, TOL_BF16)
 
 
 def test_async_host_entry_point_overlaps_streams_and_matches_the_oracle(dc):
@@ -502,7 +564,7 @@ def test_async_host_entry_point_overlaps_streams_and_matches_the_oracle(dc):
         assert dc.workspace_status(arrs[slot][2], streams[slot]) == dc.OK
         case = cases[slot]
         ref = O.chain_forward_reordered(case.x().transpose(0, 3, 1, 2), case.layers, case.residuals)
-        assert O.rel_l2(outs[slot].float().numpy().transpose(0, 3, 1, 2), ref) <= TOL_BF16
+        assert_close(outs[slot].float().numpy().transpose(0, 3, 1, 2), ref, TOL_BF16)
 
 
 def test_empty_and_degenerate_inputs_are_rejected_or_handled(dc):
