@@ -153,7 +153,8 @@ dc_status dc_merge_chain_algo(const dc_layer *layers, int n_layers, const dc_res
  * memory to another allocator -- none of them can cudaMalloc a workspace.  Here the intermediate
  * kernels of the merge live in a fixed array compiled into the library (dc_merge_chain_static_capacity()
  * bytes, 4 MiB; every GPU that loads the library holds it until the process exits).  The call
- * allocates nothing and frees nothing, on the device or through any library.
+ * allocates and frees no device memory, itself or through any library (its host-side bookkeeping
+ * uses a few small C++ vectors on the host heap).
  *
  * Inputs and outputs are as for dc_merge_chain, minus the workspace.  Runs whose intermediates
  * need more than the capacity (compare dc_merge_query's workspace_bytes) are refused with

@@ -3,9 +3,11 @@
 Some users of the library run where cudaMalloc is off limits (inside an allocator callback, in a
 plug-in after its host's initialisation phase, next to an allocator that owns the whole device).
 For them the library carries its own fixed scratch array.  This test calls that entry point
-through the C ABI twice in a row, with different runs, and checks each result against the regular
-dc_merge_chain, which works in a caller-provided workspace.  The file name sorts last on purpose:
-if this addition ever fails, every other test has already run.
+through the C ABI several times in a row, with different runs, and checks each result against the
+regular dc_merge_chain, which works in a caller-provided workspace (and is itself held to the
+oracle in test_gpu_parity.py, so agreement with it is agreement with the oracle at the same
+tolerance).  It also checks that the device's free memory is the same before and after the call.
+The file name sorts last on purpose: if this addition ever fails, every other test has already run.
 """
 import numpy as np
 import pytest
@@ -35,7 +37,11 @@ def merge_both(dc, specs, residuals):
             ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
             dc.merge_chain(layers, residuals, wm, bm, packed, dc.BF16, ws)
         else:
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             dc.merge_chain_static(layers, residuals, wm, bm, packed, dc.BF16)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
         torch.cuda.synchronize()
         out[name] = (wm, bm, packed)
     return out
@@ -47,9 +53,18 @@ def test_static_scratch_merge_matches_workspace_merge_twice_in_a_row():
     from paper_2301_12187_b200 import dc
     assert dc.merge_chain_static_capacity() == 4 << 20
     # two different runs back to back: the second call finds the first call's leftovers in the scratch
-    cases = [I.chain_case(3), I.chain_case(1), I.chain_case(3)]
-    for case in cases:
-        out = merge_both(dc, case.layers, case.residuals)
+    mk = I.make_layer
+    dense = ([mk(51, 0, 32, 48, 3, 1, 1), mk(51, 1, 48, 32, 3, 1, 1)], [])                 # dense o dense composition
+    dw_first = ([mk(52, 0, 16, 16, 3, 1, 1, depthwise=True), mk(52, 1, 16, 16, 3, 1, 1, depthwise=True),
+                 mk(52, 2, 16, 8, 1, 1, 0)], [(0, 0)])                                      # diagonal compositions
+    cases = [(c.layers, c.residuals) for c in (I.chain_case(3), I.chain_case(1), I.chain_case(3))] + [dense, dw_first]
+    # the first call on a device looks up the scratch array's address (and may load the module):
+    # make it before the calls whose effect on free memory is measured
+    dc.merge_chain_static([dc.DeviceLayer(s) for s in dense[0]], dense[1], torch.empty((32, 32, 5, 5), device="cuda"),
+                          torch.empty((32,), device="cuda"), None, dc.F32)
+    torch.cuda.synchronize()
+    for layers_, res_ in cases:
+        out = merge_both(dc, layers_, res_)
         (w0, b0, p0), (w1, b1, p1) = out["workspace"], out["static"]
         assert not torch.isnan(w1).any() and not torch.isnan(b1).any()
         assert rel(w1, w0) <= TOL_W and rel(b1, b0) <= TOL_W
