@@ -241,6 +241,27 @@ dc_status dc_block_forward(const void *x, int n, int h, int w, const dc_block *b
  */
 dc_status dc_workspace_status(void *workspace, dc_stream stream);
 
+/*
+ * As dc_workspace_status; also returns, when not NULL, the code of the wait that gave up (`where`:
+ * role in the upper bits, barrier index in the lower; 0 when nothing timed out) and the header's
+ * first detail word.
+ */
+dc_status dc_workspace_status_where(void *workspace, dc_stream stream, unsigned int *where,
+                                    unsigned int *detail);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper): enqueues a one-CTA kernel whose two
+ * roles wait, with the library's own wait routines, on a barrier that nothing completes.  After
+ * limit_us microseconds (1..100000) the waits give up, DC_ERR_TIMEOUT and the site code 0x90000 are
+ * latched in the workspace header, the second role leaves through the abort flag, and the kernel
+ * returns normally; the detail word then holds the number of roles that left their wait (2).  No
+ * copy or tensor-core work is in flight and nothing faults: the context stays usable, and the same
+ * workspace serves ordinary launches again once dc_workspace_status has cleared it.
+ * workspace: device, >= 256 bytes, 16-byte aligned.
+ */
+dc_status dc_selftest_bounded_wait(void *workspace, size_t workspace_bytes, unsigned int limit_us,
+                                   dc_stream stream);
+
 /* Host only: bytes of device workspace dc_chain_forward_host needs. */
 dc_status dc_chain_host_workspace_bytes(const dc_layer *layers, int n_layers, const dc_residual *res,
                                         int n_res, int n, int h, int w, dc_dtype dtype,

@@ -76,16 +76,23 @@ extern "C" dc_status dc_conv_forward(const void *x, int n, int h, int w, const d
                               stream, DC_ALGO_AUTO);
 }
 
-extern "C" dc_status dc_workspace_status(void *workspace, dc_stream stream) {
+extern "C" dc_status dc_workspace_status_where(void *workspace, dc_stream stream, unsigned int *where,
+                                               unsigned int *detail) {
   if (!workspace) return DC_ERR_WORKSPACE;
   DC_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
-  unsigned int st = 0;
-  DC_CUDA_OK(cudaMemcpy(&st, workspace, sizeof(st), cudaMemcpyDeviceToHost));
-  if (st != 0) {
+  unsigned int head[3] = {0, 0, 0};                    // status, site of the wait, first detail word
+  DC_CUDA_OK(cudaMemcpy(head, workspace, sizeof(head), cudaMemcpyDeviceToHost));
+  if (where) *where = head[1];
+  if (detail) *detail = head[2];
+  if (head[0] != 0) {
     DC_CUDA_OK(cudaMemset(workspace, 0, sizeof(DcWsHeader)));
     return DC_ERR_TIMEOUT;
   }
   return DC_OK;
+}
+
+extern "C" dc_status dc_workspace_status(void *workspace, dc_stream stream) {
+  return dc_workspace_status_where(workspace, stream, nullptr, nullptr);
 }
 
 // ----------------------------------------------------------------------------------------------

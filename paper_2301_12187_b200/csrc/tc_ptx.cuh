@@ -59,7 +59,8 @@ __device__ __forceinline__ uint32_t mbar_test(uint64_t *bar, uint32_t parity) {
 // Slow path of the bounded wait: parks the warp in hardware between probes.  Not inlined: the
 // tensor-core kernels are sensitive to their instruction footprint and every wait site shares it.
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                                   DcWsHeader *ws, uint32_t site) {
+                                                   DcWsHeader *ws, uint32_t site,
+                                                   unsigned long long limit_ns = kWaitLimitNs) {
   const unsigned long long t0 = globaltimer_ns();
   for (;;) {
     // a waiting warp shares its scheduler with working ones: the inner loop is probe + branch only,
@@ -68,7 +69,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parit
     for (int i = 0; i < 64; ++i)
       if (mbar_try(bar, parity, 20000u)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       atomicExch(&ws->status, (unsigned int)DC_ERR_TIMEOUT);
       ws->where = site;
@@ -79,16 +80,16 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parit
 
 // Bounded wait.  Returns false when the wait ran out (or another role already gave up).
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          DcWsHeader *ws, uint32_t site) {
+                                          DcWsHeader *ws, uint32_t site, unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_test(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, ws, site);
+  return mbar_wait_slow(bar, parity, abort_flag, ws, site, limit_ns);
 }
 
 // Every lane of a converged warp waits (so each has observed the phase itself); the warp then
 // agrees on the outcome and stays converged.
 __device__ __forceinline__ bool warp_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          DcWsHeader *ws, uint32_t site) {
-  const bool ok = mbar_wait(bar, parity, abort_flag, ws, site);
+                                          DcWsHeader *ws, uint32_t site, unsigned long long limit_ns = kWaitLimitNs) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, ws, site, limit_ns);
   return __all_sync(0xffffffffu, ok) != 0;
 }
 // true in exactly one lane of a converged warp

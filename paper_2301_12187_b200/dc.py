@@ -94,6 +94,8 @@ EXPORTS = {
     "dc_block_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Block), C.c_void_p,
                                    C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
     "dc_workspace_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "dc_workspace_status_where": (C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint), C.POINTER(C.c_uint)]),
+    "dc_selftest_bounded_wait": (C.c_int, [C.c_void_p, C.c_size_t, C.c_uint, C.c_void_p]),
     "dc_chain_host_workspace_bytes": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int,
                                                 C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]),
     "dc_chain_forward_host": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
@@ -407,6 +409,18 @@ def block_forward(x, blk: Block, y, workspace, stream=None):
 
 def workspace_status(workspace, stream=None) -> int:
     return int(lib().dc_workspace_status(_ptr(workspace), _stream(stream)))
+
+
+def workspace_status_where(workspace, stream=None) -> Tuple[int, int, int]:
+    """(status, code of the wait that gave up, first detail word); clears the header like workspace_status."""
+    where, detail = C.c_uint(0), C.c_uint(0)
+    st = int(lib().dc_workspace_status_where(_ptr(workspace), _stream(stream), C.byref(where), C.byref(detail)))
+    return st, int(where.value), int(detail.value)
+
+
+def selftest_bounded_wait(workspace, limit_us: int, stream=None):
+    _check(lib().dc_selftest_bounded_wait(_ptr(workspace), workspace.numel() * workspace.element_size(), int(limit_us),
+                                          _stream(stream)), "dc_selftest_bounded_wait")
 
 
 def host_layer_array(specs, pinned: bool = False) -> Tuple["C.Array", list]:
