@@ -262,6 +262,16 @@ dc_status dc_workspace_status_where(void *workspace, dc_stream stream, unsigned 
 dc_status dc_selftest_bounded_wait(void *workspace, size_t workspace_bytes, unsigned int limit_us,
                                    dc_stream stream);
 
+/*
+ * Host only: the layout in which dc_chain_forward_host keeps a run's parameters on the device:
+ * offsets[6 * i + j] is the byte offset of array j of layer i (j = 0 weight, 1 bias, 2 bn_gamma,
+ * 3 bn_beta, 4 bn_mean, 5 bn_var; each rounded up to 256 bytes), total the size of the block.
+ * A caller whose HOST arrays lie in one (pinned) block in exactly this layout, starting with layer
+ * 0's weights, gets them copied with a single transfer instead of one per array; absent arrays
+ * (NULL) keep their slot.  offsets may be NULL.  Only the layers' shapes are read.
+ */
+dc_status dc_chain_host_param_layout(const dc_layer *layers, int n_layers, size_t *offsets, size_t *total);
+
 /* Host only: bytes of device workspace dc_chain_forward_host needs. */
 dc_status dc_chain_host_workspace_bytes(const dc_layer *layers, int n_layers, const dc_residual *res,
                                         int n_res, int n, int h, int w, dc_dtype dtype,

@@ -207,6 +207,21 @@ extern "C" dc_status dc_chain_host_workspace_bytes(const dc_layer *layers, int n
   return DC_OK;
 }
 
+extern "C" dc_status dc_chain_host_param_layout(const dc_layer *layers, int n_layers, size_t *offsets, size_t *total) {
+  if (!layers || n_layers <= 0 || !total) return DC_ERR_INVALID_ARG;
+  size_t o = 0;
+  for (int i = 0; i < n_layers; ++i) {
+    const dc_layer &L = layers[i];
+    if (L.c_in <= 0 || L.c_out <= 0 || L.groups <= 0 || L.k <= 0 || L.c_in % L.groups) return DC_ERR_INVALID_ARG;
+    for (int j = 0; j < 6; ++j) {
+      if (offsets) offsets[6 * i + j] = o;
+      o += dc_round_up(j == 0 ? layer_weight_elems(L) * 4 : (size_t)L.c_out * 4, 256);
+    }
+  }
+  *total = o;
+  return DC_OK;
+}
+
 extern "C" dc_status dc_chain_forward_host_async(const dc_layer *layers, int n_layers, const dc_residual *res,
                                                  int n_res, const void *x_host, int n, int h, int w, dc_act act,
                                                  void *y_host, dc_dtype dtype, void *workspace,
@@ -222,18 +237,47 @@ extern "C" dc_status dc_chain_forward_host_async(const dc_layer *layers, int n_l
   size_t off = sizeof(DcWsHeader);
   auto take = [&](size_t bytes) { char *p = base + off; off += dc_round_up(bytes, 256); return p; };
   std::vector<dc_layer> dev(layers, layers + n_layers);
+  // Device layout of the parameters: per layer the weights and the five vectors, each rounded up to
+  // 256 bytes (dc_chain_host_param_layout).  When the caller's host arrays already lie in one block
+  // in that layout, one copy moves them all; otherwise one copy per array.
+  char *params_dev = base + off;
+  const char *host_base = (const char *)layers[0].weight;
+  bool one_block = host_base != nullptr;
+  size_t last_end = 0;
+  {
+    size_t o = 0;
+    for (int i = 0; i < n_layers && one_block; ++i) {
+      const dc_layer &L = layers[i];
+      const size_t wb = layer_weight_elems(L) * 4, cb = (size_t)L.c_out * 4;
+      const float *src[6] = {L.weight, L.bias, L.bn_gamma, L.bn_beta, L.bn_mean, L.bn_var};
+      for (int j = 0; j < 6; ++j) {
+        const size_t bytes = j == 0 ? wb : cb;
+        if (src[j]) {
+          if ((const char *)src[j] != host_base + o) { one_block = false; break; }
+          last_end = o + bytes;
+        }
+        o += dc_round_up(bytes, 256);
+      }
+    }
+  }
+  if (one_block) DC_CUDA_OK(cudaMemcpyAsync(params_dev, host_base, last_end, cudaMemcpyHostToDevice, st));
   for (int i = 0; i < n_layers; ++i) {
     const dc_layer &L = layers[i];
     size_t wb = layer_weight_elems(L) * 4, cb = (size_t)L.c_out * 4;
     float *dw = (float *)take(wb);
-    DC_CUDA_OK(cudaMemcpyAsync(dw, L.weight, wb, cudaMemcpyHostToDevice, st));
+    if (!L.weight) return DC_ERR_INVALID_ARG;
+    if (!one_block) DC_CUDA_OK(cudaMemcpyAsync(dw, L.weight, wb, cudaMemcpyHostToDevice, st));
     dev[i].weight = dw;
     const float *src[5] = {L.bias, L.bn_gamma, L.bn_beta, L.bn_mean, L.bn_var};
     const float **dst[5] = {&dev[i].bias, &dev[i].bn_gamma, &dev[i].bn_beta, &dev[i].bn_mean, &dev[i].bn_var};
     for (int j = 0; j < 5; ++j) {
       float *d = (float *)take(cb);
-      if (src[j]) { DC_CUDA_OK(cudaMemcpyAsync(d, src[j], cb, cudaMemcpyHostToDevice, st)); *dst[j] = d; }
-      else *dst[j] = nullptr;
+      if (src[j]) {
+        if (!one_block) DC_CUDA_OK(cudaMemcpyAsync(d, src[j], cb, cudaMemcpyHostToDevice, st));
+        *dst[j] = d;
+      } else {
+        *dst[j] = nullptr;
+      }
     }
   }
   char *merge_ws = take(hp.merge_ws);

@@ -19,6 +19,37 @@ static inline size_t dc_round_up(size_t v, size_t a) { return (v + a - 1) / a * 
 static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
 static inline int dc_floor_div2(int a) { return (a >= 0) ? a / 2 : -((-a + 1) / 2); }
 
+// Per-device host state.  SM counts and function attributes belong to a device, not to the process:
+// both are kept per device ordinal (a process may drive several GPUs through the library).  The
+// cached operations are idempotent, so two threads racing on a first use do no harm.
+constexpr int kDcMaxDevices = 64;
+static inline int dc_current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kDcMaxDevices) return -1;
+  return dev;
+}
+// SM count of the current device (148 when no device can be queried, e.g. host-only planning calls)
+static inline int dc_sm_count() {
+  static int cached[kDcMaxDevices];
+  const int dev = dc_current_device();
+  if (dev < 0) { (void)cudaGetLastError(); return 148; }
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+// Raises a kernel's dynamic shared-memory limit once per device (`done` is the call site's own table).
+template <typename K>
+static inline cudaError_t dc_set_max_smem_once(K kernel, int bytes, unsigned char (&done)[kDcMaxDevices]) {
+  const int dev = dc_current_device();
+  if (dev >= 0 && done[dev]) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && dev >= 0) done[dev] = 1;
+  return e;
+}
+
 static inline int dc_out_extent(int h, int k, int s, int p) {
   int a = h + 2 * p - k;
   return a < 0 ? 0 : a / s + 1;

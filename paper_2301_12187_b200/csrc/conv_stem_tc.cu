@@ -295,18 +295,15 @@ dc_status dc_launch_conv_stem(const void *x, int n, int h, int w, const dc_geom 
   StemParams p;
   if (!stem_plan(n, h, w, g, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
-  static bool attr_set = false;
-  if (!attr_set) {
-    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_stem_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
-    attr_set = true;
-  }
+  static unsigned char attr_done[kDcMaxDevices];
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_stem_tc, 100 * 1024, attr_done));
   // several small CTAs per SM: bounded by shared memory and by 512 tensor-memory columns per SM
   int per_sm = 200 * 1024 / (p.smem_bytes + 2048);
   if (per_sm > 512 / p.tmem_cols) per_sm = 512 / p.tmem_cols;
   if (per_sm > 8) per_sm = 8;
   if (per_sm < 1) per_sm = 1;
   const long long tiles = (long long)n * p.ho * p.xtiles;
-  const long long cap = 148ll * per_sm;
+  const long long cap = (long long)dc_sm_count() * per_sm;
   const int grid = (int)(tiles < cap ? tiles : cap);
   k_conv_stem_tc<<<grid, kStemThreads, p.smem_bytes, stream>>>(p, (const __nv_bfloat16 *)x, w_packed, bias,
                                                               (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,

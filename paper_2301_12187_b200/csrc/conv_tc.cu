@@ -368,16 +368,6 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
 }
 
 // ------------------------------------------------------------------------------------------ host
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 constexpr int kSmemBudget = 200 * 1024;
 
 // plane stride in 16-byte units is made congruent to `want` mod 8 so that the cg chunks of one
@@ -520,21 +510,18 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
 
 bool dc_conv_tc_supported(int n, int h, int w, const dc_geom *g) {
   TcParams p;
-  return tc_plan(n, h, w, g, 148, &p);
+  return tc_plan(n, h, w, g, dc_sm_count(), &p);
 }
 
 dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                             const float *bias, dc_act act, const void *residual, void *y, void *workspace,
                             cudaStream_t stream) {
   TcParams p;
-  const int n_sm = sm_count();
+  const int n_sm = dc_sm_count();
   if (!tc_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
-  static bool attr_set = false;
-  if (!attr_set) {
-    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    attr_set = true;
-  }
+  static unsigned char attr_done[kDcMaxDevices];
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc, kSmemBudget, attr_done));
   int grid = p.total_units < n_sm ? p.total_units : n_sm;
   k_conv_tc<<<grid, kThreads, p.smem_bytes, stream>>>(w_packed, p, (const __nv_bfloat16 *)x, bias,
                                                      (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,

@@ -515,16 +515,6 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
 }
 
 // ------------------------------------------------------------------------------------------ host
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 constexpr int kSmemBudget = 220 * 1024;
 constexpr int kStageLimit = 40 * 1024;
 
@@ -659,21 +649,18 @@ bool fold_plan(int n, int h, int w, const dc_geom *g, int n_sm, FoldParams *p) {
 
 bool dc_conv_fold_supported(int n, int h, int w, const dc_geom *g) {
   FoldParams p;
-  return fold_plan(n, h, w, g, 148, &p);
+  return fold_plan(n, h, w, g, dc_sm_count(), &p);
 }
 
 dc_status dc_launch_conv_fold(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                               const float *bias, dc_act act, const void *residual, void *y, void *workspace,
                               cudaStream_t stream) {
   FoldParams p;
-  const int n_sm = sm_count();
+  const int n_sm = dc_sm_count();
   if (!fold_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
-  static bool attr_set = false;
-  if (!attr_set) {
-    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_fold, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    attr_set = true;
-  }
+  static unsigned char attr_done[kDcMaxDevices];
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_fold, kSmemBudget, attr_done));
   k_conv_tc_fold<<<p.grid, kThreads, p.smem_bytes, stream>>>(p, (const __nv_bfloat16 *)x, w_packed, bias,
                                                           (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                                           (DcWsHeader *)workspace);

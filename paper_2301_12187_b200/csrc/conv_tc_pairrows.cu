@@ -513,16 +513,6 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 constexpr int kSmemBudget = 220 * 1024;
 constexpr int kStageLimit = 48 * 1024;
 constexpr int kSlack = 17 * 1024;   // a block's 128 rows may reach this far past the last stage
@@ -643,14 +633,14 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
 
 bool dc_conv_pairrows_supported(int n, int h, int w, const dc_geom *g) {
   PairParams p;
-  return pair_plan(n, h, w, g, 148, &p);
+  return pair_plan(n, h, w, g, dc_sm_count(), &p);
 }
 
 dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                                   const float *bias, dc_act act, const void *residual, void *y, void *workspace,
                                   cudaStream_t stream) {
   PairParams p;
-  const int n_sm = sm_count();
+  const int n_sm = dc_sm_count();
   if (!pair_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
   EncodeTiledFn encode = get_encode_fn();
@@ -669,11 +659,8 @@ dc_status dc_launch_conv_pairrows(const void *x, int n, int h, int w, const dc_g
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_pairrows, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    attr_set = true;
-  }
+  static unsigned char attr_done[kDcMaxDevices];
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_pairrows, kSmemBudget, attr_done));
   cudaError_t le = dc_launch_pdl(k_conv_tc_pairrows, dim3(p.grid), dim3(kThreads), (size_t)p.smem_bytes, stream, map_a, p,
                                  w_packed, bias, (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                  (DcWsHeader *)workspace);

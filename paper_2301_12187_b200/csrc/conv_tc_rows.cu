@@ -349,16 +349,6 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 constexpr int kSmemBudget = 220 * 1024;
 constexpr int kMaxLines = 128 * kMaxBlocks;      // GEMM rows of a tile
 constexpr int kSlack = 1024;
@@ -438,14 +428,14 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
 
 bool dc_conv_rows_supported(int n, int h, int w, const dc_geom *g) {
   RowsParams p;
-  return rows_plan(n, h, w, g, 148, &p);
+  return rows_plan(n, h, w, g, dc_sm_count(), &p);
 }
 
 dc_status dc_launch_conv_rows(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
                               const float *bias, dc_act act, const void *residual, void *y, void *workspace,
                               cudaStream_t stream) {
   RowsParams p;
-  const int n_sm = sm_count();
+  const int n_sm = dc_sm_count();
   if (!rows_plan(n, h, w, g, n_sm, &p)) return DC_ERR_UNSUPPORTED;
   p.act = (int)act;
   EncodeTiledFn encode = get_encode_fn();
@@ -462,11 +452,8 @@ dc_status dc_launch_conv_rows(const void *x, int n, int h, int w, const dc_geom 
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    DC_CUDA_OK(cudaFuncSetAttribute(k_conv_tc_rows, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    attr_set = true;
-  }
+  static unsigned char attr_done[kDcMaxDevices];
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_rows, kSmemBudget, attr_done));
   k_conv_tc_rows<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_a, p, w_packed, bias, (const __nv_bfloat16 *)residual,
                                                             (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;

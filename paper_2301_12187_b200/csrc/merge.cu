@@ -763,15 +763,11 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
       const int R = first.c_out * second.k * second.k;
       // few tiles: one deep slice per round trip; many tiles (more than two per SM): shallow slices,
       // so that several CTAs share an SM and one's loads overlap another's arithmetic
-      const int slice_max = gx * gy > 2 * 148 ? 64 : kDdSlice;
+      const int slice_max = gx * gy > 2 * dc_sm_count() ? 64 : kDdSlice;
       const int slice = R < slice_max ? (int)dc_round_up((size_t)R, 16) : slice_max;
       const size_t smem = (size_t)2 * slice * kDdPitch * sizeof(float);
-      static bool attr_set = false;
-      if (!attr_set) {
-        cudaFuncSetAttribute(k_compose_dense_dense, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             2 * kDdSlice * kDdPitch * (int)sizeof(float));
-        attr_set = true;
-      }
+      static unsigned char attr_done[kDcMaxDevices];
+      dc_set_max_smem_once(k_compose_dense_dense, 2 * kDdSlice * kDdPitch * (int)sizeof(float), attr_done);
       k_compose_dense_dense<<<gx * gy + nbias, 256, smem, st>>>(first, second, w, b, out.k, gx, gy, slice);
     } else {
       const int nb = blocks_for(elems, 256);
@@ -872,11 +868,8 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
   size_t batch_smem = 0;
   auto flush_blocks = [&]() {
     if (n_batch == 0) return;
-    static bool attr_set = false;
-    if (!attr_set) {
-      cudaFuncSetAttribute(k_merge_block, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-      attr_set = true;
-    }
+    static unsigned char attr_done[kDcMaxDevices];
+    dc_set_max_smem_once(k_merge_block, 200 * 1024, attr_done);
     k_merge_block<<<dim3(batch_grid, n_batch), kBlockThreads, batch_smem, st>>>(batch);
     n_batch = 0; batch_grid = 0; batch_smem = 0;
   };

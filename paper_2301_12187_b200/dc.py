@@ -96,6 +96,7 @@ EXPORTS = {
     "dc_workspace_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "dc_workspace_status_where": (C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint), C.POINTER(C.c_uint)]),
     "dc_selftest_bounded_wait": (C.c_int, [C.c_void_p, C.c_size_t, C.c_uint, C.c_void_p]),
+    "dc_chain_host_param_layout": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "dc_chain_host_workspace_bytes": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int,
                                                 C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_size_t)]),
     "dc_chain_forward_host": (C.c_int, [C.POINTER(Layer), C.c_int, C.POINTER(Residual), C.c_int, C.c_void_p,
@@ -425,28 +426,40 @@ def selftest_bounded_wait(workspace, limit_us: int, stream=None):
 
 def host_layer_array(specs, pinned: bool = False) -> Tuple["C.Array", list]:
     """dc_layer array whose pointers are HOST pointers (float32), for chain_forward_host.  With
-    pinned=True the arrays live in page-locked memory, so their copies to the device are queued
-    instead of being staged by the calling thread."""
+    pinned=True all arrays live in ONE page-locked block laid out as dc_chain_host_param_layout says,
+    so their copy to the device is a single queued transfer instead of one staged copy per array."""
     import numpy as np
     keep = []
     arr = (Layer * len(specs))()
+    for i, s in enumerate(specs):
+        arr[i] = Layer(s.c_in, s.c_out, s.groups, s.k, s.stride, s.pad, None, None, None, None, None, None,
+                       float(s.eps))
+    block = None
+    offs = (C.c_size_t * (6 * len(specs)))()
+    if pinned:
+        import torch
+        total = C.c_size_t(0)
+        _check(lib().dc_chain_host_param_layout(arr, len(specs), offs, C.byref(total)), "dc_chain_host_param_layout")
+        block = torch.zeros(int(total.value), dtype=torch.uint8).pin_memory()
+        keep.append(block)
 
-    def hp(a):
+    def hp(a, off):
         if a is None:
             return None
         a = np.ascontiguousarray(a, dtype=np.float32)
-        if pinned:
+        if block is not None:
             import torch
-            t = torch.from_numpy(a.copy()).pin_memory()
-            keep.append(t)
-            return t.data_ptr()
+            view = block[off:off + a.nbytes].view(torch.float32)
+            view.copy_(torch.from_numpy(a.reshape(-1)))
+            return block.data_ptr() + off
         keep.append(a)
         return a.ctypes.data
 
     for i, s in enumerate(specs):
         bn = s.bn or (None, None, None, None)
-        arr[i] = Layer(s.c_in, s.c_out, s.groups, s.k, s.stride, s.pad, hp(s.weight), hp(s.bias),
-                       hp(bn[0]), hp(bn[1]), hp(bn[2]), hp(bn[3]), float(s.eps))
+        arrays = (s.weight, s.bias, bn[0], bn[1], bn[2], bn[3])
+        ptrs = [hp(a, int(offs[6 * i + j])) for j, a in enumerate(arrays)]
+        arr[i].weight, arr[i].bias, arr[i].bn_gamma, arr[i].bn_beta, arr[i].bn_mean, arr[i].bn_var = ptrs
     return arr, keep
 
 

@@ -139,3 +139,22 @@ def test_host_entry_reports_its_workspace():
     arr = dc.layer_array([L(24, 144), L(144, 144, 3, 1, 1, dw=True), L(144, 24)])
     n = dc.chain_host_workspace_bytes(arr, 3, [(0, 2)], 4, 16, 16, dc.BF16)
     assert n > 2 * 4 * 16 * 16 * 24 * 2
+
+
+def test_host_parameter_layout_offsets():
+    """dc_chain_host_param_layout: 256-byte-rounded slots, six per layer, in layer order."""
+    import ctypes as C
+    from paper_2301_12187_b200 import dc, inputs as I
+    specs = [I.make_layer(0, 0, 24, 144, 1, 1, 0), I.make_layer(0, 1, 144, 144, 3, 1, 1, depthwise=True)]
+    arr, keep = dc.host_layer_array(specs)
+    offs = (C.c_size_t * 12)()
+    total = C.c_size_t(0)
+    assert dc.lib().dc_chain_host_param_layout(arr, 2, offs, C.byref(total)) == dc.OK
+    r = lambda b: (b + 255) // 256 * 256
+    want, o = [], 0
+    for s in specs:
+        for j in range(6):
+            want.append(o)
+            o += r(s.weight.size * 4 if j == 0 else s.c_out * 4)
+    assert list(offs) == want and total.value == o
+    assert dc.lib().dc_chain_host_param_layout(arr, 0, offs, C.byref(total)) == dc.ERR_INVALID_ARG

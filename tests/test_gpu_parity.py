@@ -545,7 +545,8 @@ def test_async_host_entry_point_overlaps_streams_and_matches_the_oracle(dc):
     arrs, outs, streams, cases = [], [], [], []
     for slot in range(3):
         case = I.chain_case(1, seed=20 + slot, batch=3)
-        arr, keep = dc.host_layer_array(case.layers)
+        # slots 0 and 1: one pinned parameter block in the library's layout (a single transfer); slot 2: loose arrays
+        arr, keep = dc.host_layer_array(case.layers, pinned=(slot < 2))
         n, h, w, c = case.x_shape
         nbytes = dc.chain_host_workspace_bytes(arr, len(case.layers), case.residuals, n, h, w, dc.BF16)
         ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
