@@ -175,36 +175,44 @@ class CompressedNetwork:
             dc.merge_chain(devs, res, wm, bm, packed, dc.BF16, ws)
         return len(self._merge_jobs)
 
+    def launch(self, i, cur, x):
+        """Launch group i on `cur` (the previous group's map); x is the network input (skip source -1)."""
+        op = self.ops[i]
+        if op.kind == "block":
+            dc.block_forward(cur, op.block, op.y, op.ws)
+        elif op.kind == "dw":
+            g = op.geom
+            dc.dwconv_forward(cur, g.k, g.stride, g.pad, op.packed, op.bias, op.act, op.y)
+        else:
+            res = None
+            if op.add_from == -1:
+                res = x
+            elif op.add_from >= 0:
+                res = self.ops[op.add_from].y
+            dc.conv_forward(cur, op.geom, op.packed, op.bias, op.act, res, op.y, self.conv_ws)
+        return op.y
+
     def forward(self, x):
         """Run the compressed network on x (NHWC bf16, batch == self.batch); returns the last map."""
         cur = x
-        for op in self.ops:
-            if op.kind == "block":
-                dc.block_forward(cur, op.block, op.y, op.ws)
-            elif op.kind == "dw":
-                g = op.geom
-                dc.dwconv_forward(cur, g.k, g.stride, g.pad, op.packed, op.bias, op.act, op.y)
-            else:
-                res = None
-                if op.add_from == -1:
-                    res = x
-                elif op.add_from >= 0:
-                    res = self.ops[op.add_from].y
-                dc.conv_forward(cur, op.geom, op.packed, op.bias, op.act, res, op.y, self.conv_ws)
-            cur = op.y
+        for i in range(len(self.ops)):
+            cur = self.launch(i, cur, x)
         return cur
 
-    def capture(self, x):
-        """Capture forward(x) into a CUDA graph on a side stream; replay with .replay()."""
+    def capture(self, x, keep_graph: bool = False):
+        """Capture forward(x) into a CUDA graph on a side stream; replay with .replay().  keep_graph
+        keeps the captured graph inspectable (node counts) beside its executable form."""
         torch = self.torch
         stream = torch.cuda.Stream()
         stream.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(stream):
             self.forward(x)
             stream.synchronize()
-            self.graph = torch.cuda.CUDAGraph()
+            self.graph = torch.cuda.CUDAGraph(keep_graph=keep_graph)
             with torch.cuda.graph(self.graph, stream=stream):
                 self.forward(x)
+            if keep_graph:
+                self.graph.instantiate()
         torch.cuda.current_stream().wait_stream(stream)
         return self.graph
 
@@ -215,3 +223,40 @@ class CompressedNetwork:
             if op.kind == "block":
                 st = max(st, dc.workspace_status(op.ws))
         return st
+
+
+class HostRunner:
+    """The captured network fed from pinned host buffers: a step copies its input to the device, replays
+    the forward graph and copies the last map back.  Two device input buffers and a copy stream let
+    the input copy of step i+1 run under the forward of step i; the forwards themselves are serial
+    (they share the intermediate maps)."""
+
+    def __init__(self, cn: CompressedNetwork):
+        torch = cn.torch
+        self.cn, self.torch = cn, torch
+        self.copy_stream, self.compute_stream = torch.cuda.Stream(), torch.cuda.Stream()
+        self.x = [torch.zeros(cn.in_shape, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+        self.graphs = [cn.capture(x) for x in self.x]
+        self.in_ready = [torch.cuda.Event() for _ in range(2)]
+        self.in_free = [torch.cuda.Event() for _ in range(2)]
+        self.count = 0
+
+    def submit(self, x_host, y_host):
+        """Queue one step; y_host is valid once compute_stream has been synchronised."""
+        torch = self.torch
+        b = self.count & 1
+        with torch.cuda.stream(self.copy_stream):
+            if self.count >= 2:
+                self.copy_stream.wait_event(self.in_free[b])
+            self.x[b].copy_(x_host, non_blocking=True)
+            self.in_ready[b].record(self.copy_stream)
+        with torch.cuda.stream(self.compute_stream):
+            self.compute_stream.wait_event(self.in_ready[b])
+            self.graphs[b].replay()
+            self.in_free[b].record(self.compute_stream)
+            y_host.copy_(self.cn.ops[-1].y, non_blocking=True)
+        self.count += 1
+
+    def synchronize(self):
+        self.copy_stream.synchronize()
+        self.compute_stream.synchronize()
