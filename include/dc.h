@@ -222,6 +222,13 @@ dc_status dc_dwconv_forward(const void *x, int n, int h, int w, int c, int k, in
                             const float *w_packed, const float *bias, dc_act act, void *y,
                             dc_dtype dtype, dc_stream stream);
 
+/*
+ * Synchronises `stream`, then returns DC_ERR_TIMEOUT if the bounded wait of a depthwise launch
+ * (which takes no workspace to latch it in) ran out on the current device since the last call,
+ * DC_OK otherwise; clears the flag.
+ */
+dc_status dc_dwconv_status(dc_stream stream);
+
 /* Host only: workspace bytes dc_block_forward needs for this input size. */
 dc_status dc_block_workspace_bytes(int n, int h, int w, const dc_block *blk, dc_dtype dtype,
                                    size_t *bytes);

@@ -179,7 +179,8 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
     ko->rows = 1;
     // output channels per pass: at most 128, fewer for 5x5 and 7x7 kernels, whose weight stage of one
     // (plane, tap row) step (k * 8 chunk planes of n_tile rows) must fit the shared-memory ring twice
-    const int n_tile_max = g->k <= 4 ? 128 : (g->k <= 5 ? 112 : 80);
+    // beside two activation stages and the epilogue's turn-around buffers
+    const int n_tile_max = g->k <= 4 ? 128 : (g->k <= 5 ? 96 : 64);
     ko->nnt = dc_div_up(n16, n_tile_max);
     ko->n_tile = (int)dc_round_up((size_t)dc_div_up(n16, ko->nnt), 16);
     ko->n_pad = ko->nnt * ko->n_tile;
@@ -373,4 +374,7 @@ dc_status dc_launch_conv_stem(const void *x, int n, int h, int w, const dc_geom 
                               const float *bias, dc_act act, const void *residual, void *y,
                               void *workspace, cudaStream_t stream);
 bool dc_conv_stem_supported(int n, int h, int w, const dc_geom *g);
+bool dc_dwconv_stencil_supported(int n, int h, int w, int c, int k, int stride, int pad);
+dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, int k, int stride, int pad, const float *wp,
+                                   const float *bias, dc_act act, void *y, cudaStream_t st);
 dc_status dc_validate_geom(const dc_geom *g);

@@ -445,6 +445,9 @@ static dc_status launch_dw(const void *x, int n, int h, int w, int c, int k, int
                            const float *bias, dc_act act, void *y, cudaStream_t st) {
   const int ho = dc_out_extent(h, k, stride, pad), wo = dc_out_extent(w, k, stride, pad);
   constexpr int V = DwVec<T>::V;
+  // bf16, common shapes: the shared-memory stencil (TMA-staged haloed tile)
+  if (sizeof(T) == 2 && dc_dwconv_stencil_supported(n, h, w, c, k, stride, pad))
+    return dc_launch_dwconv_stencil(x, n, h, w, c, k, stride, pad, wp, bias, act, y, st);
   if (c % V == 0 && (k == 3 || k == 5) && (stride == 1 || stride == 2) && (long long)n * ho < (1ll << 31)) {
     // stride 1: 4 outputs per thread share 6 (k = 3) input columns; stride 2 shares less, so 2 outputs
     // keep the register count down.  Threads per CTA: the row's work items, in whole warps, up to 128.

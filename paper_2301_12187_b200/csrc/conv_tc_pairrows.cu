@@ -429,6 +429,9 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
       // issue sequences of several blocks progress side by side although each shares its scheduler
       // with epilogue warps.  The warp stays converged; one elected lane issues.
       const int mw = warp - kMmaWarp;
+      // one election for the whole role: the warp stays converged and the same lane issues every
+      // instruction (an election per instruction costs ~230 cycles, several times the instruction)
+      const bool leader = elect_one();
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
       const uint32_t b_hi = (128u >> 4) | (1u << 14);            // no swizzle: 128 bytes between 8-row groups
       const uint32_t a_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128-byte swizzle: 1024 bytes between 8-row groups
@@ -460,14 +463,14 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
           for (int j = 0; j < p.nmma; ++j, b_lo += b_step) {
             const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(p.a_lo[j] + a_add);
             const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-            if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+            if (leader) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
           }
-          if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
+          if (leader) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
           slot += (uint32_t)p.mma_warps;
           while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
         }
         // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
-        if (ok && elect_one()) umma_commit(&sh.empty[s]);
+        if (ok && leader) umma_commit(&sh.empty[s]);
         c0 += nblk;
         t.step(p);
         a_row += a_stage_rows;

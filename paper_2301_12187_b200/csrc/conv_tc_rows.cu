@@ -35,6 +35,7 @@ constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
 constexpr int kThreads = 32 + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
 constexpr int kMaxBlocks = 2;                    // 128-row blocks per tile
+constexpr int kStagePitch = 80;                  // bytes per pixel in an epilogue warp's turn-around buffer (64 + 16)
 
 struct RowsParams {
   int n_img, h, w, ho, wo, c_in, c_out;
@@ -47,7 +48,7 @@ struct RowsParams {
   int lines_img;               // rbox * wbox: GEMM rows per image of a tile
   int a_stage_bytes, a_box_bytes, b_stage_bytes;
   int sa, sb, nacc, act;
-  int off_bias, off_b, off_a, smem_bytes;
+  int off_bias, off_stage, off_b, off_a, smem_bytes;
   int tmem_cols;
 };
 
@@ -175,6 +176,8 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp < kFirstEpiWarp) {
       // ================================================================== MMA issue
       const int mw = warp - kMmaWarp;
+      // one election for the whole role: the warp stays converged and the same lane issues every instruction
+      const bool leader = elect_one();
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) | (8u << 24);
       const uint32_t b_hi = (128u >> 4) | (1u << 14);                 // no swizzle: 128 bytes between 8-row groups
       const uint32_t a_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128-byte swizzle: 1024 bytes between 8-row groups
@@ -217,7 +220,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   if (sl < nsl) {
                     const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + 2u * sl);
                     const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-                    if (elect_one()) umma_bf16(d, ad, bd, idesc, accum);
+                    if (leader) umma_bf16(d, ad, bd, idesc, accum);
                     accum = 1u;
                     b_lo += b_inc;
                   }
@@ -225,13 +228,13 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               }
             }
             first = false;
-            if (elect_one()) umma_commit(&sh.b_empty[sb]);      // this warp is done with the weight stage
+            if (leader) umma_commit(&sh.b_empty[sb]);      // this warp is done with the weight stage
             if (++sb == p.sb) { sb = 0; pb ^= 1; }
           }
-          if (ok && elect_one()) umma_commit(&sh.a_empty[sa]);  // ... and with the plane
+          if (ok && leader) umma_commit(&sh.a_empty[sa]);  // ... and with the plane
           if (++sa == p.sa) { sa = 0; pa ^= 1; }
         }
-        if (ok && elect_one()) umma_commit(&sh.acc_full[set]);  // this warp's blocks of the item are complete
+        if (ok && leader) umma_commit(&sh.acc_full[set]);  // this warp's blocks of the item are complete
       }
     } else {
       // ================================================================== epilogue
@@ -240,7 +243,9 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int ew = warp - kFirstEpiWarp;
       const int q = warp & 3, par = ew >> 2;
       const uint32_t tmem_row = tmem_base + ((uint32_t)(q * 32) << 16);
+      uint8_t *stage = smem + p.off_stage + ew * (32 * kStagePitch);   // this warp's turn-around buffer
       uint32_t acc_ph[2] = {0u, 0u};
+      const bool relu6 = p.act == DC_ACT_RELU6;
 #pragma unroll 1
       for (int it = 0; it < nitems; ++it) {
         const int set = p.nacc == 2 ? (it & 1) : 0;
@@ -264,8 +269,8 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __nv_bfloat16 *dst = y + pix * p.c_out + ch0;
           const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out + ch0 : nullptr;
           const uint32_t taddr = tmem_row + (uint32_t)((set * p.mb + b) * p.n_tile);
-          // eight channels of this thread's pixel: bias, skip input, activation, one 16-byte store
-          auto store8 = [&](const uint32_t *v, int ch) {
+          // eight channels of this thread's pixel: bias, skip input, activation -> eight bf16
+          auto cook8 = [&](const uint32_t *v, int ch) {
             const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch);
             const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch + 4);
             float f[8];
@@ -273,7 +278,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
             f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
             f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
-            if (rp) {
+            if (rp && valid) {
               const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
               const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
 #pragma unroll
@@ -284,32 +289,53 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             uint4 ov;
             __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+            // ReLU6 on the rounded pairs: 0 and 6 are bf16 values and rounding is monotonic, so clamping
+            // after the conversion gives the same bits as clamping before it, in half the instructions
+            const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f), six2 = __floats2bfloat162_rn(6.f, 6.f);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              float f0 = f[2 * i], f1 = f[2 * i + 1];
-              if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
-              ob[i] = __floats2bfloat162_rn(f0, f1);
+              __nv_bfloat162 o = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+              if (relu6) o = __hmin2(__hmax2(o, zero2), six2);
+              ob[i] = o;
             }
-            *reinterpret_cast<uint4 *>(dst + ch) = ov;
+            return ov;
           };
-          // 32 accumulator columns per read while they last (one wait, four stores back to back), then 8
+          // 32 accumulator columns per read while they last.  A thread owns a pixel, so stored directly
+          // its 16-byte pieces would land c_out * 2 bytes apart from its neighbours' (half-filled
+          // sectors, 32 lines per instruction).  The warp instead turns the 32 pixels x 64 bytes around
+          // in its staging buffer (80-byte pitch: conflict-free) and writes them four lanes to a
+          // pixel: every store instruction then fills eight whole 64-byte segments.
+          const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
+          auto emit32 = [&](const uint32_t *v, int c0) {
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8)
+              *reinterpret_cast<uint4 *>(stage + lane * kStagePitch + g8 * 16) = cook8(v + 8 * g8, c0 + 8 * g8);
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int px = i * 8 + (lane >> 2), c = lane & 3;
+              const unsigned long long base = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, px);
+              if ((vmask >> px) & 1u)
+                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>((uintptr_t)base) + c0 + c * 8) =
+                    *reinterpret_cast<const uint4 *>(stage + px * kStagePitch + c * 16);
+            }
+            __syncwarp();
+          };
           int ch = 0;
 #pragma unroll 1
           for (; ch + 32 <= nch; ch += 32) {
             uint32_t v[32];
             tmem_ld32(taddr + (uint32_t)ch, v);
             tmem_ld_wait();
-            if (valid) {
-#pragma unroll
-              for (int g8 = 0; g8 < 4; ++g8) store8(v + 8 * g8, ch + 8 * g8);
-            }
+            emit32(v, ch);
           }
 #pragma unroll 1
           for (; ch < nch; ch += 8) {
             uint32_t v[8];
             tmem_ld8(taddr + (uint32_t)ch, v);
             tmem_ld_wait();
-            if (valid) store8(v, ch);
+            const uint4 ov = cook8(v, ch);
+            if (valid) *reinterpret_cast<uint4 *>(dst + ch) = ov;
           }
         }
         // this warp has read what it needs of the accumulator set
@@ -407,7 +433,8 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   // reach up to ~200 lines (25 KB) past its stage; behind the last activation stage that lands in
   // the weight stages, which are larger (what is read there only feeds rows that are dropped).
   p->off_bias = 0;
-  p->off_a = (int)dc_round_up((size_t)p->n_pad * 4, 1024);
+  p->off_stage = (int)dc_round_up((size_t)p->n_pad * 4, 128);
+  p->off_a = (int)dc_round_up((size_t)p->off_stage + kEpiWarps * 32 * kStagePitch, 1024);
   // rings: weights first (they are the larger stream), then activation planes
   int sa = 2, sb = 2;
   auto total = [&](int a, int b) {

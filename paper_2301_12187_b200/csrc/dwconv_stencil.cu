@@ -1,0 +1,249 @@
+// Depthwise convolution (bf16, k = 3 or 5, stride 1 or 2) as a shared-memory stencil on CUDA cores.
+//
+// A CTA owns a tile of output rows x the whole output width x a group of channels (x several
+// images for small maps).  One 4-D TMA load brings the haloed input patch of the tile into shared
+// memory as [image][row][column][channel]; the TMA unit writes zeros for everything outside the image,
+// so the stencil itself has no border cases.  Threads then compute from shared memory: a thread owns
+// 8 channels (one 16-byte vector) of TX neighbouring outputs of one row, so the (TX-1)*S + K input
+// vectors of a tap row are read once for all the outputs they feed, with fp32 weights and fp32
+// accumulation, and writes its results as 16-byte vectors (neighbouring threads write neighbouring
+// vectors of a pixel: whole 32-byte sectors).  Depthwise layers are bound by HBM (1.8-4.5 FLOP/B):
+// the tile is read from HBM once (neighbouring tiles share only their halo rows), and several CTAs
+// per SM overlap one tile's load with another's arithmetic and stores.  No tensor cores.
+//
+// The one wait (for the tile to land) is bounded like every wait of the library; a wait that runs
+// out sets a library-wide flag that dc_dwconv_status reports, and the CTA returns.
+#include "tc_ptx.cuh"
+
+namespace {
+using namespace tc;
+
+constexpr int kThreads = 256;
+constexpr int kV = 8;                            // channels per thread (16 bytes of bf16)
+constexpr int kTileBytes = 64 * 1024;            // patch size limit: up to three CTAs per SM by shared memory
+
+struct StencilParams {
+  int n_img, h, w, c, ho, wo, pad, act;
+  int ct, cgroups;             // channels per tile, tiles per pixel's channels
+  int rt, ytiles;              // output rows per tile, tiles per image column
+  int ni, igroups;             // images per tile, tiles over the batch
+  int in_rows, in_w;           // patch rows and columns (with halo)
+  int box_bytes, patch_bytes;  // bytes the TMA load delivers; the same rounded up to 128
+};
+
+__device__ unsigned int g_dw_status;             // DC_ERR_TIMEOUT once a wait of these kernels ran out
+
+template <int K, int S>
+__global__ void __launch_bounds__(kThreads, 2)
+k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ StencilParams p,
+                 const float *__restrict__ w, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ y) {
+  constexpr int TX = S == 1 ? 4 : 2;             // outputs per thread along a row
+  constexpr int NJ = (TX - 1) * S + K;           // input columns they read
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t abort_word;
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+  float *w_s = reinterpret_cast<float *>(smem + p.patch_bytes);          // [K*K][ct] weights, then [ct] bias
+
+  // tile of this CTA: (image group, row tile, channel group), channel groups fastest
+  int t = (int)blockIdx.x;
+  const int cg = t % p.cgroups; t /= p.cgroups;
+  const int ty = t % p.ytiles;
+  const int ig = t / p.ytiles;
+  const int c0 = cg * p.ct, y0 = ty * p.rt, img0 = ig * p.ni;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_word = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_arrive_expect_tx(&bar, (uint32_t)p.box_bytes);
+    // coordinates may be negative or reach past the tensor: those elements arrive as zeros
+    tma_load_4d(smem_u32(smem), &map_x, &bar, c0, -p.pad, y0 * S - p.pad, img0);
+  }
+  for (int i = (int)threadIdx.x; i < (K * K + 1) * p.ct; i += kThreads) {
+    const int tap = i / p.ct, ch = i - tap * p.ct;
+    w_s[i] = tap < K * K ? w[(size_t)tap * p.c + c0 + ch] : (bias ? bias[c0 + ch] : 0.f);
+  }
+  __syncthreads();
+  if (!mbar_wait(&bar, 0, &abort_word, nullptr, 0xA0000u)) {
+    atomicExch(&g_dw_status, (unsigned int)DC_ERR_TIMEOUT);
+    return;
+  }
+
+  const int cvt = p.ct / kV;                     // vectors per pixel of this tile: divides kThreads
+  const int cv = (int)threadIdx.x % cvt;         // this thread's vector, the same for all its items
+  const int xtiles = (p.wo + TX - 1) / TX;
+  const int rows_valid = p.ho - y0 < p.rt ? p.ho - y0 : p.rt;
+  const int imgs_valid = p.n_img - img0 < p.ni ? p.n_img - img0 : p.ni;
+  const int per_img = rows_valid * xtiles;
+  const int items = imgs_valid * per_img;
+  const float *bias_s = w_s + K * K * p.ct + cv * kV;
+  const size_t row_pitch = (size_t)p.in_w * p.ct, img_pitch = (size_t)p.in_rows * row_pitch;   // elements
+  const __nv_bfloat16 *patch = reinterpret_cast<const __nv_bfloat16 *>(smem) + cv * kV;
+#pragma unroll 1
+  for (int item = (int)threadIdx.x / cvt; item < items; item += kThreads / cvt) {
+    const int il = item / per_img, rem = item - il * per_img;
+    const int ry = rem / xtiles, xt = rem - ry * xtiles;
+    const int X0 = xt * TX;
+    // packed fp32 arithmetic (two multiply-adds per instruction): the layer has 4.5 FLOP per byte
+    // moved, which one scalar FMA per instruction would not keep up with
+    float2 acc[TX][kV / 2];
+    {
+      const float4 b0 = *reinterpret_cast<const float4 *>(bias_s), b1 = *reinterpret_cast<const float4 *>(bias_s + 4);
+#pragma unroll
+      for (int o = 0; o < TX; ++o) {
+        acc[o][0] = make_float2(b0.x, b0.y); acc[o][1] = make_float2(b0.z, b0.w);
+        acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
+      }
+    }
+    const __nv_bfloat16 *prow = patch + il * img_pitch + (size_t)(ry * S) * row_pitch + (size_t)(X0 * S) * p.ct;
+#pragma unroll 1
+    for (int r = 0; r < K; ++r) {
+      float2 wr[K][kV / 2];
+#pragma unroll
+      for (int sx = 0; sx < K; ++sx) {
+        const float *wp = w_s + (r * K + sx) * p.ct + cv * kV;
+        const float4 w0 = *reinterpret_cast<const float4 *>(wp), w1 = *reinterpret_cast<const float4 *>(wp + 4);
+        wr[sx][0] = make_float2(w0.x, w0.y); wr[sx][1] = make_float2(w0.z, w0.w);
+        wr[sx][2] = make_float2(w1.x, w1.y); wr[sx][3] = make_float2(w1.z, w1.w);
+      }
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        // columns past the patch's last one only feed outputs past the row's end, which are not stored
+        const int col = X0 * S + j < p.in_w ? j : 0;
+        const uint4 raw = *reinterpret_cast<const uint4 *>(prow + (size_t)r * row_pitch + (size_t)col * p.ct);
+        const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+        float2 xv[kV / 2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xv[i] = __bfloat1622float2(rb[i]);
+#pragma unroll
+        for (int o = 0; o < TX; ++o) {
+          const int sx = j - o * S;                // tap column with which input j feeds output o
+          if (sx >= 0 && sx < K) {
+#pragma unroll
+            for (int q = 0; q < kV / 2; ++q) acc[o][q] = __ffma2_rn(xv[q], wr[sx][q], acc[o][q]);
+          }
+        }
+      }
+    }
+    __nv_bfloat16 *yrow = y + (((size_t)(img0 + il) * p.ho + (size_t)(y0 + ry)) * p.wo) * p.c + c0 + cv * kV;
+#pragma unroll
+    for (int o = 0; o < TX; ++o) {
+      if (X0 + o < p.wo) {
+        uint4 ov;
+        __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float f0 = acc[o][i].x, f1 = acc[o][i].y;
+          if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
+          ob[i] = __floats2bfloat162_rn(f0, f1);
+        }
+        *reinterpret_cast<uint4 *>(yrow + (size_t)(X0 + o) * p.c) = ov;
+      }
+    }
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+bool stencil_plan(int n, int h, int w, int c, int k, int stride, int pad, StencilParams *p) {
+  if ((k != 3 && k != 5) || (stride != 1 && stride != 2) || c % kV) return false;
+  const int ho = dc_out_extent(h, k, stride, pad), wo = dc_out_extent(w, k, stride, pad);
+  if (ho <= 0 || wo <= 0) return false;
+  p->n_img = n; p->h = h; p->w = w; p->c = c; p->ho = ho; p->wo = wo; p->pad = pad;
+  p->ct = c % 64 == 0 ? 64 : (c % 32 == 0 ? 32 : (c % 16 == 0 ? 16 : 8));
+  p->cgroups = c / p->ct;
+  p->in_w = (wo - 1) * stride + k;
+  if (p->in_w > 256) return false;               // a TMA box is at most 256 elements wide
+  const long long row_bytes = (long long)p->in_w * p->ct * 2;
+  // rows per tile: as many as fit the patch limit, at least one
+  int rt = ho;
+  while (rt > 1 && ((long long)(rt - 1) * stride + k) * row_bytes > kTileBytes) --rt;
+  if (((long long)(rt - 1) * stride + k) * row_bytes > kTileBytes) return false;
+  if ((rt - 1) * stride + k > 256) rt = (256 - k) / stride + 1;
+  p->rt = rt;
+  p->ytiles = dc_div_up(ho, rt);
+  p->in_rows = (rt - 1) * stride + k;
+  // small maps: several images per tile while the grid still fills the GPU twice over
+  p->ni = 1;
+  if (p->ytiles == 1) {
+    const long long img_bytes = (long long)p->in_rows * row_bytes;
+    while (p->ni < 8 && p->ni * 2 <= n && (p->ni * 2) * img_bytes <= kTileBytes &&
+           (long long)dc_div_up(n, p->ni * 2) * p->cgroups >= 2ll * dc_sm_count())
+      p->ni *= 2;
+  }
+  p->igroups = dc_div_up(n, p->ni);
+  p->box_bytes = (int)((long long)p->ni * p->in_rows * row_bytes);
+  p->patch_bytes = (int)dc_round_up((size_t)p->box_bytes, 128);
+  if ((long long)p->igroups * p->ytiles * p->cgroups >= (1ll << 31)) return false;
+  return true;
+}
+
+}  // namespace
+
+bool dc_dwconv_stencil_supported(int n, int h, int w, int c, int k, int stride, int pad) {
+  StencilParams p;
+  return stencil_plan(n, h, w, c, k, stride, pad, &p);
+}
+
+dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, int k, int stride, int pad, const float *wp,
+                                   const float *bias, dc_act act, void *y, cudaStream_t st) {
+  StencilParams p;
+  if (!stencil_plan(n, h, w, c, k, stride, pad, &p)) return DC_ERR_UNSUPPORTED;
+  p.act = (int)act;
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return DC_ERR_CUDA;
+  CUtensorMap map_x;
+  {
+    const cuuint64_t C = (cuuint64_t)c;
+    cuuint64_t gdim[4] = {C, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+    cuuint64_t gstr[3] = {2 * C, (cuuint64_t)w * C * 2, (cuuint64_t)h * w * C * 2};
+    cuuint32_t box[4] = {(cuuint32_t)p.ct, (cuuint32_t)p.in_w, (cuuint32_t)p.in_rows, (cuuint32_t)p.ni};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = encode(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(x), gdim, gstr, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
+  }
+  const int smem = p.patch_bytes + (k * k + 1) * p.ct * 4 + 256;
+  const int grid = p.igroups * p.ytiles * p.cgroups;
+  __nv_bfloat16 *yp = (__nv_bfloat16 *)y;
+#define DC_DW_LAUNCH(KK, SS)                                                                              \
+  do {                                                                                                    \
+    static unsigned char attr_done[kDcMaxDevices];                                                        \
+    DC_CUDA_OK(dc_set_max_smem_once(k_dwconv_stencil<KK, SS>, kTileBytes + 8 * 1024, attr_done));         \
+    k_dwconv_stencil<KK, SS><<<grid, kThreads, smem, st>>>(map_x, p, wp, bias, yp);                       \
+  } while (0)
+  if (k == 3 && stride == 1) DC_DW_LAUNCH(3, 1);
+  else if (k == 3) DC_DW_LAUNCH(3, 2);
+  else if (stride == 1) DC_DW_LAUNCH(5, 1);
+  else DC_DW_LAUNCH(5, 2);
+#undef DC_DW_LAUNCH
+  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+extern "C" dc_status dc_dwconv_status(dc_stream stream) {
+  DC_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  unsigned int st = 0;
+  DC_CUDA_OK(cudaMemcpyFromSymbol(&st, g_dw_status, sizeof(st)));
+  if (st != 0) {
+    const unsigned int zero = 0;
+    DC_CUDA_OK(cudaMemcpyToSymbol(g_dw_status, &zero, sizeof(zero)));
+    return DC_ERR_TIMEOUT;
+  }
+  return DC_OK;
+}

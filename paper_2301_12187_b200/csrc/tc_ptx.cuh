@@ -71,8 +71,10 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, uint32_t parit
     if (*abort_flag) return false;
     if (globaltimer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
-      atomicExch(&ws->status, (unsigned int)DC_ERR_TIMEOUT);
-      ws->where = site;
+      if (ws) {                                  // kernels without a workspace report through their own flag
+        atomicExch(&ws->status, (unsigned int)DC_ERR_TIMEOUT);
+        ws->where = site;
+      }
       return false;
     }
   }

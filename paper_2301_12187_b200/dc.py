@@ -89,6 +89,7 @@ EXPORTS = {
                                        C.c_size_t, C.c_void_p, C.c_int]),
     "dc_dwconv_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p]),
+    "dc_dwconv_status": (C.c_int, [C.c_void_p]),
     "dc_block_workspace_bytes": (C.c_int, [C.c_int, C.c_int, C.c_int, C.POINTER(Block), C.c_int,
                                            C.POINTER(C.c_size_t)]),
     "dc_block_forward": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Block), C.c_void_p,
@@ -392,6 +393,10 @@ def dwconv_forward(x, k, stride, pad, w_packed, bias, act, y, stream=None):
     n, h, w, c = x.shape
     _check(lib().dc_dwconv_forward(_ptr(x), n, h, w, c, k, stride, pad, _ptr(w_packed), _ptr(bias), act,
                                    _ptr(y), dtype_code(x.dtype), _stream(stream)), "dc_dwconv_forward")
+
+
+def dwconv_status(stream=None) -> int:
+    return int(lib().dc_dwconv_status(_stream(stream)))
 
 
 def block_workspace_bytes(n, h, w, blk: Block, dtype: int) -> int:

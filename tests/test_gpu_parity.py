@@ -426,7 +426,11 @@ def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("c,k,s,p,n,h,w", [(32, 3, 1, 1, 2, 12, 12), (96, 3, 2, 1, 1, 15, 17),
                                            (144, 3, 1, 1, 1, 9, 30), (20, 5, 1, 2, 1, 8, 8),
-                                           (6, 3, 2, 1, 2, 7, 7), (960, 3, 1, 1, 2, 7, 7)])
+                                           (6, 3, 2, 1, 2, 7, 7), (960, 3, 1, 1, 2, 7, 7),
+                                           # the shared-memory stencil: several row tiles with a ragged last one,
+                                           # stride 2 with an odd height, 5x5 both strides, several images per tile
+                                           (32, 3, 1, 1, 3, 150, 112), (96, 3, 2, 1, 2, 41, 112), (240, 5, 2, 2, 2, 28, 28),
+                                           (384, 3, 1, 1, 21, 14, 14), (576, 5, 1, 2, 3, 14, 14), (24, 3, 1, 0, 2, 9, 20)])
 def test_dwconv(dc, dtype, c, k, s, p, n, h, w):
     spec = I.make_layer(8, 0, c, c, k, s, p, depthwise=True)
     lay = dc.DeviceLayer(spec)
@@ -442,7 +446,7 @@ def test_dwconv(dc, dtype, c, k, s, p, n, h, w):
     gy = Guarded(torch, (n, ho, wo, c), tdt, fill=float("nan"))
     y = gy.t
     dc.dwconv_forward(dev(x, tdt), k, s, p, packed, bf, dc.ACT_RELU6, y)
-    torch.cuda.synchronize()
+    assert dc.dwconv_status() == dc.OK
     gy.check("depthwise output")
     Wf, bfo = O.fold_bn(spec)
     ref = O.relu6(O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p, groups=c))
