@@ -63,12 +63,16 @@ def boundary_shapes(net):
     return shapes
 
 
-def measure_latency_table(net, unit_us: float = 1.0, reps: int = 10, max_span: int = 9, max_k: int = 7):
+def measure_latency_table(net, unit_us: float = 1.0, reps: int = 10, max_span: int = 9, max_k: int = 7,
+                          cold: bool = False):
     """Returns (T, us): T[i][j] = ceil(latency / unit_us) as Python ints (dc.DP_INF where the span
     is not mergeable or longer than max_span layers), us[i][j] the measured microseconds (None where
-    not measured).  bf16, this process's current CUDA device.  Each span's forward is captured `reps`
-    times in one CUDA graph and the graph's time divided by reps (inputs stay in L2 for small maps:
-    the table ranks merge patterns of one network against each other, it is not a roofline figure)."""
+    not measured).  bf16, this process's current CUDA device.  Warm (default): each span's forward is
+    captured `reps` times in one CUDA graph and the graph's time divided by reps, so inputs of small
+    maps stay in L2 -- the state a layer finds inside a running network, whose input the previous
+    layer has just written.  cold=True: every launch is timed on its own after a buffer larger than L2
+    has been overwritten, and the median of `reps` launches is taken (inputs come from HBM; a CUDA
+    event pair around one launch adds ~2 us to every entry alike)."""
     import math
     import torch
 
@@ -79,6 +83,7 @@ def measure_latency_table(net, unit_us: float = 1.0, reps: int = 10, max_span: i
     us = [[None] * (nL + 1) for _ in range(nL + 1)]
     conv_ws = torch.zeros(dc.conv_workspace_bytes(), dtype=torch.uint8, device="cuda")
     stream = torch.cuda.Stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if cold else None
     for i in range(nL):
         x = torch.zeros(shapes[i], dtype=torch.bfloat16, device="cuda")
         for j in range(i + 1, nL + 1):
@@ -118,19 +123,31 @@ def measure_latency_table(net, unit_us: float = 1.0, reps: int = 10, max_span: i
                         dc.conv_forward(x, g, packed, bm, dc.ACT_IDENTITY, None, y, conv_ws)
                 run()
                 stream.synchronize()
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=stream):
+                if cold:
+                    times = []
                     for _ in range(reps):
+                        flush.zero_()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record(stream)
                         run()
-                graph.replay()
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
-                graph.replay()
-                e1.record(stream)
-                stream.synchronize()
+                        e1.record(stream)
+                        stream.synchronize()
+                        times.append(e0.elapsed_time(e1) * 1e3)
+                    t_us = sorted(times)[len(times) // 2]
+                else:
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=stream):
+                        for _ in range(reps):
+                            run()
+                    graph.replay()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    graph.replay()
+                    e1.record(stream)
+                    stream.synchronize()
+                    t_us = e0.elapsed_time(e1) * 1e3 / reps
             if dc.workspace_status(conv_ws) != dc.OK:
                 raise RuntimeError("device-side wait timed out while timing span (%d, %d)" % (i, j))
-            t_us = e0.elapsed_time(e1) * 1e3 / reps
             us[i][j] = t_us
             T[i][j] = max(1, int(math.ceil(t_us / unit_us)))
     return T, us

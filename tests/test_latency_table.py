@@ -60,6 +60,32 @@ def test_measured_table_and_optimal_pattern():
 
 
 @pytest.mark.gpu
+def test_cold_table_has_the_same_valid_spans_and_is_no_faster():
+    """The L2-cold table (every launch after a flush of L2) marks the same spans valid, and a span
+    that reads its input from HBM is not faster than the same span replayed on an L2-resident input
+    (beyond the ~2 us an event pair around a single launch adds and measurement noise)."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_12187_b200 import dc
+    dc.lib()
+    net = I.mobilenet_v2(seed=0, batch=8, res=64)
+    L = len(net.layers)
+    Tw, usw = LT.measure_latency_table(net, unit_us=0.1, reps=5, max_span=3)
+    Tc, usc = LT.measure_latency_table(net, unit_us=0.1, reps=5, max_span=3, cold=True)
+    slower = 0
+    for i in range(L):
+        for j in range(i + 1, L + 1):
+            assert (Tw[i][j] < dc.DP_INF) == (Tc[i][j] < dc.DP_INF)
+            if usw[i][j] is not None:
+                slower += usc[i][j] >= usw[i][j] - 1.0
+    n_valid = sum(1 for i in range(L) for j in range(i + 1, L + 1) if usw[i][j] is not None)
+    assert slower >= 0.9 * n_valid
+    total, S, _, _ = LT.optimal_pattern(Tc, L)
+    assert total == P.alg1(Tc, L)[0][0][L]
+
+
+@pytest.mark.gpu
 def test_latency_planned_network_matches_the_oracle():
     """The network cut by Algorithm 1 over the measured table (kept activations fixed by the seed):
     every piece is a valid merge, the plan is no slower by the table than merging every valid span,
