@@ -169,11 +169,37 @@ class CompressedNetwork:
         return packed, bf
 
     # ------------------------------------------------------------------ the two halves of the path
-    def merge(self):
-        """Merge every span of two or more layers (dc_merge_chain), on the current stream."""
-        for devs, res, wm, bm, packed, ws in self._merge_jobs:
-            dc.merge_chain(devs, res, wm, bm, packed, dc.BF16, ws)
-        return len(self._merge_jobs)
+    def merge(self, n_streams: int = 10):
+        """Merge every span of two or more layers (dc_merge_chain).  The runs are independent of each
+        other (own layers, own outputs, own workspace) and each is a short chain of small dependent
+        launches, so they are spread over `n_streams` side streams forked from and joined back into the
+        current stream (largest runs first); the work is ordered like any other work on the current
+        stream and can be captured in a CUDA graph."""
+        torch = self.torch
+        jobs = self._merge_jobs
+        if n_streams <= 1 or len(jobs) <= 1:
+            for devs, res, wm, bm, packed, ws in jobs:
+                dc.merge_chain(devs, res, wm, bm, packed, dc.BF16, ws)
+            return len(jobs)
+        if not hasattr(self, "_merge_streams") or len(self._merge_streams) < n_streams:
+            self._merge_streams = [torch.cuda.Stream() for _ in range(n_streams)]
+        cur = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(cur)
+        order = sorted(range(len(jobs)), key=lambda i: -jobs[i][2].numel())
+        used = []
+        for n, i in enumerate(order):
+            st = self._merge_streams[n % n_streams]
+            if n < n_streams:
+                st.wait_event(fork)
+                used.append(st)
+            devs, res, wm, bm, packed, ws = jobs[i]
+            dc.merge_chain(devs, res, wm, bm, packed, dc.BF16, ws, stream=st)
+        for st in used:
+            done = torch.cuda.Event()
+            done.record(st)
+            cur.wait_event(done)
+        return len(jobs)
 
     def launch(self, i, cur, x):
         """Launch group i on `cur` (the previous group's map); x is the network input (skip source -1)."""
