@@ -85,21 +85,20 @@ __device__ __forceinline__ void compose_bias_block(const Piece &first, const Pie
 }
 static int bias_blocks(int c_out, int threads) { return dc_div_up(c_out * 32, threads); }
 
-// dense (second) o dense (first):  out[o][j] = sum_r A[o][r] * B[r][j] with
+// dense (second) o dense (first) for large results:  out[o][j] = sum_r A[o][r] * B[r][j] with
 //   r = (c, u2, v2),  j = (i, u', v'),  A = W2 as stored,
-//   B[r][j] = W1[c][i][u' - s1*u2][v' - s1*v2]  (0 when the tap falls outside W1).
-// 64x64 output tile, 256 threads, 4x4 outputs per thread.  The reduction is staged in slices of up
-// to kDdSlice rows: the merges are small and latency-bound, so a slice's loads (dozens per
-// thread, all independent) are issued in one go and cost one round trip to L2, where 16-deep
-// slices cost one per 16 rows.  A thread gathers one column j of B, so (i, u', v') is decoded once.
-// Blocks [0, gx*gy) are the tiles (x fastest); the blocks after them compute the bias.
-constexpr int kDdSlice = 256;
-constexpr int kDdPitch = 64 + 4;
-__global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece second, float *out, float *b_out,
-                                                             int kk, int gx, int gy, int slice) {
-  extern __shared__ __align__(16) float dd_smem[];
-  float *As = dd_smem;                       // [slice][kDdPitch]
-  float *Bs = dd_smem + slice * kDdPitch;    // [slice][kDdPitch]
+//   B[r][j] = W1[c][i][u' - s1*u2][v' - s1*v2]  (0 when the tap falls outside W1):
+// a gathered-operand SGEMM with register-staged double buffering.  Tile (16 * TM) x 64 outputs, 256 threads, TM x 4 outputs per thread, reduction slices of
+// 16 rows: while a slice is multiplied from shared memory the next one's operands are already on
+// their way into registers, so the loads' round trips to L2 hide behind the arithmetic instead of
+// alternating with it.  Same reduction order (c, u2, v2) as the other composition kernels.
+constexpr int kDtK = 16;                         // reduction rows per slice
+template <int TM>
+__global__ void __launch_bounds__(256) k_compose_dd_tiled(Piece first, Piece second, float *out, float *b_out,
+                                                          int kk, int gx, int gy) {
+  constexpr int BM = 16 * TM, PA = BM + 4, PB = 64 + 4;
+  __shared__ __align__(16) float As[2][kDtK][PA];
+  __shared__ __align__(16) float Bs[2][kDtK][PB];
   if ((int)blockIdx.x >= gx * gy) {
     compose_bias_block(first, second, b_out, (int)blockIdx.x - gx * gy);
     return;
@@ -108,85 +107,180 @@ __global__ void __launch_bounds__(256) k_compose_dense_dense(Piece first, Piece 
   const int k1 = first.k, k2 = second.k, s1 = first.stride, t2sz = k2 * k2;
   const int c0 = first.c_in, c1 = first.c_out, c2 = second.c_out;
   const int R = c1 * t2sz, J = c0 * kk * kk;
-  const int o0 = ((int)blockIdx.x / gx) * 64, j0 = ((int)blockIdx.x % gx) * 64;
-  const int t = threadIdx.x, ty = t / 16, tx = t % 16;
-  // this thread's column of B and row phase of A
-  const int jj = t & 63, j = j0 + jj;
+  const int o0 = ((int)blockIdx.x / gx) * BM, j0 = ((int)blockIdx.x % gx) * 64;
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+  // loads: A element (o = o0 + (t >> 4) + 16 q, r = t & 15), B element (r = (t >> 6) + 4 u, j = j0 + (t & 63))
+  const int ar = t & 15, ao = t >> 4;
+  const int jj = t & 63, j = j0 + jj, br = t >> 6;
   const int bi = j / (kk * kk), btp = j - bi * kk * kk, bup = btp / kk, bvp = btp - bup * kk;
-  const int arr = t & 15, arow = t >> 4;     // A: rows arow + 16q of the tile, slice row arr + 16p
-  float acc[4][4] = {};
-  for (int r0 = 0; r0 < R; r0 += slice) {
-    const int rows = R - r0 < slice ? R - r0 : slice;
-    // Operand loads are issued in batches with no branch between them (an element outside the
-    // operand reads element 0 and is zeroed afterwards): a load behind a branch would wait for the
-    // one before it, and a slice would cost dozens of round trips to L2 instead of a few.
-    // A[o][r]: consecutive threads read consecutive r of one output channel
-    for (int rb = arr; rb < rows; rb += 64) {
-      float av[4][4];
+  float av[TM], bv[4];
+  auto fetch = [&](int r0) {
+    const int ra = r0 + ar;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int rr = rb + 16 * u, r = r0 + (rr < rows ? rr : rows - 1);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int o = o0 + arow + 16 * q;
-          const bool ok = o < c2 && rr < rows;
-          const float x = second.w[ok ? (size_t)o * R + r : 0];
-          av[u][q] = ok ? ((second.ident && r == (o * k2 + ctr2) * k2 + ctr2) ? x + 1.f : x) : 0.f;
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int rr = rb + 16 * u;
-        if (rr < rows) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) As[rr * kDdPitch + arow + 16 * q] = av[u][q];
-        }
-      }
+    for (int q = 0; q < TM; ++q) {
+      const int o = o0 + ao + 16 * q;
+      const bool ok = o < c2 && ra < R;
+      const float x = second.w[ok ? (size_t)o * R + ra : 0];
+      av[q] = ok ? ((second.ident && ra == (o * k2 + ctr2) * k2 + ctr2) ? x + 1.f : x) : 0.f;
     }
-    // B[r][j]: consecutive threads read consecutive j (elements of W1 next to each other)
-    for (int rb = t >> 6; rb < rows; rb += 32) {
-      float bv[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int rr = rb + 4 * u, r = r0 + (rr < rows ? rr : rows - 1);
-        int c = r, u2 = 0, v2 = 0;
-        if (t2sz != 1) {
-          c = r / t2sz;
-          const int t2 = r - c * t2sz;
-          u2 = t2 / k2;
-          v2 = t2 - u2 * k2;
-        }
-        const int u1 = bup - s1 * u2, v1 = bvp - s1 * v2;
-        const bool ok = j < J && u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1;
-        const float x = first.w[ok ? (((size_t)c * c0 + bi) * k1 + u1) * k1 + v1 : 0];
-        bv[u] = ok ? ((first.ident && c == bi && u1 == ctr1 && v1 == ctr1) ? x + 1.f : x) : 0.f;
+    for (int u = 0; u < 4; ++u) {
+      const int r = r0 + br + 4 * u;
+      int c = r, u2 = 0, v2 = 0;
+      if (t2sz != 1) {
+        c = r / t2sz;
+        const int t2 = r - c * t2sz;
+        u2 = t2 / k2;
+        v2 = t2 - u2 * k2;
       }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int rr = rb + 4 * u;
-        if (rr < rows) Bs[rr * kDdPitch + jj] = bv[u];
-      }
+      const int u1 = bup - s1 * u2, v1 = bvp - s1 * v2;
+      const bool ok = r < R && j < J && u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1;
+      const float x = first.w[ok ? (((size_t)c * c0 + bi) * k1 + u1) * k1 + v1 : 0];
+      bv[u] = ok ? ((first.ident && c == bi && u1 == ctr1 && v1 == ctr1) ? x + 1.f : x) : 0.f;
     }
-    __syncthreads();
-#pragma unroll 4
-    for (int rr = 0; rr < rows; ++rr) {
-      const float4 a4 = *reinterpret_cast<const float4 *>(As + rr * kDdPitch + ty * 4);
-      const float4 b4 = *reinterpret_cast<const float4 *>(Bs + rr * kDdPitch + tx * 4);
-      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+  };
+  auto stage = [&](int buf) {
 #pragma unroll
-      for (int p = 0; p < 4; ++p)
+    for (int q = 0; q < TM; ++q) As[buf][ar][ao + 16 * q] = av[q];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) Bs[buf][br + 4 * u][jj] = bv[u];
+  };
+  float acc[TM][4] = {};
+  fetch(0);
+  stage(0);
+  __syncthreads();
+  int buf = 0;
+  for (int r0 = 0; r0 < R; r0 += kDtK) {
+    const bool more = r0 + kDtK < R;
+    if (more) fetch(r0 + kDtK);
+#pragma unroll
+    for (int rr = 0; rr < kDtK; ++rr) {
+      float a[TM];
+#pragma unroll
+      for (int q = 0; q < TM; q += 4) {
+        const float4 a4 = *reinterpret_cast<const float4 *>(&As[buf][rr][ty * TM + q]);
+        a[q] = a4.x; a[q + 1] = a4.y; a[q + 2] = a4.z; a[q + 3] = a4.w;
+      }
+      const float4 b4 = *reinterpret_cast<const float4 *>(&Bs[buf][rr][tx * 4]);
+      const float b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int p = 0; p < TM; ++p)
 #pragma unroll
         for (int q = 0; q < 4; ++q) acc[p][q] = fmaf(a[p], b[q], acc[p][q]);
     }
+    if (more) stage(buf ^ 1);
     __syncthreads();
+    buf ^= 1;
   }
 #pragma unroll
-  for (int p = 0; p < 4; ++p)
+  for (int p = 0; p < TM; ++p) {
+    const int o = o0 + ty * TM + p;
+    if (o >= c2) continue;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      int o = o0 + ty * 4 + p, jo = j0 + tx * 4 + q;
-      if (o < c2 && jo < J) out[(size_t)o * J + jo] = acc[p][q];
+      const int jo = j0 + tx * 4 + q;
+      if (jo < J) out[(size_t)o * J + jo] = acc[p][q];
     }
+  }
+}
+
+// dense 3x3 (stride 1) followed by dense 3x3, large channel counts (VGG-style runs): the result's
+// 5x5 kernel of one (o, i) pair is the sum over c of the full 2-D product of W2[o][c] (3x3) and
+// W1[c][i] (3x3), 81 multiply-adds per c, none of them with a structural zero -- the gathered GEMM
+// of the kernels above multiplies all 9 x 25 (tap, position) pairs, 64 % of which are zero.
+// CTA: 16 output channels x 32 input channels, 256 threads, a thread owns one o and two i (50
+// accumulators); slices of 8 intermediate channels are staged in shared memory with the next slice's
+// loads in flight (taps padded to 12 floats, read as three 16-byte vectors).  blockIdx.x walks the
+// tiles (i fastest); the blocks after them compute the bias.
+constexpr int kPolyC = 8;
+__global__ void __launch_bounds__(256) k_compose_poly33(Piece first, Piece second, float *out, float *b_out, int gx, int gy) {
+  __shared__ __align__(16) float W2s[2][16][kPolyC][12];   // [o][c][tap]
+  __shared__ __align__(16) float W1s[2][kPolyC][32][12];   // [c][i][tap]
+  if ((int)blockIdx.x >= gx * gy) {
+    compose_bias_block(first, second, b_out, (int)blockIdx.x - gx * gy);
+    return;
+  }
+  const int c0 = first.c_in, c1 = first.c_out, c2 = second.c_out;
+  const int o0 = ((int)blockIdx.x / gx) * 16, i0 = ((int)blockIdx.x % gx) * 32;
+  const int t = threadIdx.x, ol = t >> 4, il = t & 15;       // this thread's o, and i = il, il + 16
+  // loads of a slice: W2: 16 o x 8 c x 9 = 1152 floats, W1: 8 c x 32 i x 9 = 2304 floats
+  constexpr int N2 = (16 * kPolyC * 9 + 255) / 256, N1 = (kPolyC * 32 * 9) / 256;
+  float r2[N2], r1[N1];
+  auto fetch = [&](int cs) {
+#pragma unroll
+    for (int q = 0; q < N2; ++q) {
+      const int e = t + 256 * q;                 // (o, c, tap): taps of one (o, c) are contiguous in memory
+      const int tap = e % 9, oc = e / 9, cl = oc % kPolyC, o = o0 + oc / kPolyC, c = cs + cl;
+      const bool ok = e < 16 * kPolyC * 9 && o < c2 && c < c1;
+      const float x = second.w[ok ? ((size_t)o * c1 + c) * 9 + tap : 0];
+      r2[q] = ok ? ((second.ident && o == c && tap == 4) ? x + 1.f : x) : 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < N1; ++q) {
+      const int e = t + 256 * q;                 // (c, i, tap)
+      const int tap = e % 9, ci = e / 9, i = i0 + ci % 32, c = cs + ci / 32;
+      const bool ok = c < c1 && i < c0;
+      const float x = first.w[ok ? ((size_t)c * c0 + i) * 9 + tap : 0];
+      r1[q] = ok ? ((first.ident && c == i && tap == 4) ? x + 1.f : x) : 0.f;
+    }
+  };
+  auto stage = [&](int buf) {
+#pragma unroll
+    for (int q = 0; q < N2; ++q) {
+      const int e = t + 256 * q, tap = e % 9, oc = e / 9;
+      if (e < 16 * kPolyC * 9) W2s[buf][oc / kPolyC][oc % kPolyC][tap] = r2[q];
+    }
+#pragma unroll
+    for (int q = 0; q < N1; ++q) {
+      const int e = t + 256 * q, tap = e % 9, ci = e / 9;
+      W1s[buf][ci / 32][ci % 32][tap] = r1[q];
+    }
+  };
+  float acc[2][25] = {};
+  fetch(0);
+  stage(0);
+  __syncthreads();
+  int buf = 0;
+  for (int cs = 0; cs < c1; cs += kPolyC) {
+    const bool more = cs + kPolyC < c1;
+    if (more) fetch(cs + kPolyC);
+#pragma unroll 4
+    for (int cl = 0; cl < kPolyC; ++cl) {
+      float a[12], b[2][12];
+#pragma unroll
+      for (int v = 0; v < 3; ++v) {
+        *reinterpret_cast<float4 *>(a + 4 * v) = *reinterpret_cast<const float4 *>(&W2s[buf][ol][cl][4 * v]);
+        *reinterpret_cast<float4 *>(b[0] + 4 * v) = *reinterpret_cast<const float4 *>(&W1s[buf][cl][il][4 * v]);
+        *reinterpret_cast<float4 *>(b[1] + 4 * v) = *reinterpret_cast<const float4 *>(&W1s[buf][cl][il + 16][4 * v]);
+      }
+#pragma unroll
+      for (int u2 = 0; u2 < 3; ++u2)
+#pragma unroll
+        for (int v2 = 0; v2 < 3; ++v2)
+#pragma unroll
+          for (int u1 = 0; u1 < 3; ++u1)
+#pragma unroll
+            for (int v1 = 0; v1 < 3; ++v1) {
+              acc[0][(u1 + u2) * 5 + v1 + v2] = fmaf(a[u2 * 3 + v2], b[0][u1 * 3 + v1], acc[0][(u1 + u2) * 5 + v1 + v2]);
+              acc[1][(u1 + u2) * 5 + v1 + v2] = fmaf(a[u2 * 3 + v2], b[1][u1 * 3 + v1], acc[1][(u1 + u2) * 5 + v1 + v2]);
+            }
+    }
+    if (more) stage(buf ^ 1);
+    __syncthreads();
+    buf ^= 1;
+  }
+  const int o = o0 + ol;
+  if (o < c2) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int i = i0 + il + 16 * h;
+      if (i < c0) {
+        float *dst = out + ((size_t)o * c0 + i) * 25;
+#pragma unroll
+        for (int e = 0; e < 25; ++e) dst[e] = acc[h][e];
+      }
+    }
+  }
 }
 
 // dense o dense for small results (the usual case: a merged kernel has a few thousand elements):
@@ -217,7 +311,8 @@ __global__ void __launch_bounds__(256) k_compose_dd_small(Piece first, Piece sec
   float acc = 0.f;
   for (int r0 = 0; r0 < R; r0 += kDdSmallSlice) {
     const int rows = R - r0 < kDdSmallSlice ? R - r0 : kDdSmallSlice;
-    // Operand loads go out in batches with no branch between them (see k_compose_dense_dense).
+    // Operand loads go out in batches with no branch between them (an element outside the operand
+    // reads element 0 and is zeroed afterwards: a load behind a branch waits for the one before it).
     // A[o][r]: a warp reads 32 consecutive r of one output channel
     {
       float av[kDdSmallSlice / 32];
@@ -758,17 +853,17 @@ static Piece compose(const Piece &first, const Piece &second, Bump &bump, bool g
     } else if (!first.diag && !second.diag && elems <= (size_t)200000 && second.k <= 7) {
       const int gx = dc_div_up(out.c_in * out.k * out.k, 32), gy = dc_div_up(out.c_out, 8);
       k_compose_dd_small<<<gx * gy + nbias, 256, 0, st>>>(first, second, w, b, out.k, gx, gy);
+    } else if (!first.diag && !second.diag && first.k == 3 && second.k == 3 && first.stride == 1) {
+      const int gx = dc_div_up(out.c_in, 32), gy = dc_div_up(out.c_out, 16);
+      k_compose_poly33<<<gx * gy + nbias, 256, 0, st>>>(first, second, w, b, gx, gy);
     } else if (!first.diag && !second.diag) {
-      const int gx = dc_div_up(out.c_in * out.k * out.k, 64), gy = dc_div_up(out.c_out, 64);
-      const int R = first.c_out * second.k * second.k;
-      // few tiles: one deep slice per round trip; many tiles (more than two per SM): shallow slices,
-      // so that several CTAs share an SM and one's loads overlap another's arithmetic
-      const int slice_max = gx * gy > 2 * dc_sm_count() ? 64 : kDdSlice;
-      const int slice = R < slice_max ? (int)dc_round_up((size_t)R, 16) : slice_max;
-      const size_t smem = (size_t)2 * slice * kDdPitch * sizeof(float);
-      static unsigned char attr_done[kDcMaxDevices];
-      dc_set_max_smem_once(k_compose_dense_dense, 2 * kDdSlice * kDdPitch * (int)sizeof(float), attr_done);
-      k_compose_dense_dense<<<gx * gy + nbias, 256, smem, st>>>(first, second, w, b, out.k, gx, gy, slice);
+      // 128 x 64 tiles when they still give every SM two tiles, 64 x 64 otherwise
+      const int gx = dc_div_up(out.c_in * out.k * out.k, 64);
+      const int gy8 = dc_div_up(out.c_out, 128), gy4 = dc_div_up(out.c_out, 64);
+      if (gx * gy8 >= 2 * dc_sm_count())
+        k_compose_dd_tiled<8><<<gx * gy8 + nbias, 256, 0, st>>>(first, second, w, b, out.k, gx, gy8);
+      else
+        k_compose_dd_tiled<4><<<gx * gy4 + nbias, 256, 0, st>>>(first, second, w, b, out.k, gx, gy4);
     } else {
       const int nb = blocks_for(elems, 256);
       k_compose_diag<<<nb + nbias, 256, 0, st>>>(first, second, w, b, out.k, (int)elems, nb);
