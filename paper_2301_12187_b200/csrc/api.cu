@@ -29,6 +29,7 @@ extern "C" const char *dc_conv_kernel_name(int n, int h, int w, const dc_geom *g
   if (dc_conv_rows_supported(n, h, w, g)) return "k_conv_tc_rows";
   if (dc_conv_fold_supported(n, h, w, g)) return "k_conv_tc_fold";
   if (dc_conv_tc_supported(n, h, w, g)) return "k_conv_tc";
+  if (dc_conv_stem_s2_supported(n, h, w, g) && dc_conv_stem_supported(n, h, w, g)) return "k_conv_stem_s2";
   if (dc_conv_stem_supported(n, h, w, g)) return "k_conv_stem_tc";
   if (dc_conv_smallcin_supported(n, h, w, g)) return "k_conv_smallcin_bf16";
   return "k_conv_dense_bf16";
@@ -64,6 +65,8 @@ extern "C" dc_status dc_conv_forward_algo(const void *x, int n, int h, int w, co
     return dc_launch_conv_fold(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   if (tc_ok && algo != DC_ALGO_SIMT)
     return dc_launch_conv_tc(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
+  if (stem_ok && algo != DC_ALGO_SIMT && dc_conv_stem_s2_supported(n, h, w, g))
+    return dc_launch_conv_stem_s2(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   if (stem_ok && algo != DC_ALGO_SIMT)
     return dc_launch_conv_stem(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, st);
   return dc_launch_conv_simt(x, n, h, w, g, w_packed, bias, act, residual, y, dtype, st);

@@ -374,6 +374,10 @@ dc_status dc_launch_conv_stem(const void *x, int n, int h, int w, const dc_geom 
                               const float *bias, dc_act act, const void *residual, void *y,
                               void *workspace, cudaStream_t stream);
 bool dc_conv_stem_supported(int n, int h, int w, const dc_geom *g);
+dc_status dc_launch_conv_stem_s2(const void *x, int n, int h, int w, const dc_geom *g, const void *w_packed,
+                                 const float *bias, dc_act act, const void *residual, void *y,
+                                 void *workspace, cudaStream_t stream);
+bool dc_conv_stem_s2_supported(int n, int h, int w, const dc_geom *g);
 bool dc_dwconv_stencil_supported(int n, int h, int w, int c, int k, int stride, int pad);
 dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, int k, int stride, int pad, const float *wp,
                                    const float *bias, dc_act act, void *y, cudaStream_t st);

@@ -381,6 +381,13 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (3, 32, 3, 2, 1, 3, 40, 300, "k_conv_stem_tc"),         # the stem's geometry, ragged second segment
     (1, 8, 3, 1, 1, 2, 20, 20, "k_conv_stem_tc"),           # one input channel
     (3, 24, 5, 2, 2, 2, 21, 304, "k_conv_stem_tc"),         # 16-byte row chunks with a shifted second segment
+    (3, 32, 3, 2, 1, 2, 224, 224, "k_conv_stem_s2"),        # the stem itself: image rows as the operand, bands of 4 rows
+    (3, 32, 3, 2, 1, 3, 41, 304, "k_conv_stem_s2"),         # two segments per output row (the second ragged), odd height
+    (3, 40, 3, 2, 1, 2, 17, 32, "k_conv_stem_s2"),          # 40 output channels (48 operand rows), last band partial
+    (4, 16, 3, 2, 0, 2, 20, 40, "k_conv_stem_s2"),          # no padding, four channels: pixels already 8 bytes
+    (1, 8, 3, 2, 1, 2, 21, 24, "k_conv_stem_s2"),           # one input channel
+    (2, 128, 3, 2, 1, 1, 12, 16, "k_conv_stem_s2"),         # 128 output channels: one output row per band
+    (3, 32, 3, 2, 1, 64, 66, 64, "k_conv_stem_s2"),         # more bands than resident CTAs: one or two bands per CTA
     (3, 264, 3, 2, 1, 1, 20, 20, "k_conv_smallcin_bf16"),   # too many outputs for one accumulator: CUDA cores
     (24, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc_pairrows"),     # stride 2: one output per line, even/odd row boxes
     (32, 16, 5, 2, 2, 1, 30, 44, "k_conv_tc_pairrows"),     # stride 2, even padding, 5x5
