@@ -12,19 +12,35 @@
 // 128 outputs of an output row, and the threads only widen 6-byte pixels to 8 bytes.
 //
 // CTAs (256 threads, three per SM) are persistent and take bands of output rows of one image in
-// turn: one bulk copy brings a band's input rows (contiguous in memory) into one of two buffers while
-// the previous band is computed, the threads widen them, one lane issues the band's instructions (one
-// accumulator block per output row segment), and every thread reads a GEMM row back, adds the bias /
-// skip input, applies the activation and hands its pixel to the warp's turn-around buffer, from which
-// four lanes write each pixel's 64-byte pieces (whole sectors).  One thread waits on a barrier, the
-// others at the CTA barrier behind it (spinning warps would take issue slots).  Waits are bounded.
+// turn: one bulk copy brings a band's input rows (contiguous in memory) into one of two buffers while the
+// previous band is computed, the threads widen them (four 6-byte pixels per step for three channels), one
+// lane issues the band's instructions (one accumulator block per output row segment), and every
+// thread reads a GEMM row back, applies the skip input and the activation and puts its pixel into an
+// image of the band's output rows in shared memory, which leaves as one bulk copy (the rows are
+// contiguous in memory).  With a spare fourth channel the bias rides in the weights of that channel.
+// One thread waits on a barrier, the others at the CTA barrier behind it (spinning warps would take
+// issue slots).  Waits are bounded.
 #include "tc_ptx.cuh"
 
 namespace {
 using namespace tc;
 
 constexpr int kThreads = 256;                    // two warps per quarter of the accumulator lanes
-constexpr int kStagePitch = 80;                  // bytes per pixel in a warp's turn-around buffer (64 + 16)
+constexpr int kCtasPerSm = 3;
+constexpr int kTmemCols = 128;                   // accumulator columns of a CTA (512 per SM)
+constexpr int kSmemBudget = 73 * 1024;           // row, operand and output buffers of a CTA (three CTAs per SM)
+
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+  uint2 v;
+  asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts64(uint32_t a, uint32_t x, uint32_t y) {
+  asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(a), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 
 struct S2Params {
   int n_img, h, w, ho, wo, c_in, c_out, n_pad, pad, act;
@@ -39,7 +55,7 @@ struct S2Params {
   int ent[9];                  // chunk plane of tap (r, s) in the packed weights
 };
 
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restrict__ x, const void *__restrict__ w_packed,
                const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y,
                DcWsHeader *ws) {
@@ -50,13 +66,19 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_base) + 127) & ~uintptr_t(127));
   uint8_t *arow = smem + p.off_a;                // [in_rows][a_row_bytes]: 8-byte pixels, shifted right by pad
   uint8_t *bop = smem + p.off_b;                 // [3 kernel rows][2 K chunks][n_pad][16 bytes]
-  const int tid = (int)threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  uint8_t *outb = smem + p.off_stage;            // the band's output rows as they lie in memory
+  const int tid = (int)threadIdx.x, warp = tid >> 5;
   volatile uint32_t *abort_flag = &abort_s;
   const int total = p.n_img * p.bands;
+  // With a spare fourth channel every staged pixel carries 1.0 there, and the bias (split into two
+  // bf16 terms, exact to 16 mantissa bits) sits in the weights of that channel: the tensor core adds it.
+  const bool fold_bias = p.c_in <= 3;
+  const uint32_t one_hi = fold_bias ? 0x3F800000u : 0u;
 
-  // rows of band `bi` that exist in the image, as one bulk copy into raw buffer `buf`
-  auto issue_load = [&](int bi, int buf) {
-    const int img = bi / p.bands, Y0 = (bi - img * p.bands) * p.rb;
+  // rows of band `band` of image `img` that exist in the image, as one bulk copy into row buffer `buf`
+  // ([in_rows][raw_row_bytes]: rows as they are in memory)
+  auto issue_load = [&](int img, int band, int buf) {
+    const int Y0 = band * p.rb;
     const int rows_out = p.ho - Y0 < p.rb ? p.ho - Y0 : p.rb;
     const int gy0 = 2 * Y0 - p.pad;
     const int gy_first = gy0 < 0 ? 0 : gy0;
@@ -67,6 +89,9 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
     bulk_load(smem_u32(smem + p.off_raw + (size_t)buf * p.raw_buf_bytes + (size_t)(gy_first - gy0) * p.raw_row_bytes),
               reinterpret_cast<const uint8_t *>(x) + ((size_t)img * p.h + gy_first) * p.raw_row_bytes, bytes, &bar_load[buf]);
   };
+  // the bands of a CTA are gridDim.x apart: image and band advance by fixed steps
+  const int step_img = (int)gridDim.x / p.bands, step_band = (int)gridDim.x - step_img * p.bands;
+  int img = (int)blockIdx.x / p.bands, band = (int)blockIdx.x - img * p.bands;
 
   if (tid == 0) {
     abort_s = 0;
@@ -74,7 +99,7 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
     mbar_init(&bar_load[1], 1);
     mbar_init(&bar_mma, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    issue_load((int)blockIdx.x, 0);
+    issue_load(img, band, 0);
   }
   if (warp == 0) {
     tmem_alloc(&tmem_base_s, (uint32_t)p.tmem_cols);
@@ -82,143 +107,216 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
   }
   for (int i = tid; i < p.n_pad; i += kThreads) bias_s[i] = (bias && i < p.c_out) ? bias[i] : 0.f;
   // B operand from the packed weights ([chunk plane of a tap][n_pad][8 channels]): K element (pixel s, channel c)
-  // of kernel row r is W[o][c][r][s]; the fourth pixel and the fourth channel carry zeros
+  // of kernel row r is W[o][c][r][s]; the fourth pixel and the spare channels carry zeros (or the bias)
   for (int i = tid; i < 3 * 4 * p.n_pad; i += kThreads) {
     const int o = i % p.n_pad, s = (i / p.n_pad) & 3, r = i / (4 * p.n_pad);
     uint2 v = make_uint2(0u, 0u);
     if (s < 3) v = *reinterpret_cast<const uint2 *>(reinterpret_cast<const uint8_t *>(w_packed) + ((size_t)(p.ent[r * 3 + s] * p.n_pad + o)) * 16);
+    if (fold_bias && r == 0 && s < 2 && bias && o < p.c_out) {
+      const float b = bias[o];
+      const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+      const __nv_bfloat16 part = s == 0 ? hi : __float2bfloat16_rn(b - __bfloat162float(hi));
+      v.y = (v.y & 0xFFFFu) | ((uint32_t)__bfloat16_as_ushort(part) << 16);
+    }
     *reinterpret_cast<uint2 *>(bop + ((size_t)((r * 2 + (s >> 1)) * p.n_pad + o)) * 16 + (s & 1) * 8) = v;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  uint8_t *stage = smem + p.off_stage + warp * (32 * kStagePitch);
   const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
   const bool relu6 = p.act == DC_ACT_RELU6;
   const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f), six2 = __floats2bfloat162_rn(6.f, 6.f);
   const int wpix = p.w + p.pad + 4;              // pixels per operand row
+  const size_t out_row_bytes = (size_t)p.wo * p.c_out * 2;
+  // instruction and operand descriptors (no swizzle, K-major): 128 bytes between 8-row groups; A: K chunks
+  // 16 bytes apart; B: K chunks n_pad * 16 bytes apart, one descriptor per kernel row
+  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
+  const uint64_t desc_hi64 = (uint64_t)((128u >> 4) | (1u << 14)) << 32;
+  const uint32_t a_desc0 = smem_u32(arow) >> 4, a_row16 = (uint32_t)p.a_row_bytes >> 4;
+  uint64_t b_desc[3];
+#pragma unroll
+  for (int r = 0; r < 3; ++r)
+    b_desc[r] = desc_hi64 | (((smem_u32(bop) >> 4) + (uint32_t)(r * 2 * p.n_pad)) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
 
-  // ---- bands of this CTA; the next band's rows arrive while this one is computed
+  // shared-memory addresses of the widening step, 32 bits wide (the loop below is instruction bound):
+  // group j of a row = pixels 4 j .. 4 j + 3 (24 bytes) -> operand pixels 4 j + pad ..
+  const uint32_t raw_s = smem_u32(smem + p.off_raw), arow_s = smem_u32(arow), out_s = smem_u32(outb);
+  const int wj = tid & 63, wr0 = tid >> 6;
+  const int groups = p.w >> 2;                   // w is a multiple of 8 (rows are multiples of 16 bytes)
+  const uint32_t w_src0 = raw_s + (uint32_t)(wr0 * p.raw_row_bytes + wj * 24);
+  const uint32_t w_dst0 = arow_s + (uint32_t)(wr0 * p.a_row_bytes + (4 * wj + p.pad) * 8);
+  const uint32_t one = one_hi >> 16;
+  // the pixels in front of and behind a row hold the same values in every band: written once
+  for (int i = tid; i < p.in_rows * (p.pad + 4); i += kThreads) {
+    const int r = i / (p.pad + 4), q = i - r * (p.pad + 4);
+    const int pos = q < p.pad ? q : p.w + q;
+    *reinterpret_cast<uint2 *>(arow + (size_t)r * p.a_row_bytes + pos * 8) = make_uint2(0u, one_hi);
+  }
+
+  // ---- bands of this CTA; the next band's rows arrive while this one is multiplied and written
   int it = 0;
   for (int bi = (int)blockIdx.x; bi < total; bi += (int)gridDim.x, ++it) {
-    const int buf = it & 1;
-    const int img = bi / p.bands, Y0 = (bi - img * p.bands) * p.rb;
+    const int Y0 = band * p.rb;
     const int rows_out = p.ho - Y0 < p.rb ? p.ho - Y0 : p.rb;
     const int gy0 = 2 * Y0 - p.pad;              // input row of the band's first staged row
-    const uint8_t *raw = smem + p.off_raw + (size_t)buf * p.raw_buf_bytes;
+    const int buf = it & 1;
+    const int img_now = img;
+    band += step_band;
+    img += step_img;
+    if (band >= p.bands) { band -= p.bands; ++img; }
     bool done = true;
     if (tid == 0) {
       done = mbar_wait(&bar_load[buf], (uint32_t)(it >> 1) & 1u, abort_flag, ws, 0xB0000u);
-      // the other buffer was widened one band ago; the accumulators of that band have been read
-      if (done && bi + (int)gridDim.x < total) issue_load(bi + (int)gridDim.x, buf ^ 1);
+      // the other row buffer was widened one band ago: fetch the next band into it
+      if (done && bi + (int)gridDim.x < total) issue_load(img, band, buf ^ 1);
     }
-    tc_fence_before();
+    tc_fence_before();                           // the previous band's accumulators have been read
     if (!__syncthreads_and(done)) break;
-    // ---- widen: pixel px of staged row r goes to byte (px + pad) * 8 of its operand row; the padding
-    // pixels in front and behind, and rows outside the image, are zeros
-    for (int r = tid >> 7; r < p.in_rows; r += kThreads >> 7) {
-      const int gy = gy0 + r;
-      const bool row_in = gy >= 0 && gy < p.h;
-      const unsigned short *q0 = reinterpret_cast<const unsigned short *>(raw + (size_t)r * p.raw_row_bytes);
-      for (int pos = tid & 127; pos < wpix; pos += 128) {
-        const int px = pos - p.pad;
-        uint32_t v0 = 0u, v1 = 0u;
-        if (row_in && px >= 0 && px < p.w) {
-          const unsigned short *q = q0 + px * p.c_in;
-          v0 = q[0];
-          if (p.c_in > 1) v0 |= (uint32_t)q[1] << 16;
-          if (p.c_in > 2) v1 = q[2];
-          if (p.c_in > 3) v1 |= (uint32_t)q[3] << 16;
+    // ---- widen: pixel px of staged row r goes to byte (px + pad) * 8 of its operand row; rows outside
+    // the image are zeros (with 1.0 in a spare fourth channel)
+    if (p.c_in == 3) {
+      // four pixels (24 bytes) per step: three 8-byte loads, six byte permutes, four 8-byte stores
+      uint32_t src = w_src0 + (uint32_t)(buf * p.raw_buf_bytes), dst = w_dst0;
+      for (int r = wr0; r < p.in_rows; r += kThreads >> 6, src += (kThreads >> 6) * p.raw_row_bytes, dst += (kThreads >> 6) * p.a_row_bytes) {
+        const bool row_in = (unsigned)(gy0 + r) < (unsigned)p.h;
+        uint32_t sj = src, dj = dst;
+        for (int j = wj; j < groups; j += 64, sj += 64 * 24, dj += 64 * 32) {
+          uint2 a = make_uint2(0u, 0u), b = a, c = a;
+          if (row_in) {
+            a = lds64(sj);
+            b = lds64(sj + 8);
+            c = lds64(sj + 16);
+          }
+          sts64(dj, a.x, __byte_perm(a.y, one, 0x5410));
+          sts64(dj + 8, __byte_perm(a.y, b.x, 0x5432), __byte_perm(b.x, one, 0x5432));
+          sts64(dj + 16, b.y, __byte_perm(c.x, one, 0x5410));
+          sts64(dj + 24, __byte_perm(c.x, c.y, 0x5432), __byte_perm(c.y, one, 0x5432));
         }
-        *reinterpret_cast<uint2 *>(arow + (size_t)r * p.a_row_bytes + pos * 8) = make_uint2(v0, v1);
+      }
+    } else {
+      for (int r = tid >> 7; r < p.in_rows; r += kThreads >> 7) {
+        const int gy = gy0 + r;
+        const bool row_in = gy >= 0 && gy < p.h;
+        const unsigned short *q0 = reinterpret_cast<const unsigned short *>(smem + p.off_raw + (size_t)buf * p.raw_buf_bytes + (size_t)r * p.raw_row_bytes);
+        for (int pos = tid & 127; pos < wpix; pos += 128) {
+          const int px = pos - p.pad;
+          uint32_t v0 = 0u, v1 = one_hi;
+          if (row_in && px >= 0 && px < p.w) {
+            const unsigned short *q = q0 + px * p.c_in;
+            v0 = q[0];
+            if (p.c_in > 1) v0 |= (uint32_t)q[1] << 16;
+            if (p.c_in > 2) v1 |= q[2];
+            if (p.c_in > 3) v1 |= (uint32_t)q[3] << 16;
+          }
+          *reinterpret_cast<uint2 *>(arow + (size_t)r * p.a_row_bytes + pos * 8) = make_uint2(v0, v1);
+        }
       }
     }
     fence_proxy_async();                         // the rows are read by the tensor core (async proxy)
     __syncthreads();
     // ---- one lane issues the band's instructions: block (row ry, segment xt) = 3 instructions
     if (warp == 0) {
+      __syncwarp();
       if (elect_one()) {
         tc_fence_after();
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_pad >> 3) << 17) | (8u << 24);
-        const uint32_t desc_hi = (128u >> 4) | (1u << 14);     // 128 bytes between 8-row groups
-        const uint32_t a_base = smem_u32(arow) >> 4, a_row16 = (uint32_t)p.a_row_bytes >> 4;
-        const uint32_t b_base = ((smem_u32(bop) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);   // K chunks n_pad * 16 bytes apart
-        int blk = 0;
-        for (int ry = 0; ry < rows_out; ++ry)
-          for (int xt = 0; xt < p.xtiles; ++xt, ++blk) {
-            const uint32_t d = tmem_base + (uint32_t)(blk * p.n_pad);
-#pragma unroll
-            for (int r = 0; r < 3; ++r) {
-              // output X of this segment reads 32 bytes from byte 16 X of staged row 2 ry + r: K chunks 16 bytes apart
-              const uint32_t a_lo = ((a_base + (uint32_t)(2 * ry + r) * a_row16 + (uint32_t)(xt * 128)) & 0x3FFFu) | (1u << 16);
-              const uint32_t b_lo = b_base + (uint32_t)(r * 2 * p.n_pad);
-              umma_bf16(d, ((uint64_t)desc_hi << 32) | a_lo, ((uint64_t)desc_hi << 32) | b_lo, idesc, r != 0 ? 1u : 0u);
-            }
+        // output X of a segment reads 32 bytes from byte 16 X of staged row 2 ry + r (K chunks 16 bytes
+        // apart); the descriptors of a band differ in the start address only
+        uint32_t a_row = a_desc0;                // staged row 2 ry
+        uint32_t d = tmem_base;
+        for (int ry = 0; ry < rows_out; ++ry, a_row += 2 * a_row16) {
+          uint32_t a_seg = a_row;
+          for (int xt = 0; xt < p.xtiles; ++xt, a_seg += 128, d += (uint32_t)p.n_pad) {
+            umma_bf16(d, desc_hi64 | ((a_seg) & 0x3FFFu) | (1u << 16), b_desc[0], idesc, 0u);
+            umma_bf16(d, desc_hi64 | ((a_seg + a_row16) & 0x3FFFu) | (1u << 16), b_desc[1], idesc, 1u);
+            umma_bf16(d, desc_hi64 | ((a_seg + 2 * a_row16) & 0x3FFFu) | (1u << 16), b_desc[2], idesc, 1u);
           }
+        }
         umma_commit(&bar_mma);
       }
       __syncwarp();
     }
     if (tid == 0) {
+      bulk_wait_read0();                         // the previous band's store has read the output buffer
       done = mbar_wait(&bar_mma, (uint32_t)it & 1u, abort_flag, ws, 0xB0001u);
       tc_fence_before();
     }
     if (!__syncthreads_and(done)) break;
     tc_fence_after();
     // ---- read-out: thread = GEMM row = output pixel of the segment; the two warps of a lane quarter
-    // take the blocks in turn
-    for (int blk = warp >> 2; blk < rows_out * p.xtiles; blk += kThreads >> 7) {
-      const int ry = blk / p.xtiles, xt = blk - ry * p.xtiles;
-      const int X = xt * 128 + (tid & 127);
-      const bool valid = X < p.wo;
-      const size_t oi = (((size_t)img * p.ho + (Y0 + ry)) * p.wo + X) * p.c_out;
-      __nv_bfloat16 *dst = y + oi;
-      const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
-      for (int c0 = 0; c0 < p.c_out; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld32(trow + (uint32_t)(blk * p.n_pad + c0), v);
-        tmem_ld_wait();
+    // take the blocks in turn.  The band's output rows are contiguous in memory: they are put together in
+    // shared memory and leave as one bulk copy.
+    const bool plain = fold_bias && residual == nullptr;
+    int blk = 0;
+    for (int ry = 0; ry < rows_out; ++ry)
+      for (int xt = 0; xt < p.xtiles; ++xt, ++blk) {
+        if ((blk & ((kThreads >> 7) - 1)) != (warp >> 2)) continue;
+        const int X = xt * 128 + (tid & 127);
+        const bool valid = X < p.wo;
+        const uint32_t so = out_s + (uint32_t)((ry * p.wo + X) * p.c_out * 2);
+        for (int c0 = 0; c0 < p.c_out; c0 += 32) {
+          uint32_t v[32];
+          tmem_ld32(trow + (uint32_t)(blk * p.n_pad + c0), v);
+          tmem_ld_wait();
+          if (plain) {
 #pragma unroll
-        for (int g8 = 0; g8 < 4; ++g8) {
-          const int ch = c0 + 8 * g8;
-          uint4 ov = make_uint4(0u, 0u, 0u, 0u);
-          if (ch < p.c_out) {
-            float f[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g8 + i]) + bias_s[ch + i];
-            if (residual && valid) {
-              const uint4 rv = *reinterpret_cast<const uint4 *>(residual + oi + ch);
-              const __nv_bfloat162 *rbp = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+            for (int g8 = 0; g8 < 4; ++g8) {
+              uint4 ov;
+              __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                const float2 rf = __bfloat1622float2(rbp[i]);
-                f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(v[8 * g8 + 2 * i]), __uint_as_float(v[8 * g8 + 2 * i + 1]));
+                if (relu6) o2 = __hmin2(__hmax2(o2, zero2), six2);   // same bits as clamping before rounding
+                ob[i] = o2;
+              }
+              if (valid && c0 + 8 * g8 < p.c_out) sts128(so + (uint32_t)((c0 + 8 * g8) * 2), ov);
+            }
+          } else {
+            const size_t oi = (((size_t)img_now * p.ho + (Y0 + ry)) * p.wo + X) * p.c_out;
+#pragma unroll
+            for (int g8 = 0; g8 < 4; ++g8) {
+              const int ch = c0 + 8 * g8;
+              if (ch < p.c_out && valid) {
+                float f[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[8 * g8 + i]);
+                if (!fold_bias) {
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) f[i] += bias_s[ch + i];
+                }
+                if (residual) {
+                  const uint4 rv = *reinterpret_cast<const uint4 *>(residual + oi + ch);
+                  const __nv_bfloat162 *rbp = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    const float2 rf = __bfloat1622float2(rbp[i]);
+                    f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                  }
+                }
+                uint4 ov;
+                __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  __nv_bfloat162 o2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+                  if (relu6) o2 = __hmin2(__hmax2(o2, zero2), six2);
+                  ob[i] = o2;
+                }
+                sts128(so + (uint32_t)(ch * 2), ov);
               }
             }
-            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              __nv_bfloat162 o2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-              if (relu6) o2 = __hmin2(__hmax2(o2, zero2), six2);   // same bits as clamping before rounding
-              ob[i] = o2;
-            }
           }
-          *reinterpret_cast<uint4 *>(stage + lane * kStagePitch + g8 * 16) = ov;
         }
-        __syncwarp();
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int px = i * 8 + (lane >> 2), c = lane & 3;
-          const unsigned long long base = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, px);
-          if (((vmask >> px) & 1u) && c0 + c * 8 < p.c_out)
-            *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>((uintptr_t)base) + c0 + c * 8) =
-                *reinterpret_cast<const uint4 *>(stage + px * kStagePitch + c * 16);
-        }
-        __syncwarp();
       }
+    fence_proxy_async();                         // the output rows are read by the bulk copy (async proxy)
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      bulk_store(reinterpret_cast<uint8_t *>(y) + ((size_t)img_now * p.ho + Y0) * out_row_bytes, out_s,
+                 (uint32_t)((size_t)rows_out * out_row_bytes));
+      bulk_commit();
     }
   }
+  if (tid == 0) bulk_wait_all();                 // the last store has left shared memory and reached memory
   if (*abort_flag) {                             // a copy may still be in flight: give it time to land
     const unsigned long long t0 = globaltimer_ns();
     while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
@@ -247,13 +345,17 @@ bool s2_plan(int n, int h, int w, const dc_geom *g, S2Params *p) {
   p->xtiles = dc_div_up(wo, 128);
   // the last window of a row ends at pixel 2 (wo - 1) + 3 of the operand row
   if ((2 * (wo - 1) + 4) * 8 > p->a_row_bytes) return false;
-  // output rows per CTA: accumulators within 128 tensor-memory columns (four CTAs per SM), rows within ~40 KB
-  // (the read-out takes 32 columns at a time, so the last block may be read past its own columns)
+  // output rows per CTA: accumulators within the CTA's tensor-memory columns, buffers within its share of
+  // shared memory (the read-out takes 32 columns at a time, so the last block may be read past its own columns)
   const int tail = (int)dc_round_up((size_t)g->c_out, 32) - ko.n_pad;
-  int rb = (128 - tail) / (p->xtiles * ko.n_pad);
+  int rb = (kTmemCols - tail) / (p->xtiles * ko.n_pad);
   if (rb < 1) rb = 1;
-  while (rb > 1 && (2 * rb + 1) * (2 * p->raw_row_bytes + p->a_row_bytes) > 44 * 1024) --rb;
-  if (3 * (2 * p->raw_row_bytes + p->a_row_bytes) > 44 * 1024) return false;
+  auto buffers = [&](int rows) {
+    return (size_t)(2 * rows + 1) * (2 * p->raw_row_bytes + p->a_row_bytes) + (size_t)rows * wo * g->c_out * 2 +
+           3 * 2 * ko.n_pad * 16 + 1024;
+  };
+  while (rb > 1 && buffers(rb) > kSmemBudget) --rb;
+  if (buffers(rb) > kSmemBudget) return false;
   if (rb > ho) rb = ho;
   p->rb = rb;
   p->bands = dc_div_up(ho, rb);
@@ -267,10 +369,13 @@ bool s2_plan(int n, int h, int w, const dc_geom *g, S2Params *p) {
   p->off_raw = 0;
   p->raw_buf_bytes = (int)dc_round_up((size_t)p->in_rows * p->raw_row_bytes, 128);
   p->off_a = 2 * p->raw_buf_bytes;
-  // a block's 128 GEMM rows reach 2 KB + 32 bytes into (and, in the last row, past) an operand row
-  p->off_b = (int)dc_round_up((size_t)p->off_a + (size_t)p->in_rows * p->a_row_bytes + (size_t)p->xtiles * 2048 + 64, 128);
+  p->off_b = (int)dc_round_up((size_t)p->off_a + (size_t)p->in_rows * p->a_row_bytes, 128);
   p->off_stage = (int)dc_round_up((size_t)p->off_b + 3 * 2 * ko.n_pad * 16, 128);
-  p->smem_bytes = p->off_stage + (kThreads / 32) * 32 * kStagePitch + 128;
+  p->smem_bytes = p->off_stage + (int)dc_round_up((size_t)rb * wo * g->c_out * 2, 128) + 128;
+  // a block's 128 GEMM rows reach 2 KB + 32 bytes into an operand row whatever the row's length: the rows
+  // past the last output read what follows in shared memory (their results are not used); it must be there
+  const int reach = p->off_a + p->in_rows * p->a_row_bytes + p->xtiles * 2048 + 64 + 128;
+  if (p->smem_bytes < reach) p->smem_bytes = reach;
   if ((long long)n * p->bands >= (1ll << 30)) return false;
   return p->smem_bytes <= 100 * 1024;
 }
@@ -287,10 +392,12 @@ dc_status dc_launch_conv_stem_s2(const void *x, int n, int h, int w, const dc_ge
                                  cudaStream_t stream) {
   S2Params p;
   if (!s2_plan(n, h, w, g, &p)) return DC_ERR_UNSUPPORTED;
+  // rows enter and leave by bulk copies: without 16-byte aligned images the general stem kernel runs
+  if (((uintptr_t)x | (uintptr_t)y) & 15) return dc_launch_conv_stem(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, stream);
   p.act = (int)act;
   static unsigned char attr_done[kDcMaxDevices];
   DC_CUDA_OK(dc_set_max_smem_once(k_conv_stem_s2, 100 * 1024, attr_done));
-  const int total = n * p.bands, resident = 3 * dc_sm_count();
+  const int total = n * p.bands, resident = kCtasPerSm * dc_sm_count();
   k_conv_stem_s2<<<total < resident ? total : resident, kThreads, p.smem_bytes, stream>>>(p, (const __nv_bfloat16 *)x, w_packed, bias,
                                                                  (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                                                  (DcWsHeader *)workspace);
