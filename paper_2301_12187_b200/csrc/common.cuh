@@ -272,8 +272,11 @@ __host__ __device__ static inline bool dc_korder_decode(const KOrder &ko, int e,
   *pc = p;
   *ccg = ee / per;
   int rem = ee - *ccg * per;
-  *r = rem / ko.ns[p];
-  *s = ko.s0[p] + 2 * (rem - *r * ko.ns[p]);
+  // tap rows in the order even rows, odd rows: the general kernel keeps the even and the odd patch rows
+  // of a stride-2 layer apart, and the entries of a plane must come in the order of their addresses
+  const int ri = rem / ko.ns[p], ne = (ko.k + 1) >> 1;
+  *r = ri < ne ? 2 * ri : 2 * (ri - ne) + 1;
+  *s = ko.s0[p] + 2 * (rem - ri * ko.ns[p]);
   return true;
 }
 
@@ -303,7 +306,8 @@ __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc,
     int p = ((s - ko.pad) & 1);
     int per = ko.k * ko.ns[p];
     int base = (p == 0) ? 0 : ko.cg * ko.k * ko.ns[0];
-    e = base + ccg * per + r * ko.ns[p] + (s - ko.s0[p]) / 2;
+    const int ri = (r & 1) ? ((ko.k + 1) >> 1) + (r >> 1) : (r >> 1);      // even tap rows first
+    e = base + ccg * per + ri * ko.ns[p] + (s - ko.s0[p]) / 2;
   }
   return grp * ko.e_pad + e;
 }

@@ -10,7 +10,9 @@
 // address shifted by (r * patch_width + s) pixels: no im2col copy and no reload per tap.  Rows
 // of the GEMM enumerate the patch row-major INCLUDING its halo columns (pitch P), so a shifted
 // view stays a constant offset; rows that fall on halo columns are computed and dropped.
-// Stride 2 splits the patch by input-column parity (two sets of planes at half resolution).
+// Stride 2 splits the patch by input-column parity (two sets of planes at half resolution) and, inside
+// a plane, by row parity (even patch rows first): a tap then reads consecutive rows for consecutive
+// output rows, and the GEMM rows enumerate output pixels only.
 //
 // One tensor-core instruction takes K = 16 = two 16-byte chunks, addressed as "start" and
 // "start + LBO": any two chunk entries whose addresses increase can be paired, which is how
@@ -48,6 +50,7 @@ struct TcParams {
   int units_per_nt, total_units;
   int cg, ng, e_pad, cch, pcs;
   int wbox, rbox;             // patch columns (per parity), rows
+  int odd_rows_off;           // stride 2: byte offset of the odd patch rows inside a plane (even rows come first)
   int plane_stride, region_bytes, a_stage_bytes, b_stage_bytes;
   int stages, b_resident;
   int act;
@@ -206,12 +209,15 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
           const int gx = gx0 + gx_rel[i];
           const bool cv = (gx >= 0) && (gx < p.w);
           const char *src = grp_base + src_off[i];
-          uint32_t dst = stage + dst_off[i];
+          // stride 2: the even patch rows of a plane come first, then the odd ones, so that the rows one
+          // tap reads for consecutive output rows are consecutive
+          uint32_t dst_even = stage + dst_off[i], dst_odd = dst_even + (uint32_t)p.odd_rows_off;
           for (int r = 0; r < rows; ++r) {
             const bool v = cv && (r >= r_lo) && (r < r_hi);
-            cp_async16(dst, v ? (const void *)src : (const void *)x, v ? 16u : 0u);
+            const bool odd = (p.stride == 2) && (r & 1);
+            cp_async16(odd ? dst_odd : dst_even, v ? (const void *)src : (const void *)x, v ? 16u : 0u);
             src += row_stride;
-            dst += drow_stride;
+            if (odd) dst_odd += drow_stride; else dst_even += drow_stride;
           }
         }
         cp_async_arrive(&bar_full[s]);           // arrives by itself when this thread's copies have landed
@@ -426,7 +432,7 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
       p->cx0 = -g->pad; p->cy0 = -g->pad;
     } else {
       p->wbox = p->tw + dc_floor_div2(g->k - 1 - g->pad) - dc_floor_div2(-g->pad);
-      p->P = 2 * p->wbox;
+      p->P = p->wbox;
       p->cx0 = dc_floor_div2(-g->pad); p->cy0 = -g->pad;
     }
     // rows per tile: bounded by the accumulator blocks, the image, shared memory, and a target
@@ -450,6 +456,7 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   p->nxt = dc_div_up(p->wo, p->tw);
   p->mb = dc_div_up((p->th - 1) * p->P + p->tw, 128);
   if (p->mb > mb_max) return false;
+  p->odd_rows_off = (g->stride == 2) ? ((p->rbox + 1) / 2) * p->wbox * 16 : 0;
   p->plane_stride = padded_plane_units(p->rbox * p->wbox + 1, ko.cg) * 16;
   p->region_bytes = (int)dc_round_up((size_t)ko.cg * p->plane_stride, 128);
   p->a_stage_bytes = ko.pcs * p->region_bytes;
@@ -496,11 +503,15 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
       int pc, ccg, r, s;
       if (dc_korder_decode(ko, 2 * j + q, &pc, &ccg, &r, &s)) {
         int sx = (g->stride == 1) ? s : dc_floor_div2(s - g->pad) - dc_floor_div2(-g->pad);
-        off[q] = (uint32_t)(pc * p->region_bytes + ccg * p->plane_stride + (r * p->wbox + sx) * 16);
+        const int row = (g->stride == 1) ? r : (r >> 1);       // stride 2: row r / 2 of the rows of r's parity
+        off[q] = (uint32_t)(pc * p->region_bytes + ccg * p->plane_stride + (r & (g->stride - 1)) * p->odd_rows_off +
+                            (row * p->wbox + sx) * 16);
       } else if (q == 1) {
         off[1] = off[0] + 16;
       }
     }
+    // the second chunk is addressed as a 14-bit distance in 16-byte units above the first
+    if (off[1] <= off[0] || ((off[1] - off[0]) >> 4) > 0x3FFFu) return false;
     p->a_desc_lo[j] = (off[0] >> 4) | (((off[1] - off[0]) >> 4) << 16);
   }
   return true;

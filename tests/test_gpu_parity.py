@@ -393,6 +393,10 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (32, 16, 5, 2, 2, 1, 30, 44, "k_conv_tc_pairrows"),     # stride 2, even padding, 5x5
     (16, 24, 3, 2, 0, 2, 17, 36, "k_conv_tc_pairrows"),     # stride 2, no padding, odd height
     (40, 32, 3, 2, 1, 2, 28, 28, "k_conv_tc"),              # stride 2 on parity planes (more than 32 channels)
+    (96, 144, 5, 2, 2, 1, 56, 56, "k_conv_tc"),             # the widest stride-2 merged layer of the network: several tiles per image
+    (48, 64, 7, 2, 3, 1, 31, 44, "k_conv_tc"),              # 7x7 stride 2, odd height: four even and three odd tap rows
+    (48, 24, 5, 2, 1, 2, 22, 26, "k_conv_tc"),              # 5x5 stride 2 with padding 1: odd tap columns lead
+    (72, 48, 3, 2, 0, 1, 17, 150, "k_conv_tc"),             # stride 2 without padding, two column strips
     (32, 16, 1, 1, 0, 2, 20, 24, "k_conv_tc_pairrows"),     # 1x1: one instruction per 32-byte K step
     (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc_rows"),         # 1x1 expansion from few channels: one half-filled plane
     (16, 96, 1, 1, 0, 1, 40, 112, "k_conv_tc_rows"),        # 1x1 expansion from 16 channels, row tiles
