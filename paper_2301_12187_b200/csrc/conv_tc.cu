@@ -56,6 +56,7 @@ struct TcParams {
   int act;
   int cx0, cy0;               // patch origin: x = xt*tw + cx0 (parity-plane columns), y = y0*stride + cy0
   int acc_cols, tmem_cols;
+  int acc_slots;              // accumulator sets in tensor memory: 2 (epilogue of a tile under the next tile's MMAs) or 1
   int bulk_out, out_tile_bytes;
   int off_b, off_a, off_out, off_bias;  // offsets in dynamic shared memory
   int smem_bytes;
@@ -211,13 +212,24 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
           const char *src = grp_base + src_off[i];
           // stride 2: the even patch rows of a plane come first, then the odd ones, so that the rows one
           // tap reads for consecutive output rows are consecutive
-          uint32_t dst_even = stage + dst_off[i], dst_odd = dst_even + (uint32_t)p.odd_rows_off;
-          for (int r = 0; r < rows; ++r) {
-            const bool v = cv && (r >= r_lo) && (r < r_hi);
-            const bool odd = (p.stride == 2) && (r & 1);
-            cp_async16(odd ? dst_odd : dst_even, v ? (const void *)src : (const void *)x, v ? 16u : 0u);
-            src += row_stride;
-            if (odd) dst_odd += drow_stride; else dst_even += drow_stride;
+          uint32_t dst = stage + dst_off[i];
+          if (p.stride == 1) {
+            for (int r = 0; r < rows; ++r) {
+              const bool v = cv && (r >= r_lo) && (r < r_hi);
+              cp_async16(dst, v ? (const void *)src : (const void *)x, v ? 16u : 0u);
+              src += row_stride;
+              dst += drow_stride;
+            }
+          } else {
+            uint32_t dst_odd = dst + (uint32_t)p.odd_rows_off;
+            for (int r = 0; r < rows; r += 2) {
+              const bool v0 = cv && (r >= r_lo) && (r < r_hi), v1 = cv && (r + 1 >= r_lo) && (r + 1 < r_hi);
+              cp_async16(dst, v0 ? (const void *)src : (const void *)x, v0 ? 16u : 0u);
+              if (r + 1 < rows) cp_async16(dst_odd, v1 ? (const void *)(src + row_stride) : (const void *)x, v1 ? 16u : 0u);
+              src += 2 * row_stride;
+              dst += drow_stride;
+              dst_odd += drow_stride;
+            }
           }
         }
         cp_async_arrive(&bar_full[s]);           // arrives by itself when this thread's copies have landed
@@ -239,7 +251,7 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
         cur += t.th;
         const int rows = (t.th - 1) * p.P + p.tw;
         const int nblk = (rows + 127) >> 7;
-        const uint32_t a = tile_i & 1, aph = (tile_i >> 1) & 1;
+        const uint32_t a = p.acc_slots == 2 ? (tile_i & 1) : 0u, aph = p.acc_slots == 2 ? ((tile_i >> 1) & 1) : (tile_i & 1);
         if (!warp_wait(&bar_accempty[a], aph ^ 1, abort_flag, ws, 0x20000u | a)) goto mma_done;
         tc_fence_after();
         const uint32_t d0 = tmem_base + a * (uint32_t)p.acc_cols;
@@ -287,8 +299,8 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
       const int nblk = (rows + 127) >> 7;
       const int x0 = t.xt * p.tw;
       const int tw_valid = (p.wo - x0 < p.tw) ? p.wo - x0 : p.tw;
-      const uint32_t a = tile_i & 1, aph = (tile_i >> 1) & 1;
-      uint8_t *obuf = smem_out + (size_t)a * p.out_tile_bytes;
+      const uint32_t a = p.acc_slots == 2 ? (tile_i & 1) : 0u, aph = p.acc_slots == 2 ? ((tile_i >> 1) & 1) : (tile_i & 1);
+      uint8_t *obuf = smem_out + (size_t)(tile_i & 1) * p.out_tile_bytes;
       if (p.bulk_out && elected) bulk_wait_read1();   // the store that last used this buffer has read it
       // all 128 epilogue threads pass or leave together, so nobody is left alone at a named barrier
       if (!epi_all(mbar_wait(&bar_accfull[a], aph, abort_flag, ws, 0x40000u | a))) break;
@@ -406,11 +418,19 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   p->cg = ko.cg; p->ng = ko.ng; p->e_pad = ko.e_pad; p->cch = ko.cch; p->pcs = ko.pcs;
   p->nnt = dc_div_up(ko.n_pad, 256);
   p->n_tile = (int)dc_round_up((size_t)dc_div_up(ko.n_pad, p->nnt), 16);
-  int mb_max = 256 / p->n_tile;
-  if (mb_max > 8) mb_max = 8;
-  if (mb_max < 1) return false;
   p->b_stage_bytes = ko.e_pad * p->n_tile * 16;
   p->b_resident = (ko.ng == 1 && p->nnt == 1) ? 1 : 0;
+  // Two accumulator sets let the epilogue of a tile run under the next tile's MMAs.  Wide outputs leave
+  // room for one 128-row block per set only; when the weights are streamed per (tile, channel group)
+  // as well, one set of up to three blocks is better: a weight stage then serves three times the rows.
+  int mb_max = 256 / p->n_tile;
+  p->acc_slots = 2;
+  if (mb_max < 2 && !p->b_resident && 512 / p->n_tile >= 2) {
+    p->acc_slots = 1;
+    mb_max = 512 / p->n_tile;
+  }
+  if (mb_max > 8) mb_max = 8;
+  if (mb_max < 1) return false;
 
   if (flat) {
     long long pixels = (long long)n * h * w;
@@ -438,7 +458,7 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
     // rows per tile: bounded by the accumulator blocks, the image, shared memory, and a target
     // of about six tiles per CTA so that load, MMA and epilogue overlap
     long long total_rows = (long long)n * ho * dc_div_up(wo, p->tw) * p->nnt;
-    int th_target = (int)(total_rows / ((long long)n_sm * 6));
+    int th_target = (int)(total_rows / ((long long)n_sm * (p->acc_slots == 2 ? 6 : 2)));
     if (th_target < 1) th_target = 1;
     int th = (mb_max * 128 - p->tw) / p->P + 1;
     if (th < 1) return false;
@@ -462,7 +482,7 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
   p->a_stage_bytes = ko.pcs * p->region_bytes;
   p->acc_cols = p->mb * p->n_tile;
   int cols = 32;
-  while (cols < 2 * p->acc_cols) cols *= 2;
+  while (cols < p->acc_slots * p->acc_cols) cols *= 2;
   if (cols > 512) return false;
   p->tmem_cols = cols;
   long long units = (long long)p->n_img * p->nxt * p->ho;
