@@ -33,6 +33,17 @@ struct StencilParams {
 
 __device__ unsigned int g_dw_status;             // DC_ERR_TIMEOUT once a wait of these kernels ran out
 
+__device__ __forceinline__ uint4 lds_u4(uint32_t a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float4 lds_f4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+  return v;
+}
+
 template <int K, int S>
 __global__ void __launch_bounds__(kThreads, 2)
 k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ StencilParams p,
@@ -77,9 +88,12 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int imgs_valid = p.n_img - img0 < p.ni ? p.n_img - img0 : p.ni;
   const int per_img = rows_valid * xtiles;
   const int items = imgs_valid * per_img;
-  const float *bias_s = w_s + K * K * p.ct + cv * kV;
-  const size_t row_pitch = (size_t)p.in_w * p.ct, img_pitch = (size_t)p.in_rows * row_pitch;   // elements
-  const __nv_bfloat16 *patch = reinterpret_cast<const __nv_bfloat16 *>(smem) + cv * kV;
+  // shared-memory addresses as 32-bit offsets (the loop below is bound by its instruction stream)
+  const uint32_t ct2 = (uint32_t)p.ct * 2u, ct4 = (uint32_t)p.ct * 4u;
+  const uint32_t w_sa = smem_u32(w_s) + (uint32_t)(cv * kV) * 4u;         // this thread's 8 channels of tap 0
+  const uint32_t bias_sa = w_sa + (uint32_t)(K * K) * ct4;
+  const uint32_t row_pitch = (uint32_t)p.in_w * ct2, img_pitch = (uint32_t)p.in_rows * row_pitch;   // bytes
+  const uint32_t patch_sa = smem_u32(smem) + (uint32_t)(cv * kV) * 2u;
 #pragma unroll 1
   for (int item = (int)threadIdx.x / cvt; item < items; item += kThreads / cvt) {
     const int il = item / per_img, rem = item - il * per_img;
@@ -89,29 +103,31 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // moved, which one scalar FMA per instruction would not keep up with
     float2 acc[TX][kV / 2];
     {
-      const float4 b0 = *reinterpret_cast<const float4 *>(bias_s), b1 = *reinterpret_cast<const float4 *>(bias_s + 4);
+      const float4 b0 = lds_f4(bias_sa), b1 = lds_f4(bias_sa + 16u);
 #pragma unroll
       for (int o = 0; o < TX; ++o) {
         acc[o][0] = make_float2(b0.x, b0.y); acc[o][1] = make_float2(b0.z, b0.w);
         acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
       }
     }
-    const __nv_bfloat16 *prow = patch + il * img_pitch + (size_t)(ry * S) * row_pitch + (size_t)(X0 * S) * p.ct;
+    // columns past the patch's last one only feed outputs past the row's end, which are not stored
+    uint32_t col_off[NJ];
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) col_off[j] = (X0 * S + j < p.in_w ? (uint32_t)j : 0u) * ct2;
+    uint32_t prow = patch_sa + (uint32_t)il * img_pitch + (uint32_t)(ry * S) * row_pitch + (uint32_t)(X0 * S) * ct2;
+    uint32_t wrow = w_sa;
 #pragma unroll 1
-    for (int r = 0; r < K; ++r) {
+    for (int r = 0; r < K; ++r, prow += row_pitch, wrow += (uint32_t)K * ct4) {
       float2 wr[K][kV / 2];
 #pragma unroll
       for (int sx = 0; sx < K; ++sx) {
-        const float *wp = w_s + (r * K + sx) * p.ct + cv * kV;
-        const float4 w0 = *reinterpret_cast<const float4 *>(wp), w1 = *reinterpret_cast<const float4 *>(wp + 4);
+        const float4 w0 = lds_f4(wrow + (uint32_t)sx * ct4), w1 = lds_f4(wrow + (uint32_t)sx * ct4 + 16u);
         wr[sx][0] = make_float2(w0.x, w0.y); wr[sx][1] = make_float2(w0.z, w0.w);
         wr[sx][2] = make_float2(w1.x, w1.y); wr[sx][3] = make_float2(w1.z, w1.w);
       }
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
-        // columns past the patch's last one only feed outputs past the row's end, which are not stored
-        const int col = X0 * S + j < p.in_w ? j : 0;
-        const uint4 raw = *reinterpret_cast<const uint4 *>(prow + (size_t)r * row_pitch + (size_t)col * p.ct);
+        const uint4 raw = lds_u4(prow + col_off[j]);
         const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&raw);
         float2 xv[kV / 2];
 #pragma unroll
