@@ -71,6 +71,35 @@ def test_static_scratch_merge_matches_workspace_merge_twice_in_a_row():
         assert torch.equal(p0, p1)
 
 
+def test_static_scratch_merge_inside_a_captured_graph():
+    """After a first call outside capture (it looks up the scratch array's address), the call only queues
+    kernels on the stream: captured in a CUDA graph and replayed, it gives the same bits every time."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2301_12187_b200 import dc
+    case = I.chain_case(1)
+    layers = [dc.DeviceLayer(s) for s in case.layers]
+    g, ws_bytes = dc.merge_query(layers, case.residuals)
+    ref_w = torch.empty((g.c_out, g.c_in, g.k, g.k), dtype=torch.float32, device="cuda")
+    ref_b = torch.empty((g.c_out,), dtype=torch.float32, device="cuda")
+    ref_p = torch.zeros(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
+    dc.merge_chain(layers, case.residuals, ref_w, ref_b, ref_p, dc.BF16, torch.empty(ws_bytes, dtype=torch.uint8, device="cuda"))
+    wm, bm, packed = torch.empty_like(ref_w), torch.empty_like(ref_b), torch.zeros_like(ref_p)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        dc.merge_chain_static(layers, case.residuals, wm, bm, packed, dc.BF16)       # warm-up, outside capture
+        st.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            dc.merge_chain_static(layers, case.residuals, wm, bm, packed, dc.BF16)
+        for _ in range(2):
+            wm.fill_(float("nan")); bm.fill_(float("nan")); packed.zero_()
+            graph.replay()
+            st.synchronize()
+            assert rel(wm, ref_w) <= TOL_W and rel(bm, ref_b) <= TOL_W
+            assert torch.equal(packed, ref_p)
+
+
 def test_static_scratch_merge_refuses_runs_beyond_its_capacity():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
