@@ -90,7 +90,8 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_base) + 1023) & ~uintptr_t(1023));
   uint8_t *smem_b = smem + p.off_b;
   uint8_t *smem_a = smem + p.off_a;              // 1024-byte aligned stages (the swizzle pattern repeats every 1024 bytes)
-  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
+  uint8_t *smem_ones = smem + p.off_bias;        // 8 lines of the constant operand (1024-byte aligned)
+  uint8_t *smem_bias = smem_ones + 1024;         // [n_pad][16 bytes]: bias as two bf16 terms, then n_tile zero rows
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile uint32_t *abort_flag = &sh.abort;
@@ -165,8 +166,27 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
       tmem_relinquish();
     } else if (warp >= kFirstEpiWarp) {
-      for (int t = (int)threadIdx.x - kFirstEpiWarp * 32; t < p.n_pad; t += kEpiWarps * 32)
-        bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
+      // The bias is added by the tensor core: one instruction per block multiplies a constant operand
+      // (1.0 in the first two K elements of every line) with [bias as bf16, its bf16 remainder, 0, ...]
+      // per output channel (exact to 16 mantissa bits) before the block's other instructions accumulate.
+      // The constant operand is one 8-line group read sixteen times (group stride 0); with the 128-byte
+      // swizzle the first 16-byte chunk of line r sits at chunk r.
+      const int t0 = (int)threadIdx.x - kFirstEpiWarp * 32;
+      for (int t = t0; t < 64; t += kEpiWarps * 32) {
+        const int r = t >> 3, c = t & 7;
+        reinterpret_cast<uint4 *>(smem_ones)[t] = make_uint4(c == r ? 0x3F803F80u : 0u, 0u, 0u, 0u);
+      }
+      for (int t = t0; t < p.n_pad + p.n_tile; t += kEpiWarps * 32) {
+        uint32_t w0 = 0u;
+        if (bias && t < p.c_out) {
+          const float b = bias[t];
+          const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+          w0 = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+        }
+        reinterpret_cast<uint4 *>(smem_bias)[t] = make_uint4(w0, 0u, 0u, 0u);
+      }
+      fence_proxy_async();                       // both are read by the tensor core (async proxy)
     }
     tc_fence_before();
     bar_sync(kBarConsumers, kConsumerThreads);
@@ -182,6 +202,8 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t b_hi = (128u >> 4) | (1u << 14);                 // no swizzle: 128 bytes between 8-row groups
       const uint32_t a_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // 128-byte swizzle: 1024 bytes between 8-row groups
       const uint32_t a_row0 = smem_u32(smem_a) >> 4, b_row0 = smem_u32(smem_b) >> 4;
+      const uint32_t bias_row0 = smem_u32(smem_bias) >> 4, zero_row = bias_row0 + (uint32_t)p.n_pad;
+      const uint64_t ones_desc = ((uint64_t)((1u << 14) | (2u << 29)) << 32) | (uint64_t)(((smem_u32(smem_ones) >> 4) & 0x3FFFu) | (1u << 16));
       int sa = 0, sb = 0;
       uint32_t pa = 0, pb = 0;
       uint32_t acc_ph[2] = {1u, 1u};             // parity this warp waits for on acc_empty (first use passes)
@@ -192,7 +214,16 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!warp_wait(&sh.acc_empty[set], acc_ph[set], abort_flag, ws, 0x30000u | set)) break;
         acc_ph[set] ^= 1u;
         tc_fence_after();
-        bool first = true;
+        {
+          // bias first (needs no load): it also initialises the accumulators of this warp's blocks
+          Item iq;
+          iq.of(p, item0 + it);
+          const uint32_t bias_row = bias_row0 + (uint32_t)(iq.nt * p.n_tile);
+          const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)((bias_row & 0x3FFFu) | ((zero_row - bias_row) << 16));
+#pragma unroll 1
+          for (int b = mw; b < p.mb; b += kMmaWarps)
+            if (leader) umma_bf16(tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile), ones_desc, bd, idesc, 0u);
+        }
 #pragma unroll 1
         for (int g = 0; g < p.planes && ok; ++g) {
           if (!warp_wait(&sh.a_full[sa], pa, abort_flag, ws, 0x40000u | sa)) { ok = false; break; }
@@ -212,7 +243,6 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               uint32_t a_lo = ((a_stage + (uint32_t)(b * 1024 + r * p.wbox * 8)) & 0x3FFFu) | (1u << 16);
               uint32_t b_lo = (b_stage & 0x3FFFu) | ((uint32_t)p.n_tile << 16);
               const uint32_t b_inc = 2u * (uint32_t)p.n_tile;
-              uint32_t accum = first ? 0u : 1u;
 #pragma unroll 1
               for (int s = 0; s < p.k; ++s, a_lo += 8u) {
 #pragma unroll
@@ -220,14 +250,12 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   if (sl < nsl) {
                     const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + 2u * sl);
                     const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-                    if (leader) umma_bf16(d, ad, bd, idesc, accum);
-                    accum = 1u;
+                    if (leader) umma_bf16(d, ad, bd, idesc, 1u);
                     b_lo += b_inc;
                   }
                 }
               }
             }
-            first = false;
             if (leader) umma_commit(&sh.b_empty[sb]);      // this warp is done with the weight stage
             if (++sb == p.sb) { sb = 0; pb ^= 1; }
           }
@@ -269,15 +297,11 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __nv_bfloat16 *dst = y + pix * p.c_out + ch0;
           const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out + ch0 : nullptr;
           const uint32_t taddr = tmem_row + (uint32_t)((set * p.mb + b) * p.n_tile);
-          // eight channels of this thread's pixel: bias, skip input, activation -> eight bf16
+          // eight channels of this thread's pixel: skip input, activation -> eight bf16
           auto cook8 = [&](const uint32_t *v, int ch) {
-            const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch);
-            const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch0 + ch + 4);
             float f[8];
-            f[0] = __uint_as_float(v[0]) + b0.x; f[1] = __uint_as_float(v[1]) + b0.y;
-            f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
-            f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
-            f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[i]);     // the bias is in the accumulator already
             if (rp && valid) {
               const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
               const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
@@ -433,7 +457,7 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   // reach up to ~200 lines (25 KB) past its stage; behind the last activation stage that lands in
   // the weight stages, which are larger (what is read there only feeds rows that are dropped).
   p->off_bias = 0;
-  p->off_stage = (int)dc_round_up((size_t)p->n_pad * 4, 128);
+  p->off_stage = (int)dc_round_up((size_t)1024 + (size_t)(p->n_pad + p->n_tile) * 16, 128);   // constant operand, bias rows, zero rows
   p->off_a = (int)dc_round_up((size_t)p->off_stage + kEpiWarps * 32 * kStagePitch, 1024);
   // rings: weights first (they are the larger stream), then activation planes
   int sa = 2, sb = 2;
