@@ -184,13 +184,9 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
 #pragma unroll
           for (int ch = 0; ch < CO8; ch += 8) {
             if (ch < p.c_out) {
-              float f[8];
-              const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
-              const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
-              f[0] = __uint_as_float(v[ch]) + b0.x; f[1] = __uint_as_float(v[ch + 1]) + b0.y;
-              f[2] = __uint_as_float(v[ch + 2]) + b0.z; f[3] = __uint_as_float(v[ch + 3]) + b0.w;
-              f[4] = __uint_as_float(v[ch + 4]) + b1.x; f[5] = __uint_as_float(v[ch + 5]) + b1.y;
-              f[6] = __uint_as_float(v[ch + 6]) + b1.z; f[7] = __uint_as_float(v[ch + 7]) + b1.w;
+              float f[8];                          // the bias is in the accumulator already
+#pragma unroll
+              for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[ch + i]);
               if (RES) {
                 const uint4 rv = *reinterpret_cast<const uint4 *>(rp + e * p.c_out + ch);
                 const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
@@ -285,17 +281,13 @@ __device__ __noinline__ void epilogue_wide(const PairParams &p, Shared &sh, DcWs
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.slot_empty[slot]);
         }
-        const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
-        const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           const uint32_t *v = e ? v1 : v0;
           if (e ? valid1 : valid0) {
-            float f[8];
-            f[0] = __uint_as_float(v[0]) + b0.x; f[1] = __uint_as_float(v[1]) + b0.y;
-            f[2] = __uint_as_float(v[2]) + b0.z; f[3] = __uint_as_float(v[3]) + b0.w;
-            f[4] = __uint_as_float(v[4]) + b1.x; f[5] = __uint_as_float(v[5]) + b1.y;
-            f[6] = __uint_as_float(v[6]) + b1.z; f[7] = __uint_as_float(v[7]) + b1.w;
+            float f[8];                            // the bias is in the accumulator already
+#pragma unroll
+            for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[i]);
             if (rp) {
               const uint4 rv = *reinterpret_cast<const uint4 *>(rp + e * p.c_out + ch);
               const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
@@ -347,7 +339,9 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
   uint8_t *smem_b = smem + p.off_b;
   uint8_t *smem_a = smem + p.off_a;              // 1024-byte aligned stages (the swizzle pattern repeats every 1024 bytes)
   uint8_t *smem_out = smem + p.off_out;
-  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
+  float *bias_s = nullptr;                       // (the read-out no longer adds the bias)
+  uint8_t *smem_ones = smem + p.off_bias;        // 8 lines of the constant operand (1024-byte aligned)
+  uint8_t *smem_bias = smem_ones + 1024;         // [n_pad][16 bytes]: bias as two bf16 terms, then n_pad zero rows
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile uint32_t *abort_flag = &sh.abort;
@@ -415,8 +409,28 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
       tmem_alloc(&sh.tmem_base, (uint32_t)p.tmem_cols);
       tmem_relinquish();
     } else if (warp >= kFirstEpiWarp) {
-      const int t = (int)threadIdx.x - kFirstEpiWarp * 32;
-      if (t < p.co8) bias_s[t] = (bias && t < p.c_out) ? bias[t] : 0.f;
+      // The bias is added by the tensor core: one instruction per block multiplies a constant operand
+      // (1.0 in the first two K elements of every line) with [bias as bf16, its bf16 remainder, 0, ...]
+      // per accumulator column (exact to 16 mantissa bits) before the block's other instructions
+      // accumulate.  The constant operand is one 8-line group read sixteen times (group stride 0); with
+      // the 128-byte swizzle the first 16-byte chunk of line r sits at chunk r.  Column n belongs to
+      // output channel n mod co8 (the second pixel's columns follow the first's).
+      const int t0 = (int)threadIdx.x - kFirstEpiWarp * 32;
+      const int ncol = (p.stride == 1 ? 2 : 1) * p.co8;
+      for (int t = t0; t < 64; t += kEpiWarps * 32)
+        reinterpret_cast<uint4 *>(smem_ones)[t] = make_uint4((t & 7) == (t >> 3) ? 0x3F803F80u : 0u, 0u, 0u, 0u);
+      for (int t = t0; t < 2 * p.n_pad; t += kEpiWarps * 32) {
+        uint32_t w0 = 0u;
+        const int ch = t < ncol ? (t >= p.co8 ? t - p.co8 : t) : p.c_out;
+        if (bias && ch < p.c_out) {
+          const float b = bias[ch];
+          const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+          w0 = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+        }
+        reinterpret_cast<uint4 *>(smem_bias)[t] = make_uint4(w0, 0u, 0u, 0u);
+      }
+      fence_proxy_async();                       // both are read by the tensor core (async proxy)
     }
     tc_fence_before();
     bar_sync(kBarConsumers, kConsumerThreads);
@@ -438,6 +452,8 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
       const uint32_t b_lo0 = ((smem_u32(smem_b) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16);
       const uint32_t b_step = 2u * (uint32_t)p.n_pad;
       const uint32_t a_row0 = smem_u32(smem_a) >> 4, a_stage_rows = (uint32_t)p.a_stage_bytes >> 4;
+      const uint64_t ones_desc = ((uint64_t)((1u << 14) | (2u << 29)) << 32) | (uint64_t)(((smem_u32(smem_ones) >> 4) & 0x3FFFu) | (1u << 16));
+      const uint64_t bias_desc = ((uint64_t)b_hi << 32) | (uint64_t)(((smem_u32(smem_bias) >> 4) & 0x3FFFu) | ((uint32_t)p.n_pad << 16));
       bool ok = warp_wait(&sh.weights, 0, abort_flag, ws, 0x70000u);
       int s = 0;                                 // stage and its phase, accumulator slot and its phase
       uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
@@ -459,11 +475,12 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
           const uint32_t a_add = a_row + (uint32_t)(b * 1024);    // 128 rows of 128 bytes, in 16-byte units
           uint32_t b_lo = b_lo0;
+          if (leader) umma_bf16(d, ones_desc, bias_desc, idesc, 0u);     // the bias initialises the accumulator
 #pragma unroll 2
           for (int j = 0; j < p.nmma; ++j, b_lo += b_step) {
             const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(p.a_lo[j] + a_add);
             const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-            if (leader) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+            if (leader) umma_bf16(d, ad, bd, idesc, 1u);
           }
           if (leader) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
           slot += (uint32_t)p.mma_warps;
@@ -566,8 +583,8 @@ bool pair_plan(int n, int h, int w, const dc_geom *g, int n_sm, PairParams *p) {
   p->bulk_out = (p->nxt == 1 && ko.co8 <= 32) ? 1 : 0;     // wider outputs are stored straight from registers
   p->out_buf_bytes = p->bulk_out ? (int)dc_round_up((size_t)(S == 1 ? 64 : 32) * g->c_out * 2, 128) : 0;
   p->off_b = 0;
-  p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 128);
-  p->off_a = (int)dc_round_up((size_t)p->off_bias + 1024, 1024);
+  p->off_bias = (int)dc_round_up((size_t)p->b_bytes, 1024);                       // constant operand, bias rows, zero rows
+  p->off_a = (int)dc_round_up((size_t)p->off_bias + 1024 + 2 * (size_t)p->n_pad * 16, 1024);
   // the output staging buffers follow the stages and double as the room a block's last rows may
   // reach into past the last stage (what is read there only feeds rows that are dropped)
   const long long tail_bytes = kEpiWarps * p->out_buf_bytes > kSlack ? kEpiWarps * p->out_buf_bytes : kSlack;
