@@ -99,8 +99,12 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
     mbar_init(&bar_load[1], 1);
     mbar_init(&bar_mma, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    issue_load(img, band, 0);
   }
+  // Nothing above touched global memory; everything below may.  Tensor memory is allocated after this
+  // point on purpose: a CTA that held columns while it waits here for the previous kernel could keep a
+  // CTA of that kernel on the same SM from getting its own.
+  dc_pdl_enter();
+  if (tid == 0) issue_load(img, band, 0);
   if (warp == 0) {
     tmem_alloc(&tmem_base_s, (uint32_t)p.tmem_cols);
     tmem_relinquish();
@@ -398,8 +402,8 @@ dc_status dc_launch_conv_stem_s2(const void *x, int n, int h, int w, const dc_ge
   static unsigned char attr_done[kDcMaxDevices];
   DC_CUDA_OK(dc_set_max_smem_once(k_conv_stem_s2, 100 * 1024, attr_done));
   const int total = n * p.bands, resident = kCtasPerSm * dc_sm_count();
-  k_conv_stem_s2<<<total < resident ? total : resident, kThreads, p.smem_bytes, stream>>>(p, (const __nv_bfloat16 *)x, w_packed, bias,
-                                                                 (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
-                                                                 (DcWsHeader *)workspace);
-  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+  const cudaError_t le = dc_launch_pdl(k_conv_stem_s2, dim3(total < resident ? total : resident), dim3(kThreads),
+                                       (size_t)p.smem_bytes, stream, p, (const __nv_bfloat16 *)x, w_packed, bias,
+                                       (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }

@@ -119,6 +119,10 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
     for (int a = 0; a < 2; ++a) { mbar_init(&bar_accfull[a], 1); mbar_init(&bar_accempty[a], 128); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // Nothing above touched global memory; everything below may.  Tensor memory is allocated after this
+  // point on purpose: a CTA that held columns while it waits here for the previous kernel could keep a
+  // CTA of that kernel on the same SM from getting its own.
+  dc_pdl_enter();
   if (warp == 4) {
     tmem_alloc(&tmem_base_s, (uint32_t)p.tmem_cols);
     tmem_relinquish();
@@ -554,8 +558,8 @@ dc_status dc_launch_conv_tc(const void *x, int n, int h, int w, const dc_geom *g
   static unsigned char attr_done[kDcMaxDevices];
   DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc, kSmemBudget, attr_done));
   int grid = p.total_units < n_sm ? p.total_units : n_sm;
-  k_conv_tc<<<grid, kThreads, p.smem_bytes, stream>>>(w_packed, p, (const __nv_bfloat16 *)x, bias,
-                                                     (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
-                                                     (DcWsHeader *)workspace);
-  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+  const cudaError_t le = dc_launch_pdl(k_conv_tc, dim3(grid), dim3(kThreads), (size_t)p.smem_bytes, stream, w_packed, p,
+                                       (const __nv_bfloat16 *)x, bias, (const __nv_bfloat16 *)residual,
+                                       (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }

@@ -109,6 +109,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     else if (t == 96) { sh.abort = 0; prefetch_tensormap(&map_a); did = true; }
     if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  dc_pdl_enter();                                // nothing above touched global memory; everything below may
   __syncthreads();
 
   if (warp == 0) {
@@ -505,7 +506,8 @@ dc_status dc_launch_conv_rows(const void *x, int n, int h, int w, const dc_geom 
   }
   static unsigned char attr_done[kDcMaxDevices];
   DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_rows, kSmemBudget, attr_done));
-  k_conv_tc_rows<<<p.grid, kThreads, p.smem_bytes, stream>>>(map_a, p, w_packed, bias, (const __nv_bfloat16 *)residual,
-                                                            (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
-  return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+  const cudaError_t le = dc_launch_pdl(k_conv_tc_rows, dim3(p.grid), dim3(kThreads), (size_t)p.smem_bytes, stream, map_a, p,
+                                       w_packed, bias, (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
+                                       (DcWsHeader *)workspace);
+  return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }

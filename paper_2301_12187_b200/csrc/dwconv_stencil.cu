@@ -67,6 +67,9 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     mbar_init(&bar, 1);
     abort_word = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  dc_pdl_enter();                                // nothing above touched global memory; everything below may
+  if (threadIdx.x == 0) {
     mbar_arrive_expect_tx(&bar, (uint32_t)p.box_bytes);
     // coordinates may be negative or reach past the tensor: those elements arrive as zeros
     tma_load_4d(smem_u32(smem), &map_x, &bar, c0, -p.pad, y0 * S - p.pad, img0);
@@ -242,7 +245,8 @@ dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, in
   do {                                                                                                    \
     static unsigned char attr_done[kDcMaxDevices];                                                        \
     DC_CUDA_OK(dc_set_max_smem_once(k_dwconv_stencil<KK, SS>, kTileBytes + 8 * 1024, attr_done));         \
-    k_dwconv_stencil<KK, SS><<<grid, kThreads, smem, st>>>(map_x, p, wp, bias, yp);                       \
+    if (dc_launch_pdl(k_dwconv_stencil<KK, SS>, dim3(grid), dim3(kThreads), (size_t)smem, st, map_x, p, wp, bias, yp) != cudaSuccess) \
+      return DC_ERR_CUDA;                                                                                 \
   } while (0)
   if (k == 3 && stride == 1) DC_DW_LAUNCH(3, 1);
   else if (k == 3) DC_DW_LAUNCH(3, 2);
