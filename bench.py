@@ -382,9 +382,11 @@ def measure_network(args, peaks, peak_src):
             cn.merge()
     g_fwd = cn.capture(x, keep_graph=True)
     n_launch = count_kernel_nodes_of(g_fwd)
+    g_step = cn.capture_step(x)
     with torch.cuda.stream(stream):
         fwd = replay_stats(g_fwd, stream, 1)
         merge = replay_stats(g_merge, stream, 1)
+        step = replay_stats(g_step, stream, 1)
         # one launch group at a time: a graph of three launches of the group on the maps the forward left
         groups = []
         cur = x
@@ -449,9 +451,11 @@ def measure_network(args, peaks, peak_src):
     return {
         "config": {"workload": "cfg4_mbv2_full_batch128", "launch_groups": len(cn.ops), "kernel_launches": n_launch,
                    "merged_spans": sum(1 for op in cn.ops if op.merged), "plan_seed": 0, "plan": plan_name,
-                   "step": "all dc_merge_chain calls + forward graph", "l2": "activation maps (0.1-0.6 GB each) exceed L2"},
-        "value": 128 / ((fwd["median"] + merge["median"]) * 1e-6), "unit": "images/s",
-        "ms_per_step": (fwd["median"] + merge["median"]) * 1e-3,
+                   "step": "all dc_merge_chain calls + forward in one graph (a launch group waits for the merge of its own span only)",
+                   "l2": "activation maps (0.1-0.6 GB each) exceed L2"},
+        "value": 128 / (step["median"] * 1e-6), "unit": "images/s",
+        "ms_per_step": step["median"] * 1e-3,
+        "step_ms": {k: (v * 1e-3 if k in ("median", "min", "max") else v) for k, v in step.items()},
         "forward_ms": {k: (v * 1e-3 if k in ("median", "min", "max") else v) for k, v in fwd.items()},
         "forward_images_per_s": 128 / fwd_s, "merge_latency_us": merge, "roofline": roof, "groups": table,
         "e2e": {"value": 128 / (e2e_ms * 1e-3), "unit": "images/s", "ms_per_step": e2e_ms,

@@ -33,6 +33,7 @@ class _Op:
         self.out_shape = None
         self.y = None
         self.merged = False
+        self.merge_job = -1       # index into the network's merge jobs (merged spans only)
 
 
 class CompressedNetwork:
@@ -115,6 +116,7 @@ class CompressedNetwork:
                     op.bias = torch.empty((g.c_out,), dtype=torch.float32, device="cuda")
                     op.packed = torch.empty(dc.packed_bytes(g, dc.BF16), dtype=torch.uint8, device="cuda")
                     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+                    op.merge_job = len(self._merge_jobs)
                     self._merge_jobs.append((devs, list(po.residuals), wm, op.bias, op.packed, ws))
                     op.keep = [wm, ws]
                 g = op.geom
@@ -200,6 +202,49 @@ class CompressedNetwork:
             done.record(st)
             cur.wait_event(done)
         return len(jobs)
+
+    def step(self, x, n_streams: int = 10):
+        """The whole path once: every merge, then the forward, as one piece of work on the current stream.
+        The merges run on side streams in the order the forward needs them, and a launch group waits only
+        for the merge of its own span.  (Measured on cfg4: 1.13 ms, the same as the merges followed by the
+        forward, 0.24 + 0.88 ms: the forward's persistent kernels fill every SM, so the merges' small
+        launches get their turn between them either way; high-priority merge streams did not change it.)"""
+        torch = self.torch
+        jobs = self._merge_jobs
+        if not hasattr(self, "_merge_streams") or len(self._merge_streams) < n_streams:
+            self._merge_streams = [torch.cuda.Stream() for _ in range(n_streams)]
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        done = []
+        for j, (devs, res, wm, bm, packed, ws) in enumerate(jobs):
+            st = self._merge_streams[j % n_streams]
+            if j < n_streams:
+                st.wait_event(fork)
+            dc.merge_chain(devs, res, wm, bm, packed, dc.BF16, ws, stream=st)
+            ev = torch.cuda.Event()
+            ev.record(st)
+            done.append(ev)
+        cur = x
+        for i, op in enumerate(self.ops):
+            if op.merge_job >= 0:
+                main.wait_event(done[op.merge_job])
+            cur = self.launch(i, cur, x)
+        return cur
+
+    def capture_step(self, x):
+        """Capture step(x) into a CUDA graph; replay with .replay()."""
+        torch = self.torch
+        stream = torch.cuda.Stream()
+        stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(stream):
+            self.step(x)
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                self.step(x)
+        torch.cuda.current_stream().wait_stream(stream)
+        return graph
 
     def launch(self, i, cur, x):
         """Launch group i on `cur` (the previous group's map); x is the network input (skip source -1)."""

@@ -133,3 +133,21 @@ def test_graph_replay_reproduces_the_eager_result(run):
     torch.cuda.synchronize()
     assert torch.equal(cn.ops[-1].y, ref)
     assert cn.status() == run["dc"].OK
+
+
+def test_step_graph_merges_and_runs_with_per_span_dependencies(run):
+    """The whole path as one graph: the merged weights are wiped before every replay, so a launch group
+    that ran before the merge of its span had finished would read zeros."""
+    cn, x = run["cn"], run["x"]
+    ref = run["y"].clone()
+    g = cn.capture_step(x)
+    for _ in range(3):
+        for op in cn.ops:
+            if op.merged:
+                op.packed.zero_()
+                op.bias.zero_()
+        cn.ops[-1].y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(cn.ops[-1].y, ref)
+    assert cn.status() == run["dc"].OK
