@@ -106,12 +106,12 @@ struct Walk {
 
 // Epilogue of one warp: tensor-memory lane quadrant q of every block c = grp mod groups, where grp
 // counts the warps of the same quadrant.  Nothing is shared with other warps: the thread of GEMM
-// row m owns the two output pixels of pair m, adds bias and skip input, applies the activation,
-// converts to bf16 and stages them; the warp's valid pixels are consecutive in the NHWC output (only
+// row m owns the two output pixels of pair m, adds the skip input (the bias is in the accumulator
+// already), applies the activation, converts to bf16 and stages them; the warp's valid pixels are consecutive in the NHWC output (only
 // halo pairs and the tail of the block or tile drop out), so they leave as one bulk copy.
 // ACT and RES are compile-time so the per-pixel code carries no runtime switches.
 template <int CO8, int ACT, int RES>
-__device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+__device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, DcWsHeader *ws,
                                               uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
                                               int tile0, int ntiles) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -200,9 +200,11 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
               __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                float f0 = f[2 * i], f1 = f[2 * i + 1];
-                if (ACT) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
-                ob[i] = __floats2bfloat162_rn(f0, f1);
+                // ReLU6 on the rounded pair: 0 and 6 are bf16 values and rounding is monotonic, so this gives
+                // the same bits as clamping before the conversion, in half the instructions
+                __nv_bfloat162 o2 = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+                if (ACT) o2 = __hmin2(__hmax2(o2, __floats2bfloat162_rn(0.f, 0.f)), __floats2bfloat162_rn(6.f, 6.f));
+                ob[i] = o2;
               }
               // in the staging buffer the warp's pixels are packed: the second follows the first only if there is one
               *reinterpret_cast<uint4 *>(dst + ((e && (valid0 || !p.bulk_out) ? p.c_out : 0) + ch) * 2) = ov;
@@ -232,7 +234,7 @@ __device__ __forceinline__ void epilogue_role(const PairParams &p, Shared &sh, D
 // The same for more than 32 output channels: the channels are walked 8 at a time in a run-time
 // loop (any c_out that is a multiple of 8), and a thread stores its pixels' channels straight to
 // global memory (2 * c_out contiguous bytes per pixel; no staging buffer of that size per warp).
-__device__ __noinline__ void epilogue_wide(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+__device__ __noinline__ void epilogue_wide(const PairParams &p, Shared &sh, DcWsHeader *ws,
                                            const __nv_bfloat16 *residual, __nv_bfloat16 *y, int tile0, int ntiles) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int grp = (warp - kFirstEpiWarp) >> 2;
@@ -318,14 +320,14 @@ __device__ __noinline__ void epilogue_wide(const PairParams &p, Shared &sh, DcWs
 }
 
 template <int CO8>
-__device__ __forceinline__ void epilogue_dispatch(const PairParams &p, Shared &sh, DcWsHeader *ws, const float *bias_s,
+__device__ __forceinline__ void epilogue_dispatch(const PairParams &p, Shared &sh, DcWsHeader *ws,
                                                   uint8_t *smem_out, const __nv_bfloat16 *residual, __nv_bfloat16 *y,
                                                   int tile0, int ntiles) {
   const int v = (p.act == DC_ACT_RELU6 ? 1 : 0) | (residual ? 2 : 0);
-  if (v == 0) epilogue_role<CO8, 0, 0>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
-  else if (v == 1) epilogue_role<CO8, 1, 0>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
-  else if (v == 2) epilogue_role<CO8, 0, 1>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
-  else epilogue_role<CO8, 1, 1>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles);
+  if (v == 0) epilogue_role<CO8, 0, 0>(p, sh, ws, smem_out, residual, y, tile0, ntiles);
+  else if (v == 1) epilogue_role<CO8, 1, 0>(p, sh, ws, smem_out, residual, y, tile0, ntiles);
+  else if (v == 2) epilogue_role<CO8, 0, 1>(p, sh, ws, smem_out, residual, y, tile0, ntiles);
+  else epilogue_role<CO8, 1, 1>(p, sh, ws, smem_out, residual, y, tile0, ntiles);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -339,7 +341,6 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
   uint8_t *smem_b = smem + p.off_b;
   uint8_t *smem_a = smem + p.off_a;              // 1024-byte aligned stages (the swizzle pattern repeats every 1024 bytes)
   uint8_t *smem_out = smem + p.off_out;
-  float *bias_s = nullptr;                       // (the read-out no longer adds the bias)
   uint8_t *smem_ones = smem + p.off_bias;        // 8 lines of the constant operand (1024-byte aligned)
   uint8_t *smem_bias = smem_ones + 1024;         // [n_pad][16 bytes]: bias as two bf16 terms, then n_pad zero rows
 
@@ -494,12 +495,12 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (++s == p.stages) { s = 0; ph ^= 1; a_row = a_row0; }
       }
     } else {
-      if (p.co8 > 32) epilogue_wide(p, sh, ws, bias_s, residual, y, tile0, ntiles);
+      if (p.co8 > 32) epilogue_wide(p, sh, ws, residual, y, tile0, ntiles);
       else switch (p.co8) {
-        case 8: epilogue_dispatch<8>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
-        case 16: epilogue_dispatch<16>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
-        case 24: epilogue_dispatch<24>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
-        default: epilogue_dispatch<32>(p, sh, ws, bias_s, smem_out, residual, y, tile0, ntiles); break;
+        case 8: epilogue_dispatch<8>(p, sh, ws, smem_out, residual, y, tile0, ntiles); break;
+        case 16: epilogue_dispatch<16>(p, sh, ws, smem_out, residual, y, tile0, ntiles); break;
+        case 24: epilogue_dispatch<24>(p, sh, ws, smem_out, residual, y, tile0, ntiles); break;
+        default: epilogue_dispatch<32>(p, sh, ws, smem_out, residual, y, tile0, ntiles); break;
       }
     }
     // ---- consumer teardown
