@@ -299,21 +299,26 @@ class CompressedNetwork:
 class HostRunner:
     """The captured network fed from pinned host buffers: a step copies its input to the device, replays
     the forward graph and copies the last map back.  Two device input buffers and a copy stream let
-    the input copy of step i+1 run under the forward of step i; the forwards themselves are serial
-    (they share the intermediate maps)."""
+    the input copy of step i+1 run under the forward of step i; the last map is copied to one of two
+    device staging buffers behind the forward (a few microseconds) and goes to the host from there on a
+    third stream, under the next forward.  The forwards themselves are serial (they share the
+    intermediate maps)."""
 
     def __init__(self, cn: CompressedNetwork):
         torch = cn.torch
         self.cn, self.torch = cn, torch
-        self.copy_stream, self.compute_stream = torch.cuda.Stream(), torch.cuda.Stream()
+        self.copy_stream, self.compute_stream, self.out_stream = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         self.x = [torch.zeros(cn.in_shape, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+        self.y = [torch.zeros(cn.out_shape, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
         self.graphs = [cn.capture(x) for x in self.x]
         self.in_ready = [torch.cuda.Event() for _ in range(2)]
         self.in_free = [torch.cuda.Event() for _ in range(2)]
+        self.out_ready = [torch.cuda.Event() for _ in range(2)]
+        self.out_free = [torch.cuda.Event() for _ in range(2)]
         self.count = 0
 
     def submit(self, x_host, y_host):
-        """Queue one step; y_host is valid once compute_stream has been synchronised."""
+        """Queue one step; y_host is valid once synchronize() has returned."""
         torch = self.torch
         b = self.count & 1
         with torch.cuda.stream(self.copy_stream):
@@ -325,9 +330,23 @@ class HostRunner:
             self.compute_stream.wait_event(self.in_ready[b])
             self.graphs[b].replay()
             self.in_free[b].record(self.compute_stream)
-            y_host.copy_(self.cn.ops[-1].y, non_blocking=True)
+            if self.count >= 2:
+                self.compute_stream.wait_event(self.out_free[b])
+            self.y[b].copy_(self.cn.ops[-1].y, non_blocking=True)
+            self.out_ready[b].record(self.compute_stream)
+        with torch.cuda.stream(self.out_stream):
+            self.out_stream.wait_event(self.out_ready[b])
+            y_host.copy_(self.y[b], non_blocking=True)
+            self.out_free[b].record(self.out_stream)
         self.count += 1
+
+    def join(self):
+        """Make compute_stream wait for the copies queued so far (so that an event recorded on it afterwards
+        marks the end of every queued step)."""
+        self.compute_stream.wait_stream(self.copy_stream)
+        self.compute_stream.wait_stream(self.out_stream)
 
     def synchronize(self):
         self.copy_stream.synchronize()
         self.compute_stream.synchronize()
+        self.out_stream.synchronize()

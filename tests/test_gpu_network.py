@@ -151,3 +151,23 @@ def test_step_graph_merges_and_runs_with_per_span_dependencies(run):
         torch.cuda.synchronize()
         assert torch.equal(cn.ops[-1].y, ref)
     assert cn.status() == run["dc"].OK
+
+
+def test_host_runner_returns_every_steps_own_result(run):
+    """Steps fed from pinned host buffers with the copies running under neighbouring forwards: each step's
+    output is the forward of its own input (two inputs alternate, five steps in flight)."""
+    from paper_2301_12187_b200.network import HostRunner
+    cn, x = run["cn"], run["x"]
+    x2 = torch.flip(x, dims=[0]).contiguous()
+    ref = [cn.forward(x).clone(), cn.forward(x2).clone()]
+    torch.cuda.synchronize()
+    assert not torch.equal(ref[0], ref[1])
+    runner = HostRunner(cn)
+    xs = [x.cpu().pin_memory(), x2.cpu().pin_memory()]
+    ys = [torch.zeros(cn.out_shape, dtype=torch.bfloat16).pin_memory() for _ in range(5)]
+    for i in range(5):
+        runner.submit(xs[i & 1], ys[i])
+    runner.synchronize()
+    for i in range(5):
+        assert torch.equal(ys[i], ref[i & 1].cpu()), "step %d" % i
+    assert cn.status() == run["dc"].OK
