@@ -294,7 +294,7 @@ class ChainBench:
                      "images_per_s_kernel_only": n / (conv["median"] * 1e-6)})
         return {"conv_forward_us": conv, "merge_latency_us": merge, "step_us": step, "roofline": roof}
 
-    def e2e(self, world, barrier, steps):
+    def e2e(self, world, barrier, steps, n_slots=3):
         """End to end through the host-buffer entry point: every step copies its input (and the run's
         parameters, one pinned block) from pinned host memory, merges, runs the forward and copies the
         output back.  Steps rotate over three streams, each with its own workspace and pinned buffers,
@@ -304,7 +304,6 @@ class ChainBench:
         n, h, w, c = case.x_shape
         arr, keep = dc.host_layer_array(case.layers, pinned=True)
         ws_bytes = dc.chain_host_workspace_bytes(arr, len(case.layers), case.residuals, n, h, w, dc.BF16)
-        n_slots = 3
         e_ws = [torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda") for _ in range(n_slots)]
         e_x = [self.x_host.clone().pin_memory() for _ in range(n_slots)]
         e_y = [torch.empty(self.yshape, dtype=torch.bfloat16).pin_memory() for _ in range(n_slots)]
@@ -338,7 +337,7 @@ class ChainBench:
                 raise RuntimeError("device-side wait timed out during the end-to-end run (%s)" % self.name)
         param_bytes = sum(int(s.weight.size) * 4 + 4 * int(s.c_out) * 4 for s in case.layers)
         return ms, {"h2d_bytes_per_step": int(2 * n * h * w * c + param_bytes), "d2h_bytes_per_step": int(2 * np.prod(self.yshape)),
-                    "steps": steps, "api": "dc_chain_forward_host_async (pinned host buffers, one parameter block, 3 streams in flight)"}
+                    "steps": steps, "api": "dc_chain_forward_host_async (pinned host buffers, one parameter block, %d streams in flight)" % n_slots}
 
     def config(self):
         g = self.g
@@ -644,7 +643,7 @@ def run_ours(args):
             t_end = time.time()
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     figs = hb.kernel_figures(peaks, peak_src)
-    e2e_ms, e2e_info = hb.e2e(world, barrier, max(9, min(args.steps, 60)))
+    e2e_ms, e2e_info = hb.e2e(world, barrier, max(9, min(args.steps, 60)), args.e2e_streams)
     times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
     R.max_over_ranks(times, world)
     ms_total, e2e_ms = float(times[0]), float(times[1])
@@ -676,7 +675,7 @@ def run_ours(args):
         for name in ("cfg2", "cfg3"):
             cb = ChainBench(name, R.replica_seed(0, rank), stream)
             f = cb.kernel_figures(peaks, peak_src)
-            ms, info = cb.e2e(world, barrier, 30)
+            ms, info = cb.e2e(world, barrier, 30, args.e2e_streams)
             per[name] = chain_entry(cb, f, ms, info, world, cpu_baseline(cb.case, seconds_cap=8.0) if want_cpu else None)
             cb.free()
         entry, net, cn = measure_network(args, peaks, peak_src)
@@ -707,6 +706,7 @@ def main():
                     help="all: cfg1 as the headline line plus cfg1..cfg4 under per_config (one GPU); cfgN: that workload alone")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-streams", type=int, default=3, help="steps in flight in the end-to-end measurement of the chain workloads")
     ap.add_argument("--plan", default="spans", choices=["spans", "latency"],
                     help="cfg4: merge every valid span, or cut by Algorithm 1 over the measured latency table")
     args = ap.parse_args()
