@@ -312,6 +312,30 @@ __host__ __device__ static inline int dc_korder_encode(const KOrder &ko, int cc,
   return grp * ko.e_pad + e;
 }
 
+// Position (in 16-byte chunks of 8 channels) of row `row` of chunk plane `plane` in the packed weights.
+// Planes are [n_pad rows][8 channels] one after the other, except in rows order with several output-
+// channel passes: there a pass's n_tile rows of all planes are contiguous ([pass][plane][n_tile rows]),
+// so that the planes of one (64-channel plane, tap row) step of one pass are one contiguous block.
+__host__ __device__ static inline size_t dc_packed_chunk(const KOrder &ko, int plane, int row) {
+  if (ko.rows && ko.nnt > 1) {
+    const int pass = row / ko.n_tile;
+    return ((size_t)pass * ko.e_pad + plane) * ko.n_tile + (row - pass * ko.n_tile);
+  }
+  return (size_t)plane * ko.n_pad + row;
+}
+// the inverse: chunk position -> (plane, row)
+__host__ __device__ static inline void dc_packed_unchunk(const KOrder &ko, int idx8, int *plane, int *row) {
+  if (ko.rows && ko.nnt > 1) {
+    const int per_pass = ko.e_pad * ko.n_tile;
+    const int pass = idx8 / per_pass, rem = idx8 - pass * per_pass;
+    *plane = rem / ko.n_tile;
+    *row = pass * ko.n_tile + (rem - *plane * ko.n_tile);
+    return;
+  }
+  *plane = idx8 / ko.n_pad;
+  *row = idx8 - *plane * ko.n_pad;
+}
+
 // row of output channel o (and tap column s) inside a chunk plane of the packed weights
 __host__ __device__ static inline int dc_korder_row(const KOrder &ko, int s, int o) {
   return ko.fold ? s * ko.co8 + o : o;   // pair order: the first pixel's rows are 0..co8-1

@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(128) k_conv_dense_bf16(const __nv_bfloat16 *__
         const __nv_bfloat16 *xp = x + (((size_t)img * h + yy) * wd + xx) * g.c_in;
         for (int cc = 0; cc < ko.cch; ++cc) {
           const int plane = dc_korder_encode(ko, cc, u, v);
-          const uint4 wv = *reinterpret_cast<const uint4 *>(w + ((size_t)plane * ko.n_pad + dc_korder_row(ko, v, o)) * 8);
+          const uint4 wv = *reinterpret_cast<const uint4 *>(w + dc_packed_chunk(ko, plane, dc_korder_row(ko, v, o)) * 8);
           const __nv_bfloat16 *wb = reinterpret_cast<const __nv_bfloat16 *>(&wv);
           if (vec) {
             const uint4 xv = *reinterpret_cast<const uint4 *>(xp + cc * 8);
@@ -139,7 +139,7 @@ k_conv_smallcin_bf16(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *_
     float wv = 0.f;
     if (o0 + o < g.c_out) {
       const int plane = dc_korder_encode(ko, c / 8, u, v);
-      wv = __bfloat162float(w[((size_t)plane * ko.n_pad + dc_korder_row(ko, v, o0 + o)) * 8 + (c & 7)]);
+      wv = __bfloat162float(w[dc_packed_chunk(ko, plane, dc_korder_row(ko, v, o0 + o)) * 8 + (c & 7)]);
     }
     w_s[i] = wv;
   }

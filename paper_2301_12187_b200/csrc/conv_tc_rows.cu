@@ -44,6 +44,7 @@ struct RowsParams {
   int tiles_y, img_groups;
   int grid, items_per, items_rem;    // CTAs; CTA b takes items_per (+1 if b < items_rem) work items
   int n_tile, nnt, n_pad;      // output channels per pass, passes, nnt * n_tile
+  int planes_all;              // chunk planes of the packed weights (all 64-channel planes and taps)
   int mb;                      // blocks per tile
   int lines_img;               // rbox * wbox: GEMM rows per image of a tile
   int a_stage_bytes, a_box_bytes, b_stage_bytes;
@@ -145,16 +146,11 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const size_t plane0 = (size_t)g * p.k * p.k * 8 + (size_t)r * nplanes;
             if (lane == 0) mbar_arrive_expect_tx(&sh.b_full[sb], (uint32_t)(nplanes * p.n_tile * 16));
             __syncwarp();
-            if (p.nnt == 1) {
-              if (lane == 0)
-                bulk_load(dst, wsrc + plane0 * p.n_pad * 16, (uint32_t)(nplanes * p.n_tile * 16), &sh.b_full[sb]);
-            } else {
-              // a pass takes n_tile of the n_pad rows of every plane
-              for (int pl = lane; pl < nplanes; pl += 32)
-                bulk_load(dst + (uint32_t)(pl * p.n_tile * 16),
-                          wsrc + ((plane0 + pl) * p.n_pad + (size_t)q.nt * p.n_tile) * 16, (uint32_t)(p.n_tile * 16),
-                          &sh.b_full[sb]);
-            }
+            // the planes of a step are contiguous in the packed weights, with several passes too (there a
+            // pass's rows of all planes are stored together): one bulk copy
+            if (lane == 0)
+              bulk_load(dst, wsrc + ((size_t)q.nt * p.planes_all + plane0) * p.n_tile * 16, (uint32_t)(nplanes * p.n_tile * 16),
+                        &sh.b_full[sb]);
             if (++sb == p.sb) { sb = 0; pb ^= 1; }
           }
         }
@@ -416,6 +412,7 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->k = g->k; p->pad = g->pad;
   p->planes = dc_div_up(g->c_in, 64);
   p->n_tile = ko.n_tile; p->nnt = ko.nnt; p->n_pad = ko.n_pad;
+  p->planes_all = ko.e_pad;
   // tile: as many rows as fit kMaxLines GEMM rows; whole small images several at a time
   p->nxt = 1;
   while (dc_div_up(wo, p->nxt) + g->k - 1 > kMaxLines / g->k) ++p->nxt;   // at least one output row per tile

@@ -467,7 +467,8 @@ __global__ void k_pack_dw(const float *w, float *out, int c, int k) {
 __global__ void k_pack_bf16(const float *w, __nv_bfloat16 *out, int c_out, KOrder ko) {
   const int total = ko.ng * ko.e_pad * ko.n_pad * 8;
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
-    int c8 = idx % 8, o = (idx / 8) % ko.n_pad, plane = idx / (8 * ko.n_pad);
+    int c8 = idx % 8, o, plane;
+    dc_packed_unchunk(ko, idx / 8, &plane, &o);
     int grp = plane / ko.e_pad, e = plane - grp * ko.e_pad;
     int pc, ccg, r, s;
     float v = 0.f;
@@ -519,7 +520,8 @@ __device__ __forceinline__ void deliver_packed_bf16_chunks(const Piece &acc, __n
   const int c_out = acc.c_out, kk = acc.k * acc.k, ctr = ((acc.k - 1) / 2) * (acc.k + 1);
   const int total8 = ko.ng * ko.e_pad * ko.n_pad;
   for (int idx8 = start; idx8 < total8; idx8 += stride) {
-    const int plane = idx8 / ko.n_pad, o_row = idx8 - plane * ko.n_pad;
+    int plane, o_row;
+    dc_packed_unchunk(ko, idx8, &plane, &o_row);
     const int grp = plane / ko.e_pad, e = plane - grp * ko.e_pad;
     int pc, ccg0, r, s0;
     bool live = dc_korder_decode(ko, e, &pc, &ccg0, &r, &s0);
@@ -607,7 +609,8 @@ __global__ void k_deliver(Piece acc, float *w_merged, float *b_merged, void *pac
     __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(packed);
     const int total = ko.ng * ko.e_pad * ko.n_pad * 8;
     for (int idx = blk * blockDim.x + threadIdx.x; idx < total; idx += nb_p * blockDim.x) {
-      int c8 = idx % 8, o = (idx / 8) % ko.n_pad, plane = idx / (8 * ko.n_pad);
+      int c8 = idx % 8, o, plane;
+      dc_packed_unchunk(ko, idx / 8, &plane, &o);
       int grp = plane / ko.e_pad, e = plane - grp * ko.e_pad;
       int pc, ccg, r, sx;
       float v = 0.f;
