@@ -400,6 +400,8 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (32, 16, 1, 1, 0, 2, 20, 24, "k_conv_tc_pairrows"),     # 1x1: one instruction per 32-byte K step
     (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc_rows"),         # 1x1 expansion from few channels: one half-filled plane
     (16, 96, 1, 1, 0, 1, 40, 112, "k_conv_tc_rows"),        # 1x1 expansion from 16 channels, row tiles
+    (32, 192, 3, 1, 1, 2, 28, 28, "k_conv_tc_rows"),        # 3x3 from few channels to more outputs than the pair rows take
+    (16, 136, 5, 1, 2, 1, 12, 20, "k_conv_tc_rows"),        # the same with 16 channels and a 5x5 kernel, two passes
     (32, 40, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with 40 outputs: general kernel
     (16, 128, 3, 1, 1, 1, 12, 16, "k_conv_tc_pairrows"),    # N = 256: two accumulator slots, run-time channel loop
     (32, 64, 3, 2, 1, 1, 28, 28, "k_conv_tc_pairrows"),     # stride 2, 64 output channels
