@@ -309,16 +309,14 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               }
             }
             uint4 ov;
-            __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
-            // ReLU6 on the rounded pairs: 0 and 6 are bf16 values and rounding is monotonic, so clamping
-            // after the conversion gives the same bits as clamping before it, in half the instructions
-            const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.f, 0.f), six2 = __floats2bfloat162_rn(6.f, 6.f);
+            uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
+            // ReLU6 on the rounded pairs: 0 and 6 are bf16 values and rounding is monotonic, so clamping in and
+            // after the conversion gives the same values as clamping before it: the conversion clamps at zero
+            // itself, one packed minimum against (6, 6) does the rest
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              __nv_bfloat162 o = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-              if (relu6) o = __hmin2(__hmax2(o, zero2), six2);
-              ob[i] = o;
-            }
+            for (int i = 0; i < 4; ++i)
+              ow[i] = relu6 ? min_bf16x2(pack_bf16x2_relu(f[2 * i], f[2 * i + 1]), 0x40C040C0u)
+                            : pack_bf16x2(f[2 * i], f[2 * i + 1]);
             return ov;
           };
           // 32 accumulator columns per read while they last.  A thread owns a pixel, so stored directly
@@ -327,6 +325,12 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // in its staging buffer (80-byte pitch: conflict-free) and writes them four lanes to a
           // pixel: every store instruction then fills eight whole 64-byte segments.
           const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
+          // the four pixels this lane helps to store (pixel i * 8 + lane / 4 of the warp's 32): their addresses
+          // come from the lanes that own them, once per block
+          unsigned long long px_base[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            px_base[i] = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, i * 8 + (lane >> 2));
           auto emit32 = [&](const uint32_t *v, int c0) {
 #pragma unroll
             for (int g8 = 0; g8 < 4; ++g8)
@@ -335,9 +339,8 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int px = i * 8 + (lane >> 2), c = lane & 3;
-              const unsigned long long base = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, px);
               if ((vmask >> px) & 1u)
-                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>((uintptr_t)base) + c0 + c * 8) =
+                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>((uintptr_t)px_base[i]) + c0 + c * 8) =
                     *reinterpret_cast<const uint4 *>(stage + px * kStagePitch + c * 16);
             }
             __syncwarp();

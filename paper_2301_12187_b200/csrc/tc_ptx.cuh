@@ -177,6 +177,26 @@ __device__ __forceinline__ bool epi_all(bool ok) {
   return all != 0;
 }
 
+// two floats -> packed bf16 (lo in the low half), round to nearest even; the second form clamps negative
+// values to zero in the same instruction (ReLU): zero is a bf16 value and rounding is monotonic, so this
+// gives the same bits as max(x, 0) before the conversion
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+// min of packed bf16 pairs
+__device__ __forceinline__ uint32_t min_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+
 // named barrier `id` over `count` threads
 __device__ __forceinline__ void bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
