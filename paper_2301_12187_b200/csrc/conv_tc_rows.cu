@@ -20,6 +20,7 @@
 // warps 1-2 MMA issue (blocks alternate between them), warps 3-10 epilogue (two per tensor-memory
 // lane quadrant, blocks alternate).  A work item is (tile, output-channel pass); CTAs (one per SM)
 // take contiguous runs of items.  All waits are bounded (tc::mbar_wait).
+#include <type_traits>
 #include "tc_ptx.cuh"
 
 namespace {
@@ -295,11 +296,12 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out + ch0 : nullptr;
           const uint32_t taddr = tmem_row + (uint32_t)((set * p.mb + b) * p.n_tile);
           // eight channels of this thread's pixel: skip input, activation -> eight bf16
-          auto cook8 = [&](const uint32_t *v, int ch) {
+          // (RELU and RES are compile-time: the per-pixel code carries no run-time switches)
+          auto cook8 = [&](auto RELU, auto RES, const uint32_t *v, int ch) {
             float f[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[i]);     // the bias is in the accumulator already
-            if (rp && valid) {
+            if (decltype(RES)::value && valid) {
               const uint4 rv = *reinterpret_cast<const uint4 *>(rp + ch);
               const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
 #pragma unroll
@@ -315,8 +317,8 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // itself, one packed minimum against (6, 6) does the rest
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              ow[i] = relu6 ? min_bf16x2(pack_bf16x2_relu(f[2 * i], f[2 * i + 1]), 0x40C040C0u)
-                            : pack_bf16x2(f[2 * i], f[2 * i + 1]);
+              ow[i] = decltype(RELU)::value ? min_bf16x2(pack_bf16x2_relu(f[2 * i], f[2 * i + 1]), 0x40C040C0u)
+                                            : pack_bf16x2(f[2 * i], f[2 * i + 1]);
             return ov;
           };
           // 32 accumulator columns per read while they last.  A thread owns a pixel, so stored directly
@@ -331,10 +333,10 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 4; ++i)
             px_base[i] = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, i * 8 + (lane >> 2));
-          auto emit32 = [&](const uint32_t *v, int c0) {
+          auto emit32 = [&](auto RELU, auto RES, const uint32_t *v, int c0) {
 #pragma unroll
             for (int g8 = 0; g8 < 4; ++g8)
-              *reinterpret_cast<uint4 *>(stage + lane * kStagePitch + g8 * 16) = cook8(v + 8 * g8, c0 + 8 * g8);
+              *reinterpret_cast<uint4 *>(stage + lane * kStagePitch + g8 * 16) = cook8(RELU, RES, v + 8 * g8, c0 + 8 * g8);
             __syncwarp();
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -345,22 +347,28 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             __syncwarp();
           };
-          int ch = 0;
+          auto channels = [&](auto RELU, auto RES) {
+            int ch = 0;
 #pragma unroll 1
-          for (; ch + 32 <= nch; ch += 32) {
-            uint32_t v[32];
-            tmem_ld32(taddr + (uint32_t)ch, v);
-            tmem_ld_wait();
-            emit32(v, ch);
-          }
+            for (; ch + 32 <= nch; ch += 32) {
+              uint32_t v[32];
+              tmem_ld32(taddr + (uint32_t)ch, v);
+              tmem_ld_wait();
+              emit32(RELU, RES, v, ch);
+            }
 #pragma unroll 1
-          for (; ch < nch; ch += 8) {
-            uint32_t v[8];
-            tmem_ld8(taddr + (uint32_t)ch, v);
-            tmem_ld_wait();
-            const uint4 ov = cook8(v, ch);
-            if (valid) *reinterpret_cast<uint4 *>(dst + ch) = ov;
-          }
+            for (; ch < nch; ch += 8) {
+              uint32_t v[8];
+              tmem_ld8(taddr + (uint32_t)ch, v);
+              tmem_ld_wait();
+              const uint4 ov = cook8(RELU, RES, v, ch);
+              if (valid) *reinterpret_cast<uint4 *>(dst + ch) = ov;
+            }
+          };
+          using T = std::true_type;
+          using F = std::false_type;
+          if (relu6) { if (rp) channels(T{}, T{}); else channels(T{}, F{}); }
+          else { if (rp) channels(F{}, T{}); else channels(F{}, F{}); }
         }
         // this warp has read what it needs of the accumulator set
         tc_fence_before();
