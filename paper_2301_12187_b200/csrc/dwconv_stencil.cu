@@ -46,7 +46,7 @@ __device__ __forceinline__ float4 lds_f4(uint32_t a) {
   return v;
 }
 
-template <int K, int S>
+template <int K, int S, int ACT>
 __global__ void __launch_bounds__(kThreads, 4)
 k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ StencilParams p,
                  const float *__restrict__ w, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ y) {
@@ -153,13 +153,12 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     for (int o = 0; o < TX; ++o) {
       if (X0 + o < p.wo) {
         uint4 ov;
-        __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+        uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
+        // ReLU6 (compile-time): the conversion clamps at zero itself, one packed minimum against (6, 6) does
+        // the rest -- the same values as clamping before rounding, since 0 and 6 are bf16 values
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          float f0 = acc[o][i].x, f1 = acc[o][i].y;
-          if (p.act == DC_ACT_RELU6) { f0 = fminf(fmaxf(f0, 0.f), 6.f); f1 = fminf(fmaxf(f1, 0.f), 6.f); }
-          ob[i] = __floats2bfloat162_rn(f0, f1);
-        }
+        for (int i = 0; i < 4; ++i)
+          ow[i] = ACT ? min_bf16x2(pack_bf16x2_relu(acc[o][i].x, acc[o][i].y), 0x40C040C0u) : pack_bf16x2(acc[o][i].x, acc[o][i].y);
         *reinterpret_cast<uint4 *>(yrow + (size_t)(X0 + o) * p.c) = ov;
       }
     }
@@ -245,17 +244,23 @@ dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, in
   const int smem = p.patch_bytes + (k * k + 1) * p.ct * 4 + 256;
   const int grid = p.igroups * p.ytiles * p.cgroups;
   __nv_bfloat16 *yp = (__nv_bfloat16 *)y;
-#define DC_DW_LAUNCH(KK, SS)                                                                              \
+#define DC_DW_LAUNCH1(KK, SS, AA)                                                                         \
   do {                                                                                                    \
     static unsigned char attr_done[kDcMaxDevices];                                                        \
-    DC_CUDA_OK(dc_set_max_smem_once(k_dwconv_stencil<KK, SS>, kTileBytes + 8 * 1024, attr_done));         \
-    if (dc_launch_pdl(k_dwconv_stencil<KK, SS>, dim3(grid), dim3(kThreads), (size_t)smem, st, map_x, p, wp, bias, yp) != cudaSuccess) \
+    DC_CUDA_OK(dc_set_max_smem_once(k_dwconv_stencil<KK, SS, AA>, kTileBytes + 8 * 1024, attr_done));     \
+    if (dc_launch_pdl(k_dwconv_stencil<KK, SS, AA>, dim3(grid), dim3(kThreads), (size_t)smem, st, map_x, p, wp, bias, yp) != cudaSuccess) \
       return DC_ERR_CUDA;                                                                                 \
+  } while (0)
+#define DC_DW_LAUNCH(KK, SS)                                                                              \
+  do {                                                                                                    \
+    if (act == DC_ACT_RELU6) DC_DW_LAUNCH1(KK, SS, 1);                                                    \
+    else DC_DW_LAUNCH1(KK, SS, 0);                                                                        \
   } while (0)
   if (k == 3 && stride == 1) DC_DW_LAUNCH(3, 1);
   else if (k == 3) DC_DW_LAUNCH(3, 2);
   else if (stride == 1) DC_DW_LAUNCH(5, 1);
   else DC_DW_LAUNCH(5, 2);
+#undef DC_DW_LAUNCH1
 #undef DC_DW_LAUNCH
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
