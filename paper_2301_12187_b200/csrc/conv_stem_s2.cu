@@ -55,6 +55,9 @@ struct S2Params {
   int ent[9];                  // chunk plane of tap (r, s) in the packed weights
 };
 
+// PLAIN: at most three input channels (the bias rides in the weights) and no skip input; RELU: ReLU6 in
+// that case (compile-time, so that the per-pixel code of the common case carries no run-time switches)
+template <int PLAIN, int RELU>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restrict__ x, const void *__restrict__ w_packed,
                const float *__restrict__ bias, const __nv_bfloat16 *__restrict__ residual, __nv_bfloat16 *__restrict__ y,
@@ -250,7 +253,6 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
     // ---- read-out: thread = GEMM row = output pixel of the segment; the two warps of a lane quarter
     // take the blocks in turn.  The band's output rows are contiguous in memory: they are put together in
     // shared memory and leave as one bulk copy.
-    const bool plain = fold_bias && residual == nullptr;
     int blk = 0;
     for (int ry = 0; ry < rows_out; ++ry)
       for (int xt = 0; xt < p.xtiles; ++xt, ++blk) {
@@ -262,16 +264,17 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
           uint32_t v[32];
           tmem_ld32(trow + (uint32_t)(blk * p.n_pad + c0), v);
           tmem_ld_wait();
-          if (plain) {
+          if (PLAIN) {
 #pragma unroll
             for (int g8 = 0; g8 < 4; ++g8) {
               uint4 ov;
-              __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+              uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
+              // ReLU6: the conversion clamps at zero itself, one packed minimum against (6, 6) does the rest
+              // (the same values as clamping before rounding, since 0 and 6 are bf16 values)
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(v[8 * g8 + 2 * i]), __uint_as_float(v[8 * g8 + 2 * i + 1]));
-                if (relu6) o2 = __hmin2(__hmax2(o2, zero2), six2);   // same bits as clamping before rounding
-                ob[i] = o2;
+                const float f0 = __uint_as_float(v[8 * g8 + 2 * i]), f1 = __uint_as_float(v[8 * g8 + 2 * i + 1]);
+                ow[i] = RELU ? min_bf16x2(pack_bf16x2_relu(f0, f1), 0x40C040C0u) : pack_bf16x2(f0, f1);
               }
               if (valid && c0 + 8 * g8 < p.c_out) sts128(so + (uint32_t)((c0 + 8 * g8) * 2), ov);
             }
@@ -399,11 +402,20 @@ dc_status dc_launch_conv_stem_s2(const void *x, int n, int h, int w, const dc_ge
   // rows enter and leave by bulk copies: without 16-byte aligned images the general stem kernel runs
   if (((uintptr_t)x | (uintptr_t)y) & 15) return dc_launch_conv_stem(x, n, h, w, g, w_packed, bias, act, residual, y, workspace, stream);
   p.act = (int)act;
-  static unsigned char attr_done[kDcMaxDevices];
-  DC_CUDA_OK(dc_set_max_smem_once(k_conv_stem_s2, 100 * 1024, attr_done));
   const int total = n * p.bands, resident = kCtasPerSm * dc_sm_count();
-  const cudaError_t le = dc_launch_pdl(k_conv_stem_s2, dim3(total < resident ? total : resident), dim3(kThreads),
-                                       (size_t)p.smem_bytes, stream, p, (const __nv_bfloat16 *)x, w_packed, bias,
-                                       (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y, (DcWsHeader *)workspace);
+  const bool plain = g->c_in <= 3 && residual == nullptr;
+  cudaError_t le;
+#define DC_STEM_LAUNCH(PP, RR)                                                                                      \
+  do {                                                                                                              \
+    static unsigned char attr_done[kDcMaxDevices];                                                                  \
+    DC_CUDA_OK(dc_set_max_smem_once(k_conv_stem_s2<PP, RR>, 100 * 1024, attr_done));                                \
+    le = dc_launch_pdl(k_conv_stem_s2<PP, RR>, dim3(total < resident ? total : resident), dim3(kThreads),            \
+                       (size_t)p.smem_bytes, stream, p, (const __nv_bfloat16 *)x, w_packed, bias,                   \
+                       (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y, (DcWsHeader *)workspace);               \
+  } while (0)
+  if (!plain) DC_STEM_LAUNCH(0, 0);
+  else if (act == DC_ACT_RELU6) DC_STEM_LAUNCH(1, 1);
+  else DC_STEM_LAUNCH(1, 0);
+#undef DC_STEM_LAUNCH
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
