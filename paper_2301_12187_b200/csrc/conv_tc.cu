@@ -32,6 +32,7 @@
 // owns the tensor-memory allocation, warps 5-8 epilogue.  Accumulators are double buffered so the
 // epilogue of tile i overlaps the MMAs of tile i+1.  Every wait is bounded: when one runs out the
 // CTA latches DC_ERR_TIMEOUT in the caller's workspace and leaves.
+#include <type_traits>
 #include "tc_ptx.cuh"
 
 namespace {
@@ -319,45 +320,56 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
         __nv_bfloat16 *gout = y + pix * p.c_out;
         const __nv_bfloat16 *gres = residual ? residual + pix * p.c_out : nullptr;
         uint8_t *sout = obuf + (size_t)(yy * p.tw + xx) * p.c_out * 2;
-        for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
-          if (ch_base + c0 >= p.c_out) break;    // uniform across the warp
-          uint32_t v[32];
-          const bool wide = (c0 + 32 <= p.n_tile);
-          if (wide) tmem_ld32(taddr + (uint32_t)c0, v);
-          else tmem_ld16(taddr + (uint32_t)c0, v);
-          tmem_ld_wait();
-          if (valid) {
+        // activation and skip input are compile-time in the per-pixel code (four instantiations, picked once
+        // per block); the pixel goes to the staged tile or straight to memory through one generic pointer
+        uint8_t *const pdst = p.bulk_out ? sout : reinterpret_cast<uint8_t *>(gout);
+        auto channels = [&](auto RELU, auto RES) {
+          for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
+            if (ch_base + c0 >= p.c_out) break;    // uniform across the warp
+            uint32_t v[32];
+            const bool wide = (c0 + 32 <= p.n_tile);
+            if (wide) tmem_ld32(taddr + (uint32_t)c0, v);
+            else tmem_ld16(taddr + (uint32_t)c0, v);
+            tmem_ld_wait();
+            if (valid) {
 #pragma unroll
-            for (int e8 = 0; e8 < 4; ++e8) {
-              const int ch = ch_base + c0 + e8 * 8;
-              if ((e8 < 2 || wide) && ch < p.c_out) {
-                const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
-                const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
-                float f[8];
-                f[0] = __uint_as_float(v[e8 * 8 + 0]) + b0.x; f[1] = __uint_as_float(v[e8 * 8 + 1]) + b0.y;
-                f[2] = __uint_as_float(v[e8 * 8 + 2]) + b0.z; f[3] = __uint_as_float(v[e8 * 8 + 3]) + b0.w;
-                f[4] = __uint_as_float(v[e8 * 8 + 4]) + b1.x; f[5] = __uint_as_float(v[e8 * 8 + 5]) + b1.y;
-                f[6] = __uint_as_float(v[e8 * 8 + 6]) + b1.z; f[7] = __uint_as_float(v[e8 * 8 + 7]) + b1.w;
-                if (gres) {
-                  const uint4 rv = *reinterpret_cast<const uint4 *>(gres + ch);
-                  const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
+              for (int e8 = 0; e8 < 4; ++e8) {
+                const int ch = ch_base + c0 + e8 * 8;
+                if ((e8 < 2 || wide) && ch < p.c_out) {
+                  const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
+                  const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
+                  float f[8];
+                  f[0] = __uint_as_float(v[e8 * 8 + 0]) + b0.x; f[1] = __uint_as_float(v[e8 * 8 + 1]) + b0.y;
+                  f[2] = __uint_as_float(v[e8 * 8 + 2]) + b0.z; f[3] = __uint_as_float(v[e8 * 8 + 3]) + b0.w;
+                  f[4] = __uint_as_float(v[e8 * 8 + 4]) + b1.x; f[5] = __uint_as_float(v[e8 * 8 + 5]) + b1.y;
+                  f[6] = __uint_as_float(v[e8 * 8 + 6]) + b1.z; f[7] = __uint_as_float(v[e8 * 8 + 7]) + b1.w;
+                  if (decltype(RES)::value) {
+                    const uint4 rv = *reinterpret_cast<const uint4 *>(gres + ch);
+                    const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
 #pragma unroll
-                  for (int i = 0; i < 4; ++i) {
-                    const float2 rf = __bfloat1622float2(rb[i]);
-                    f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                    for (int i = 0; i < 4; ++i) {
+                      const float2 rf = __bfloat1622float2(rb[i]);
+                      f[2 * i] += rf.x; f[2 * i + 1] += rf.y;
+                    }
                   }
-                }
-                uint4 ov;
-                __nv_bfloat162 *ob = reinterpret_cast<__nv_bfloat162 *>(&ov);
+                  uint4 ov;
+                  uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
+                  // ReLU6: the conversion clamps at zero itself, one packed minimum against (6, 6) does the rest
+                  // (the same values as clamping before rounding, since 0 and 6 are bf16 values)
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                  ob[i] = __floats2bfloat162_rn(dc_act_apply(f[2 * i], p.act), dc_act_apply(f[2 * i + 1], p.act));
-                if (p.bulk_out) *reinterpret_cast<uint4 *>(sout + ch * 2) = ov;
-                else *reinterpret_cast<uint4 *>(gout + ch) = ov;
+                  for (int i = 0; i < 4; ++i)
+                    ow[i] = decltype(RELU)::value ? min_bf16x2(pack_bf16x2_relu(f[2 * i], f[2 * i + 1]), 0x40C040C0u)
+                                                  : pack_bf16x2(f[2 * i], f[2 * i + 1]);
+                  *reinterpret_cast<uint4 *>(pdst + ch * 2) = ov;
+                }
               }
             }
           }
-        }
+        };
+        using T = std::true_type;
+        using F = std::false_type;
+        if (p.act == DC_ACT_RELU6) { if (gres) channels(T{}, T{}); else channels(T{}, F{}); }
+        else { if (gres) channels(F{}, T{}); else channels(F{}, F{}); }
       }
       tc_fence_before();
       mbar_arrive(&bar_accempty[a]);
