@@ -48,6 +48,7 @@ struct RowsParams {
   int planes_all;              // chunk planes of the packed weights (all 64-channel planes and taps)
   int mb;                      // blocks per tile
   int lines_img;               // rbox * wbox: GEMM rows per image of a tile
+  uint32_t inv_lines, inv_wbox; // ceil(2^20 / lines_img), ceil(2^20 / wbox)
   int a_stage_bytes, a_box_bytes, b_stage_bytes;
   int sa, sb, nacc, act;
   int off_bias, off_stage, off_b, off_a, smem_bytes;
@@ -288,12 +289,14 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
         for (int b = par; b < p.mb; b += 2) {
           const int pos = b * 128 + q * 32 + lane;
-          const int il = pos / p.lines_img, rem = pos - il * p.lines_img;
-          const int yy = rem / p.wbox, xx = rem - yy * p.wbox;
+          // pos < 512 and the divisors are at most 256: multiplying by the rounded-up reciprocal is exact
+          const int il = (int)(((uint32_t)pos * p.inv_lines) >> 20), rem = pos - il * p.lines_img;
+          const int yy = (int)(((uint32_t)rem * p.inv_wbox) >> 20), xx = rem - yy * p.wbox;
           const bool valid = il < p.ni && iq.img0 + il < p.n_img && yy < th_valid && xx < tw_valid;
-          const size_t pix = ((size_t)(iq.img0 + il) * p.ho + (size_t)(y0 + yy)) * p.wo + (size_t)(x0 + xx);
-          __nv_bfloat16 *dst = y + pix * p.c_out + ch0;
-          const __nv_bfloat16 *rp = residual ? residual + pix * p.c_out + ch0 : nullptr;
+          // (the plan keeps the pixel count of the output below 2^31)
+          const int pix = ((iq.img0 + il) * p.ho + (y0 + yy)) * p.wo + (x0 + xx);
+          __nv_bfloat16 *dst = y + (size_t)pix * p.c_out + ch0;
+          const __nv_bfloat16 *rp = residual ? residual + (size_t)pix * p.c_out + ch0 : nullptr;
           const uint32_t taddr = tmem_row + (uint32_t)((set * p.mb + b) * p.n_tile);
           // eight channels of this thread's pixel: skip input, activation -> eight bf16
           // (RELU and RES are compile-time: the per-pixel code carries no run-time switches)
@@ -330,9 +333,12 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // the four pixels this lane helps to store (pixel i * 8 + lane / 4 of the warp's 32): their addresses
           // come from the lanes that own them, once per block
           unsigned long long px_base[4];
+          bool px_on[4];
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
+          for (int i = 0; i < 4; ++i) {
             px_base[i] = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, i * 8 + (lane >> 2));
+            px_on[i] = (vmask >> (i * 8 + (lane >> 2))) & 1u;
+          }
           auto emit32 = [&](auto RELU, auto RES, const uint32_t *v, int c0) {
 #pragma unroll
             for (int g8 = 0; g8 < 4; ++g8)
@@ -341,7 +347,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int px = i * 8 + (lane >> 2), c = lane & 3;
-              if ((vmask >> px) & 1u)
+              if (px_on[i])
                 *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>((uintptr_t)px_base[i]) + c0 + c * 8) =
                     *reinterpret_cast<const uint4 *>(stage + px * kStagePitch + c * 16);
             }
@@ -417,7 +423,7 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   if (!ko.rows) return false;
   const int ho = dc_out_extent(h, g->k, 1, g->pad), wo = dc_out_extent(w, g->k, 1, g->pad);
   if (ho <= 0 || wo <= 0) return false;
-  if ((long long)n * h * w * g->c_in >= (1ll << 40)) return false;
+  if ((long long)n * h * w * g->c_in >= (1ll << 40) || (long long)n * ho * wo >= (1ll << 31)) return false;
   p->n_img = n; p->h = h; p->w = w; p->ho = ho; p->wo = wo;
   p->c_in = g->c_in; p->c_out = g->c_out;
   p->k = g->k; p->pad = g->pad;
@@ -436,6 +442,8 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->th = th;
   p->rbox = th + g->k - 1;
   p->lines_img = p->rbox * p->wbox;
+  p->inv_lines = ((1u << 20) + (uint32_t)p->lines_img - 1) / (uint32_t)p->lines_img;
+  p->inv_wbox = ((1u << 20) + (uint32_t)p->wbox - 1) / (uint32_t)p->wbox;
   p->ni = 1;
   if (th == ho && p->nxt == 1) {
     p->ni = kMaxLines / p->lines_img;
