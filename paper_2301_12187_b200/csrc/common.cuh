@@ -175,7 +175,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
   // ordered (plane g of 64 channels, tap row r, tap column s, 16-channel step, half): the planes of
   // one (g, r) step are contiguous, which is the unit the kernel streams.
   if (g->groups == 1 && g->stride == 1 && g->k <= 7 &&
-      (ko->cch >= 5 ? g->c_out >= (g->k == 1 ? 32 : 48)
+      (ko->cch >= 5 ? g->c_out >= 32
                     : ((g->k == 1 && ko->cch >= 2 && g->c_out >= 48) || (g->k >= 3 && ko->cch >= 2 && ko->co8 > 128))) &&
       g->c_in % 8 == 0 && g->c_out % 8 == 0) {
     const int n16 = (int)dc_round_up((size_t)g->c_out, 16);

@@ -51,6 +51,7 @@ struct RowsParams {
   uint32_t inv_lines, inv_wbox; // ceil(2^20 / lines_img), ceil(2^20 / wbox)
   int a_stage_bytes, a_box_bytes, b_stage_bytes;
   int sa, sb, nacc, act;
+  int b_resident;              // all weights stay in shared memory (one copy per CTA)
   int off_bias, off_stage, off_b, off_a, smem_bytes;
   int tmem_cols;
 };
@@ -58,6 +59,7 @@ struct RowsParams {
 struct Shared {
   uint64_t a_full[kMaxA], a_empty[kMaxA];
   uint64_t b_full[kMaxB], b_empty[kMaxB];
+  uint64_t b_all;              // resident weights have landed
   uint64_t acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   uint32_t abort;
@@ -83,6 +85,10 @@ struct Item {
   }
 };
 
+// RESIDENT: all weights of the layer (a single output-channel pass, at most 96 KB) stay in shared memory:
+// one copy per CTA instead of one stream per work item.  Compile-time, so that the streaming version's
+// loops carry no switches.
+template <bool RESIDENT>
 __global__ void __launch_bounds__(kThreads, 1)
 k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ RowsParams p,
                const void *__restrict__ w_packed, const float *__restrict__ bias,
@@ -109,7 +115,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (t < p.sa) { mbar_init(&sh.a_full[t], 1); mbar_init(&sh.a_empty[t], kMmaWarps); did = true; }
     else if (t >= 32 && t < 32 + p.sb) { mbar_init(&sh.b_full[t - 32], 1); mbar_init(&sh.b_empty[t - 32], kMmaWarps); did = true; }
     else if (t >= 64 && t < 66) { mbar_init(&sh.acc_full[t - 64], kMmaWarps); mbar_init(&sh.acc_empty[t - 64], kEpiWarps); did = true; }
-    else if (t == 96) { sh.abort = 0; prefetch_tensormap(&map_a); did = true; }
+    else if (t == 96) { sh.abort = 0; mbar_init(&sh.b_all, 1); prefetch_tensormap(&map_a); did = true; }
     if (did) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   dc_pdl_enter();                                // nothing above touched global memory; everything below may
@@ -125,6 +131,11 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int sa = 0, sb = 0;
       uint32_t pa = 0, pb = 0;
       bool ok = true;
+      if (RESIDENT && lane == 0) {               // the whole packed buffer once
+        const uint32_t all = (uint32_t)(p.planes_all * p.n_tile * 16);
+        mbar_arrive_expect_tx(&sh.b_all, all);
+        bulk_load(b_base0, wsrc, all, &sh.b_all);
+      }
 #pragma unroll 1
       for (int it = 0; it < nitems && ok; ++it) {
         Item q;
@@ -142,7 +153,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int nsl = plane_steps(p, g);
           const int nplanes = p.k * nsl * 2;     // chunk planes of one (g, r) step
 #pragma unroll 1
-          for (int r = 0; r < p.k; ++r) {
+          for (int r = 0; r < p.k && !RESIDENT; ++r) {
             if (!warp_wait(&sh.b_empty[sb], pb ^ 1, abort_flag, ws, 0x20000u | sb)) { ok = false; break; }
             const uint32_t dst = b_base0 + (uint32_t)sb * (uint32_t)p.b_stage_bytes;
             const size_t plane0 = (size_t)g * p.k * p.k * 8 + (size_t)r * nplanes;
@@ -207,6 +218,10 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t pa = 0, pb = 0;
       uint32_t acc_ph[2] = {1u, 1u};             // parity this warp waits for on acc_empty (first use passes)
       bool ok = true;
+      if (RESIDENT) {
+        ok = warp_wait(&sh.b_all, 0, abort_flag, ws, 0x70000u);
+        tc_fence_after();
+      }
 #pragma unroll 1
       for (int it = 0; it < nitems && ok; ++it) {
         const int set = p.nacc == 2 ? (it & 1) : 0;
@@ -231,9 +246,14 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int nsl = plane_steps(p, g);
 #pragma unroll 1
           for (int r = 0; r < p.k; ++r) {
-            if (!warp_wait(&sh.b_full[sb], pb, abort_flag, ws, 0x50000u | sb)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t b_stage = b_row0 + (uint32_t)sb * ((uint32_t)p.b_stage_bytes >> 4);
+            uint32_t b_stage;
+            if (RESIDENT) {
+              b_stage = b_row0 + (uint32_t)((g * p.k * p.k * 8 + r * p.k * nsl * 2) * p.n_tile);   // planes before this step
+            } else {
+              if (!warp_wait(&sh.b_full[sb], pb, abort_flag, ws, 0x50000u | sb)) { ok = false; break; }
+              tc_fence_after();
+              b_stage = b_row0 + (uint32_t)sb * ((uint32_t)p.b_stage_bytes >> 4);
+            }
 #pragma unroll 1
             for (int b = mw; b < p.mb; b += kMmaWarps) {
               const uint32_t d = tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile);
@@ -255,8 +275,10 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
               }
             }
-            if (leader) umma_commit(&sh.b_empty[sb]);      // this warp is done with the weight stage
-            if (++sb == p.sb) { sb = 0; pb ^= 1; }
+            if (!RESIDENT) {
+              if (leader) umma_commit(&sh.b_empty[sb]);    // this warp is done with the weight stage
+              if (++sb == p.sb) { sb = 0; pb ^= 1; }
+            }
           }
           if (ok && leader) umma_commit(&sh.a_empty[sa]);  // ... and with the plane
           if (++sa == p.sa) { sa = 0; pa ^= 1; }
@@ -478,13 +500,19 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->off_a = (int)dc_round_up((size_t)p->off_stage + kEpiWarps * 32 * kStagePitch, 1024);
   // rings: weights first (they are the larger stream), then activation planes
   int sa = 2, sb = 2;
+  // Small weights of a single pass with many input channels stay resident: then a work item streams its
+  // activation planes only.  (For layers of one or two planes the weight stream is small beside the
+  // activations and the resident version measured no faster.)
+  const long long b_all = (long long)dc_round_up((size_t)ko.e_pad * p->n_tile * 16, 1024);
+  p->b_resident = (p->nnt == 1 && p->planes >= 3 && b_all <= 96 * 1024) ? 1 : 0;
   auto total = [&](int a, int b) {
-    const long long wbytes = (long long)b * p->b_stage_bytes;
+    const long long wbytes = p->b_resident ? b_all : (long long)b * p->b_stage_bytes;
     const long long tail = wbytes >= 26 * 1024 ? kSlack : 26 * 1024 - wbytes + kSlack;   // room for the overrun
     return 1024ll + p->off_a + wbytes + (long long)a * p->a_stage_bytes + tail;
   };
+  if (p->b_resident && total(sa, sb) > kSmemBudget) p->b_resident = 0;
   if (total(sa, sb) > kSmemBudget) return false;
-  while (sb < kMaxB && total(sa, sb + 1) <= kSmemBudget) ++sb;
+  while (!p->b_resident && sb < kMaxB && total(sa, sb + 1) <= kSmemBudget) ++sb;
   while (sa < kMaxA && total(sa + 1, sb) <= kSmemBudget) ++sa;
   p->sa = sa; p->sb = sb;
   p->off_b = p->off_a + sa * p->a_stage_bytes;
@@ -521,8 +549,10 @@ dc_status dc_launch_conv_rows(const void *x, int n, int h, int w, const dc_geom 
     if (r != CUDA_SUCCESS) return DC_ERR_CUDA;
   }
   static unsigned char attr_done[kDcMaxDevices];
-  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_rows, kSmemBudget, attr_done));
-  const cudaError_t le = dc_launch_pdl(k_conv_tc_rows, dim3(p.grid), dim3(kThreads), (size_t)p.smem_bytes, stream, map_a, p,
+  static unsigned char attr_done_r[kDcMaxDevices];
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_rows<false>, kSmemBudget, attr_done));
+  DC_CUDA_OK(dc_set_max_smem_once(k_conv_tc_rows<true>, kSmemBudget, attr_done_r));
+  const cudaError_t le = dc_launch_pdl(p.b_resident ? k_conv_tc_rows<true> : k_conv_tc_rows<false>, dim3(p.grid), dim3(kThreads), (size_t)p.smem_bytes, stream, map_a, p,
                                        w_packed, bias, (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y,
                                        (DcWsHeader *)workspace);
   return le == cudaSuccess && cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;

@@ -99,7 +99,8 @@ def test_kernel_name_query_follows_the_dispatch_rules():
     assert dc.conv_kernel_name(128, 56, 56, dc.geom(96, 144, 1, 5, 2, 2), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 14, 14, dc.geom(96, 576, 1, 1, 1, 0), dc.BF16) == "k_conv_tc_rows"
     assert dc.conv_kernel_name(128, 7, 7, dc.geom(160, 960, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_rows"
-    assert dc.conv_kernel_name(128, 28, 28, dc.geom(144, 32, 1, 3, 1, 1), dc.BF16) == "k_conv_tc"
+    assert dc.conv_kernel_name(128, 28, 28, dc.geom(144, 32, 1, 3, 1, 1), dc.BF16) == "k_conv_tc_rows"
+    assert dc.conv_kernel_name(128, 28, 28, dc.geom(144, 24, 1, 3, 1, 1), dc.BF16) == "k_conv_tc"
     assert dc.conv_kernel_name(128, 224, 224, dc.geom(3, 32, 1, 3, 2, 1), dc.BF16) == "k_conv_stem_s2"
     assert dc.conv_kernel_name(2, 17, 33, dc.geom(3, 40, 1, 3, 2, 1), dc.BF16) == "k_conv_stem_tc"
     assert dc.conv_kernel_name(1, 20, 20, dc.geom(3, 264, 1, 3, 2, 1), dc.BF16) == "k_conv_smallcin_bf16"

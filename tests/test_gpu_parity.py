@@ -411,7 +411,8 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
     (128, 128, 5, 1, 2, 2, 14, 14, "k_conv_tc_rows"),       # 5x5 with 128 outputs: two passes of 64 (weight stage limit)
     (96, 96, 7, 1, 3, 1, 14, 14, "k_conv_tc_rows"),         # 7x7: passes of at most 80 output channels
-    (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc"),             # many channels, few outputs: general kernel
+    (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc_rows"),        # many channels, 32 outputs: rows kernel with resident weights
+    (200, 24, 3, 1, 1, 2, 14, 14, "k_conv_tc"),             # many channels, fewer than 32 outputs: general kernel
     (192, 32, 1, 1, 0, 2, 28, 28, "k_conv_tc_rows"),        # 1x1 projection to 32 channels
 ])
 def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, w, kernel):
