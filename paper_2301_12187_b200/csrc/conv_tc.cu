@@ -107,7 +107,8 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
   uint8_t *smem_a = smem + p.off_a;
   uint8_t *smem_out = smem + p.off_out;
   uint8_t *smem_zero = smem_a + (size_t)p.stages * p.a_stage_bytes;   // always-zero plane + slack
-  float *bias_s = reinterpret_cast<float *>(smem + p.off_bias);
+  uint8_t *smem_ones = smem + p.off_bias;        // 8 GEMM rows of the constant operand: (1, 1, 0, ..) in 16 bytes each
+  uint8_t *smem_bias = smem_ones + 128;          // [nnt * n_tile][16 bytes]: bias as two bf16 terms, then n_tile zero rows
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile uint32_t *abort_flag = &abort_s;
@@ -130,7 +131,21 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
   }
   if (threadIdx.x >= 5 * 32) {
     const int t = threadIdx.x - 5 * 32;
-    for (int i = t; i < p.nnt * p.n_tile; i += 128) bias_s[i] = (bias && i < p.c_out) ? bias[i] : 0.f;
+    // The bias is added by the tensor core: one instruction per block multiplies a constant operand (1.0 in
+    // the first two K elements of every GEMM row; one 8-row group read sixteen times, group stride 0; its
+    // second K chunk is the zero plane) with [bias as bf16, its bf16 remainder, 0, ...] per output channel
+    // (exact to 16 mantissa bits) before the block's other instructions accumulate.
+    if (t < 8) reinterpret_cast<uint4 *>(smem_ones)[t] = make_uint4(0x3F803F80u, 0u, 0u, 0u);
+    for (int i = t; i < (p.nnt + 1) * p.n_tile; i += 128) {
+      uint32_t w0 = 0u;
+      if (bias && i < p.c_out) {
+        const float b = bias[i];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+        w0 = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+      }
+      reinterpret_cast<uint4 *>(smem_bias)[i] = make_uint4(w0, 0u, 0u, 0u);
+    }
     // the zero plane: second chunk of the padding entry, and the landing zone of reads past the last stage
     uint4 *z = reinterpret_cast<uint4 *>(smem_zero);
     for (int i = t; i < (p.mb * 2048 + 1024) / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -260,6 +275,15 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
         if (!warp_wait(&bar_accempty[a], aph ^ 1, abort_flag, ws, 0x20000u | a)) goto mma_done;
         tc_fence_after();
         const uint32_t d0 = tmem_base + a * (uint32_t)p.acc_cols;
+        {
+          // the bias initialises the accumulators of the tile's blocks (it needs no load)
+          const uint32_t ones_a = smem_u32(smem_ones), bias_a = smem_u32(smem_bias) + (uint32_t)(t.nt * p.n_tile * 16);
+          const uint32_t zero_rows = smem_u32(smem_bias) + (uint32_t)(p.nnt * p.n_tile * 16);
+          const uint64_t ad = ((uint64_t)(1u << 14) << 32) | (uint64_t)(((ones_a >> 4) & 0x3FFFu) | (((zero_addr - ones_a) >> 4) << 16));
+          const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(((bias_a >> 4) & 0x3FFFu) | (((zero_rows - bias_a) >> 4) << 16));
+          for (int b = 0; b < nblk; ++b)
+            if (elect_one()) umma_bf16(d0 + (uint32_t)(b * p.n_tile), ad, bd, idesc, 0u);
+        }
         for (int grp = 0; grp < p.ng; ++grp, ++it) {
           const int s = it % p.stages;
           const uint32_t ph = (it / p.stages) & 1;
@@ -283,7 +307,7 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
               if (odd_entries && (uint32_t)j == last) lo = pad_lo;
               const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
               const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
-              if (elect_one()) umma_bf16(d, ad, bd, idesc, (grp | j) != 0 ? 1u : 0u);
+              if (elect_one()) umma_bf16(d, ad, bd, idesc, 1u);
             }
           }
           if (elect_one()) umma_commit(&bar_empty[s]);   // stage s may be refilled once these MMAs finish
@@ -336,13 +360,9 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
               for (int e8 = 0; e8 < 4; ++e8) {
                 const int ch = ch_base + c0 + e8 * 8;
                 if ((e8 < 2 || wide) && ch < p.c_out) {
-                  const float4 b0 = *reinterpret_cast<const float4 *>(bias_s + ch);
-                  const float4 b1 = *reinterpret_cast<const float4 *>(bias_s + ch + 4);
-                  float f[8];
-                  f[0] = __uint_as_float(v[e8 * 8 + 0]) + b0.x; f[1] = __uint_as_float(v[e8 * 8 + 1]) + b0.y;
-                  f[2] = __uint_as_float(v[e8 * 8 + 2]) + b0.z; f[3] = __uint_as_float(v[e8 * 8 + 3]) + b0.w;
-                  f[4] = __uint_as_float(v[e8 * 8 + 4]) + b1.x; f[5] = __uint_as_float(v[e8 * 8 + 5]) + b1.y;
-                  f[6] = __uint_as_float(v[e8 * 8 + 6]) + b1.z; f[7] = __uint_as_float(v[e8 * 8 + 7]) + b1.w;
+                  float f[8];                      // the bias is in the accumulator already
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(v[e8 * 8 + i]);
                   if (decltype(RES)::value) {
                     const uint4 rv = *reinterpret_cast<const uint4 *>(gres + ch);
                     const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&rv);
@@ -513,7 +533,7 @@ bool tc_plan(int n, int h, int w, const dc_geom *g, int n_sm, TcParams *p) {
 
   // shared memory: [weights][bias][output tiles x2][activation stages][slack]
   const int slack = p->mb * 2048 + 1024;
-  const int bias_bytes = (int)dc_round_up((size_t)p->nnt * p->n_tile * 4, 128);
+  const int bias_bytes = (int)dc_round_up((size_t)128 + (size_t)(p->nnt + 1) * p->n_tile * 16, 128);   // constant operand, bias rows, zero rows
   int stages = kMaxStages;
   for (;; --stages) {
     if (stages < 2) return false;
