@@ -33,6 +33,9 @@ struct StencilParams {
   int box_bytes, patch_bytes;  // bytes the TMA load delivers; the same rounded up to 128
 };
 
+// outputs of one row that a thread computes together (the kernel's register tile and the patch width depend on it)
+__host__ __device__ constexpr int outputs_per_item(int k, int stride) { return (stride == 1 ? 4 : 2) * (k == 3 ? 2 : 1); }
+
 __device__ unsigned int g_dw_status;             // DC_ERR_TIMEOUT once a wait of these kernels ran out
 
 __device__ __forceinline__ uint4 lds_u4(uint32_t a) {
@@ -51,7 +54,7 @@ __global__ void __launch_bounds__(kThreads, 4)
 k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ StencilParams p,
                  const float *__restrict__ w, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ y) {
   // outputs per thread along a row: 8 / 4 for 3x3 (4 / 2 measured 10 % and 3 % slower), 4 / 2 for 5x5 (registers)
-  constexpr int TX = (S == 1 ? 4 : 2) * (K == 3 ? 2 : 1);
+  constexpr int TX = outputs_per_item(K, S);
   constexpr int NJ = (TX - 1) * S + K;           // input columns they read
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar;
@@ -100,6 +103,9 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const uint32_t bias_sa = w_sa + (uint32_t)(K * K) * ct4;
   const uint32_t row_pitch = (uint32_t)p.in_w * ct2, img_pitch = (uint32_t)p.in_rows * row_pitch;   // bytes
   const uint32_t patch_sa = smem_u32(smem) + (uint32_t)(cv * kV) * 2u;
+  uint32_t joff[NJ];                             // byte offsets of an item's input columns (the patch is as wide as a row's last item reads)
+#pragma unroll
+  for (int j = 0; j < NJ; ++j) joff[j] = (uint32_t)j * ct2;
 #pragma unroll 1
   for (int item = (int)threadIdx.x / cvt; item < items; item += kThreads / cvt) {
     const int il = item / per_img, rem = item - il * per_img;
@@ -116,10 +122,6 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
       }
     }
-    // columns past the patch's last one only feed outputs past the row's end, which are not stored
-    uint32_t col_off[NJ];
-#pragma unroll
-    for (int j = 0; j < NJ; ++j) col_off[j] = (X0 * S + j < p.in_w ? (uint32_t)j : 0u) * ct2;
     uint32_t prow = patch_sa + (uint32_t)il * img_pitch + (uint32_t)(ry * S) * row_pitch + (uint32_t)(X0 * S) * ct2;
     uint32_t wrow = w_sa;
 #pragma unroll 1
@@ -133,7 +135,7 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
       }
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
-        const uint4 raw = lds_u4(prow + col_off[j]);
+        const uint4 raw = lds_u4(prow + joff[j]);
         const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&raw);
         float2 xv[kV / 2];
 #pragma unroll
@@ -189,7 +191,10 @@ bool stencil_plan(int n, int h, int w, int c, int k, int stride, int pad, Stenci
   // channels per tile: 32 (64-byte lines for the TMA unit; 16 measured 20 % slower, 64 leaves fewer rows per tile)
   p->ct = c % 32 == 0 ? 32 : (c % 16 == 0 ? 16 : 8);
   p->cgroups = c / p->ct;
-  p->in_w = (wo - 1) * stride + k;
+  // patch columns: up to the last input column of the last thread item of a row (an item is tx outputs wide;
+  // what lies past the image is zero-filled by the TMA unit), so that the stencil needs no column clamp
+  const int tx = outputs_per_item(k, stride);
+  p->in_w = (dc_div_up(wo, tx) * tx - 1) * stride + k;
   if (p->in_w > 256) return false;               // a TMA box is at most 256 elements wide
   const long long row_bytes = (long long)p->in_w * p->ct * 2;
   // rows per tile: as many as fit the patch limit, at least one
