@@ -49,13 +49,16 @@ __device__ __forceinline__ float4 lds_f4(uint32_t a) {
   return v;
 }
 
-template <int K, int S, int ACT>
+template <int K, int S, int ACT, int CT>
 __global__ void __launch_bounds__(kThreads, 4)
 k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ StencilParams p,
                  const float *__restrict__ w, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ y) {
   // outputs per thread along a row: 8 / 4 for 3x3 (4 / 2 measured 10 % and 3 % slower), 4 / 2 for 5x5 (registers)
   constexpr int TX = outputs_per_item(K, S);
   constexpr int NJ = (TX - 1) * S + K;           // input columns they read
+  // channels per tile: compile-time for the common 32 (every shared-memory offset of the stencil is then an
+  // immediate of its load), run-time otherwise
+  const int ct = CT ? CT : p.ct;
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bar;
   __shared__ uint32_t abort_word;
@@ -67,7 +70,7 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int cg = t % p.cgroups; t /= p.cgroups;
   const int ty = t % p.ytiles;
   const int ig = t / p.ytiles;
-  const int c0 = cg * p.ct, y0 = ty * p.rt, img0 = ig * p.ni;
+  const int c0 = cg * ct, y0 = ty * p.rt, img0 = ig * p.ni;
 
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
@@ -80,8 +83,8 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     // coordinates may be negative or reach past the tensor: those elements arrive as zeros
     tma_load_4d(smem_u32(smem), &map_x, &bar, c0, -p.pad, y0 * S - p.pad, img0);
   }
-  for (int i = (int)threadIdx.x; i < (K * K + 1) * p.ct; i += kThreads) {
-    const int tap = i / p.ct, ch = i - tap * p.ct;
+  for (int i = (int)threadIdx.x; i < (K * K + 1) * ct; i += kThreads) {
+    const int tap = i / ct, ch = i - tap * ct;
     w_s[i] = tap < K * K ? w[(size_t)tap * p.c + c0 + ch] : (bias ? bias[c0 + ch] : 0.f);
   }
   __syncthreads();
@@ -90,80 +93,90 @@ k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     return;
   }
 
-  const int cvt = p.ct / kV;                     // vectors per pixel of this tile: divides kThreads
+  const int cvt = ct / kV;                       // vectors per pixel of this tile: divides kThreads
   const int cv = (int)threadIdx.x % cvt;         // this thread's vector, the same for all its items
   const int xtiles = (p.wo + TX - 1) / TX;
   const int rows_valid = p.ho - y0 < p.rt ? p.ho - y0 : p.rt;
   const int imgs_valid = p.n_img - img0 < p.ni ? p.n_img - img0 : p.ni;
-  const int per_img = rows_valid * xtiles;
-  const int items = imgs_valid * per_img;
   // shared-memory addresses as 32-bit offsets (the loop below is bound by its instruction stream)
-  const uint32_t ct2 = (uint32_t)p.ct * 2u, ct4 = (uint32_t)p.ct * 4u;
+  const uint32_t ct2 = (uint32_t)ct * 2u, ct4 = (uint32_t)ct * 4u;
   const uint32_t w_sa = smem_u32(w_s) + (uint32_t)(cv * kV) * 4u;         // this thread's 8 channels of tap 0
-  const uint32_t bias_sa = w_sa + (uint32_t)(K * K) * ct4;
   const uint32_t row_pitch = (uint32_t)p.in_w * ct2, img_pitch = (uint32_t)p.in_rows * row_pitch;   // bytes
   const uint32_t patch_sa = smem_u32(smem) + (uint32_t)(cv * kV) * 2u;
-  uint32_t joff[NJ];                             // byte offsets of an item's input columns (the patch is as wide as a row's last item reads)
-#pragma unroll
-  for (int j = 0; j < NJ; ++j) joff[j] = (uint32_t)j * ct2;
+  const size_t c2 = (size_t)p.c * 2;             // bytes from one output pixel to the next
+  // items (image, row, group of TX outputs) of this thread: the first one by division, the following ones by
+  // adding the decomposed step with carries (two divisions per item cost more than the rest of its index work)
+  const int step = kThreads / cvt;
+  const int d_il = step / (rows_valid * xtiles), d_rem = step - d_il * rows_valid * xtiles;
+  const int d_ry = d_rem / xtiles, d_xt = d_rem - d_ry * xtiles;
+  int il, ry, xt;
+  {
+    const int item = (int)threadIdx.x / cvt;
+    il = item / (rows_valid * xtiles);
+    const int rem = item - il * rows_valid * xtiles;
+    ry = rem / xtiles;
+    xt = rem - ry * xtiles;
+  }
 #pragma unroll 1
-  for (int item = (int)threadIdx.x / cvt; item < items; item += kThreads / cvt) {
-    const int il = item / per_img, rem = item - il * per_img;
-    const int ry = rem / xtiles, xt = rem - ry * xtiles;
+  while (il < imgs_valid) {
     const int X0 = xt * TX;
     // packed fp32 arithmetic (two multiply-adds per instruction): the layer has 4.5 FLOP per byte
     // moved, which one scalar FMA per instruction would not keep up with
     float2 acc[TX][kV / 2];
+    float2 bz[kV / 2];
     {
-      const float4 b0 = lds_f4(bias_sa), b1 = lds_f4(bias_sa + 16u);
-#pragma unroll
-      for (int o = 0; o < TX; ++o) {
-        acc[o][0] = make_float2(b0.x, b0.y); acc[o][1] = make_float2(b0.z, b0.w);
-        acc[o][2] = make_float2(b1.x, b1.y); acc[o][3] = make_float2(b1.z, b1.w);
-      }
+      const float4 b0 = lds_f4(w_sa + (uint32_t)(K * K) * ct4), b1 = lds_f4(w_sa + (uint32_t)(K * K) * ct4 + 16u);
+      bz[0] = make_float2(b0.x, b0.y); bz[1] = make_float2(b0.z, b0.w);
+      bz[2] = make_float2(b1.x, b1.y); bz[3] = make_float2(b1.z, b1.w);
     }
     uint32_t prow = patch_sa + (uint32_t)il * img_pitch + (uint32_t)(ry * S) * row_pitch + (uint32_t)(X0 * S) * ct2;
-    uint32_t wrow = w_sa;
-#pragma unroll 1
-    for (int r = 0; r < K; ++r, prow += row_pitch, wrow += (uint32_t)K * ct4) {
+    // tap rows unrolled: the first one starts every accumulator from the bias (no copy of it), and with a
+    // compile-time tile width the weights' and inputs' offsets are immediates
+#pragma unroll
+    for (int r = 0; r < K; ++r, prow += row_pitch) {
       float2 wr[K][kV / 2];
 #pragma unroll
       for (int sx = 0; sx < K; ++sx) {
-        const float4 w0 = lds_f4(wrow + (uint32_t)sx * ct4), w1 = lds_f4(wrow + (uint32_t)sx * ct4 + 16u);
+        const uint32_t wa = w_sa + (uint32_t)(r * K + sx) * ct4;
+        const float4 w0 = lds_f4(wa), w1 = lds_f4(wa + 16u);
         wr[sx][0] = make_float2(w0.x, w0.y); wr[sx][1] = make_float2(w0.z, w0.w);
         wr[sx][2] = make_float2(w1.x, w1.y); wr[sx][3] = make_float2(w1.z, w1.w);
       }
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
-        const uint4 raw = lds_u4(prow + joff[j]);
-        const __nv_bfloat162 *rb = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-        float2 xv[kV / 2];
+        const uint4 raw = lds_u4(prow + (uint32_t)j * ct2);
+        const uint32_t *rw = reinterpret_cast<const uint32_t *>(&raw);
+        float2 xv[kV / 2];                       // bf16 -> fp32: the 16 bits moved to the top of a word
 #pragma unroll
-        for (int i = 0; i < 4; ++i) xv[i] = __bfloat1622float2(rb[i]);
+        for (int i = 0; i < 4; ++i) xv[i] = make_float2(__uint_as_float(rw[i] << 16), __uint_as_float(rw[i] & 0xFFFF0000u));
 #pragma unroll
         for (int o = 0; o < TX; ++o) {
           const int sx = j - o * S;                // tap column with which input j feeds output o
           if (sx >= 0 && sx < K) {
 #pragma unroll
-            for (int q = 0; q < kV / 2; ++q) acc[o][q] = __ffma2_rn(xv[q], wr[sx][q], acc[o][q]);
+            for (int q = 0; q < kV / 2; ++q) acc[o][q] = __ffma2_rn(xv[q], wr[sx][q], r == 0 && sx == 0 ? bz[q] : acc[o][q]);
           }
         }
       }
     }
-    __nv_bfloat16 *yrow = y + (((size_t)(img0 + il) * p.ho + (size_t)(y0 + ry)) * p.wo) * p.c + c0 + cv * kV;
+    uint8_t *yp = reinterpret_cast<uint8_t *>(y + (((size_t)(img0 + il) * p.ho + (size_t)(y0 + ry)) * p.wo + (size_t)X0) * p.c + c0 + cv * kV);
+    const int n_out = p.wo - X0;                 // outputs of this item inside the row (the last item may hang over)
 #pragma unroll
-    for (int o = 0; o < TX; ++o) {
-      if (X0 + o < p.wo) {
-        uint4 ov;
-        uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
-        // ReLU6 (compile-time): the conversion clamps at zero itself, one packed minimum against (6, 6) does
-        // the rest -- the same values as clamping before rounding, since 0 and 6 are bf16 values
+    for (int o = 0; o < TX; ++o, yp += c2) {
+      uint4 ov;
+      uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
+      // ReLU6 (compile-time): the conversion clamps at zero itself, one packed minimum against (6, 6) does
+      // the rest -- the same values as clamping before rounding, since 0 and 6 are bf16 values
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          ow[i] = ACT ? min_bf16x2(pack_bf16x2_relu(acc[o][i].x, acc[o][i].y), 0x40C040C0u) : pack_bf16x2(acc[o][i].x, acc[o][i].y);
-        *reinterpret_cast<uint4 *>(yrow + (size_t)(X0 + o) * p.c) = ov;
-      }
+      for (int i = 0; i < 4; ++i)
+        ow[i] = ACT ? min_bf16x2(pack_bf16x2_relu(acc[o][i].x, acc[o][i].y), 0x40C040C0u) : pack_bf16x2(acc[o][i].x, acc[o][i].y);
+      if (o < n_out) *reinterpret_cast<uint4 *>(yp) = ov;
     }
+    xt += d_xt;
+    if (xt >= xtiles) { xt -= xtiles; ++ry; }
+    ry += d_ry;
+    if (ry >= rows_valid) { ry -= rows_valid; ++il; }
+    il += d_il;
   }
 }
 
@@ -249,12 +262,17 @@ dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, in
   const int smem = p.patch_bytes + (k * k + 1) * p.ct * 4 + 256;
   const int grid = p.igroups * p.ytiles * p.cgroups;
   __nv_bfloat16 *yp = (__nv_bfloat16 *)y;
-#define DC_DW_LAUNCH1(KK, SS, AA)                                                                         \
+#define DC_DW_LAUNCH2(KK, SS, AA, CC)                                                                        \
   do {                                                                                                    \
     static unsigned char attr_done[kDcMaxDevices];                                                        \
-    DC_CUDA_OK(dc_set_max_smem_once(k_dwconv_stencil<KK, SS, AA>, kTileBytes + 8 * 1024, attr_done));     \
-    if (dc_launch_pdl(k_dwconv_stencil<KK, SS, AA>, dim3(grid), dim3(kThreads), (size_t)smem, st, map_x, p, wp, bias, yp) != cudaSuccess) \
+    DC_CUDA_OK(dc_set_max_smem_once(k_dwconv_stencil<KK, SS, AA, CC>, kTileBytes + 8 * 1024, attr_done));     \
+    if (dc_launch_pdl(k_dwconv_stencil<KK, SS, AA, CC>, dim3(grid), dim3(kThreads), (size_t)smem, st, map_x, p, wp, bias, yp) != cudaSuccess) \
       return DC_ERR_CUDA;                                                                                 \
+  } while (0)
+#define DC_DW_LAUNCH1(KK, SS, AA)                                                                         \
+  do {                                                                                                    \
+    if (p.ct == 32) DC_DW_LAUNCH2(KK, SS, AA, 32);                                                        \
+    else DC_DW_LAUNCH2(KK, SS, AA, 0);                                                                    \
   } while (0)
 #define DC_DW_LAUNCH(KK, SS)                                                                              \
   do {                                                                                                    \
@@ -265,6 +283,7 @@ dc_status dc_launch_dwconv_stencil(const void *x, int n, int h, int w, int c, in
   else if (k == 3) DC_DW_LAUNCH(3, 2);
   else if (stride == 1) DC_DW_LAUNCH(5, 1);
   else DC_DW_LAUNCH(5, 2);
+#undef DC_DW_LAUNCH2
 #undef DC_DW_LAUNCH1
 #undef DC_DW_LAUNCH
   return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
