@@ -85,7 +85,7 @@ struct Item {
   }
 };
 
-// RESIDENT: all weights of the layer (a single output-channel pass, at most 96 KB) stay in shared memory:
+// RESIDENT: all weights of the layer (a single output-channel pass, at most 128 KB) stay in shared memory:
 // one copy per CTA instead of one stream per work item.  Compile-time, so that the streaming version's
 // loops carry no switches.
 template <bool RESIDENT>
@@ -292,7 +292,11 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int ew = warp - kFirstEpiWarp;
       const int q = warp & 3, par = ew >> 2;
       const uint32_t tmem_row = tmem_base + ((uint32_t)(q * 32) << 16);
-      uint8_t *stage = smem + p.off_stage + ew * (32 * kStagePitch);   // this warp's turn-around buffer
+      // this warp's turn-around buffer, as 32-bit shared addresses: where this lane writes its pixel, and where it
+      // reads the piece it stores of pixel lane / 4 (the three other pixels lie 8 * kStagePitch bytes apart)
+      const uint32_t stage = smem_u32(smem + p.off_stage + ew * (32 * kStagePitch));
+      const uint32_t stage_wr = stage + (uint32_t)lane * kStagePitch;
+      const uint32_t stage_rd = stage + (uint32_t)(lane >> 2) * kStagePitch + (uint32_t)(lane & 3) * 16u;
       uint32_t acc_ph[2] = {0u, 0u};
       const bool relu6 = p.act == DC_ACT_RELU6;
 #pragma unroll 1
@@ -354,24 +358,21 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
           // the four pixels this lane helps to store (pixel i * 8 + lane / 4 of the warp's 32): their addresses
           // come from the lanes that own them, once per block
-          unsigned long long px_base[4];
+          uint8_t *px_ptr[4];                              // + 16 bytes per lane of the four that share a pixel
           bool px_on[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            px_base[i] = __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, i * 8 + (lane >> 2));
+            px_ptr[i] = reinterpret_cast<uint8_t *>((uintptr_t)__shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)dst, i * 8 + (lane >> 2))) + (lane & 3) * 16;
             px_on[i] = (vmask >> (i * 8 + (lane >> 2))) & 1u;
           }
           auto emit32 = [&](auto RELU, auto RES, const uint32_t *v, int c0) {
 #pragma unroll
-            for (int g8 = 0; g8 < 4; ++g8)
-              *reinterpret_cast<uint4 *>(stage + lane * kStagePitch + g8 * 16) = cook8(RELU, RES, v + 8 * g8, c0 + 8 * g8);
+            for (int g8 = 0; g8 < 4; ++g8) sts_u4(stage_wr + (uint32_t)g8 * 16u, cook8(RELU, RES, v + 8 * g8, c0 + 8 * g8));
             __syncwarp();
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const int px = i * 8 + (lane >> 2), c = lane & 3;
-              if (px_on[i])
-                *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>((uintptr_t)px_base[i]) + c0 + c * 8) =
-                    *reinterpret_cast<const uint4 *>(stage + px * kStagePitch + c * 16);
+              const uint4 piece = lds_u4(stage_rd + (uint32_t)(i * 8 * kStagePitch));
+              if (px_on[i]) *reinterpret_cast<uint4 *>(px_ptr[i] + (size_t)c0 * 2) = piece;
             }
             __syncwarp();
           };
@@ -452,15 +453,23 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->planes = dc_div_up(g->c_in, 64);
   p->n_tile = ko.n_tile; p->nnt = ko.nnt; p->n_pad = ko.n_pad;
   p->planes_all = ko.e_pad;
-  // tile: as many rows as fit kMaxLines GEMM rows; whole small images several at a time
-  p->nxt = 1;
-  while (dc_div_up(wo, p->nxt) + g->k - 1 > kMaxLines / g->k) ++p->nxt;   // at least one output row per tile
-  p->tw = dc_div_up(wo, p->nxt);
-  p->nxt = dc_div_up(wo, p->tw);
+  // tile: as many rows as fit kMaxLines GEMM rows; whole small images several at a time.  Rows may be cut into
+  // strips: of the first few strip counts that fit, the one with the fewest tiles per image wins (28 x 28 with a
+  // 3 x 3 kernel: two strips of 14 columns x 14 rows make 4 tiles where full rows x 6 make 5)
+  int nxt0 = 1;
+  while (dc_div_up(wo, nxt0) + g->k - 1 > kMaxLines / g->k) ++nxt0;       // at least one output row per tile
+  int th = 0, best_tiles = 0;
+  p->nxt = 0;
+  for (int cand = nxt0; cand <= nxt0 + 3 && cand <= wo; ++cand) {
+    const int tw_c = dc_div_up(wo, cand), nxt_c = dc_div_up(wo, tw_c);
+    int th_c = kMaxLines / (tw_c + g->k - 1) - (g->k - 1);
+    if (th_c < 1) continue;
+    if (th_c > ho) th_c = ho;
+    const int tiles_c = nxt_c * dc_div_up(ho, th_c);
+    if (p->nxt == 0 || tiles_c < best_tiles) { p->nxt = nxt_c; p->tw = tw_c; th = th_c; best_tiles = tiles_c; }
+  }
+  if (p->nxt == 0) return false;
   p->wbox = p->tw + g->k - 1;
-  int th = kMaxLines / p->wbox - (g->k - 1);
-  if (th < 1) return false;
-  if (th > ho) th = ho;
   p->th = th;
   p->rbox = th + g->k - 1;
   p->lines_img = p->rbox * p->wbox;
@@ -500,11 +509,12 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->off_a = (int)dc_round_up((size_t)p->off_stage + kEpiWarps * 32 * kStagePitch, 1024);
   // rings: weights first (they are the larger stream), then activation planes
   int sa = 2, sb = 2;
-  // Small weights of a single pass with many input channels stay resident: then a work item streams its
-  // activation planes only.  (For layers of one or two planes the weight stream is small beside the
-  // activations and the resident version measured no faster.)
+  // Small weights of a single pass stay resident where a work item would otherwise stream more weight than
+  // activation bytes (many input planes, or a k x k kernel on few): then it streams its activation planes only.
+  // (For 1 x 1 layers of one or two planes the weight stream is small beside the activations and the resident
+  // version measured no faster.)
   const long long b_all = (long long)dc_round_up((size_t)ko.e_pad * p->n_tile * 16, 1024);
-  p->b_resident = (p->nnt == 1 && p->planes >= 3 && b_all <= 96 * 1024) ? 1 : 0;
+  p->b_resident = (p->nnt == 1 && b_all <= 128 * 1024 && (p->planes >= 3 || b_all >= 2ll * p->a_stage_bytes)) ? 1 : 0;
   auto total = [&](int a, int b) {
     const long long wbytes = p->b_resident ? b_all : (long long)b * p->b_stage_bytes;
     const long long tail = wbytes >= 26 * 1024 ? kSlack : 26 * 1024 - wbytes + kSlack;   // room for the overrun
