@@ -937,7 +937,7 @@ static dc_status merge_walk(const dc_layer *layers, int n, const dc_residual *re
       t.n = cnt;
       if (go) {
         int bx = blocks_for(max_total, 256);
-        dim3 grid(bx > 64 ? 64 : bx, cnt);
+        dim3 grid(bx > 1024 ? 1024 : bx, cnt);       // a few elements per thread: the launch is short beside its chain
         k_fold_bn<<<grid, 256, 0, st>>>(t);
       }
       cnt = 0;
