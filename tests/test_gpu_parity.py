@@ -400,7 +400,7 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (32, 16, 1, 1, 0, 2, 20, 24, "k_conv_tc_pairrows"),     # 1x1: one instruction per 32-byte K step
     (32, 96, 1, 1, 0, 2, 20, 24, "k_conv_tc_rows"),         # 1x1 expansion from few channels: one half-filled plane
     (16, 96, 1, 1, 0, 1, 40, 112, "k_conv_tc_rows"),        # 1x1 expansion from 16 channels, row tiles
-    (32, 192, 3, 1, 1, 2, 28, 28, "k_conv_tc_rows"),        # 3x3 from few channels to more outputs than the pair rows take
+    (32, 192, 3, 1, 1, 2, 28, 28, "k_conv_tc_rows"),        # 3x3 from few channels to more outputs than the pair rows take: two column strips, 110 KB of resident weights
     (16, 136, 5, 1, 2, 1, 12, 20, "k_conv_tc_rows"),        # the same with 16 channels and a 5x5 kernel, two passes
     (32, 40, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with 40 outputs: general kernel
     (16, 128, 3, 1, 1, 1, 12, 16, "k_conv_tc_pairrows"),    # N = 256: two accumulator slots, run-time channel loop
@@ -411,7 +411,9 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
     (128, 128, 5, 1, 2, 2, 14, 14, "k_conv_tc_rows"),       # 5x5 with 128 outputs: two passes of 64 (weight stage limit)
     (96, 96, 7, 1, 3, 1, 14, 14, "k_conv_tc_rows"),         # 7x7: passes of at most 80 output channels
-    (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc_rows"),        # many channels, 32 outputs: rows kernel with resident weights
+    (144, 32, 3, 1, 1, 1, 28, 28, "k_conv_tc_rows"),        # many channels, 32 outputs: rows kernel with resident weights, two strips of 14 x 14
+    (80, 48, 3, 1, 1, 2, 14, 27, "k_conv_tc_rows"),         # ragged strips (14 + 13 columns), whole height per tile
+    (64, 64, 3, 1, 1, 1, 33, 45, "k_conv_tc_rows"),         # three strips of 15 columns, row tiles of 13, 13 and 7
     (200, 24, 3, 1, 1, 2, 14, 14, "k_conv_tc"),             # many channels, fewer than 32 outputs: general kernel
     (192, 32, 1, 1, 0, 2, 28, 28, "k_conv_tc_rows"),        # 1x1 projection to 32 channels
 ])
@@ -435,6 +437,31 @@ def test_each_forward_kernel_against_the_oracle(dc, c_in, c_out, k, s, p, n, h, 
     assert_close(nchw(y), lin, TOL_BF16)
     y = run_conv(dc, dev(x, torch.bfloat16), g, packed, bf, dc.ACT_RELU6, residual=dev(r, torch.bfloat16))
     assert_close(nchw(y), O.relu6(lin + r.transpose(0, 3, 1, 2)), TOL_BF16)
+
+
+@pytest.mark.parametrize("c,k,s,p,n,h,w", [(64, 3, 1, 1, 2, 19, 21), (48, 3, 2, 1, 1, 20, 30), (32, 5, 1, 2, 1, 11, 13)])
+def test_dwconv_stencil_without_activation(dc, c, k, s, p, n, h, w):
+    """The stencil's instantiations without ReLU6 (tile widths 32 and 16, widths that are no multiple of a
+    thread's item): negative and large outputs must come through unclamped."""
+    spec = I.make_layer(18, 0, c, c, k, s, p, depthwise=True)
+    lay = dc.DeviceLayer(spec)
+    wf = torch.empty_like(lay.weight)
+    bf = torch.empty(c, device="cuda")
+    dc.fold_bn(lay, wf, bf)
+    g = dc.geom(c, c, c, k, s, p)
+    packed = torch.empty(dc.packed_bytes(g, dc.F32) // 4, dtype=torch.float32, device="cuda")
+    dc.pack_weights(wf, g, dc.F32, packed)
+    x = 4.0 * I.make_input(19, (n, h, w, c), bf16=True)
+    x = I.round_bf16(x)
+    ho, wo = O.out_extent(h, k, s, p), O.out_extent(w, k, s, p)
+    gy = Guarded(torch, (n, ho, wo, c), torch.bfloat16, fill=float("nan"))
+    dc.dwconv_forward(dev(x, torch.bfloat16), k, s, p, packed, bf, dc.ACT_IDENTITY, gy.t)
+    assert dc.dwconv_status() == dc.OK
+    gy.check("depthwise output")
+    Wf, bfo = O.fold_bn(spec)
+    ref = O.conv_direct(x.transpose(0, 3, 1, 2), Wf, bfo, k, s, p, groups=c)
+    assert ref.min() < -1.0 and ref.max() > 6.5        # the case does exercise what ReLU6 would have cut
+    assert_close(nchw(gy.t), ref, TOL_BF16, bf16=True)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
