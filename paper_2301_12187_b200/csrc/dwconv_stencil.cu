@@ -33,8 +33,15 @@ struct StencilParams {
   int box_bytes, patch_bytes;  // bytes the TMA load delivers; the same rounded up to 128
 };
 
-// outputs of one row that a thread computes together (the kernel's register tile and the patch width depend on it)
-__host__ __device__ constexpr int outputs_per_item(int k, int stride) { return (stride == 1 ? 4 : 2) * (k == 3 ? 2 : 1); }
+// Outputs of one row that a thread computes together (the kernel's register tile and the patch width depend on
+// it).  Stride 1: an ODD count.  The two items of a quarter warp (4 lanes = the 64 bytes of a 32-channel pixel
+// each) then read pixels of different parity, i.e. the two halves of the 128 bytes that the 32 banks span; with
+// 8 outputs per item all eight items of a warp read from the same 16 banks and every 16-byte load took two
+// wavefronts (112 x 112 x 32: 49 us with 8, 42 us with 7; 5x5 at 28 x 28 x 240: 96 us with 4, 48 us with 5).
+// Stride 2 moves an item by an even number of pixels whatever the count.
+__host__ __device__ constexpr int outputs_per_item(int k, int stride) {
+  return stride == 1 ? (k == 3 ? 7 : 5) : (k == 3 ? 4 : 2);
+}
 
 __device__ unsigned int g_dw_status;             // DC_ERR_TIMEOUT once a wait of these kernels ran out
 
@@ -48,7 +55,6 @@ template <int K, int S, int ACT, int CT>
 __global__ void __launch_bounds__(kThreads, 4)
 k_dwconv_stencil(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ StencilParams p,
                  const float *__restrict__ w, const float *__restrict__ bias, __nv_bfloat16 *__restrict__ y) {
-  // outputs per thread along a row: 8 / 4 for 3x3 (4 / 2 measured 10 % and 3 % slower), 4 / 2 for 5x5 (registers)
   constexpr int TX = outputs_per_item(K, S);
   constexpr int NJ = (TX - 1) * S + K;           // input columns they read
   // channels per tile: compile-time for the common 32 (every shared-memory offset of the stencil is then an
