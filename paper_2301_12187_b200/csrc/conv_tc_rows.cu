@@ -36,7 +36,7 @@ constexpr int kConsumerThreads = (kMmaWarps + kEpiWarps) * 32;
 constexpr int kThreads = 32 + kConsumerThreads;
 constexpr int kBarConsumers = 7;                 // named barrier of all consumer warps
 constexpr int kMaxBlocks = 2;                    // 128-row blocks per tile
-constexpr int kStagePitch = 80;                  // bytes per pixel in an epilogue warp's turn-around buffer (64 + 16)
+constexpr int kStagePitch = 64;                  // bytes per pixel in an epilogue warp's turn-around buffer (pieces XOR-swizzled)
 
 struct RowsParams {
   int n_img, h, w, ho, wo, c_in, c_out;
@@ -295,8 +295,12 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // this warp's turn-around buffer, as 32-bit shared addresses: where this lane writes its pixel, and where it
       // reads the piece it stores of pixel lane / 4 (the three other pixels lie 8 * kStagePitch bytes apart)
       const uint32_t stage = smem_u32(smem + p.off_stage + ew * (32 * kStagePitch));
-      const uint32_t stage_wr = stage + (uint32_t)lane * kStagePitch;
-      const uint32_t stage_rd = stage + (uint32_t)(lane >> 2) * kStagePitch + (uint32_t)(lane & 3) * 16u;
+      // 16-byte piece g of pixel px sits at piece g ^ ((px >> 1) & 3) of the pixel's 64 bytes: the eight lanes of a
+      // quarter warp then touch eight different 16-byte bank groups both when every lane writes piece g of its own
+      // pixel and when four lanes read the four pieces of each of two neighbouring pixels
+      const uint32_t stage_wr = stage + (uint32_t)lane * kStagePitch, swz_wr = (uint32_t)((lane >> 1) & 3);
+      const uint32_t stage_rd = stage + (uint32_t)(lane >> 2) * kStagePitch +
+                                (uint32_t)((lane & 3) ^ ((lane >> 3) & 3)) * 16u;
       uint32_t acc_ph[2] = {0u, 0u};
       const bool relu6 = p.act == DC_ACT_RELU6;
 #pragma unroll 1
@@ -353,7 +357,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // 32 accumulator columns per read while they last.  A thread owns a pixel, so stored directly
           // its 16-byte pieces would land c_out * 2 bytes apart from its neighbours' (half-filled
           // sectors, 32 lines per instruction).  The warp instead turns the 32 pixels x 64 bytes around
-          // in its staging buffer (80-byte pitch: conflict-free) and writes them four lanes to a
+          // in its staging buffer (64-byte pitch, pieces XOR-swizzled: conflict-free both ways) and writes them four lanes to a
           // pixel: every store instruction then fills eight whole 64-byte segments.
           const uint32_t vmask = __ballot_sync(0xffffffffu, valid);
           // the four pixels this lane helps to store (pixel i * 8 + lane / 4 of the warp's 32): their addresses
@@ -367,7 +371,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           auto emit32 = [&](auto RELU, auto RES, const uint32_t *v, int c0) {
 #pragma unroll
-            for (int g8 = 0; g8 < 4; ++g8) sts_u4(stage_wr + (uint32_t)g8 * 16u, cook8(RELU, RES, v + 8 * g8, c0 + 8 * g8));
+            for (int g8 = 0; g8 < 4; ++g8) sts_u4(stage_wr + (((uint32_t)g8 ^ swz_wr) << 4), cook8(RELU, RES, v + 8 * g8, c0 + 8 * g8));
             __syncwarp();
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
