@@ -162,6 +162,8 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
   }
 
   // ---- bands of this CTA; the next band's rows arrive while this one is multiplied and written
+  const int wrot = (wj >> 2) & 3;                // widen: rotation of a lane's four pixels
+  const int rot = (tid >> 1) & 3;                // rotation of this lane's output pieces (read-out)
   int it = 0;
   for (int bi = (int)blockIdx.x; bi < total; bi += (int)gridDim.x, ++it) {
     const int Y0 = band * p.rb;
@@ -195,10 +197,16 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
             b = lds64(sj + 8);
             c = lds64(sj + 16);
           }
-          sts64(dj, a.x, __byte_perm(a.y, one, 0x5410));
-          sts64(dj + 8, __byte_perm(a.y, b.x, 0x5432), __byte_perm(b.x, one, 0x5432));
-          sts64(dj + 16, b.y, __byte_perm(c.x, one, 0x5410));
-          sts64(dj + 24, __byte_perm(c.x, c.y, 0x5432), __byte_perm(c.y, one, 0x5432));
+          // the four widened pixels leave as four 8-byte stores (the row starts `pad` pixels in, so 16-byte
+          // stores would be misaligned).  A lane's 32 bytes start 32 bytes after its neighbour's: stored in the
+          // same order by every lane, lanes j, j + 4, j + 8, j + 12 of a half warp would hit the same banks, so
+          // lane j stores its pixel (t + j / 4) mod 4 in turn t (rotated in registers as in the read-out)
+          uint2 px[4] = {make_uint2(a.x, __byte_perm(a.y, one, 0x5410)), make_uint2(__byte_perm(a.y, b.x, 0x5432), __byte_perm(b.x, one, 0x5432)),
+                         make_uint2(b.y, __byte_perm(c.x, one, 0x5410)), make_uint2(__byte_perm(c.x, c.y, 0x5432), __byte_perm(c.y, one, 0x5432))};
+          if (wrot & 1) { const uint2 t0 = px[0]; px[0] = px[1]; px[1] = px[2]; px[2] = px[3]; px[3] = t0; }
+          if (wrot & 2) { const uint2 t0 = px[0], t1 = px[1]; px[0] = px[2]; px[1] = px[3]; px[2] = t0; px[3] = t1; }
+#pragma unroll
+          for (int t = 0; t < 4; ++t) sts64(dj + (uint32_t)(((t + wrot) & 3) * 8), px[t].x, px[t].y);
         }
       }
     } else {
@@ -265,10 +273,14 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
           tmem_ld32(trow + (uint32_t)(blk * p.n_pad + c0), v);
           tmem_ld_wait();
           if (PLAIN) {
+            // A lane owns a pixel, and with 32 output channels a pixel is 64 bytes: piece g of eight neighbouring
+            // lanes would fall on two 16-byte bank groups (four wavefronts per quarter warp).  Lane L therefore
+            // stores its piece (t + L / 2) mod 4 in turn t: the eight lanes then hit eight different groups.  The
+            // pieces are rotated in registers by two conditional moves (by one, then by two).
+            uint4 ov[4];
 #pragma unroll
             for (int g8 = 0; g8 < 4; ++g8) {
-              uint4 ov;
-              uint32_t *ow = reinterpret_cast<uint32_t *>(&ov);
+              uint32_t *ow = reinterpret_cast<uint32_t *>(&ov[g8]);
               // ReLU6: the conversion clamps at zero itself, one packed minimum against (6, 6) does the rest
               // (the same values as clamping before rounding, since 0 and 6 are bf16 values)
 #pragma unroll
@@ -276,7 +288,13 @@ k_conv_stem_s2(const __grid_constant__ S2Params p, const __nv_bfloat16 *__restri
                 const float f0 = __uint_as_float(v[8 * g8 + 2 * i]), f1 = __uint_as_float(v[8 * g8 + 2 * i + 1]);
                 ow[i] = RELU ? min_bf16x2(pack_bf16x2_relu(f0, f1), 0x40C040C0u) : pack_bf16x2(f0, f1);
               }
-              if (valid && c0 + 8 * g8 < p.c_out) sts128(so + (uint32_t)((c0 + 8 * g8) * 2), ov);
+            }
+            if (rot & 1) { const uint4 t0 = ov[0]; ov[0] = ov[1]; ov[1] = ov[2]; ov[2] = ov[3]; ov[3] = t0; }
+            if (rot & 2) { const uint4 t0 = ov[0], t1 = ov[1]; ov[0] = ov[2]; ov[1] = ov[3]; ov[2] = t0; ov[3] = t1; }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              const int g8 = (t + rot) & 3;       // the piece that now sits in ov[t]
+              if (valid && c0 + 8 * g8 < p.c_out) sts128(so + (uint32_t)((c0 + 8 * g8) * 2), ov[t]);
             }
           } else {
             const size_t oi = (((size_t)img_now * p.ho + (Y0 + ry)) * p.wo + X) * p.c_out;
