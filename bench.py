@@ -6,8 +6,9 @@ convolutions (dc_merge_chain: BN fold, composition, skip fold, repack) and run t
 convolution forward over the batch (dc_conv_forward).  Headline workload: the MobileNetV2-1.0
 inverted-residual block at 56x56, batch 64, bf16 (1x1 24->144, dw3x3, 1x1 144->24, skip folded ->
 one 3x3 conv 24->24).  The default run also measures the stride-2 merge (cfg2), the cross-block
-merge (cfg3) and the full depth-compressed MobileNetV2-1.0 (cfg4) and reports them under
-`per_config` of the same JSON line.
+merge (cfg3) and the full depth-compressed MobileNetV2-1.0 (cfg4: with every valid span of a seeded
+pattern merged, and cut by Algorithm 1 over the latency table measured on the spot) and reports them
+under `per_config` of the same JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|cfg1|cfg2|cfg3|cfg4] [--impl reference]
 
@@ -682,6 +683,13 @@ def run_ours(args):
         if want_cpu:
             entry["cpu_baseline"] = cpu_baseline_network(net, cn)
         per["cfg4"] = entry
+        # the same network cut by Algorithm 1 over the latency table measured here (the paper's own way to pick
+        # the merge pattern; the plan above merges every valid span of a fixed seeded pattern instead)
+        del cn, net
+        import copy
+        args_lat = copy.copy(args)
+        args_lat.plan = "latency"
+        per["cfg4_latency_plan"] = measure_network(args_lat, peaks, peak_src)[0]
         out["per_config"] = per
     print(json.dumps(out))
 
@@ -703,7 +711,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--workload", default="all", choices=["all"] + sorted(WORKLOADS),
-                    help="all: cfg1 as the headline line plus cfg1..cfg4 under per_config (one GPU); cfgN: that workload alone")
+                    help="all: cfg1 as the headline line plus cfg1..cfg4 (cfg4 under both plans) under per_config (one GPU); cfgN: that workload alone")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-streams", type=int, default=3, help="steps in flight in the end-to-end measurement of the chain workloads")
