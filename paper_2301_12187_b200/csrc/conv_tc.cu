@@ -265,6 +265,9 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
       const uint32_t desc_hi = (128u >> 4) | (1u << 14);
       const int npairs = p.e_pad / 2;
       const uint32_t zero_addr = smem_u32(smem_zero);
+      // one election for the whole role: the same lane issues every instruction, a stage's instructions in one
+      // stretch (an election and a branch per instruction cost the warp several times the instruction itself)
+      const bool leader = elect_one();
       uint32_t it = 0, tile_i = 0;
       for (int cur = cta_begin; cur < cta_end; ++tile_i) {
         const Tile t = decode_tile(p, cur, cta_end);
@@ -281,8 +284,9 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
           const uint32_t zero_rows = smem_u32(smem_bias) + (uint32_t)(p.nnt * p.n_tile * 16);
           const uint64_t ad = ((uint64_t)(1u << 14) << 32) | (uint64_t)(((ones_a >> 4) & 0x3FFFu) | (((zero_addr - ones_a) >> 4) << 16));
           const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(((bias_a >> 4) & 0x3FFFu) | (((zero_rows - bias_a) >> 4) << 16));
-          for (int b = 0; b < nblk; ++b)
-            if (elect_one()) umma_bf16(d0 + (uint32_t)(b * p.n_tile), ad, bd, idesc, 0u);
+          if (leader)
+            for (int b = 0; b < nblk; ++b) umma_bf16(d0 + (uint32_t)(b * p.n_tile), ad, bd, idesc, 0u);
+          __syncwarp();
         }
         for (int grp = 0; grp < p.ng; ++grp, ++it) {
           const int s = it % p.stages;
@@ -298,21 +302,25 @@ k_conv_tc(const void *__restrict__ w_packed, const __grid_constant__ TcParams p,
           const uint32_t last = (uint32_t)(npairs - 1);
           const uint32_t first_off = (p.a_desc_lo[last] & 0x3FFFu) << 4;
           const uint32_t pad_lo = (first_off >> 4) | (((zero_addr - a_base - first_off) >> 4) << 16);
-          for (int b = 0; b < nblk; ++b) {
-            const uint32_t d = d0 + (uint32_t)(b * p.n_tile);
-            const uint32_t a_add = (a_base >> 4) + (uint32_t)b * 128u;
+          if (leader) {
+            for (int b = 0; b < nblk; ++b) {
+              const uint32_t d = d0 + (uint32_t)(b * p.n_tile);
+              const uint32_t a_add = (a_base >> 4) + (uint32_t)b * 128u;
 #pragma unroll 4
-            for (int j = 0; j < npairs; ++j) {
-              uint32_t lo = p.a_desc_lo[j];
-              if (odd_entries && (uint32_t)j == last) lo = pad_lo;
-              const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
-              const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
-              if (elect_one()) umma_bf16(d, ad, bd, idesc, 1u);
+              for (int j = 0; j < npairs; ++j) {
+                uint32_t lo = p.a_desc_lo[j];
+                if (odd_entries && (uint32_t)j == last) lo = pad_lo;
+                const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(lo + a_add);
+                const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
+                umma_bf16(d, ad, bd, idesc, 1u);
+              }
             }
+            umma_commit(&bar_empty[s]);          // stage s may be refilled once these MMAs finish
           }
-          if (elect_one()) umma_commit(&bar_empty[s]);   // stage s may be refilled once these MMAs finish
+          __syncwarp();
         }
-        if (elect_one()) umma_commit(&bar_accfull[a]);   // accumulator a is complete
+        if (leader) umma_commit(&bar_accfull[a]);        // accumulator a is complete
+        __syncwarp();
       }
     }
   mma_done:;

@@ -453,6 +453,8 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
       const uint32_t b_step = 2u * (uint32_t)p.n_pad;
       const uint32_t a_row0 = smem_u32(smem_a) >> 4, a_stage_rows = (uint32_t)p.a_stage_bytes >> 4;
       bool ok = warp_wait(&sh.weights, 0, abort_flag, ws, 0x70000u);
+      // one election for the whole role: the same lane issues a block's instructions in one stretch
+      const bool leader = elect_one();
       int s = 0;                                 // stage and its phase, accumulator slot and its phase
       uint32_t ph = 0, slot = (uint32_t)mw, sph = 1, a_row = a_row0;
       while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
@@ -473,20 +475,24 @@ k_conv_tc_fold(const __grid_constant__ FoldParams p, const __nv_bfloat16 *__rest
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
           const uint32_t a_add = a_row + (uint32_t)(b * p.blk_rows);
           // statically indexed so that the table entries are read straight from the constant bank
+          if (leader) {
 #pragma unroll
-          for (int j = 0; j < kMaxPairs; ++j) {
-            if (j < p.npairs) {
-              const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(p.a_desc_lo[j] + a_add);
-              const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
-              if (elect_one()) umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+            for (int j = 0; j < kMaxPairs; ++j) {
+              if (j < p.npairs) {
+                const uint64_t ad = ((uint64_t)desc_hi << 32) | (uint64_t)(p.a_desc_lo[j] + a_add);
+                const uint64_t bd = ((uint64_t)desc_hi << 32) | (uint64_t)(b_lo0 + (uint32_t)j * b_step);
+                umma_bf16(d, ad, bd, idesc, j != 0 ? 1u : 0u);
+              }
             }
+            umma_commit(&sh.slot_full[slot]);    // the block's accumulator is complete
           }
-          if (elect_one()) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
+          __syncwarp();
           slot += (uint32_t)p.mma_warps;
           while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
         }
         // this warp's share of the stage: free once its MMAs have finished (at once if it had none)
-        if (ok && elect_one()) umma_commit(&sh.empty[s]);
+        if (ok && leader) umma_commit(&sh.empty[s]);
+        __syncwarp();
         c0 += nblk;
         t.step(p);
         a_row += a_stage_rows;

@@ -476,14 +476,18 @@ k_conv_tc_pairrows(const __grid_constant__ CUtensorMap map_a, const __grid_const
           const uint32_t d = tmem_base + slot * (uint32_t)p.n_pad;
           const uint32_t a_add = a_row + (uint32_t)(b * 1024);    // 128 rows of 128 bytes, in 16-byte units
           uint32_t b_lo = b_lo0;
-          if (leader) umma_bf16(d, ones_desc, bias_desc, idesc, 0u);     // the bias initialises the accumulator
+          // one lane issues the block's instructions in one stretch (no branch per instruction)
+          if (leader) {
+            umma_bf16(d, ones_desc, bias_desc, idesc, 0u);               // the bias initialises the accumulator
 #pragma unroll 2
-          for (int j = 0; j < p.nmma; ++j, b_lo += b_step) {
-            const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(p.a_lo[j] + a_add);
-            const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-            if (leader) umma_bf16(d, ad, bd, idesc, 1u);
+            for (int j = 0; j < p.nmma; ++j, b_lo += b_step) {
+              const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(p.a_lo[j] + a_add);
+              const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
+              umma_bf16(d, ad, bd, idesc, 1u);
+            }
+            umma_commit(&sh.slot_full[slot]);    // the block's accumulator is complete
           }
-          if (leader) umma_commit(&sh.slot_full[slot]);   // the block's accumulator is complete
+          __syncwarp();
           slot += (uint32_t)p.mma_warps;
           while (slot >= (uint32_t)p.slots) { slot -= (uint32_t)p.slots; sph ^= 1; }
         }

@@ -26,8 +26,9 @@
 namespace {
 using namespace tc;
 
-constexpr int kMaxA = 3;                         // activation plane stages
-constexpr int kMaxB = 4;                         // weight stages
+constexpr int kMaxA = 8;                         // activation plane stages
+constexpr int kMaxB = 12;                        // weight stages
+constexpr int kFirstA = 3, kFirstB = 4;          // depths reached first (weights, then activations), before the rings deepen in turn
 constexpr int kMmaWarp = 1;
 constexpr int kMmaWarps = 2;
 constexpr int kFirstEpiWarp = kMmaWarp + kMmaWarps;
@@ -254,27 +255,41 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tc_fence_after();
               b_stage = b_row0 + (uint32_t)sb * ((uint32_t)p.b_stage_bytes >> 4);
             }
+            // One lane issues the step's instructions in one stretch and the warp meets again behind it: with a
+            // branch around every single instruction the warp diverged and met again each time, ~130 cycles per
+            // instruction where the instruction itself takes ~50.  (Measured the same: every lane executing the
+            // instruction under the leader's predicate, no branch at all.)
+            if (leader) {
 #pragma unroll 1
-            for (int b = mw; b < p.mb; b += kMmaWarps) {
-              const uint32_t d = tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile);
-              // descriptors advance by adds only: +8 (one line) per tap column, +2 (32 bytes) per K step on
-              // the activation side, two chunk planes per instruction on the weight side
-              uint32_t a_lo = ((a_stage + (uint32_t)(b * 1024 + r * p.wbox * 8)) & 0x3FFFu) | (1u << 16);
-              uint32_t b_lo = (b_stage & 0x3FFFu) | ((uint32_t)p.n_tile << 16);
-              const uint32_t b_inc = 2u * (uint32_t)p.n_tile;
+              for (int b = mw; b < p.mb; b += kMmaWarps) {
+                const uint32_t d = tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile);
+                // descriptors advance by adds only: +8 (one line) per tap column, +2 (32 bytes) per K step on
+                // the activation side, two chunk planes per instruction on the weight side
+                uint32_t a_lo = ((a_stage + (uint32_t)(b * 1024 + r * p.wbox * 8)) & 0x3FFFu) | (1u << 16);
+                uint32_t b_lo = (b_stage & 0x3FFFu) | ((uint32_t)p.n_tile << 16);
+                const uint32_t b_inc = 2u * (uint32_t)p.n_tile;
+                if (nsl == 4) {                  // a full plane of 64 channels
 #pragma unroll 1
-              for (int s = 0; s < p.k; ++s, a_lo += 8u) {
+                  for (int s = 0; s < p.k; ++s, a_lo += 8u) {
 #pragma unroll
-                for (int sl = 0; sl < 4; ++sl) {
-                  if (sl < nsl) {
-                    const uint64_t ad = ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + 2u * sl);
-                    const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)b_lo;
-                    if (leader) umma_bf16(d, ad, bd, idesc, 1u);
-                    b_lo += b_inc;
+                    for (int sl = 0; sl < 4; ++sl) {
+                      umma_bf16(d, ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + 2u * sl), ((uint64_t)b_hi << 32) | (uint64_t)b_lo, idesc, 1u);
+                      b_lo += b_inc;
+                    }
+                  }
+                } else {
+#pragma unroll 1
+                  for (int s = 0; s < p.k; ++s, a_lo += 8u) {
+#pragma unroll 1
+                    for (int sl = 0; sl < nsl; ++sl) {
+                      umma_bf16(d, ((uint64_t)a_hi << 32) | (uint64_t)(a_lo + 2u * sl), ((uint64_t)b_hi << 32) | (uint64_t)b_lo, idesc, 1u);
+                      b_lo += b_inc;
+                    }
                   }
                 }
               }
             }
+            __syncwarp();
             if (!RESIDENT) {
               if (leader) umma_commit(&sh.b_empty[sb]);    // this warp is done with the weight stage
               if (++sb == p.sb) { sb = 0; pb ^= 1; }
@@ -481,10 +496,23 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->inv_wbox = ((1u << 20) + (uint32_t)p->wbox - 1) / (uint32_t)p->wbox;
   p->ni = 1;
   if (th == ho && p->nxt == 1) {
-    p->ni = kMaxLines / p->lines_img;
-    if (p->ni > n) p->ni = n;
-    if (p->ni > 8) p->ni = 8;
-    if (p->ni < 1) p->ni = 1;
+    int ni_max = kMaxLines / p->lines_img;
+    if (ni_max > n) ni_max = n;
+    if (ni_max > 8) ni_max = 8;
+    if (ni_max < 1) ni_max = 1;
+    // Fewer images per tile where that fills the machine: a work item takes in its activation planes and its
+    // pass's weights from L2, and the launch lasts as long as the CTA with the most items.  Cost of a choice =
+    // items per CTA x (bytes of an item + 64 KB for the item's own chain of waits); a smaller count must win
+    // by a tenth.  960 -> 160, 1 x 1, 128 images of 7 x 7: two images per tile (128 items) instead of five (52).
+    const long long w_item = (long long)ko.e_pad * p->n_tile * 16;
+    long long best_cost = 0;
+    p->ni = ni_max;
+    for (int c = ni_max; c >= 1; --c) {
+      const long long items_c = (long long)dc_div_up(n, c) * p->nnt;
+      const long long per_cta = (items_c + n_sm - 1) / n_sm;
+      const long long cost = per_cta * ((long long)c * p->lines_img * 128 * p->planes + w_item + 64 * 1024);
+      if (c == ni_max || cost * 10 < best_cost * 9) { best_cost = cost; p->ni = c; }
+    }
   }
   if (p->wbox > 256 || p->rbox > 256) return false;
   p->tiles_y = dc_div_up(ho, th);
@@ -526,8 +554,16 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   };
   if (p->b_resident && total(sa, sb) > kSmemBudget) p->b_resident = 0;
   if (total(sa, sb) > kSmemBudget) return false;
-  while (!p->b_resident && sb < kMaxB && total(sa, sb + 1) <= kSmemBudget) ++sb;
-  while (sa < kMaxA && total(sa + 1, sb) <= kSmemBudget) ++sa;
+  while (!p->b_resident && sb < kFirstB && total(sa, sb + 1) <= kSmemBudget) ++sb;
+  while (sa < kFirstA && total(sa + 1, sb) <= kSmemBudget) ++sa;
+  // Layers of many input planes with small stages (deep 1 x 1 layers: 10-30 KB per step) are bound by the
+  // bytes in flight (a stage comes back ~1 us after it was asked for), so what shared memory is left deepens
+  // both rings in turn.
+  for (bool grew = true; grew;) {
+    grew = false;
+    if (!p->b_resident && sb < kMaxB && total(sa, sb + 1) <= kSmemBudget) { ++sb; grew = true; }
+    if (sa < kMaxA && total(sa + 1, sb) <= kSmemBudget) { ++sa; grew = true; }
+  }
   p->sa = sa; p->sb = sb;
   p->off_b = p->off_a + sa * p->a_stage_bytes;
   p->smem_bytes = (int)total(sa, sb);

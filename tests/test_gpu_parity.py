@@ -405,8 +405,11 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (32, 40, 1, 1, 0, 2, 20, 24, "k_conv_tc"),              # 1x1 with 40 outputs: general kernel
     (16, 128, 3, 1, 1, 1, 12, 16, "k_conv_tc_pairrows"),    # N = 256: two accumulator slots, run-time channel loop
     (32, 64, 3, 2, 1, 1, 28, 28, "k_conv_tc_pairrows"),     # stride 2, 64 output channels
-    (160, 200, 3, 1, 1, 5, 7, 7, "k_conv_tc_rows"),         # three planes (the last half full), two passes, three images per tile
-    (96, 64, 1, 1, 0, 7, 7, 7, "k_conv_tc_rows"),           # 1x1: five images per tile, the last group partial
+    (160, 200, 3, 1, 1, 5, 7, 7, "k_conv_tc_rows"),         # three planes (the last half full), two passes; few images: one per tile
+    (96, 64, 1, 1, 0, 7, 7, 7, "k_conv_tc_rows"),           # 1x1 at 7 x 7, few images: one per tile
+    (96, 64, 1, 1, 0, 733, 7, 7, "k_conv_tc_rows"),         # 1x1, a machine's worth of images: five per tile (147 tiles), the last group of three
+    (160, 200, 3, 1, 1, 300, 7, 7, "k_conv_tc_rows"),       # 3x3 at 7 x 7 with more tiles than CTAs: three images per tile, two passes
+    (960, 160, 1, 1, 0, 128, 7, 7, "k_conv_tc_rows"),       # deep projection of the network: two images per tile fill the machine (five would leave two thirds idle)
     (64, 48, 5, 1, 2, 1, 20, 70, "k_conv_tc_rows"),         # 5x5, two column strips, row tiles
     (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
     (128, 128, 5, 1, 2, 2, 14, 14, "k_conv_tc_rows"),       # 5x5 with 128 outputs: two passes of 64 (weight stage limit)
