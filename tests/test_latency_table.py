@@ -170,3 +170,69 @@ def test_plan_from_boundaries_builds_the_same_ops_as_the_span_planner():
     with pytest.raises(ValueError):
         I.plan_from_boundaries(net, acts, [0, kept, kept + 2] + list(range(kept + 3, L + 1)),
                                lambda a, c: LT.span_residuals(net, a, c) if c - a > 1 else [])
+
+
+@pytest.mark.gpu
+def test_latency_planned_network_at_full_size_per_launch_group():
+    """The bench's second cfg4 plan at its own size (batch 128, 224 x 224): the table is measured on the
+    spot, Algorithm 1 cuts the network with the seed's kept activations fixed, and every launch group's
+    output (NaN-filled, between sentinel bands) is compared on images 0, 63 and 127 with the oracle applied
+    to the GPU's own previous map: rel-L2 and the element-wise bound, 3 x for an unmerged block."""
+    import numpy as np
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from oracle import dc_oracle as O
+    from paper_2301_12187_b200 import dc
+    from paper_2301_12187_b200.network import CompressedNetwork
+    from parity_util import Guarded, assert_close
+    dc.lib()
+    net = I.mobilenet_v2(seed=0, batch=128)
+    L = len(net.layers)
+    acts = I.removed_activations(net, seed=0)
+    T, _ = LT.measure_latency_table(net, unit_us=0.1, reps=3, max_span=9)
+    ops, bounds, total = LT.latency_optimal_plan(net, acts, T)
+    assert bounds[0] == 0 and bounds[-1] == L
+    cn = CompressedNetwork(net, acts, ops)
+    guards = []
+    for op in cn.ops:
+        gy = Guarded(torch, tuple(op.out_shape), torch.bfloat16, fill=float("nan"))
+        op.y = gy.t
+        guards.append(gy)
+    cn.merge()
+    x = torch.from_numpy(I.make_input(0, net.x_shape, bf16=True)).to("cuda", dtype=torch.bfloat16)
+    cn.forward(x)
+    torch.cuda.synchronize()
+    assert cn.status() == dc.OK
+
+    def nchw(t):
+        return t.float().cpu().numpy().astype(np.float64).transpose(0, 3, 1, 2)
+
+    sel = [0, 63, 127]
+    prev = x
+    for op, gy in zip(cn.ops, guards):
+        what = "+".join(net.layers[i].name for i in op.layers)
+        gy.check("output of " + what)
+        specs = [net.layers[i] for i in op.layers]
+        cur = nchw(prev[sel])
+        if op.kind == "block":
+            ref = cur
+            for s in specs:
+                Wf, bf = O.fold_bn(s)
+                ref = O.conv_direct(ref, Wf, bf, s.k, s.stride, s.pad, s.groups)
+                if s.act == "relu6":
+                    ref = O.relu6(ref)
+            if net.blocks[specs[0].block]["residual"]:
+                ref = ref + cur
+        else:
+            po = cn.plan_ops[op.plan_index[0]]
+            ref = O.chain_forward_reordered(cur, specs, po.residuals)
+            if op.add_from == -1:
+                ref = ref + nchw(x[sel])
+            elif op.add_from >= 0:
+                ref = ref + nchw(cn.ops[op.add_from].y[sel])
+            if po.act == "relu6":
+                ref = O.relu6(ref)
+        k = 3.0 if op.kind == "block" else 1.0
+        assert_close(nchw(op.y[sel]), ref, k * 2e-2, scale=k, what=what)
+        prev = op.y
