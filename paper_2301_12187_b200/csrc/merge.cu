@@ -192,8 +192,11 @@ __global__ void __launch_bounds__(256) k_compose_dd_tiled(Piece first, Piece sec
 // accumulators); slices of 8 intermediate channels are staged in shared memory with the next slice's
 // loads in flight (taps padded to 12 floats, read as three 16-byte vectors).  blockIdx.x walks the
 // tiles (i fastest); the blocks after them compute the bias.
+// At most 128 registers per thread, so that two CTAs share an SM and one's loads hide behind the other's
+// arithmetic (c = 512: 1.31 -> 0.97 ms).  Tiles of 8 output channels in CTAs of 128 threads, for results with
+// fewer tiles than two per SM, were measured and spill (c = 256: 209 -> 302 us): not kept.
 constexpr int kPolyC = 8;
-__global__ void __launch_bounds__(256) k_compose_poly33(Piece first, Piece second, float *out, float *b_out, int gx, int gy) {
+__global__ void __launch_bounds__(256, 2) k_compose_poly33(Piece first, Piece second, float *out, float *b_out, int gx, int gy) {
   __shared__ __align__(16) float W2s[2][16][kPolyC][12];   // [o][c][tap]
   __shared__ __align__(16) float W1s[2][kPolyC][32][12];   // [c][i][tap]
   if ((int)blockIdx.x >= gx * gy) {
