@@ -113,15 +113,22 @@ __global__ void __launch_bounds__(256) k_compose_dd_tiled(Piece first, Piece sec
   const int ar = t & 15, ao = t >> 4;
   const int jj = t & 63, j = j0 + jj, br = t >> 6;
   const int bi = j / (kk * kk), btp = j - bi * kk * kk, bup = btp / kk, bvp = btp - bup * kk;
+  // fetch() only issues the loads (from a safe address where the element is structurally zero) and keeps what
+  // decides the element's value as two bit masks; the values are first touched in stage(), behind the
+  // arithmetic on the current slice, so the loads' round trips hide behind it.  (With the selects in fetch()
+  // every warp waited for its loads before it started on the slice.)
   float av[TM], bv[4];
+  uint32_t a_ok, a_id, b_ok, b_id;
   auto fetch = [&](int r0) {
     const int ra = r0 + ar;
+    a_ok = a_id = b_ok = b_id = 0u;
 #pragma unroll
     for (int q = 0; q < TM; ++q) {
       const int o = o0 + ao + 16 * q;
       const bool ok = o < c2 && ra < R;
-      const float x = second.w[ok ? (size_t)o * R + ra : 0];
-      av[q] = ok ? ((second.ident && ra == (o * k2 + ctr2) * k2 + ctr2) ? x + 1.f : x) : 0.f;
+      av[q] = second.w[ok ? (size_t)o * R + ra : 0];
+      a_ok |= (ok ? 1u : 0u) << q;
+      a_id |= ((ok && second.ident && ra == (o * k2 + ctr2) * k2 + ctr2) ? 1u : 0u) << q;
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -135,15 +142,18 @@ __global__ void __launch_bounds__(256) k_compose_dd_tiled(Piece first, Piece sec
       }
       const int u1 = bup - s1 * u2, v1 = bvp - s1 * v2;
       const bool ok = r < R && j < J && u1 >= 0 && u1 < k1 && v1 >= 0 && v1 < k1;
-      const float x = first.w[ok ? (((size_t)c * c0 + bi) * k1 + u1) * k1 + v1 : 0];
-      bv[u] = ok ? ((first.ident && c == bi && u1 == ctr1 && v1 == ctr1) ? x + 1.f : x) : 0.f;
+      bv[u] = first.w[ok ? (((size_t)c * c0 + bi) * k1 + u1) * k1 + v1 : 0];
+      b_ok |= (ok ? 1u : 0u) << u;
+      b_id |= ((ok && first.ident && c == bi && u1 == ctr1 && v1 == ctr1) ? 1u : 0u) << u;
     }
   };
   auto stage = [&](int buf) {
 #pragma unroll
-    for (int q = 0; q < TM; ++q) As[buf][ar][ao + 16 * q] = av[q];
+    for (int q = 0; q < TM; ++q)
+      As[buf][ar][ao + 16 * q] = ((a_ok >> q) & 1u) ? (((a_id >> q) & 1u) ? av[q] + 1.f : av[q]) : 0.f;
 #pragma unroll
-    for (int u = 0; u < 4; ++u) Bs[buf][br + 4 * u][jj] = bv[u];
+    for (int u = 0; u < 4; ++u)
+      Bs[buf][br + 4 * u][jj] = ((b_ok >> u) & 1u) ? (((b_id >> u) & 1u) ? bv[u] + 1.f : bv[u]) : 0.f;
   };
   float acc[TM][4] = {};
   fetch(0);
@@ -208,35 +218,42 @@ __global__ void __launch_bounds__(256, 2) k_compose_poly33(Piece first, Piece se
   const int t = threadIdx.x, ol = t >> 4, il = t & 15;       // this thread's o, and i = il, il + 16
   // loads of a slice: W2: 16 o x 8 c x 9 = 1152 floats, W1: 8 c x 32 i x 9 = 2304 floats
   constexpr int N2 = (16 * kPolyC * 9 + 255) / 256, N1 = (kPolyC * 32 * 9) / 256;
+  // fetch() only issues the loads and notes in bit masks what decides each element's value; the values are
+  // first touched in stage(), behind the arithmetic on the current slice (see k_compose_dd_tiled).
   float r2[N2], r1[N1];
+  uint32_t ok2, id2, ok1, id1;
   auto fetch = [&](int cs) {
+    ok2 = id2 = ok1 = id1 = 0u;
 #pragma unroll
     for (int q = 0; q < N2; ++q) {
       const int e = t + 256 * q;                 // (o, c, tap): taps of one (o, c) are contiguous in memory
       const int tap = e % 9, oc = e / 9, cl = oc % kPolyC, o = o0 + oc / kPolyC, c = cs + cl;
       const bool ok = e < 16 * kPolyC * 9 && o < c2 && c < c1;
-      const float x = second.w[ok ? ((size_t)o * c1 + c) * 9 + tap : 0];
-      r2[q] = ok ? ((second.ident && o == c && tap == 4) ? x + 1.f : x) : 0.f;
+      r2[q] = second.w[ok ? ((size_t)o * c1 + c) * 9 + tap : 0];
+      ok2 |= (ok ? 1u : 0u) << q;
+      id2 |= ((ok && second.ident && o == c && tap == 4) ? 1u : 0u) << q;
     }
 #pragma unroll
     for (int q = 0; q < N1; ++q) {
       const int e = t + 256 * q;                 // (c, i, tap)
       const int tap = e % 9, ci = e / 9, i = i0 + ci % 32, c = cs + ci / 32;
       const bool ok = c < c1 && i < c0;
-      const float x = first.w[ok ? ((size_t)c * c0 + i) * 9 + tap : 0];
-      r1[q] = ok ? ((first.ident && c == i && tap == 4) ? x + 1.f : x) : 0.f;
+      r1[q] = first.w[ok ? ((size_t)c * c0 + i) * 9 + tap : 0];
+      ok1 |= (ok ? 1u : 0u) << q;
+      id1 |= ((ok && first.ident && c == i && tap == 4) ? 1u : 0u) << q;
     }
   };
   auto stage = [&](int buf) {
 #pragma unroll
     for (int q = 0; q < N2; ++q) {
       const int e = t + 256 * q, tap = e % 9, oc = e / 9;
-      if (e < 16 * kPolyC * 9) W2s[buf][oc / kPolyC][oc % kPolyC][tap] = r2[q];
+      if (e < 16 * kPolyC * 9)
+        W2s[buf][oc / kPolyC][oc % kPolyC][tap] = ((ok2 >> q) & 1u) ? (((id2 >> q) & 1u) ? r2[q] + 1.f : r2[q]) : 0.f;
     }
 #pragma unroll
     for (int q = 0; q < N1; ++q) {
       const int e = t + 256 * q, tap = e % 9, ci = e / 9;
-      W1s[buf][ci / 32][ci % 32][tap] = r1[q];
+      W1s[buf][ci / 32][ci % 32][tap] = ((ok1 >> q) & 1u) ? (((id1 >> q) & 1u) ? r1[q] + 1.f : r1[q]) : 0.f;
     }
   };
   float acc[2][25] = {};
