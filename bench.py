@@ -10,7 +10,7 @@ merge (cfg3) and the full depth-compressed MobileNetV2-1.0 (cfg4: with every val
 pattern merged, and cut by Algorithm 1 over the latency table measured on the spot) and reports them
 under `per_config` of the same JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|cfg1|cfg2|cfg3|cfg4] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload all|cfg1|cfg2|cfg3|cfg4|vgg] [--impl reference]
 
 Prints one JSON line (rank 0).  `value` = images/s with inputs resident in HBM; `e2e` = the same
 through the host-buffer entry point with the copies inside the timed region; `roofline` = the
@@ -212,11 +212,11 @@ class ChainBench:
     step, of the conv forward alone and of the merge alone."""
     MERGES_PER_GRAPH = 10            # a one-merge graph would time the graph launch, not the merge
 
-    def __init__(self, name, seed, stream):
+    def __init__(self, name, seed, stream, case=None):
         import torch
         from paper_2301_12187_b200 import dc, inputs as I
         self.torch, self.dc, self.name, self.stream = torch, dc, name, stream
-        case = self.case = I.chain_case(WORKLOADS[name], seed=seed)
+        case = self.case = case if case is not None else I.chain_case(WORKLOADS[name], seed=seed)
         n, h, w, c = case.x_shape
         self.layers = [dc.DeviceLayer(s) for s in case.layers]
         g, merge_ws_bytes = dc.merge_query(self.layers, case.residuals)
@@ -611,6 +611,29 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    if args.workload == "vgg":
+        # VGG-style runs (two dense 3x3 layers of 64..512 channels -> one 5x5 layer): merge latency and the merged
+        # layer's forward by the same protocol (graph replays, L2-cold by rotation), kernel figures only
+        from paper_2301_12187_b200 import inputs as I
+        stream = torch.cuda.Stream()
+        per = {}
+        for c in sorted(I.VGG_MAPS):
+            cb = ChainBench("vgg_c%d" % c, R.replica_seed(0, rank), stream, case=I.vgg_case(c, seed=R.replica_seed(0, rank)))
+            f = cb.kernel_figures(peaks, peak_src)
+            f["config"] = cb.config()
+            per[cb.name] = f
+            cb.free()
+        if rank == 0:
+            head = per["vgg_c512"]
+            print(json.dumps({"metric": METRIC, "value": head["roofline"]["images_per_s_kernel_only"] * world, "unit": "images/s",
+                              "n_gpus": world, "steps": head["conv_forward_us"]["replays"], "warmup": KERNEL_WARMUPS,
+                              "ms_per_step": head["step_us"]["median"] * 1e-3, "higher_is_better": True, "scaling": "weak",
+                              "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": head["config"],
+                              "roofline": head["roofline"], "per_config": per}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     headline = "cfg1" if args.workload == "all" else args.workload
     stream = torch.cuda.Stream()
     hb = ChainBench(headline, R.replica_seed(0, rank), stream)
@@ -710,7 +733,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=200)
-    ap.add_argument("--workload", default="all", choices=["all"] + sorted(WORKLOADS),
+    ap.add_argument("--workload", default="all", choices=["all", "vgg"] + sorted(WORKLOADS),
                     help="all: cfg1 as the headline line plus cfg1..cfg4 (cfg4 under both plans) under per_config (one GPU); cfgN: that workload alone")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -182,6 +182,18 @@ def chain_case(idx: int, seed: int = 0, batch: Optional[int] = None) -> ChainCas
     raise ValueError("chain_case index must be 0..3")
 
 
+VGG_MAPS = {64: 224, 128: 112, 256: 56, 512: 28}       # channel width -> feature-map side of that VGG stage
+
+
+def vgg_case(c: int, seed: int = 0, batch: int = 32) -> ChainCase:
+    """Two dense 3x3 layers c -> c -> c (stride 1, padding 1, BN each) with an identity in between, on the
+    feature map of the VGG stage of that width: the run that merges into one 5x5 layer."""
+    L = [make_layer(seed, 0, c, c, 3, 1, 1, act=None, name="conv_a"),
+         make_layer(seed, 1, c, c, 3, 1, 1, act=None, name="conv_b")]
+    hw = VGG_MAPS[c]
+    return ChainCase("vgg_c%d" % c, "bf16", L, [], (batch, hw, hw, c), seed)
+
+
 # --------------------------------------------------------------------------- MobileNetV2-1.0
 
 
