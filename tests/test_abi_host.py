@@ -160,3 +160,17 @@ def test_host_parameter_layout_offsets():
             o += r(s.weight.size * 4 if j == 0 else s.c_out * 4)
     assert list(offs) == want and total.value == o
     assert dc.lib().dc_chain_host_param_layout(arr, 0, offs, C.byref(total)) == dc.ERR_INVALID_ARG
+
+
+def test_vgg_style_cases_have_the_shapes_of_their_stage():
+    """Host logic of the bench's VGG-style workload: two dense 3x3 layers of equal width with no activation
+    between them, on the map of that width's stage; by the oracle's geometry rule they merge into a 5x5
+    layer with padding 2 (two 3x3 -> 5x5)."""
+    from oracle import dc_oracle as O
+    from paper_2301_12187_b200 import inputs as I
+    assert sorted(I.VGG_MAPS) == [64, 128, 256, 512]
+    for c, hw in I.VGG_MAPS.items():
+        case = I.vgg_case(c, seed=3, batch=2)
+        assert case.x_shape == (2, hw, hw, c) and case.dtype == "bf16" and case.residuals == []
+        assert [(s.c_in, s.c_out, s.k, s.stride, s.pad, s.groups, s.act) for s in case.layers] == [(c, c, 3, 1, 1, 1, None)] * 2
+        assert O.compose_geometry(case.layers) == (5, 1, 2)
