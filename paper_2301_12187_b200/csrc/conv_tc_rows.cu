@@ -45,6 +45,7 @@ struct RowsParams {
   int tw, th, nxt, wbox, rbox, ni;   // tile: outputs per row, rows, strips per row, patch width / rows, images
   int tiles_y, img_groups;
   int grid, items_per, items_rem;    // CTAs; CTA b takes items_per (+1 if b < items_rem) work items
+  int split;                         // the counts above are 128-row blocks instead: a CTA's run may begin and end inside an item
   int n_tile, nnt, n_pad;      // output channels per pass, passes, nnt * n_tile
   int planes_all;              // chunk planes of the packed weights (all 64-channel planes and taps)
   int mb;                      // blocks per tile
@@ -107,8 +108,20 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   volatile uint32_t *abort_flag = &sh.abort;
 
   const int bid = (int)blockIdx.x;
-  const int nitems = p.items_per + (bid < p.items_rem ? 1 : 0);
-  const int item0 = bid * p.items_per + (bid < p.items_rem ? bid : p.items_rem);
+  // This CTA's run of work items.  When the plan balances by blocks (split), the run is counted in 128-row
+  // blocks: its first item starts at block blk_first and its last one ends before blk_end; the tile and the
+  // weights of such an item are still staged whole.
+  int nitems = p.items_per + (bid < p.items_rem ? 1 : 0);
+  int item0 = bid * p.items_per + (bid < p.items_rem ? bid : p.items_rem);
+  int blk_first = 0, blk_end = p.mb;
+  if (p.split) {
+    const int u0 = item0, u1 = item0 + nitems - 1;           // first and last block of the run
+    item0 = u0 / p.mb;
+    const int item1 = u1 / p.mb;
+    nitems = item1 - item0 + 1;
+    blk_first = u0 - item0 * p.mb;
+    blk_end = u1 - item1 * p.mb + 1;
+  }
 
   {
     const int t = (int)threadIdx.x;
@@ -226,6 +239,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll 1
       for (int it = 0; it < nitems && ok; ++it) {
         const int set = p.nacc == 2 ? (it & 1) : 0;
+        const int blk_lo = it == 0 ? blk_first : 0, blk_hi = it == nitems - 1 ? blk_end : p.mb;   // this run's blocks of the item
         if (!warp_wait(&sh.acc_empty[set], acc_ph[set], abort_flag, ws, 0x30000u | set)) break;
         acc_ph[set] ^= 1u;
         tc_fence_after();
@@ -236,7 +250,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t bias_row = bias_row0 + (uint32_t)(iq.nt * p.n_tile);
           const uint64_t bd = ((uint64_t)b_hi << 32) | (uint64_t)((bias_row & 0x3FFFu) | ((zero_row - bias_row) << 16));
 #pragma unroll 1
-          for (int b = mw; b < p.mb; b += kMmaWarps)
+          for (int b = blk_lo + mw; b < blk_hi; b += kMmaWarps)
             if (leader) umma_bf16(tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile), ones_desc, bd, idesc, 0u);
         }
 #pragma unroll 1
@@ -261,7 +275,7 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // instruction under the leader's predicate, no branch at all.)
             if (leader) {
 #pragma unroll 1
-              for (int b = mw; b < p.mb; b += kMmaWarps) {
+              for (int b = blk_lo + mw; b < blk_hi; b += kMmaWarps) {
                 const uint32_t d = tmem_base + (uint32_t)((set * p.mb + b) * p.n_tile);
                 // descriptors advance by adds only: +8 (one line) per tap column, +2 (32 bytes) per K step on
                 // the activation side, two chunk planes per instruction on the weight side
@@ -331,8 +345,9 @@ k_conv_tc_rows(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int th_valid = p.ho - y0 < p.th ? p.ho - y0 : p.th;
         const int ch0 = iq.nt * p.n_tile;
         const int nch = p.c_out - ch0 < p.n_tile ? p.c_out - ch0 : p.n_tile;   // multiple of 8
+        const int blk_lo = it == 0 ? blk_first : 0, blk_hi = it == nitems - 1 ? blk_end : p.mb;   // this run's blocks of the item
 #pragma unroll 1
-        for (int b = par; b < p.mb; b += 2) {
+        for (int b = blk_lo + par; b < blk_hi; b += 2) {
           const int pos = b * 128 + q * 32 + lane;
           // pos < 512 and the divisors are at most 256: multiplying by the rounded-up reciprocal is exact
           const int il = (int)(((uint32_t)pos * p.inv_lines) >> 20), rem = pos - il * p.lines_img;
@@ -530,6 +545,21 @@ bool rows_plan(int n, int h, int w, const dc_geom *g, int n_sm, RowsParams *p) {
   p->grid = items < n_sm ? (int)items : n_sm;
   p->items_per = (int)(items / p->grid);
   p->items_rem = (int)(items % p->grid);
+  // Where whole items leave some CTAs a block more than an even split would (160 -> 960, 3 x 3 at 7 x 7: 344
+  // items of two blocks on 148 SMs, three items = six blocks on 48 of them against five by blocks), the runs are
+  // cut by blocks: an item at a run's end is then shared by two CTAs, each staging its tile and weights.
+  p->split = 0;
+  if (p->mb > 1) {
+    const long long units = items * p->mb;
+    const int grid_u = units < n_sm ? (int)units : n_sm;
+    const long long whole = (items / p->grid + (items % p->grid ? 1 : 0)) * p->mb, cut = units / grid_u + (units % grid_u ? 1 : 0);
+    if (cut * 8 <= whole * 7 && units < (1ll << 30)) {     // worth it from an eighth less (a shared item is staged twice)
+      p->split = 1;
+      p->grid = grid_u;
+      p->items_per = (int)(units / grid_u);
+      p->items_rem = (int)(units % grid_u);
+    }
+  }
   p->a_box_bytes = p->ni * p->lines_img * 128;
   p->a_stage_bytes = (int)dc_round_up((size_t)p->a_box_bytes, 1024);
   p->b_stage_bytes = (int)dc_round_up((size_t)g->k * 4 * 2 * p->n_tile * 16, 1024);
