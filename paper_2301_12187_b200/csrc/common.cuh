@@ -183,7 +183,7 @@ static inline void dc_korder_init(KOrder *ko, const dc_geom *g) {
     // output channels per pass: at most 128, fewer for 5x5 and 7x7 kernels, whose weight stage of one
     // (plane, tap row) step (k * 8 chunk planes of n_tile rows) must fit the shared-memory ring twice
     // beside two activation stages and the epilogue's turn-around buffers
-    const int n_tile_max = g->k <= 4 ? 128 : (g->k <= 5 ? 96 : 64);
+    const int n_tile_max = (g->k == 1 && g->c_in >= 512 && g->c_out > 256) ? 256 : (g->k <= 4 ? 128 : (g->k <= 5 ? 96 : 64));
     ko->nnt = dc_div_up(n16, n_tile_max);
     ko->n_tile = (int)dc_round_up((size_t)dc_div_up(n16, ko->nnt), 16);
     ko->n_pad = ko->nnt * ko->n_tile;
