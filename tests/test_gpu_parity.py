@@ -410,6 +410,7 @@ def test_single_conv_bf16_with_explicit_skip(dc, c_in, c_out, k, s, p, n, h, w, 
     (96, 64, 1, 1, 0, 733, 7, 7, "k_conv_tc_rows"),         # 1x1, a machine's worth of images: five per tile (147 tiles), the last group of three
     (160, 200, 3, 1, 1, 300, 7, 7, "k_conv_tc_rows"),       # 3x3 at 7 x 7 with more items than CTAs: three images per tile, two passes, runs cut by blocks (items shared by two CTAs)
     (960, 160, 1, 1, 0, 128, 7, 7, "k_conv_tc_rows"),       # deep projection of the network: two images per tile fill the machine (five would leave two thirds idle)
+    (512, 512, 1, 1, 0, 6, 7, 7, "k_conv_tc_rows"),          # deep 1x1 with more than 256 outputs: two passes of 256 channels, one accumulator set
     (64, 48, 5, 1, 2, 1, 20, 70, "k_conv_tc_rows"),         # 5x5, two column strips, row tiles
     (384, 64, 3, 1, 1, 2, 14, 14, "k_conv_tc_rows"),        # six planes, whole image per tile
     (128, 128, 5, 1, 2, 2, 14, 14, "k_conv_tc_rows"),       # 5x5 with 128 outputs: two passes of 64 (weight stage limit)
